@@ -1,0 +1,329 @@
+"""Seeded synthetic inputs shaped like the paper's DeiT / ViT / Swin workloads.
+
+This module holds NONE of the method's integer arithmetic: it draws float
+tensors with numpy, quantises them with the plain uniform quantiser of the
+paper's background section (round(x / s) + z, clipped), and runs an fp64
+"shadow" forward pass only to pick the scale of every intermediate tensor
+(the job PTQ calibration does on real images).  Both the CUDA library and the
+CPU oracle are fed from here; each side then derives its own integer constants
+with its own ``*_prepare`` functions.
+
+The inputs stand in for ImageNet / COCO activations and trained weights, which
+are not available: logits ~ N(0, 3^2) with 1 % of each row set to +12, GELU
+inputs ~ N(-0.3, 1.2^2) with a 0.5 % Laplace(0, 4) tail, LayerNorm inputs
+~ N(0, 1) with 2 % of the channels scaled by 20, weights ~ N(0, 0.02^2).
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+
+import numpy as np
+
+# ------------------------------------------------------------------ shapes
+
+
+@dataclass(frozen=True)
+class BlockShape:
+    name: str
+    B: int        # images (or windows, for Swin)
+    N: int        # tokens per attention problem
+    D: int        # embedding dim
+    H: int        # heads
+    dh: int       # head dim
+    Dh: int       # MLP hidden dim
+    has_bias: bool = False   # relative-position bias [H, N, N]
+
+    @property
+    def T(self) -> int:
+        return self.B * self.N
+
+    def gemm_ops(self) -> int:
+        """2 * sum(M*N*K) of the real (unpadded) contractions of one block."""
+        T, D, Dh, N, dh = self.T, self.D, self.Dh, self.N, self.dh
+        lin = T * D * (3 * D) + T * D * D + 2 * T * D * Dh
+        att = 2 * self.B * self.H * N * N * dh
+        return 2 * (lin + att)
+
+
+CONFIGS = {
+    "cfg0": BlockShape("DeiT-Tiny b1", 1, 197, 192, 3, 64, 768),
+    "cfg1": BlockShape("DeiT-Small b64", 64, 197, 384, 6, 64, 1536),
+    "cfg2": BlockShape("ViT-Base b128", 128, 197, 768, 12, 64, 3072),
+    "cfg3": BlockShape("Swin-Tiny stage1 b64", 64 * 64, 49, 96, 3, 32, 384, True),
+}
+
+# Swin-Tiny backbone at detection resolution (config 4): token grid 200 x 304.
+SWIN_T_STAGES = [
+    dict(dim=96, heads=3, depth=2, grid=(200, 304)),
+    dict(dim=192, heads=6, depth=2, grid=(100, 152)),
+    dict(dim=384, heads=12, depth=6, grid=(50, 76)),
+    dict(dim=768, heads=24, depth=2, grid=(25, 38)),
+]
+
+
+def _rng(seed: int, stream: int) -> np.random.Generator:
+    """Independent sub-stream ``stream`` of ``seed`` (fixed spawn order)."""
+    return np.random.default_rng(np.random.SeedSequence(seed).spawn(stream + 1)[stream])
+
+
+# ------------------------------------------------------------------ stand-alone non-linear inputs
+
+def softmax_logits(rows: int, n: int, seed: int = 0) -> np.ndarray:
+    """fp64 logits [rows, n]: N(0, 3^2); ceil(1 % of n) random positions per row set to +12."""
+    g = _rng(seed, 0)
+    x = g.normal(0.0, 3.0, size=(rows, n))
+    k = max(1, math.ceil(0.01 * n))
+    pos = np.argsort(g.random((rows, n)), axis=1)[:, :k]
+    np.put_along_axis(x, pos, 12.0, axis=1)
+    return x
+
+
+def quantize_scores(logits: np.ndarray, scale: float) -> np.ndarray:
+    return np.round(logits / scale).astype(np.int32)
+
+
+SOFTMAX_SCALE_ACC = 3.0e-4          # accumulator-like scale: floor(1/S) = 3333
+SOFTMAX_SCALE_8BIT = 12.0 / 127.0   # 8-bit-like scale: floor(1/S) = 10
+
+
+def gelu_values(n: int, seed: int = 0) -> np.ndarray:
+    """fp64 GELU inputs: N(-0.3, 1.2^2), 0.5 % replaced by Laplace(0, 4)."""
+    g = _rng(seed, 1)
+    x = g.normal(-0.3, 1.2, size=n)
+    tail = g.random(n) < 0.005
+    x[tail] = g.laplace(0.0, 4.0, size=int(tail.sum()))
+    return x
+
+
+def quantize_sym(x: np.ndarray, bits: int, dtype=np.int32):
+    """Symmetric per-tensor quantiser: scale = max|x| / (2^(bits-1) - 1)."""
+    qmax = (1 << (bits - 1)) - 1
+    scale = float(np.abs(x).max()) / qmax
+    q = np.clip(np.round(x / scale), -qmax - 1, qmax).astype(dtype)
+    return q, scale
+
+
+def ln_values(rows: int, dim: int, seed: int = 0):
+    """fp64 LayerNorm inputs [rows, dim]: N(0,1) with a fixed random 2 % of channels x20,
+    plus gamma ~ N(1, 0.1^2), beta ~ N(0, 0.1^2)."""
+    g = _rng(seed, 2)
+    x = g.normal(0.0, 1.0, size=(rows, dim))
+    k = max(1, round(0.02 * dim))
+    ch = g.choice(dim, size=k, replace=False)
+    x[:, ch] *= 20.0
+    gamma = g.normal(1.0, 0.1, size=dim).astype(np.float32)
+    beta = g.normal(0.0, 0.1, size=dim).astype(np.float32)
+    return x, gamma, beta, np.sort(ch)
+
+
+def ptf_shifts(xq: np.ndarray) -> np.ndarray:
+    """Per-channel power-of-two factors alpha_c in {0..3}: the channels are quantised
+    at scale S * 2^alpha_c; pick alpha from each channel's range (host-side calibration)."""
+    amax = np.abs(xq.astype(np.int64)).max(axis=0).astype(np.float64)
+    ref = max(1.0, float(np.median(amax)))
+    a = np.clip(np.floor(np.log2(np.maximum(amax, 1.0) / ref)), 0, 3)
+    return a.astype(np.uint8)
+
+
+def affine_out_quant(y: np.ndarray, bits: int = 8):
+    """Asymmetric output quantiser from the range of an fp64 reference:
+    scale = (max - min) / (2^bits - 1), zero point placed in the signed range."""
+    lo, hi = float(y.min()), float(y.max())
+    lo, hi = min(lo, 0.0), max(hi, 0.0)
+    scale = (hi - lo) / ((1 << bits) - 1)
+    zp = int(round(-lo / scale)) - (1 << (bits - 1))
+    return scale, zp
+
+
+# ------------------------------------------------------------------ fp64 references (for calibration / error reports)
+
+def gelu_ref(x):
+    from math import erf
+    v = np.vectorize(erf)
+    return 0.5 * x * (1.0 + v(x / math.sqrt(2.0)))
+
+
+def layernorm_ref(x, gamma, beta):
+    mu = x.mean(axis=-1, keepdims=True)
+    sd = x.std(axis=-1, keepdims=True)
+    sd = np.where(sd == 0, 1.0, sd)
+    return (x - mu) / sd * gamma + beta
+
+
+def softmax_ref(x):
+    e = np.exp(x - x.max(axis=-1, keepdims=True))
+    return e / e.sum(axis=-1, keepdims=True)
+
+
+# ------------------------------------------------------------------ weights
+
+def quantize_weight(w: np.ndarray, bits: int = 8):
+    """Symmetric per-output-channel weight quantiser.  Returns (int8 values, scales[N])."""
+    qmax = (1 << (bits - 1)) - 1
+    s = np.abs(w).max(axis=1) / qmax
+    s = np.where(s == 0, 1.0, s)
+    q = np.clip(np.round(w / s[:, None]), -qmax - 1, qmax).astype(np.int8)
+    return q, s
+
+
+def pack_int4(q: np.ndarray) -> np.ndarray:
+    """Pack int4 values [N, K] two per byte: element k in byte k//2, even k in the low nibble."""
+    assert q.shape[1] % 2 == 0
+    u = (q.astype(np.int16) & 15).astype(np.uint8)
+    return (u[:, 0::2] | (u[:, 1::2] << 4)).astype(np.uint8)
+
+
+# ------------------------------------------------------------------ encoder block
+
+@dataclass
+class LinearSpec:
+    w: np.ndarray            # int8 [N, K] (unpacked values, also for 4-bit)
+    w_packed: np.ndarray     # what the library is given: int8 [N,K] or uint8 [N,K/2]
+    bias: np.ndarray         # int32 [N], input zero-point already folded in
+    ratio: np.ndarray        # fp64 [N]: S_x * S_w[n] / S_out
+    out_zp: int = 0
+    res_ratio: float | None = None   # S_res / S_out of the residual branch (before the 2^-16 widening)
+    res_zp: int = 0
+
+
+@dataclass
+class BlockSpec:
+    shape: BlockShape
+    w_bits: int
+    x: np.ndarray                                  # int8 [T, D]
+    ln1: dict = field(default_factory=dict)        # gamma, beta (float32), out_scale, out_zp
+    ln2: dict = field(default_factory=dict)
+    qkv: LinearSpec | None = None
+    proj: LinearSpec | None = None
+    fc1: LinearSpec | None = None                  # ratio = S_x*S_w[n] / S_gelu_in
+    fc2: LinearSpec | None = None
+    softmax_scale: float = 0.0                     # scale of the int32 scores (1/sqrt(dh) folded in)
+    pv_ratio: float = 0.0                          # 2^-7 * S_v / S_attn
+    gelu: dict = field(default_factory=dict)       # in_scale, in_bits, out_scale, out_zp
+    attn_bias: np.ndarray | None = None            # int32 [H, N, N] at the score scale
+    mask_id: np.ndarray | None = None              # uint8 [B, N]
+
+
+def make_block(shape: BlockShape, seed: int = 0, w_bits: int = 8, gelu_in_bits: int = 16,
+               calib_images: int = 2, mask_id: np.ndarray | None = None) -> BlockSpec:
+    """Draw one encoder block (weights, input) and calibrate every intermediate scale
+    with an fp64 shadow forward over the first ``calib_images`` attention problems."""
+    g = _rng(seed, 3)
+    T, D, H, dh, Dh, N = shape.T, shape.D, shape.H, shape.dh, shape.Dh, shape.N
+    # block input: the LayerNorm-input distribution
+    xin, g1, b1, _ = ln_values(T, D, seed)
+    x, Sx = quantize_sym(xin, 8, np.int8)
+    del xin
+    Tc = min(T, calib_images * N)
+    Bc = Tc // N
+    xc = x[:Tc].astype(np.float64) * Sx
+
+    def draw_w(n, k, gain=1.0):
+        return g.normal(0.0, 0.02, size=(n, k)) * gain, g.normal(0.0, 0.02, size=n) * gain
+
+    def qlin(wf, bf, S_in, w_bits_):
+        wq, Sw = quantize_weight(wf, w_bits_)
+        bq = np.round(bf / (S_in * Sw)).astype(np.int32)
+        wp = pack_int4(wq) if w_bits_ == 4 else wq
+        return wq, Sw, bq, wp
+
+    spec = BlockSpec(shape=shape, w_bits=w_bits, x=x)
+    # ---- LN1
+    h1 = layernorm_ref(xc, g1, b1)
+    S_h1 = float(np.abs(h1).max()) / 127.0
+    spec.ln1 = dict(gamma=g1, beta=b1, out_scale=S_h1, out_zp=0)
+    h1 = np.clip(np.round(h1 / S_h1), -128, 127) * S_h1
+    # ---- QKV; a gain on the q/k rows puts the logits on config 0's N(0, 3^2) spread
+    wf, bf = draw_w(3 * D, D)
+    q0 = h1 @ wf[:D].T + bf[:D]
+    k0 = h1 @ wf[D:2 * D].T + bf[D:2 * D]
+    lg = np.einsum("bnhd,bmhd->bhnm", q0.reshape(Bc, N, H, dh), k0.reshape(Bc, N, H, dh)) / math.sqrt(dh)
+    gain = math.sqrt(3.0 / float(lg.std()))
+    wf[:2 * D] *= gain
+    bf[:2 * D] *= gain
+    wq, Sw, bq, wp = qlin(wf, bf, S_h1, w_bits)
+    qkv = h1 @ (wq * Sw[:, None]).T + bq * (S_h1 * Sw)
+    S_qkv = float(np.abs(qkv).max()) / 127.0
+    spec.qkv = LinearSpec(wq, wp, bq, S_h1 * Sw / S_qkv)
+    qkv = np.clip(np.round(qkv / S_qkv), -128, 127) * S_qkv
+    # ---- attention
+    spec.softmax_scale = S_qkv * S_qkv / math.sqrt(dh)
+    qh = qkv[:, :D].reshape(Bc, N, H, dh)
+    kh = qkv[:, D:2 * D].reshape(Bc, N, H, dh)
+    vh = qkv[:, 2 * D:].reshape(Bc, N, H, dh)
+    lg = np.einsum("bnhd,bmhd->bhnm", qh, kh) / math.sqrt(dh)
+    if shape.has_bias:
+        bias_f = g.normal(0.0, 1.0, size=(H, N, N))
+        spec.attn_bias = np.round(bias_f / spec.softmax_scale).astype(np.int32)
+        lg = lg + spec.attn_bias[None] * spec.softmax_scale
+    if mask_id is not None:
+        spec.mask_id = np.ascontiguousarray(mask_id, dtype=np.uint8)
+        mm = spec.mask_id[:Bc, :, None] != spec.mask_id[:Bc, None, :]
+        lg = np.where(mm[:, None], -1e9, lg)
+    P = softmax_ref(lg)
+    att = np.einsum("bhnm,bmhd->bnhd", P, vh).reshape(Tc, D)
+    S_att = float(np.abs(att).max()) / 127.0
+    spec.pv_ratio = (2.0 ** -7) * S_qkv / S_att
+    att = np.clip(np.round(att / S_att), -128, 127) * S_att
+    # ---- proj + residual
+    wf, bf = draw_w(D, D)
+    wq, Sw, bq, wp = qlin(wf, bf, S_att, w_bits)
+    x1 = att @ (wq * Sw[:, None]).T + bq * (S_att * Sw) + xc
+    S_x1 = float(np.abs(x1).max()) / 127.0
+    spec.proj = LinearSpec(wq, wp, bq, S_att * Sw / S_x1, 0, Sx / S_x1, 0)
+    x1 = np.clip(np.round(x1 / S_x1), -128, 127) * S_x1
+    # ---- LN2
+    g2 = g.normal(1.0, 0.1, size=D).astype(np.float32)
+    b2 = g.normal(0.0, 0.1, size=D).astype(np.float32)
+    h2 = layernorm_ref(x1, g2, b2)
+    S_h2 = float(np.abs(h2).max()) / 127.0
+    spec.ln2 = dict(gamma=g2, beta=b2, out_scale=S_h2, out_zp=0)
+    h2 = np.clip(np.round(h2 / S_h2), -128, 127) * S_h2
+    # ---- FC1 + GELU; a gain puts the GELU input on config 0's N(-0.3, 1.2^2) spread
+    wf, bf = draw_w(Dh, D)
+    a0 = h2 @ wf.T + bf
+    gain = 1.2 / float(a0.std())
+    wf *= gain
+    bf = bf * gain - 0.3
+    wq, Sw, bq, wp = qlin(wf, bf, S_h2, w_bits)
+    a = h2 @ (wq * Sw[:, None]).T + bq * (S_h2 * Sw)
+    # widest GELU input (<= gelu_in_bits) whose per-channel requant ratio stays below 1/4
+    while True:
+        qmax_in = (1 << (gelu_in_bits - 1)) - 1
+        S_gin = float(np.abs(a).max()) / qmax_in
+        if gelu_in_bits == 8 or float((S_h2 * Sw / S_gin).max()) < 0.25:
+            break
+        gelu_in_bits -= 1
+    spec.fc1 = LinearSpec(wq, wp, bq, S_h2 * Sw / S_gin)
+    hid = gelu_ref(a)
+    S_hid, zp_hid = affine_out_quant(hid, 8)
+    spec.gelu = dict(in_scale=S_gin, in_bits=gelu_in_bits, out_scale=S_hid, out_zp=zp_hid)
+    hid_q = np.clip(np.round(hid / S_hid) + zp_hid, -128, 127)
+    hid = (hid_q - zp_hid) * S_hid
+    # ---- FC2 + residual; the hidden zero point is folded into the bias
+    wf, bf = draw_w(D, Dh)
+    wq, Sw, bq, wp = qlin(wf, bf, S_hid, w_bits)
+    bq = (bq.astype(np.int64) - zp_hid * wq.astype(np.int64).sum(axis=1)).astype(np.int32)
+    yf = hid_q @ (wq * Sw[:, None]).T * S_hid + bq * (S_hid * Sw) + x1
+    S_y = float(np.abs(yf).max()) / 127.0
+    spec.fc2 = LinearSpec(wq, wp, bq, S_hid * Sw / S_y, 0, S_x1 / S_y, 0)
+    return spec
+
+
+# ------------------------------------------------------------------ Swin shifted-window labels
+
+def swin_mask_ids(window: int = 7, shift: int = 3) -> np.ndarray:
+    """Region label of every token of the last window in each direction after a cyclic shift:
+    tokens with different labels must not attend to each other.  Returns the 4 label
+    patterns [4, window*window] (interior, right edge, bottom edge, corner)."""
+    def lab(n_edge):
+        a = np.zeros(window, dtype=np.uint8)
+        if n_edge:
+            a[window - shift:] = 1
+        return a
+    out = []
+    for eh in (0, 1):
+        for ew in (0, 1):
+            out.append((lab(eh)[:, None] * 2 + lab(ew)[None, :]).reshape(-1))
+    return np.stack(out).astype(np.uint8)
