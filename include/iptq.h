@@ -1,0 +1,240 @@
+/*
+ * iptq.h -- C ABI of the B200 (sm_100a) library for the integer-only non-linear
+ * layers of IPTQ-ViT and the INT8 blocks they are fused into.
+ *
+ * Conventions (all entry points)
+ *   - Every function returns an iptq_status (0 = IPTQ_OK).  Argument errors are
+ *     detected on the host and reported before anything is launched.
+ *   - "dev" pointers are DEVICE memory owned by the caller; they must stay alive
+ *     until the work enqueued on `stream` has completed.  "host" pointers are
+ *     host memory and are only read/written during the call.
+ *   - Work is enqueued on the caller's stream; no call synchronises except
+ *     iptq_check().  No call allocates device memory: scratch comes from the
+ *     caller's workspace `ws` (device, 256-byte aligned, size from the matching
+ *     *_workspace_bytes()).  The first 256 bytes of a workspace hold the status
+ *     block that device-side bounded waits write to (see iptq_check()).
+ *   - Tensors are dense row-major, base pointers 16-byte aligned.
+ *   - ">>" on negative values is an arithmetic shift (floor).  Quantised
+ *     tensors follow the uniform quantiser of Sec. 3.1 ("Background"): an
+ *     integer array plus (scale, zero point, bit-width) passed as arguments.
+ *   - Float scales appear only in the host-side *_prepare() functions, which
+ *     turn them into the plain-old-data integer constants the kernels consume.
+ */
+#ifndef IPTQ_H
+#define IPTQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* iptq_stream_t;   /* same type as cudaStream_t */
+
+typedef enum {
+    IPTQ_OK = 0,
+    IPTQ_ERR_NULL = 1,         /* a required pointer is NULL */
+    IPTQ_ERR_SHAPE = 2,        /* a size is zero/negative/unsupported */
+    IPTQ_ERR_ALIGN = 3,        /* a pointer or stride breaks the alignment contract */
+    IPTQ_ERR_BITS = 4,         /* unsupported bit-width */
+    IPTQ_ERR_SCALE_RANGE = 5,  /* a scale/ratio falls outside what the integer constants can hold */
+    IPTQ_ERR_VARIANT = 6,      /* unknown approximation variant */
+    IPTQ_ERR_WORKSPACE = 7,    /* workspace missing or too small */
+    IPTQ_ERR_TIMEOUT = 8,      /* a bounded device-side wait gave up (reported by iptq_check) */
+    IPTQ_ERR_CUDA = 9          /* a CUDA runtime/driver call failed */
+} iptq_status;
+
+/* Candidate approximation functions per layer type (Sec. 3.2, "Overall Pipeline"). */
+typedef enum {
+    IPTQ_SM_BITEXP = 0,    /* Efficient Bit-Softmax, Eqs. (13)-(15) (the paper's own; default) */
+    IPTQ_SM_SHIFTMAX = 1,  /* bit-shifting candidate, Eqs. (7)-(10) */
+    IPTQ_SM_POLY = 2       /* polynomial candidate (second-order integer exp) */
+} iptq_softmax_variant;
+typedef enum {
+    IPTQ_GELU_POLY4 = 0,   /* Data-aware Poly-GELU, Eqs. (3), (5) (the paper's own; default) */
+    IPTQ_GELU_POLY2 = 1,   /* polynomial candidate (second-order erf), Eq. (2) */
+    IPTQ_GELU_SHIFT = 2    /* bit-shifting candidate: x * sigmoid(1.702 x) with the shift exponential */
+} iptq_gelu_variant;
+typedef enum {
+    IPTQ_LN_SHIFT = 0,     /* bit-shifting candidate: fixed 10-step shift/add square root (default) */
+    IPTQ_LN_NEWTON = 1,    /* polynomial candidate: integer square root iterated to convergence */
+    IPTQ_LN_PTF = 2        /* logarithm candidate: per-channel power-of-two factors on the input */
+} iptq_ln_variant;
+
+/* The per-layer table of Sec. 3.2: which candidate each activation layer of one block runs. */
+typedef struct {
+    iptq_softmax_variant sm;
+    iptq_gelu_variant gelu;
+    iptq_ln_variant ln1, ln2;
+} iptq_variant_table;
+
+/*
+ * Dyadic requantisation R (the integer-only pipelines of Sec. 2 use a dyadic
+ * multiplier; the paper gives no formula, this is the library's definition):
+ *   R(y) = clamp(((hi32(y * mult) + 2^(shift-1)) >> shift) + zp, qmin, qmax)
+ * hi32(p) = floor(p / 2^32) of the exact 64-bit product; the real ratio is
+ * mult * 2^-(32 + shift), mult in [2^30, 2^31), shift in [1, 31].
+ */
+typedef struct {
+    int32_t mult, shift, zp, qmin, qmax;
+} iptq_requant;
+
+/* host: ratio must be in [2^-33, 1/4) -> IPTQ_ERR_SCALE_RANGE otherwise. */
+int iptq_requant_prepare(double ratio, int32_t zp, int32_t qmin, int32_t qmax, iptq_requant* out /*host*/);
+/* host: per-output-channel ratios[n] -> mult[n], shift[n] (all host arrays). */
+int iptq_channel_requant_prepare(const double* ratios, int n, int32_t* mult, int8_t* shift);
+
+/* ------------------------------------------------------------------ Softmax
+ * Sec. 3.4 ("Efficient Bit-exp for Integer-only Softmax"), Eqs. (6)-(15).
+ * Per row of int32 scores s at scale S: mx = max s; d = min(mx - s, dcap);
+ * Qp = -d + (-d >> 1) - (-d >> 4) (Eq. (7)); (q, r) = divmod(-Qp, x0), x0 = floor(1/S)
+ * (Eq. (8)); e = ((Phi(-r) + x0) << nsh) >> q with Phi(u) = (u>>1)+(u>>3)+(u>>4)
+ * (Eqs. (9), (13), (14)); p = (floor(2^M / sum e) * e) >> (M - (out_bits-1)) (Eq. (15)).
+ * Output: uint8 probabilities at scale 2^-(out_bits-1), values in [0, 2^(out_bits-1)].
+ */
+typedef struct {
+    int32_t variant, out_bits, row_len;
+    int32_t x0, nsh, M, dcap;
+    int32_t qln2, qb, qc, norm_l, norm_r;    /* IPTQ_SM_POLY only */
+    /* derived, for the kernels: floor(v / x0) == umulhi(v, div_mul) >> div_shift for 0 <= v < 2^31 */
+    uint32_t div_mul; int32_t div_shift;
+    int32_t f_shl, p_shr;                    /* p = umulhi(f << f_shl, e) >> p_shr */
+} iptq_softmax_consts;
+
+/* host.  in_scale: scale of the scores (1/sqrt(d_head) folded in); needs 8 <= floor(1/in_scale) < 2^24
+ * and row_len * (x0 << nsh) < 2^31 (IPTQ_ERR_SCALE_RANGE); out_bits in [4, 8]; 1 <= row_len <= 1024. */
+int iptq_softmax_prepare(double in_scale, int row_len, int out_bits, iptq_softmax_variant variant,
+                         iptq_softmax_consts* out /*host*/);
+/* scores: dev int32 [rows, row_len], |score| < 2^30.  probs: dev uint8 [rows, row_len].
+ * bias: nullable dev int32 [bias_period, row_len] at the score scale; row i adds bias row (i % bias_period).
+ * consts: host.  No workspace. */
+int iptq_softmax(const int32_t* scores, uint8_t* probs, int64_t rows, int row_len, const int32_t* bias,
+                 int64_t bias_period, const iptq_softmax_consts* consts, iptq_stream_t stream);
+
+/* ------------------------------------------------------------------ GELU
+ * Sec. 3.3 ("Data-aware Poly-GELU"), Eqs. (1)-(5): GELU(x) ~ x/2 [1 + L(x/sqrt 2)],
+ * L(u) = sign(u) [a (min(|u|, -b) + b)^4 + 1], a = -0.019913, b = -2.698088.
+ * Integer form per element (x: in_bits-bit value at scale S, S' = S/sqrt 2, Bq = floor(|b|/S')):
+ *   m = min(|x|, Bq); t = Bq - m; t2 = (t*t) >> sh2; E = C - t2*t2; G = sgn(x)*E + C;
+ *   y = x * (G >> gs); out = R(y).     (IPTQ_GELU_POLY2: E = C - t2.)
+ */
+typedef struct {
+    int32_t variant, in_bits;
+    int32_t Bq, sh2, C, gs;
+    int32_t x0, nsh, dcap;                   /* IPTQ_GELU_SHIFT only */
+    uint32_t div_mul; int32_t div_shift;     /* IPTQ_GELU_SHIFT only: division by x0 */
+    iptq_requant out;
+} iptq_gelu_consts;
+
+/* host.  in_bits in [8, 16], out_bits in [4, 8]; floor(|b| / S') must be in [1, 2^15). */
+int iptq_gelu_prepare(double in_scale, int in_bits, double out_scale, int out_zp, int out_bits,
+                      iptq_gelu_variant variant, iptq_gelu_consts* out /*host*/);
+/* x: dev int32 [n] (clamped to in_bits inside); y: dev int8 [n]; consts: host. */
+int iptq_gelu(const int32_t* x, int8_t* y, int64_t n, const iptq_gelu_consts* consts, iptq_stream_t stream);
+
+/* ------------------------------------------------------------------ LayerNorm
+ * Sec. 3.2 names the LayerNorm candidates; the paper defines none, so the integer
+ * algorithm is the library's: s1 = sum x, s2 = sum x^2, u_c = D x_c - s1, V = D s2 - s1^2,
+ * r = isqrt_variant(V), F = floor(2^40 / r), n_c = (u_c F) >> 30 (Q10, 0 when r = 0),
+ * y_c = n_c gamma_q[c] + beta_q[c], out = R(y_c).  The input scale cancels.
+ */
+typedef struct {
+    int32_t variant, dim;
+    iptq_requant out;
+} iptq_ln_consts;
+
+/* host.  gamma/beta: host float [dim]; gamma_q/beta_q: host int32 [dim] outputs
+ * (gamma_q = round(gamma / S_g), S_g = max|gamma| / 32767; beta_q = round(beta / (2^-10 S_g))).
+ * 2 <= dim <= 4096, dim % 4 == 0. */
+int iptq_layernorm_prepare(int dim, const float* gamma, const float* beta, double out_scale, int out_zp,
+                           int out_bits, iptq_ln_variant variant, int32_t* gamma_q, int32_t* beta_q,
+                           iptq_ln_consts* out /*host*/);
+/* x, y: dev int8 [rows, dim]; gamma_q, beta_q: dev int32 [dim];
+ * ptf_shift: dev uint8 [dim] in 0..3, used (and required) only by IPTQ_LN_PTF; consts: host. */
+int iptq_layernorm(const int8_t* x, int8_t* y, int64_t rows, int dim, const int32_t* gamma_q,
+                   const int32_t* beta_q, const uint8_t* ptf_shift, const iptq_ln_consts* consts,
+                   iptq_stream_t stream);
+
+/* ------------------------------------------------------------------ INT8 GEMM carrier
+ * Linear ops run in integer arithmetic (Sec. 3.1): acc[m,n] = sum_k x[m,k] w[n,k] + bias[n];
+ * y = clamp(R_n(acc) + R_res((residual - residual_rq.zp) << 16) + out_zp, -128, 127), where R_n uses
+ * (mult[n], shift[n]) without zero point/clamp and the residual term is present only if residual != NULL.
+ * x: dev int8 [M, K]; w: dev int8 [N, K] (w_bits = 8) or packed int4 [N, K/2] (w_bits = 4: element k in
+ * byte k/2, even k in the low nibble, two's complement); bias: nullable dev int32 [N] (input zero point
+ * folded in by the caller); mult: dev int32 [N]; shift: dev int8 [N]; residual: nullable dev int8 [M, N];
+ * residual_rq: host; y: dev int8 [M, N].  K % 16 == 0, N % 16 == 0, K <= 4096.
+ * ws: required (status block; plus N*K bytes of unpack scratch when w_bits = 4).
+ */
+size_t iptq_linear_workspace_bytes(int64_t M, int N, int K, int w_bits);
+int iptq_linear(const int8_t* x, const void* w, int w_bits, const int32_t* bias, const int32_t* mult,
+                const int8_t* shift, int32_t out_zp, const int8_t* residual, const iptq_requant* residual_rq,
+                int8_t* y, int64_t M, int N, int K, void* ws, size_t ws_bytes, iptq_stream_t stream);
+
+/* ------------------------------------------------------------------ fused attention
+ * QK^T (INT8 -> int32, kept on chip) -> (+ bias) -> integer Softmax of Sec. 3.4 -> uint8 P -> P.V
+ * (INT8 -> int32) -> R(out_rq) -> int8, heads re-interleaved.  No int32 intermediate reaches HBM.
+ * q, k, v: dev int8 [B, H, N, dh] (zero point 0); out: dev int8 [B, N, H*dh];
+ * bias: nullable dev int32 [H, N, N] at the score scale; mask_id: nullable dev uint8 [B, N]: the pair
+ * (i, j) is masked (probability 0, excluded from max and sum) iff mask_id[b,i] != mask_id[b,j].
+ * N <= 256, dh in {32, 64}; sm (host) prepared with row_len = N; out_rq: host.  ws: status block only.
+ */
+size_t iptq_attention_workspace_bytes(int64_t B, int H, int N, int dh);
+int iptq_attention_block(const int8_t* q, const int8_t* k, const int8_t* v, int8_t* out, int64_t B, int H,
+                         int N, int dh, const int32_t* bias, const uint8_t* mask_id,
+                         const iptq_softmax_consts* sm, const iptq_requant* out_rq, void* ws, size_t ws_bytes,
+                         iptq_stream_t stream);
+
+/* ------------------------------------------------------------------ fused MLP
+ * FC1 (INT8 GEMM) with the integer GELU of Sec. 3.3 applied in the int32 epilogue:
+ *   xin = clamp(R_n(acc1; m1[n], s1[n]), in_bits range); h = R(gelu_core(xin))  -> int8 [M, Dh]
+ * then, unless w2 == NULL (stop after GELU, y is [M, Dh]), FC2 as iptq_linear with (b2, m2, s2, out_zp,
+ * residual) -> y int8 [M, D].  The hidden tensor lives in the workspace.  w1: [Dh, D], w2: [D, Dh].
+ */
+size_t iptq_mlp_workspace_bytes(int64_t M, int D, int Dh, int w_bits);
+int iptq_mlp_block(const int8_t* x, const void* w1, const int32_t* b1, const int32_t* m1, const int8_t* s1,
+                   const iptq_gelu_consts* gelu, const void* w2, const int32_t* b2, const int32_t* m2,
+                   const int8_t* s2, int32_t out_zp, const int8_t* residual, const iptq_requant* residual_rq,
+                   int8_t* y, int64_t M, int D, int Dh, int w_bits, void* ws, size_t ws_bytes,
+                   iptq_stream_t stream);
+
+/* ------------------------------------------------------------------ one encoder block
+ * LN1 -> QKV GEMM -> fused attention -> proj GEMM (+ residual x) -> LN2 -> fused MLP (+ residual),
+ * each layer running the variant its consts name (the per-layer table of Sec. 3.2).
+ * All array members are dev pointers, all consts/requant members host pointers.
+ * w_qkv: [3D, D], rows ordered [q | k | v], head h in rows h*dh .. h*dh+dh-1 of each third.
+ */
+typedef struct {
+    int64_t B; int32_t N, D, H, dh, Dh, w_bits;
+    iptq_variant_table table;      /* informative: must agree with the consts below */
+    const int32_t *ln1_gamma, *ln1_beta; const uint8_t* ln1_ptf; const iptq_ln_consts* ln1;
+    const void* w_qkv; const int32_t *b_qkv, *m_qkv; const int8_t* s_qkv;
+    const int32_t* attn_bias; const uint8_t* mask_id;
+    const iptq_softmax_consts* sm; const iptq_requant* pv_rq;
+    const void* w_proj; const int32_t *b_proj, *m_proj; const int8_t* s_proj; int32_t proj_zp;
+    const iptq_requant* res1_rq;
+    const int32_t *ln2_gamma, *ln2_beta; const uint8_t* ln2_ptf; const iptq_ln_consts* ln2;
+    const void* w_fc1; const int32_t *b_fc1, *m_fc1; const int8_t* s_fc1; const iptq_gelu_consts* gelu;
+    const void* w_fc2; const int32_t *b_fc2, *m_fc2; const int8_t* s_fc2; int32_t fc2_zp;
+    const iptq_requant* res2_rq;
+} iptq_block_params;
+
+size_t iptq_encoder_block_workspace_bytes(const iptq_block_params* p /*host*/);
+/* x, y: dev int8 [B*N, D]. */
+int iptq_encoder_block(const int8_t* x, int8_t* y, const iptq_block_params* p /*host*/, void* ws, size_t ws_bytes,
+                       iptq_stream_t stream);
+
+/* ------------------------------------------------------------------ status
+ * iptq_workspace_init: zero the status block (enqueued on the stream); call once per workspace.
+ * iptq_check: synchronise the stream and return IPTQ_ERR_TIMEOUT if any kernel that used `ws`
+ * abandoned a bounded wait, IPTQ_ERR_CUDA if the stream reports an error, else IPTQ_OK. */
+int iptq_workspace_init(void* ws, size_t ws_bytes, iptq_stream_t stream);
+int iptq_check(iptq_stream_t stream, const void* ws);
+const char* iptq_strerror(int status);
+/* Number of kernels the library has launched so far in this process (for launch accounting). */
+int64_t iptq_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IPTQ_H */

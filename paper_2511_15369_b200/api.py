@@ -1,0 +1,341 @@
+"""Thin Python binding of the iptq C-ABI library (``include/iptq.h``).
+
+Argument marshalling only: torch is used for device memory and streams; every step of the
+path runs in the library's CUDA kernels.  The binding fails loudly when ``libiptq.so`` is
+missing -- there is no CPU or eager fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libiptq.so")
+
+SM_BITEXP, SM_SHIFTMAX, SM_POLY = 0, 1, 2
+GELU_POLY4, GELU_POLY2, GELU_SHIFT = 0, 1, 2
+LN_SHIFT, LN_NEWTON, LN_PTF = 0, 1, 2
+
+OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_BITS, ERR_SCALE_RANGE, ERR_VARIANT, ERR_WORKSPACE, ERR_TIMEOUT, ERR_CUDA = range(10)
+
+
+class Requant(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("mult", "shift", "zp", "qmin", "qmax")]
+
+
+class SoftmaxConsts(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("variant", "out_bits", "row_len", "x0", "nsh", "M", "dcap",
+                                         "qln2", "qb", "qc", "norm_l", "norm_r")] + \
+               [("div_mul", C.c_uint32), ("div_shift", C.c_int32), ("f_shl", C.c_int32), ("p_shr", C.c_int32)]
+
+
+class GeluConsts(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("variant", "in_bits", "Bq", "sh2", "C", "gs", "x0", "nsh", "dcap")] + \
+               [("div_mul", C.c_uint32), ("div_shift", C.c_int32), ("out", Requant)]
+
+
+class LnConsts(C.Structure):
+    _fields_ = [("variant", C.c_int32), ("dim", C.c_int32), ("out", Requant)]
+
+
+class VariantTable(C.Structure):
+    _fields_ = [("sm", C.c_int), ("gelu", C.c_int), ("ln1", C.c_int), ("ln2", C.c_int)]
+
+
+class BlockParams(C.Structure):
+    _fields_ = [
+        ("B", C.c_int64), ("N", C.c_int32), ("D", C.c_int32), ("H", C.c_int32), ("dh", C.c_int32),
+        ("Dh", C.c_int32), ("w_bits", C.c_int32),
+        ("table", VariantTable),
+        ("ln1_gamma", C.c_void_p), ("ln1_beta", C.c_void_p), ("ln1_ptf", C.c_void_p), ("ln1", C.c_void_p),
+        ("w_qkv", C.c_void_p), ("b_qkv", C.c_void_p), ("m_qkv", C.c_void_p), ("s_qkv", C.c_void_p),
+        ("attn_bias", C.c_void_p), ("mask_id", C.c_void_p),
+        ("sm", C.c_void_p), ("pv_rq", C.c_void_p),
+        ("w_proj", C.c_void_p), ("b_proj", C.c_void_p), ("m_proj", C.c_void_p), ("s_proj", C.c_void_p),
+        ("proj_zp", C.c_int32),
+        ("res1_rq", C.c_void_p),
+        ("ln2_gamma", C.c_void_p), ("ln2_beta", C.c_void_p), ("ln2_ptf", C.c_void_p), ("ln2", C.c_void_p),
+        ("w_fc1", C.c_void_p), ("b_fc1", C.c_void_p), ("m_fc1", C.c_void_p), ("s_fc1", C.c_void_p),
+        ("gelu", C.c_void_p),
+        ("w_fc2", C.c_void_p), ("b_fc2", C.c_void_p), ("m_fc2", C.c_void_p), ("s_fc2", C.c_void_p),
+        ("fc2_zp", C.c_int32),
+        ("res2_rq", C.c_void_p),
+    ]
+
+
+class IptqError(RuntimeError):
+    def __init__(self, status, what):
+        self.status = status
+        msg = lib().iptq_strerror(status).decode() if _lib is not None else "?"
+        super().__init__("%s: iptq status %d (%s)" % (what, status, msg))
+
+
+_lib = None
+_vp = C.c_void_p
+
+
+def lib():
+    """Load ``libiptq.so`` (built in-tree by ``paper_2511_15369_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("libiptq.so is missing: run `python -m paper_2511_15369_b200.build` "
+                              "(the library has no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        L.iptq_strerror.restype = C.c_char_p
+        L.iptq_strerror.argtypes = [C.c_int]
+        L.iptq_launch_count.restype = C.c_int64
+        L.iptq_requant_prepare.argtypes = [C.c_double, C.c_int32, C.c_int32, C.c_int32, C.POINTER(Requant)]
+        L.iptq_channel_requant_prepare.argtypes = [_vp, C.c_int, _vp, _vp]
+        L.iptq_softmax_prepare.argtypes = [C.c_double, C.c_int, C.c_int, C.c_int, C.POINTER(SoftmaxConsts)]
+        L.iptq_softmax.argtypes = [_vp, _vp, C.c_int64, C.c_int, _vp, C.c_int64, C.POINTER(SoftmaxConsts), _vp]
+        L.iptq_gelu_prepare.argtypes = [C.c_double, C.c_int, C.c_double, C.c_int, C.c_int, C.c_int,
+                                        C.POINTER(GeluConsts)]
+        L.iptq_gelu.argtypes = [_vp, _vp, C.c_int64, C.POINTER(GeluConsts), _vp]
+        L.iptq_layernorm_prepare.argtypes = [C.c_int, _vp, _vp, C.c_double, C.c_int, C.c_int, C.c_int, _vp, _vp,
+                                             C.POINTER(LnConsts)]
+        L.iptq_layernorm.argtypes = [_vp, _vp, C.c_int64, C.c_int, _vp, _vp, _vp, C.POINTER(LnConsts), _vp]
+        L.iptq_linear_workspace_bytes.restype = C.c_size_t
+        L.iptq_linear_workspace_bytes.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
+        L.iptq_linear.argtypes = [_vp, _vp, C.c_int, _vp, _vp, _vp, C.c_int32, _vp, C.POINTER(Requant), _vp,
+                                  C.c_int64, C.c_int, C.c_int, _vp, C.c_size_t, _vp]
+        L.iptq_attention_workspace_bytes.restype = C.c_size_t
+        L.iptq_attention_workspace_bytes.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
+        L.iptq_attention_block.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, C.c_int, C.c_int, C.c_int, _vp, _vp,
+                                           C.POINTER(SoftmaxConsts), C.POINTER(Requant), _vp, C.c_size_t, _vp]
+        L.iptq_mlp_workspace_bytes.restype = C.c_size_t
+        L.iptq_mlp_workspace_bytes.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
+        L.iptq_mlp_block.argtypes = [_vp, _vp, _vp, _vp, _vp, C.POINTER(GeluConsts), _vp, _vp, _vp, _vp, C.c_int32,
+                                     _vp, C.POINTER(Requant), _vp, C.c_int64, C.c_int, C.c_int, C.c_int, _vp,
+                                     C.c_size_t, _vp]
+        L.iptq_encoder_block_workspace_bytes.restype = C.c_size_t
+        L.iptq_encoder_block_workspace_bytes.argtypes = [C.POINTER(BlockParams)]
+        L.iptq_encoder_block.argtypes = [_vp, _vp, C.POINTER(BlockParams), _vp, C.c_size_t, _vp]
+        L.iptq_workspace_init.argtypes = [_vp, C.c_size_t, _vp]
+        L.iptq_check.argtypes = [_vp, _vp]
+        _lib = L
+    return _lib
+
+
+def exported_symbols():
+    """Names declared in include/iptq.h (used by the CPU-side load test)."""
+    return ["iptq_requant_prepare", "iptq_channel_requant_prepare", "iptq_softmax_prepare", "iptq_softmax",
+            "iptq_gelu_prepare", "iptq_gelu", "iptq_layernorm_prepare", "iptq_layernorm",
+            "iptq_linear_workspace_bytes", "iptq_linear", "iptq_attention_workspace_bytes", "iptq_attention_block",
+            "iptq_mlp_workspace_bytes", "iptq_mlp_block", "iptq_encoder_block_workspace_bytes",
+            "iptq_encoder_block", "iptq_workspace_init", "iptq_check", "iptq_strerror", "iptq_launch_count"]
+
+
+def _chk(rc, what):
+    if rc != 0:
+        raise IptqError(rc, what)
+
+
+def _dp(t):
+    """Device pointer of a contiguous CUDA tensor (None -> NULL)."""
+    if t is None:
+        return None
+    assert isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous(), "expected a contiguous CUDA tensor"
+    return t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ref(s):
+    return None if s is None else C.byref(s)
+
+
+def launch_count() -> int:
+    return int(lib().iptq_launch_count())
+
+
+# ------------------------------------------------------------------ host-side prepare
+
+def requant_prepare(ratio, zp=0, qmin=-128, qmax=127) -> Requant:
+    r = Requant()
+    _chk(lib().iptq_requant_prepare(float(ratio), zp, qmin, qmax, C.byref(r)), "iptq_requant_prepare")
+    return r
+
+
+def channel_requant_prepare(ratios):
+    ratios = np.ascontiguousarray(ratios, dtype=np.float64)
+    mult = np.empty(ratios.shape[0], dtype=np.int32)
+    shift = np.empty(ratios.shape[0], dtype=np.int8)
+    _chk(lib().iptq_channel_requant_prepare(ratios.ctypes.data, ratios.shape[0], mult.ctypes.data,
+                                            shift.ctypes.data), "iptq_channel_requant_prepare")
+    return mult, shift
+
+
+def softmax_prepare(in_scale, row_len, out_bits=8, variant=SM_BITEXP) -> SoftmaxConsts:
+    c = SoftmaxConsts()
+    _chk(lib().iptq_softmax_prepare(float(in_scale), row_len, out_bits, variant, C.byref(c)), "iptq_softmax_prepare")
+    return c
+
+
+def gelu_prepare(in_scale, in_bits, out_scale, out_zp=0, out_bits=8, variant=GELU_POLY4) -> GeluConsts:
+    c = GeluConsts()
+    _chk(lib().iptq_gelu_prepare(float(in_scale), in_bits, float(out_scale), out_zp, out_bits, variant,
+                                 C.byref(c)), "iptq_gelu_prepare")
+    return c
+
+
+def layernorm_prepare(gamma, beta, out_scale, out_zp=0, out_bits=8, variant=LN_SHIFT):
+    g = np.ascontiguousarray(gamma, dtype=np.float32)
+    b = np.ascontiguousarray(beta, dtype=np.float32)
+    gq = np.empty(g.shape[0], dtype=np.int32)
+    bq = np.empty(g.shape[0], dtype=np.int32)
+    c = LnConsts()
+    _chk(lib().iptq_layernorm_prepare(g.shape[0], g.ctypes.data, b.ctypes.data, float(out_scale), out_zp, out_bits,
+                                      variant, gq.ctypes.data, bq.ctypes.data, C.byref(c)), "iptq_layernorm_prepare")
+    return gq, bq, c
+
+
+# ------------------------------------------------------------------ workspace
+
+class Workspace:
+    """A caller-owned device scratch buffer whose first 256 bytes are the status block."""
+
+    def __init__(self, nbytes: int, device="cuda"):
+        nbytes = max(int(nbytes), 256)
+        self.buf = torch.empty(nbytes + 256, dtype=torch.uint8, device=device)
+        off = (-self.buf.data_ptr()) % 256
+        self.ptr = self.buf.data_ptr() + off
+        self.nbytes = nbytes
+        _chk(lib().iptq_workspace_init(self.ptr, self.nbytes, _stream()), "iptq_workspace_init")
+
+    def check(self):
+        _chk(lib().iptq_check(_stream(), self.ptr), "iptq_check")
+
+
+# ------------------------------------------------------------------ device entry points
+
+def softmax(scores, consts: SoftmaxConsts, bias=None, out=None):
+    rows, n = scores.shape
+    if out is None:
+        out = torch.empty((rows, n), dtype=torch.uint8, device=scores.device)
+    period = bias.shape[0] if bias is not None else 1
+    _chk(lib().iptq_softmax(_dp(scores), _dp(out), rows, n, _dp(bias), period, C.byref(consts), _stream()),
+         "iptq_softmax")
+    return out
+
+
+def gelu(x, consts: GeluConsts, out=None):
+    if out is None:
+        out = torch.empty(x.shape, dtype=torch.int8, device=x.device)
+    _chk(lib().iptq_gelu(_dp(x), _dp(out), x.numel(), C.byref(consts), _stream()), "iptq_gelu")
+    return out
+
+
+def layernorm(x, gamma_q, beta_q, consts: LnConsts, ptf_shift=None, out=None):
+    rows, dim = x.shape
+    if out is None:
+        out = torch.empty((rows, dim), dtype=torch.int8, device=x.device)
+    _chk(lib().iptq_layernorm(_dp(x), _dp(out), rows, dim, _dp(gamma_q), _dp(beta_q), _dp(ptf_shift),
+                              C.byref(consts), _stream()), "iptq_layernorm")
+    return out
+
+
+def linear_workspace_bytes(M, N, K, w_bits=8):
+    return int(lib().iptq_linear_workspace_bytes(M, N, K, w_bits))
+
+
+def linear(x, w, bias, mult, shift, ws: Workspace, out_zp=0, residual=None, residual_rq=None, w_bits=8, out=None):
+    M, K = x.shape
+    N = w.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.int8, device=x.device)
+    _chk(lib().iptq_linear(_dp(x), _dp(w), w_bits, _dp(bias), _dp(mult), _dp(shift), out_zp, _dp(residual),
+                           _ref(residual_rq), _dp(out), M, N, K, ws.ptr, ws.nbytes, _stream()), "iptq_linear")
+    return out
+
+
+def attention_workspace_bytes(B, H, N, dh):
+    return int(lib().iptq_attention_workspace_bytes(B, H, N, dh))
+
+
+def attention_block(q, k, v, sm: SoftmaxConsts, out_rq: Requant, ws: Workspace, bias=None, mask_id=None, out=None):
+    B, H, N, dh = q.shape
+    if out is None:
+        out = torch.empty((B, N, H * dh), dtype=torch.int8, device=q.device)
+    _chk(lib().iptq_attention_block(_dp(q), _dp(k), _dp(v), _dp(out), B, H, N, dh, _dp(bias), _dp(mask_id),
+                                    C.byref(sm), C.byref(out_rq), ws.ptr, ws.nbytes, _stream()),
+         "iptq_attention_block")
+    return out
+
+
+def mlp_workspace_bytes(M, D, Dh, w_bits=8):
+    return int(lib().iptq_mlp_workspace_bytes(M, D, Dh, w_bits))
+
+
+def mlp_block(x, w1, b1, m1, s1, gelu_c: GeluConsts, ws: Workspace, w2=None, b2=None, m2=None, s2=None, out_zp=0,
+              residual=None, residual_rq=None, w_bits=8, out=None):
+    M, D = x.shape
+    Dh = w1.shape[0]
+    if out is None:
+        out = torch.empty((M, D if w2 is not None else Dh), dtype=torch.int8, device=x.device)
+    _chk(lib().iptq_mlp_block(_dp(x), _dp(w1), _dp(b1), _dp(m1), _dp(s1), C.byref(gelu_c), _dp(w2), _dp(b2),
+                              _dp(m2), _dp(s2), out_zp, _dp(residual), _ref(residual_rq), _dp(out), M, D, Dh,
+                              w_bits, ws.ptr, ws.nbytes, _stream()), "iptq_mlp_block")
+    return out
+
+
+class EncoderBlock:
+    """Device-resident parameters of one integer encoder block, prepared from a ``synth.BlockSpec``
+    (or any object with the same fields) with the library's own ``*_prepare`` functions."""
+
+    def __init__(self, spec, table=(SM_BITEXP, GELU_POLY4, LN_SHIFT, LN_SHIFT), device="cuda"):
+        sh = spec.shape
+        self.shape = sh
+        self.keep = []          # host structs and device tensors referenced by raw pointers
+        p = BlockParams()
+        p.B, p.N, p.D, p.H, p.dh, p.Dh, p.w_bits = sh.B, sh.N, sh.D, sh.H, sh.dh, sh.Dh, spec.w_bits
+        p.table = VariantTable(*table)
+        sm_v, gelu_v, ln1_v, ln2_v = table
+
+        def dev(a):
+            if a is None:
+                return None
+            t = torch.from_numpy(np.ascontiguousarray(a)).to(device)
+            self.keep.append(t)
+            return t.data_ptr()
+
+        def host(s):
+            self.keep.append(s)
+            return C.addressof(s)
+
+        for name, lnspec, var in (("ln1", spec.ln1, ln1_v), ("ln2", spec.ln2, ln2_v)):
+            gq, bq, c = layernorm_prepare(lnspec["gamma"], lnspec["beta"], lnspec["out_scale"], lnspec["out_zp"], 8, var)
+            setattr(p, name + "_gamma", dev(gq))
+            setattr(p, name + "_beta", dev(bq))
+            setattr(p, name + "_ptf", dev(lnspec.get("ptf")))
+            setattr(p, name, host(c))
+        for name, ls in (("qkv", spec.qkv), ("proj", spec.proj), ("fc1", spec.fc1), ("fc2", spec.fc2)):
+            m, s = channel_requant_prepare(ls.ratio)
+            setattr(p, "w_" + name, dev(ls.w_packed))
+            setattr(p, "b_" + name, dev(ls.bias))
+            setattr(p, "m_" + name, dev(m))
+            setattr(p, "s_" + name, dev(s))
+        p.attn_bias = dev(spec.attn_bias)
+        p.mask_id = dev(spec.mask_id)
+        p.sm = host(softmax_prepare(spec.softmax_scale, sh.N, 8, sm_v))
+        p.pv_rq = host(requant_prepare(spec.pv_ratio))
+        p.proj_zp, p.fc2_zp = spec.proj.out_zp, spec.fc2.out_zp
+        p.res1_rq = host(requant_prepare(spec.proj.res_ratio / 65536.0, zp=spec.proj.res_zp))
+        p.res2_rq = host(requant_prepare(spec.fc2.res_ratio / 65536.0, zp=spec.fc2.res_zp))
+        gl = spec.gelu
+        p.gelu = host(gelu_prepare(gl["in_scale"], gl["in_bits"], gl["out_scale"], gl["out_zp"], 8, gelu_v))
+        self.params = p
+        self.ws = Workspace(int(lib().iptq_encoder_block_workspace_bytes(C.byref(p))), device)
+
+    def __call__(self, x, out=None):
+        T, D = x.shape
+        if out is None:
+            out = torch.empty((T, D), dtype=torch.int8, device=x.device)
+        _chk(lib().iptq_encoder_block(_dp(x), _dp(out), C.byref(self.params), self.ws.ptr, self.ws.nbytes,
+                                      _stream()), "iptq_encoder_block")
+        return out

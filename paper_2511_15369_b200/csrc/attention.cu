@@ -1,0 +1,381 @@
+// Fused integer attention: S = Q K^T (tcgen05 INT8 -> int32 in TMEM) -> (+bias, mask) -> integer Softmax of
+// Sec. 3.4 (Eqs. (6)-(15)) computed straight out of TMEM, one thread per query row -> uint8 P written to
+// shared memory in the tensor-core operand layout -> O = P V (u8 x s8 -> int32 in TMEM) -> dyadic requant ->
+// int8, heads re-interleaved.  Neither S nor P ever reaches HBM.
+//
+// The integer Softmax cannot be computed "online" (flash style): the floor in Eq. (9) depends on the final row
+// maximum and P depends on floor(2^M / sum) before it multiplies V, so the whole score row stays in TMEM
+// (<= 256 columns) and is swept three times (max; exponentials + sum, written back to TMEM; probabilities).
+//
+// Work item = (batch, head, 128-row query tile).  6 warps per CTA: warp 0 = TMA producer (2-stage ring of
+// Q/K/V tiles), warp 1 = MMA issuer, warps 2..5 = softmax + output epilogue (warp w owns TMEM lanes 32*(w%4)..).
+// Two CTAs fit on an SM so that one CTA's tensor-core / copy latency hides behind the other's integer ALU work.
+#include <algorithm>
+
+#include "tc_common.cuh"
+
+namespace iptq {
+
+constexpr int ATT_THREADS = 192;
+constexpr int ATT_STAGES = 2;
+
+struct AttnParams {
+    int B, H, N, dh;
+    int mtiles;            // ceil(N / 128)
+    int npad_s;            // N rounded up to 16: UMMA N of QK^T, TMEM columns of S
+    int kpad;              // N rounded up to 32: UMMA K extent of P V
+    int q_bytes, k_bytes, v_bytes, stage_bytes;
+    int p_off, bar_off;
+    uint32_t tmem_cols;
+    const int32_t* bias;   // [H, N, N] or null
+    const uint8_t* mask_id;// [B, N] or null
+    int8_t* out;           // [B, N, H*dh]
+    ExpDev ex; int M, f_shl, p_shr;
+    RequantDev orq;
+    StatusBlock* status;
+};
+
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+template <int DH, int VARIANT, bool HAS_BIAS, bool HAS_MASK>
+__global__ void __launch_bounds__(ATT_THREADS, 2)
+attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                 const __grid_constant__ CUtensorMap map_v, const AttnParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sP = smem + p.p_off;
+    uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + p.bar_off);   // [ATT_STAGES]
+    uint64_t* kv_empty = kv_full + ATT_STAGES;                            // [ATT_STAGES]
+    uint64_t* s_full = kv_empty + ATT_STAGES;
+    uint64_t* p_ready = s_full + 1;
+    uint64_t* o_full = p_ready + 1;
+    uint64_t* t_empty = o_full + 1;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(t_empty + 1);
+    CtaControl* ctl = reinterpret_cast<CtaControl*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int items = p.B * p.H * p.mtiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < ATT_STAGES; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
+        mbar_init(s_full, 1);
+        mbar_init(p_ready, 128);
+        mbar_init(o_full, 1);
+        mbar_init(t_empty, 128);
+        ctl->abort = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&map_q);
+        prefetch_tensormap(&map_k);
+        prefetch_tensormap(&map_v);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, p.tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (elect_one()) {
+            int s = 0; uint32_t ph = 0;
+            for (int it = blockIdx.x; it < items; it += gridDim.x) {
+                const int mt = it % p.mtiles;
+                const int bh = it / p.mtiles;
+                const int h = bh % p.H, b = bh / p.H;
+                if (!mbar_wait(&kv_empty[s], ph ^ 1u, ctl, p.status, 11)) break;
+                uint8_t* st = smem + s * p.stage_bytes;
+                mbar_expect_tx(&kv_full[s], (uint32_t)((128 + p.npad_s + p.kpad) * DH));   // bytes of the three full boxes
+                tma_load_4d(st, &map_q, &kv_full[s], 0, mt * 128, h, b);
+                tma_load_4d(st + p.q_bytes, &map_k, &kv_full[s], 0, 0, h, b);
+                tma_load_4d(st + p.q_bytes + p.k_bytes, &map_v, &kv_full[s], 0, 0, h, b);
+                if (++s == ATT_STAGES) { s = 0; ph ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (elect_one()) {
+            const uint32_t idesc_s = umma_idesc_i8(128, p.npad_s, true, true, false, false);
+            const uint32_t idesc_o = umma_idesc_i8(128, DH, false, true, false, true);     // u8 P (K-major) x s8 V (MN-major)
+            int s = 0; uint32_t ph = 0;
+            uint32_t iph = 0;                                  // parity of the per-item barriers
+            for (int it = blockIdx.x; it < items; it += gridDim.x, iph ^= 1u) {
+                if (!mbar_wait(t_empty, iph ^ 1u, ctl, p.status, 12)) break;     // previous O has been read
+                if (!mbar_wait(&kv_full[s], ph, ctl, p.status, 13)) break;
+                tc_fence_after_sync();
+                const uint32_t q_addr = smem_u32(smem + s * p.stage_bytes);
+                const uint32_t k_addr = q_addr + p.q_bytes;
+                const uint32_t v_addr = k_addr + p.k_bytes;
+                // S = Q K^T: both operands K-major with DH-byte rows (DH-byte swizzle, 8-row groups 8*DH apart)
+#pragma unroll
+                for (int k = 0; k < DH / 32; ++k) {
+                    const uint64_t da = umma_smem_desc(q_addr + k * 32, 16, 8 * DH, DH);
+                    const uint64_t db = umma_smem_desc(k_addr + k * 32, 16, 8 * DH, DH);
+                    umma_i8(tmem_base, da, db, idesc_s, k != 0 ? 1u : 0u);
+                }
+                umma_commit(s_full);
+                if (!mbar_wait(p_ready, iph, ctl, p.status, 14)) break;          // P is in shared memory, S is dead
+                tc_fence_after_sync();
+                const uint32_t p_addr = smem_u32(sP);
+                for (int ks = 0; ks < p.kpad / 32; ++ks) {
+                    // A = P: K-major, 128-byte swizzle, column blocks of 128 keys are 16 KB apart
+                    const uint64_t da = umma_smem_desc(p_addr + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, 128);
+                    // B = V [keys, DH]: MN-major (DH contiguous), DH-byte swizzle, 8-key groups 8*DH apart
+                    const uint64_t db = umma_smem_desc(v_addr + ks * 32 * DH, 8 * DH, 8 * DH, DH);
+                    umma_i8(tmem_base, da, db, idesc_o, ks != 0 ? 1u : 0u);
+                }
+                umma_commit(&kv_empty[s]);                     // the stage may be refilled
+                umma_commit(o_full);
+                if (++s == ATT_STAGES) { s = 0; ph ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ softmax + output warps (thread = query row)
+        const int quad = warp & 3;
+        const int rloc = quad * 32 + lane;                     // row inside the 128-row tile
+        const uint32_t trow = tmem_base + ((uint32_t)(quad * 32) << 16);
+        const uint32_t p_row = smem_u32(sP) + (uint32_t)((rloc >> 3) * 1024 + (rloc & 7) * 128);
+        const int HD = p.H * DH;
+        uint32_t iph = 0;
+        for (int it = blockIdx.x; it < items; it += gridDim.x, iph ^= 1u) {
+            const int mt = it % p.mtiles;
+            const int bh = it / p.mtiles;
+            const int h = bh % p.H, b = bh / p.H;
+            const int row = mt * 128 + rloc;
+            const bool valid = row < p.N;
+            const int32_t* brow = HAS_BIAS ? p.bias + ((size_t)h * p.N + (valid ? row : 0)) * p.N : nullptr;
+            const uint8_t* mrow = HAS_MASK ? p.mask_id + (size_t)b * p.N : nullptr;
+            const unsigned my_id = (HAS_MASK && valid) ? mrow[row] : 0u;
+
+            if (!mbar_wait(s_full, iph, ctl, p.status, 15)) break;
+            tc_fence_after_sync();
+            // ---- sweep 1: row maximum over the real, unmasked columns (Eq. (6))
+            int mx = INT_MIN;
+#pragma unroll 1
+            for (int c0 = 0; c0 < p.npad_s; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld16(trow + c0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int col = c0 + j;
+                    int s = (int)r[j];
+                    if (HAS_BIAS && col < p.N) s += __ldg(brow + col);
+                    bool use = col < p.N;
+                    if (HAS_MASK && use && valid) use = (mrow[col] == my_id);
+                    if (use) mx = max(mx, s);
+                }
+            }
+            // ---- sweep 2: integer exponentials (Eqs. (7)-(14)) and their sum; e goes back to TMEM
+            unsigned sum = 0;
+#pragma unroll 1
+            for (int c0 = 0; c0 < p.npad_s; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld16(trow + c0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int col = c0 + j;
+                    int s = (int)r[j];
+                    if (HAS_BIAS && col < p.N) s += __ldg(brow + col);
+                    bool use = col < p.N;
+                    if (HAS_MASK && use && valid) use = (mrow[col] == my_id);
+                    const unsigned d = min((unsigned)(mx - s), (unsigned)p.ex.dcap);
+                    const unsigned e = use ? exp_core<VARIANT>(d, p.ex) : 0u;
+                    sum += e;
+                    r[j] = e;
+                }
+                tmem_st16(trow + c0, r);
+            }
+            tmem_wait_st();
+            // ---- sweep 3: IntDiv (Eq. (15)) -> uint8 probabilities in the UMMA A-operand layout
+            const unsigned f = intdiv_factor(sum, p.M) << p.f_shl;
+#pragma unroll 1
+            for (int c0 = 0; c0 < p.npad_s; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld16(trow + c0, r);
+                tmem_wait_ld();
+                uint32_t w[4];
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    uint32_t acc = 0;
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) acc |= ((__umulhi(f, r[q4 * 4 + t]) >> p.p_shr) & 255u) << (8 * t);
+                    w[q4] = acc;
+                }
+                const int chunk = (c0 & 127) >> 4;
+                st_shared_v4(p_row + (uint32_t)((c0 >> 7) * 16384 + ((chunk ^ (rloc & 7)) << 4)), w[0], w[1], w[2], w[3]);
+            }
+            fence_proxy_async_smem();            // generic-proxy stores -> visible to the tensor core's reads
+            tc_fence_before_sync();
+            mbar_arrive(p_ready);
+
+            // ---- output: O = P V from TMEM -> requant -> int8
+            if (!mbar_wait(o_full, iph, ctl, p.status, 16)) break;
+            tc_fence_after_sync();
+            int8_t* orow = p.out + ((size_t)b * p.N + (valid ? row : 0)) * HD + h * DH;
+#pragma unroll
+            for (int c0 = 0; c0 < DH; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld16(trow + c0, r);
+                tmem_wait_ld();
+                int o[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) o[j] = requant_full((int)r[j], p.orq);
+                if (valid) {
+                    int4 pk;
+                    pk.x = (int)pack4_s8(o[0], o[1], o[2], o[3]);
+                    pk.y = (int)pack4_s8(o[4], o[5], o[6], o[7]);
+                    pk.z = (int)pack4_s8(o[8], o[9], o[10], o[11]);
+                    pk.w = (int)pack4_s8(o[12], o[13], o[14], o[15]);
+                    *reinterpret_cast<int4*>(orow + c0) = pk;
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(t_empty);
+        }
+    }
+
+    // ------------------------------------------------------------ teardown (also reached after an abort)
+    __syncwarp();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (ctl->abort) {
+        for (int i = 0; i < 64; ++i) __nanosleep(2000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, p.tmem_cols);
+    }
+}
+
+// ---------------------------------------------------------------- launcher (strided q/k/v so that the encoder
+// block can read heads straight out of the fused QKV activation)
+struct AttnArgs {
+    const int8_t *q, *k, *v;
+    int64_t tok_stride, head_stride, batch_stride;     // in bytes (= elements)
+    int8_t* out;
+    int64_t B; int H, N, dh;
+    const int32_t* bias; const uint8_t* mask_id;
+    const iptq_softmax_consts* sm; const iptq_requant* out_rq;
+    StatusBlock* status;
+};
+
+template <int DH, int VARIANT>
+static int launch_attn(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const AttnParams& p,
+                       int smem_bytes, cudaStream_t st)
+{
+    const int items = p.B * p.H * p.mtiles;
+    const int grid = std::min(items, 2 * sm_count());
+#define IPTQ_ATT_LAUNCH(HB, HM)                                                                                   \
+    do {                                                                                                          \
+        auto kern = attention_kernel<DH, VARIANT, HB, HM>;                                                        \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)  \
+            return IPTQ_ERR_CUDA;                                                                                 \
+        kern<<<grid, ATT_THREADS, smem_bytes, st>>>(mq, mk, mv, p);                                               \
+    } while (0)
+    if (p.bias && p.mask_id) IPTQ_ATT_LAUNCH(true, true);
+    else if (p.bias) IPTQ_ATT_LAUNCH(true, false);
+    else if (p.mask_id) IPTQ_ATT_LAUNCH(false, true);
+    else IPTQ_ATT_LAUNCH(false, false);
+#undef IPTQ_ATT_LAUNCH
+    note_launch();
+    return last_launch_status();
+}
+
+template <int DH>
+static int launch_attn_v(int variant, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                         const AttnParams& p, int smem_bytes, cudaStream_t st)
+{
+    switch (variant) {
+        case IPTQ_SM_BITEXP: return launch_attn<DH, IPTQ_SM_BITEXP>(mq, mk, mv, p, smem_bytes, st);
+        case IPTQ_SM_SHIFTMAX: return launch_attn<DH, IPTQ_SM_SHIFTMAX>(mq, mk, mv, p, smem_bytes, st);
+        case IPTQ_SM_POLY: return launch_attn<DH, IPTQ_SM_POLY>(mq, mk, mv, p, smem_bytes, st);
+        default: return IPTQ_ERR_VARIANT;
+    }
+}
+
+int attention_launch(const AttnArgs& a, cudaStream_t st)
+{
+    if (!a.sm || !a.out_rq) return IPTQ_ERR_NULL;
+    if (a.B < 0 || a.B > (1 << 24) || a.H < 1 || a.H > 1024 || a.N < 1 || a.N > 256) return IPTQ_ERR_SHAPE;
+    if (a.dh != 32 && a.dh != 64) return IPTQ_ERR_SHAPE;
+    if (a.sm->row_len != a.N) return IPTQ_ERR_SHAPE;
+    if (a.sm->out_bits < 4 || a.sm->out_bits > 8) return IPTQ_ERR_BITS;
+    if (a.sm->x0 < 8 || a.sm->M < 31 || a.sm->M > 40) return IPTQ_ERR_SCALE_RANGE;
+    int rc = check_requant(a.out_rq);
+    if (rc != IPTQ_OK) return rc;
+    if (!a.status) return IPTQ_ERR_WORKSPACE;
+    if (a.B == 0) return IPTQ_OK;
+    if (!a.q || !a.k || !a.v || !a.out) return IPTQ_ERR_NULL;
+    if (!aligned16(a.q) || !aligned16(a.k) || !aligned16(a.v) || !aligned16(a.out) ||
+        (a.bias && (reinterpret_cast<uintptr_t>(a.bias) & 3u)) || (a.tok_stride & 15) || (a.head_stride & 15) ||
+        (a.batch_stride & 15))
+        return IPTQ_ERR_ALIGN;
+    if (a.B * a.H * ((a.N + 127) / 128) > (int64_t)1 << 30) return IPTQ_ERR_SHAPE;
+
+    AttnParams p;
+    p.B = (int)a.B; p.H = a.H; p.N = a.N; p.dh = a.dh;
+    p.mtiles = (a.N + 127) / 128;
+    p.npad_s = (a.N + 15) & ~15;
+    p.kpad = (a.N + 31) & ~31;
+    auto up1k = [](int v) { return (v + 1023) & ~1023; };
+    p.q_bytes = up1k(128 * a.dh);
+    p.k_bytes = up1k(p.npad_s * a.dh);
+    p.v_bytes = up1k(p.kpad * a.dh);
+    p.stage_bytes = p.q_bytes + p.k_bytes + p.v_bytes;
+    p.p_off = ATT_STAGES * p.stage_bytes;
+    const int p_bytes = ((p.kpad + 127) / 128) * 16384;
+    p.bar_off = p.p_off + p_bytes;
+    const int smem_bytes = p.bar_off + 128 + 1024;
+    p.tmem_cols = 32;
+    while ((int)p.tmem_cols < std::max(p.npad_s, a.dh)) p.tmem_cols <<= 1;
+    p.bias = a.bias; p.mask_id = a.mask_id; p.out = a.out;
+    p.ex = to_dev_exp(*a.sm);
+    p.M = a.sm->M; p.f_shl = a.sm->f_shl; p.p_shr = a.sm->p_shr;
+    p.orq = to_dev(*a.out_rq);
+    p.status = a.status;
+
+    // q/k/v as 4-D tensors (dh, N, H, B); rows past N read as zero, which is what the padding needs.
+    CUtensorMap mq, mk, mv;
+    const uint64_t dims[4] = {(uint64_t)a.dh, (uint64_t)a.N, (uint64_t)a.H, (uint64_t)a.B};
+    const uint64_t str[3] = {(uint64_t)a.tok_stride, (uint64_t)a.head_stride, (uint64_t)a.batch_stride};
+    const uint32_t box_q[4] = {(uint32_t)a.dh, 128u, 1u, 1u};
+    const uint32_t box_k[4] = {(uint32_t)a.dh, (uint32_t)p.npad_s, 1u, 1u};
+    const uint32_t box_v[4] = {(uint32_t)a.dh, (uint32_t)p.kpad, 1u, 1u};
+    if ((rc = make_tensor_map_u8(&mq, a.q, 4, dims, str, box_q, a.dh)) != IPTQ_OK) return rc;
+    if ((rc = make_tensor_map_u8(&mk, a.k, 4, dims, str, box_k, a.dh)) != IPTQ_OK) return rc;
+    if ((rc = make_tensor_map_u8(&mv, a.v, 4, dims, str, box_v, a.dh)) != IPTQ_OK) return rc;
+    if (a.dh == 64) return launch_attn_v<64>(a.sm->variant, mq, mk, mv, p, smem_bytes, st);
+    return launch_attn_v<32>(a.sm->variant, mq, mk, mv, p, smem_bytes, st);
+}
+
+}  // namespace iptq
+
+using namespace iptq;
+
+extern "C" {
+
+size_t iptq_attention_workspace_bytes(int64_t, int, int, int) { return kStatusBytes; }
+
+int iptq_attention_block(const int8_t* q, const int8_t* k, const int8_t* v, int8_t* out, int64_t B, int H,
+                         int N, int dh, const int32_t* bias, const uint8_t* mask_id,
+                         const iptq_softmax_consts* sm, const iptq_requant* out_rq, void* ws, size_t ws_bytes,
+                         iptq_stream_t stream)
+{
+    if (!ws || ws_bytes < kStatusBytes) return IPTQ_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(ws) & 255u) return IPTQ_ERR_ALIGN;
+    AttnArgs a{q, k, v, (int64_t)dh, (int64_t)N * dh, (int64_t)H * N * dh, out, B, H, N, dh, bias, mask_id, sm, out_rq,
+               static_cast<StatusBlock*>(ws)};
+    return attention_launch(a, stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,466 @@
+// INT8 x INT8 -> INT32 GEMM on the 5th-generation tensor cores (tcgen05.mma.kind::i8, TMEM accumulators,
+// TMA-fed shared-memory pipeline) with the integer epilogues of the path applied straight out of TMEM:
+//   - per-channel dyadic requantisation (QKV, proj, FC2), optionally with the int8 residual branch;
+//   - FC1: requantise to the GELU input scale, integer GELU (Sec. 3.3, Eqs. (3), (5)), requantise to int8.
+// No int32 intermediate is written to HBM.
+//
+// One persistent CTA per SM, 10 warps: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM),
+// warps 2..9 = epilogue (two warps per TMEM lane quadrant, each taking half of the tile's columns).
+// The accumulator is double-buffered in TMEM so that the epilogue of tile i overlaps the mainloop of tile i+1.
+#include <algorithm>
+#include <mutex>
+
+#include "tc_common.cuh"
+
+namespace iptq {
+
+// ---------------------------------------------------------------- host: tensor map encoding
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+int make_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides,
+                       const uint32_t* box, int swizzle_bytes)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return IPTQ_ERR_CUDA;
+    cuuint64_t gdim[5], gstr[5];
+    cuuint32_t bx[5], estr[5];
+    for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bx[i] = box[i]; estr[i] = 1; }
+    for (int i = 0; i + 1 < rank; ++i) {
+        gstr[i] = strides[i];
+        if (strides[i] & 15u) return IPTQ_ERR_ALIGN;
+    }
+    if (reinterpret_cast<uintptr_t>(base) & 15u) return IPTQ_ERR_ALIGN;
+    CUtensorMapSwizzle sw = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                          : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                          : swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr, bx, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? IPTQ_OK : IPTQ_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------- kernel
+enum { EPI_REQUANT = 0, EPI_RESIDUAL = 1, EPI_GELU = 2 };
+
+constexpr int BM = 128;          // rows per tile = TMEM lanes
+constexpr int BK = 128;          // bytes of K per stage = one 128-byte swizzle row = 4 MMA k-steps
+constexpr int STAGES = 4;
+constexpr int EPI_WARPS = 8;
+constexpr int GEMM_THREADS = 32 * (2 + EPI_WARPS);
+
+struct GemmParams {
+    int M, N, K;
+    int num_m_tiles, num_n_tiles;
+    const int32_t* bias; const int32_t* mult; const int8_t* shift;
+    int out_zp;
+    const int8_t* residual;
+    int res_mult, res_rnd, res_shift, res_zp;
+    int8_t* y;
+    GeluDev gelu;
+    StatusBlock* status;
+};
+
+template <int BN>
+struct GemmSmem {
+    static constexpr int A_BYTES = BM * BK;
+    static constexpr int B_BYTES = BN * BK;
+    static constexpr int COLS_PER_WARP = BN / 2;
+    static constexpr int OFF_A = 0;
+    static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
+    static constexpr int OFF_CP = OFF_B + STAGES * B_BYTES;                      // [EPI_WARPS][COLS_PER_WARP] int4
+    static constexpr int OFF_BAR = OFF_CP + EPI_WARPS * COLS_PER_WARP * 16;
+    static constexpr int OFF_END = OFF_BAR + (2 * STAGES + 4) * 8 + 16;
+    static constexpr int TOTAL = OFF_END + 1024;                                 // slack for 1024-byte alignment
+};
+
+template <int BN, int EPI, int GELU_VARIANT>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const GemmParams p)
+{
+    using L = GemmSmem<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sA = smem + L::OFF_A;
+    uint8_t* sB = smem + L::OFF_B;
+    int4* sCP = reinterpret_cast<int4*>(smem + L::OFF_CP);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
+    uint64_t* empty_bar = full_bar + STAGES;
+    uint64_t* acc_full = empty_bar + STAGES;      // [2]
+    uint64_t* acc_empty = acc_full + 2;           // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    CtaControl* ctl = reinterpret_cast<CtaControl*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int num_tiles = p.num_m_tiles * p.num_n_tiles;
+    const int kblocks = (p.K + BK - 1) / BK;
+    constexpr uint32_t TMEM_COLS = 2 * BN;        // two accumulator buffers (power of two for BN in {64, 128})
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EPI_WARPS); }
+        ctl->abort = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_b);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (elect_one()) {
+            int s = 0; uint32_t ph = 0;
+            for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+                const int m0 = (t / p.num_n_tiles) * BM;
+                const int n0 = (t % p.num_n_tiles) * BN;
+                bool ok = true;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait(&empty_bar[s], ph ^ 1u, ctl, p.status, 1)) { ok = false; break; }
+                    mbar_expect_tx(&full_bar[s], L::A_BYTES + L::B_BYTES);
+                    tma_load_2d(sA + s * L::A_BYTES, &map_a, &full_bar[s], kb * BK, m0);
+                    tma_load_2d(sB + s * L::B_BYTES, &map_b, &full_bar[s], kb * BK, n0);
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (elect_one()) {
+            constexpr uint32_t idesc = umma_idesc_i8(BM, BN, true, true, false, false);
+            int s = 0; uint32_t ph = 0;
+            int it = 0;
+            for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+                const int ab = it & 1;
+                const uint32_t abph = (uint32_t)(it >> 1) & 1u;
+                if (!mbar_wait(&acc_empty[ab], abph ^ 1u, ctl, p.status, 2)) break;
+                tc_fence_after_sync();
+                const uint32_t tacc = tmem_base + (uint32_t)(ab * BN);
+                bool ok = true;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait(&full_bar[s], ph, ctl, p.status, 3)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t a_addr = smem_u32(sA + s * L::A_BYTES);
+                    const uint32_t b_addr = smem_u32(sB + s * L::B_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / 32; ++k) {
+                        // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart; a k-step is 32 bytes
+                        const uint64_t da = umma_smem_desc(a_addr + k * 32, 16, 1024, 128);
+                        const uint64_t db = umma_smem_desc(b_addr + k * 32, 16, 1024, 128);
+                        umma_i8(tacc, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(&empty_bar[s]);               // frees the stage once these MMAs have read it
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(&acc_full[ab]);                   // accumulator complete
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue warps
+        const int ew = warp - 2;                              // 0..7
+        const int quad = warp & 3;                            // TMEM lane quadrant this warp may access
+        const int half = ew >> 2;                             // which half of the tile's columns
+        int4* cp = sCP + ew * L::COLS_PER_WARP;
+        int it = 0;
+        for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+            const int ab = it & 1;
+            const uint32_t abph = (uint32_t)(it >> 1) & 1u;
+            const int m0 = (t / p.num_n_tiles) * BM;
+            const int n0 = (t % p.num_n_tiles) * BN + half * L::COLS_PER_WARP;
+            // per-column constants of this warp's columns: (bias, mult, 2^(shift-1), shift)
+            __syncwarp();
+            for (int c = lane; c < L::COLS_PER_WARP; c += 32) {
+                const int n = n0 + c;
+                int4 v = make_int4(0, 1 << 30, 1, 1);
+                if (n < p.N) {
+                    const int sh = (int)__ldg(p.shift + n);
+                    v = make_int4(p.bias ? __ldg(p.bias + n) : 0, __ldg(p.mult + n), 1 << (sh - 1), sh);
+                }
+                cp[c] = v;
+            }
+            __syncwarp();
+            if (!mbar_wait(&acc_full[ab], abph, ctl, p.status, 4)) break;
+            tc_fence_after_sync();
+            const int row = m0 + quad * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * BN + half * L::COLS_PER_WARP);
+#pragma unroll 1
+            for (int c0 = 0; c0 < L::COLS_PER_WARP; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld16(taddr + c0, r);
+                tmem_wait_ld();
+                if (n0 + c0 >= p.N) continue;                 // N is a multiple of 16: whole chunk in or out
+                int o[16];
+                int4 resv = make_int4(0, 0, 0, 0);
+                if (EPI == EPI_RESIDUAL && row < p.M)
+                    resv = __ldg(reinterpret_cast<const int4*>(p.residual + (size_t)row * p.N + n0 + c0));
+                const int resw[4] = {resv.x, resv.y, resv.z, resv.w};
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int4 k4 = cp[c0 + j];
+                    int v = requant_core((int)r[j] + k4.x, k4.y, k4.z, k4.w);
+                    if (EPI == EPI_GELU) {
+                        v = gelu_core<GELU_VARIANT>(v, p.gelu);               // clamps to in_bits first
+                        v = requant_full(v, p.gelu.out);
+                    } else {
+                        if (EPI == EPI_RESIDUAL) {
+                            const int rb = (int)(int8_t)(resw[j >> 2] >> (8 * (j & 3)));
+                            v += requant_core((rb - p.res_zp) << 16, p.res_mult, p.res_rnd, p.res_shift);
+                        }
+                        v += p.out_zp;
+                    }
+                    o[j] = v;
+                }
+                if (row < p.M) {
+                    int4 pk;
+                    pk.x = (int)pack4_sat_s8(o[0], o[1], o[2], o[3]);
+                    pk.y = (int)pack4_sat_s8(o[4], o[5], o[6], o[7]);
+                    pk.z = (int)pack4_sat_s8(o[8], o[9], o[10], o[11]);
+                    pk.w = (int)pack4_sat_s8(o[12], o[13], o[14], o[15]);
+                    *reinterpret_cast<int4*>(p.y + (size_t)row * p.N + n0 + c0) = pk;
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[ab]);
+        }
+    }
+
+    // ------------------------------------------------------------ teardown (also reached after an abort)
+    __syncwarp();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (ctl->abort) {
+        // give copies that are still in flight time to land before shared memory is released
+        for (int i = 0; i < 64; ++i) __nanosleep(2000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ---------------------------------------------------------------- W4: unpack nibbles to int8
+__global__ void unpack_int4_kernel(const uint8_t* __restrict__ packed, int8_t* __restrict__ out, int64_t nbytes)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nbytes; i += stride) {
+        const unsigned b = packed[i];
+        const int lo = (int)(b & 15u), hi = (int)(b >> 4);
+        char2 v;
+        v.x = (char)(lo >= 8 ? lo - 16 : lo);                 // element 2i   (low nibble)
+        v.y = (char)(hi >= 8 ? hi - 16 : hi);                 // element 2i+1 (high nibble)
+        reinterpret_cast<char2*>(out)[i] = v;
+    }
+}
+
+int unpack_int4_launch(const void* packed, int8_t* out, int64_t n_elems, cudaStream_t st)
+{
+    const int64_t nbytes = n_elems / 2;
+    const int grid = (int)std::min<int64_t>((nbytes + 255) / 256, (int64_t)sm_count() * 8);
+    unpack_int4_kernel<<<grid, 256, 0, st>>>(static_cast<const uint8_t*>(packed), out, nbytes);
+    note_launch();
+    return last_launch_status();
+}
+
+// ---------------------------------------------------------------- launcher
+struct LinearArgs {
+    const int8_t* x; const int8_t* w;                          // w already int8 [N, K]
+    const int32_t* bias; const int32_t* mult; const int8_t* shift;
+    int32_t out_zp;
+    const int8_t* residual; const iptq_requant* residual_rq;
+    const iptq_gelu_consts* gelu;                              // non-null: FC1 + GELU epilogue
+    int8_t* y;
+    int64_t M; int N, K;
+    StatusBlock* status;
+};
+
+template <int BN, int EPI, int GV>
+static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, cudaStream_t st)
+{
+    using L = GemmSmem<BN>;
+    auto kern = gemm_i8_kernel<BN, EPI, GV>;
+    static bool configured = false;           // one attribute call per instantiation is enough per process/device
+    if (!configured) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) != cudaSuccess)
+            return IPTQ_ERR_CUDA;
+        configured = true;
+    }
+    const int tiles = p.num_m_tiles * p.num_n_tiles;
+    const int grid = std::min(tiles, sm_count());
+    kern<<<grid, GEMM_THREADS, L::TOTAL, st>>>(ma, mb, p);
+    note_launch();
+    return last_launch_status();
+}
+
+int linear_launch(const LinearArgs& a, cudaStream_t st)
+{
+    if (!a.x || !a.w || !a.mult || !a.shift || !a.y) return IPTQ_ERR_NULL;
+    if (a.M < 0 || a.M > (int64_t)1 << 30 || a.N < 16 || a.K < 16 || a.K > 4096 || (a.N & 15) || (a.K & 15))
+        return IPTQ_ERR_SHAPE;
+    if (!aligned16(a.x) || !aligned16(a.w) || !aligned16(a.y) || (a.residual && !aligned16(a.residual)) ||
+        (a.bias && (reinterpret_cast<uintptr_t>(a.bias) & 3u)) || (reinterpret_cast<uintptr_t>(a.mult) & 3u))
+        return IPTQ_ERR_ALIGN;
+    if (a.residual) { int rc = check_requant(a.residual_rq); if (rc != IPTQ_OK) return rc; }
+    if (a.gelu) {
+        if (a.gelu->in_bits < 8 || a.gelu->in_bits > 16) return IPTQ_ERR_BITS;
+        if (a.gelu->variant < 0 || a.gelu->variant > 2) return IPTQ_ERR_VARIANT;
+        int rc = check_requant(&a.gelu->out); if (rc != IPTQ_OK) return rc;
+    }
+    if (!a.status) return IPTQ_ERR_WORKSPACE;
+    if (a.M == 0) return IPTQ_OK;
+
+    constexpr int BN = 128;
+    GemmParams p;
+    p.M = (int)a.M; p.N = a.N; p.K = a.K;
+    p.num_m_tiles = (int)((a.M + BM - 1) / BM);
+    p.num_n_tiles = (a.N + BN - 1) / BN;
+    p.bias = a.bias; p.mult = a.mult; p.shift = a.shift; p.out_zp = a.out_zp;
+    p.residual = a.residual;
+    p.res_mult = p.res_rnd = p.res_shift = p.res_zp = 0;
+    if (a.residual) {
+        p.res_mult = a.residual_rq->mult; p.res_shift = a.residual_rq->shift;
+        p.res_rnd = 1 << (a.residual_rq->shift - 1); p.res_zp = a.residual_rq->zp;
+    }
+    p.y = a.y;
+    p.status = a.status;
+    if (a.gelu) p.gelu = to_dev(*a.gelu);
+    else { iptq_gelu_consts z{}; z.in_bits = 8; z.out.shift = 1; p.gelu = to_dev(z); }
+
+    CUtensorMap ma, mb;
+    {
+        const uint64_t dims[2] = {(uint64_t)a.K, (uint64_t)a.M};
+        const uint64_t str[1] = {(uint64_t)a.K};
+        const uint32_t box[2] = {BK, BM};
+        int rc = make_tensor_map_u8(&ma, a.x, 2, dims, str, box, 128);
+        if (rc != IPTQ_OK) return rc;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)a.K, (uint64_t)a.N};
+        const uint64_t str[1] = {(uint64_t)a.K};
+        const uint32_t box[2] = {BK, BN};
+        int rc = make_tensor_map_u8(&mb, a.w, 2, dims, str, box, 128);
+        if (rc != IPTQ_OK) return rc;
+    }
+    if (a.gelu) {
+        switch (a.gelu->variant) {
+            case IPTQ_GELU_POLY4: return launch_gemm<BN, EPI_GELU, IPTQ_GELU_POLY4>(ma, mb, p, st);
+            case IPTQ_GELU_POLY2: return launch_gemm<BN, EPI_GELU, IPTQ_GELU_POLY2>(ma, mb, p, st);
+            default: return launch_gemm<BN, EPI_GELU, IPTQ_GELU_SHIFT>(ma, mb, p, st);
+        }
+    }
+    if (a.residual) return launch_gemm<BN, EPI_RESIDUAL, 0>(ma, mb, p, st);
+    return launch_gemm<BN, EPI_REQUANT, 0>(ma, mb, p, st);
+}
+
+static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
+
+}  // namespace iptq
+
+using namespace iptq;
+
+extern "C" {
+
+size_t iptq_linear_workspace_bytes(int64_t M, int N, int K, int w_bits)
+{
+    (void)M;
+    size_t b = kStatusBytes;
+    if (w_bits == 4 && N > 0 && K > 0) b += align256((size_t)N * (size_t)K);
+    return b;
+}
+
+int iptq_linear(const int8_t* x, const void* w, int w_bits, const int32_t* bias, const int32_t* mult,
+                const int8_t* shift, int32_t out_zp, const int8_t* residual, const iptq_requant* residual_rq,
+                int8_t* y, int64_t M, int N, int K, void* ws, size_t ws_bytes, iptq_stream_t stream)
+{
+    if (w_bits != 8 && w_bits != 4) return IPTQ_ERR_BITS;
+    if (!ws) return IPTQ_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(ws) & 255u) return IPTQ_ERR_ALIGN;
+    if (N < 1 || K < 1) return IPTQ_ERR_SHAPE;
+    if (ws_bytes < iptq_linear_workspace_bytes(M, N, K, w_bits)) return IPTQ_ERR_WORKSPACE;
+    if (!w) return IPTQ_ERR_NULL;
+    const int8_t* w8 = static_cast<const int8_t*>(w);
+    if (w_bits == 4) {
+        if (K & 1) return IPTQ_ERR_SHAPE;
+        int8_t* scratch = static_cast<int8_t*>(ws) + kStatusBytes;
+        int rc = unpack_int4_launch(w, scratch, (int64_t)N * K, stream);
+        if (rc != IPTQ_OK) return rc;
+        w8 = scratch;
+    }
+    LinearArgs a{x, w8, bias, mult, shift, out_zp, residual, residual_rq, nullptr, y, M, N, K,
+                 static_cast<StatusBlock*>(ws)};
+    return linear_launch(a, stream);
+}
+
+size_t iptq_mlp_workspace_bytes(int64_t M, int D, int Dh, int w_bits)
+{
+    size_t b = kStatusBytes;
+    if (M > 0 && Dh > 0) b += align256((size_t)M * (size_t)Dh);               // hidden activations
+    if (w_bits == 4 && D > 0 && Dh > 0) b += 2 * align256((size_t)D * (size_t)Dh);
+    return b;
+}
+
+int iptq_mlp_block(const int8_t* x, const void* w1, const int32_t* b1, const int32_t* m1, const int8_t* s1,
+                   const iptq_gelu_consts* gelu, const void* w2, const int32_t* b2, const int32_t* m2,
+                   const int8_t* s2, int32_t out_zp, const int8_t* residual, const iptq_requant* residual_rq,
+                   int8_t* y, int64_t M, int D, int Dh, int w_bits, void* ws, size_t ws_bytes,
+                   iptq_stream_t stream)
+{
+    if (w_bits != 8 && w_bits != 4) return IPTQ_ERR_BITS;
+    if (!gelu || !w1) return IPTQ_ERR_NULL;
+    if (!ws) return IPTQ_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(ws) & 255u) return IPTQ_ERR_ALIGN;
+    if (M < 0 || D < 1 || Dh < 1) return IPTQ_ERR_SHAPE;
+    if (ws_bytes < iptq_mlp_workspace_bytes(M, D, Dh, w_bits)) return IPTQ_ERR_WORKSPACE;
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    StatusBlock* status = reinterpret_cast<StatusBlock*>(base);
+    int8_t* hidden = reinterpret_cast<int8_t*>(base + kStatusBytes);
+    size_t off = kStatusBytes + align256((size_t)M * (size_t)Dh);
+    const int8_t* w1_8 = static_cast<const int8_t*>(w1);
+    const int8_t* w2_8 = static_cast<const int8_t*>(w2);
+    if (w_bits == 4) {
+        int8_t* u1 = reinterpret_cast<int8_t*>(base + off);
+        int rc = unpack_int4_launch(w1, u1, (int64_t)D * Dh, stream);
+        if (rc != IPTQ_OK) return rc;
+        w1_8 = u1;
+        if (w2) {
+            int8_t* u2 = reinterpret_cast<int8_t*>(base + off + align256((size_t)D * (size_t)Dh));
+            rc = unpack_int4_launch(w2, u2, (int64_t)D * Dh, stream);
+            if (rc != IPTQ_OK) return rc;
+            w2_8 = u2;
+        }
+    }
+    // FC1 with the GELU epilogue; without FC2 the activations go straight to y
+    LinearArgs fc1{x, w1_8, b1, m1, s1, 0, nullptr, nullptr, gelu, w2 ? hidden : y, M, Dh, D, status};
+    int rc = linear_launch(fc1, stream);
+    if (rc != IPTQ_OK || !w2) return rc;
+    LinearArgs fc2{hidden, w2_8, b2, m2, s2, out_zp, residual, residual_rq, nullptr, y, M, D, Dh, status};
+    return linear_launch(fc2, stream);
+}
+
+}  // extern "C"

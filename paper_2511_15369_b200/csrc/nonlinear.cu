@@ -1,0 +1,359 @@
+// Stand-alone integer Softmax / GELU / LayerNorm kernels (row- and element-wise, HBM/ALU bound).
+#include <climits>
+
+#include "iptq_common.cuh"
+
+namespace iptq {
+
+constexpr unsigned kFull = 0xffffffffu;
+
+// ------------------------------------------------------------------------------------------------
+// Softmax: one warp per row, the row lives in registers (NITER values per lane), row max / row sum
+// by warp reduction, one fp64 division per row for floor(2^M / sum).
+// ------------------------------------------------------------------------------------------------
+struct SoftmaxDev {
+    ExpDev ex;
+    int M, f_shl, p_shr;
+};
+
+template <int VARIANT, int NITER, bool HAS_BIAS>
+__global__ void __launch_bounds__(256)
+softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ probs, int64_t rows, int n,
+                    const int32_t* __restrict__ bias, int64_t bias_period, const SoftmaxDev c)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t row = warp; row < rows; row += nwarps) {
+        const int32_t* sr = scores + row * n;
+        const int32_t* br = HAS_BIAS ? bias + (row % bias_period) * n : nullptr;
+        int v[NITER];
+        int mx = INT_MIN;
+#pragma unroll
+        for (int k = 0; k < NITER; ++k) {
+            const int j = lane + 32 * k;
+            if (j < n) {
+                int s = __ldg(sr + j);
+                if (HAS_BIAS) s += __ldg(br + j);
+                v[k] = s;
+                mx = max(mx, s);
+            } else {
+                v[k] = 0;
+            }
+        }
+        mx = __reduce_max_sync(kFull, mx);                      // Eq. (6)
+        unsigned e[NITER];
+        unsigned sum = 0;
+#pragma unroll
+        for (int k = 0; k < NITER; ++k) {
+            const int j = lane + 32 * k;
+            unsigned d = min((unsigned)(mx - v[k]), (unsigned)c.ex.dcap);
+            unsigned ev = exp_core<VARIANT>(d, c.ex);
+            e[k] = j < n ? ev : 0u;
+            sum += e[k];
+        }
+        sum = __reduce_add_sync(kFull, sum);
+        const unsigned f = intdiv_factor(sum, c.M) << c.f_shl;  // Eq. (15)
+        uint8_t* pr = probs + row * n;
+#pragma unroll
+        for (int k = 0; k < NITER; ++k) {
+            const int j = lane + 32 * k;
+            if (j < n) pr[j] = (uint8_t)(__umulhi(f, e[k]) >> c.p_shr);
+        }
+    }
+}
+
+template <int VARIANT, int NITER>
+static int launch_softmax2(const int32_t* s, uint8_t* p, int64_t rows, int n, const int32_t* bias, int64_t period,
+                           const SoftmaxDev& c, cudaStream_t st)
+{
+    const int threads = 256;
+    const int64_t want = (rows + 7) / 8;
+    const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 8);
+    if (bias) softmax_rows_kernel<VARIANT, NITER, true><<<grid, threads, 0, st>>>(s, p, rows, n, bias, period, c);
+    else      softmax_rows_kernel<VARIANT, NITER, false><<<grid, threads, 0, st>>>(s, p, rows, n, bias, period, c);
+    note_launch();
+    return last_launch_status();
+}
+
+template <int VARIANT>
+static int launch_softmax1(const int32_t* s, uint8_t* p, int64_t rows, int n, const int32_t* bias, int64_t period,
+                           const SoftmaxDev& c, cudaStream_t st)
+{
+    const int it = (n + 31) / 32;
+    switch (it) {
+        case 1: return launch_softmax2<VARIANT, 1>(s, p, rows, n, bias, period, c, st);
+        case 2: return launch_softmax2<VARIANT, 2>(s, p, rows, n, bias, period, c, st);
+        case 3: return launch_softmax2<VARIANT, 3>(s, p, rows, n, bias, period, c, st);
+        case 4: return launch_softmax2<VARIANT, 4>(s, p, rows, n, bias, period, c, st);
+        case 5: return launch_softmax2<VARIANT, 5>(s, p, rows, n, bias, period, c, st);
+        case 6: return launch_softmax2<VARIANT, 6>(s, p, rows, n, bias, period, c, st);
+        case 7: return launch_softmax2<VARIANT, 7>(s, p, rows, n, bias, period, c, st);
+        case 8: return launch_softmax2<VARIANT, 8>(s, p, rows, n, bias, period, c, st);
+        default:
+            if (it <= 16) return launch_softmax2<VARIANT, 16>(s, p, rows, n, bias, period, c, st);
+            return launch_softmax2<VARIANT, 32>(s, p, rows, n, bias, period, c, st);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// GELU: element-wise; each warp iteration covers 512 elements with four coalesced 16-byte loads per
+// lane and four coalesced 4-byte stores.
+// ------------------------------------------------------------------------------------------------
+template <int VARIANT>
+__device__ __forceinline__ int gelu_elem(int x, const GeluDev& c)
+{
+    return requant_full(gelu_core<VARIANT>(x, c), c.out);
+}
+
+template <int VARIANT>
+__global__ void __launch_bounds__(256)
+gelu_kernel(const int32_t* __restrict__ x, int8_t* __restrict__ y, int64_t n, const GeluDev c)
+{
+    const int64_t nvec = n >> 2;                                 // int4 / 4-byte groups
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int4* xv = reinterpret_cast<const int4*>(x);
+    unsigned* yv = reinterpret_cast<unsigned*>(y);
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    // four independent groups per iteration for memory-level parallelism
+    for (; i + 3 * stride < nvec; i += 4 * stride) {
+        int4 a[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) a[u] = __ldcs(xv + i + u * stride);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            unsigned o = pack4_s8(gelu_elem<VARIANT>(a[u].x, c), gelu_elem<VARIANT>(a[u].y, c),
+                                  gelu_elem<VARIANT>(a[u].z, c), gelu_elem<VARIANT>(a[u].w, c));
+            __stcs(yv + i + u * stride, o);
+        }
+    }
+    for (; i < nvec; i += stride) {
+        int4 a = __ldcs(xv + i);
+        yv[i] = pack4_s8(gelu_elem<VARIANT>(a.x, c), gelu_elem<VARIANT>(a.y, c), gelu_elem<VARIANT>(a.z, c),
+                         gelu_elem<VARIANT>(a.w, c));
+    }
+    // ragged tail (n % 4 elements)
+    const int64_t t = (nvec << 2) + (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < n) y[t] = (int8_t)gelu_elem<VARIANT>(x[t], c);
+}
+
+// ------------------------------------------------------------------------------------------------
+// LayerNorm: one warp per row; the row lives in registers as packed int8 words (NW per lane).
+// ------------------------------------------------------------------------------------------------
+struct LnDev {
+    int variant, dim;
+    RequantDev out;
+};
+
+__device__ __forceinline__ unsigned long long isqrt_floor(unsigned long long V)
+{
+    // V < 2^53: start from the fp64 square root and fix the last unit
+    unsigned long long r = (unsigned long long)sqrt((double)V);
+    while (r * r > V) --r;
+    while ((r + 1) * (r + 1) <= V) ++r;
+    return r;
+}
+
+__device__ __forceinline__ unsigned long long isqrt_variant(unsigned long long V, int variant)
+{
+    if (V == 0) return 0;
+    if (variant == IPTQ_LN_SHIFT) {
+        // fixed 10 steps of r <- (r + V / r) >> 1 from 2^ceil(bitlen(V) / 2); no convergence test
+        const int w = 64 - __clzll((long long)V);
+        unsigned long long r = 1ull << ((w + 1) >> 1);
+#pragma unroll 1
+        for (int it = 0; it < 10; ++it) r = (r + V / r) >> 1;
+        return r;
+    }
+    return isqrt_floor(V);
+}
+
+template <int NW, bool PTF>
+__global__ void __launch_bounds__(256)
+layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int64_t rows,
+                      const int32_t* __restrict__ gamma_q, const int32_t* __restrict__ beta_q,
+                      const uint8_t* __restrict__ ptf, const LnDev c)
+{
+    const int lane = threadIdx.x & 31;
+    const int D = c.dim;
+    const int words = D >> 2;
+    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    // per-lane channel parameters stay in registers across rows when they fit
+    constexpr bool KEEP = NW <= 8;
+    int4 g[KEEP ? NW : 1], b[KEEP ? NW : 1];
+    unsigned sh[NW];
+#pragma unroll
+    for (int k = 0; k < NW; ++k) {
+        const int wi = lane + 32 * k;
+        sh[k] = 0;
+        if (wi < words) {
+            if (KEEP) {
+                g[k] = __ldg(reinterpret_cast<const int4*>(gamma_q) + wi);
+                b[k] = __ldg(reinterpret_cast<const int4*>(beta_q) + wi);
+            }
+            if (PTF) sh[k] = __ldg(reinterpret_cast<const unsigned*>(ptf) + wi);
+        }
+    }
+    for (int64_t row = warp; row < rows; row += nwarps) {
+        const int* xr = reinterpret_cast<const int*>(x + row * D);
+        int w[NW];
+        int s1 = 0;
+        unsigned s2 = 0;
+#pragma unroll
+        for (int k = 0; k < NW; ++k) {
+            const int wi = lane + 32 * k;
+            w[k] = wi < words ? __ldcs(xr + wi) : 0;
+            if (!PTF) {
+                s1 = __dp4a(w[k], 0x01010101, s1);
+                s2 = (unsigned)__dp4a(w[k], w[k], (int)s2);
+            } else {
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const int xv = ((int)(int8_t)(w[k] >> (8 * t))) << ((sh[k] >> (8 * t)) & 3);
+                    s1 += xv;
+                    s2 += (unsigned)(xv * xv);
+                }
+            }
+        }
+        s1 = __reduce_add_sync(kFull, s1);
+        s2 = __reduce_add_sync(kFull, s2);
+        const long long V = (long long)D * (long long)s2 - (long long)s1 * (long long)s1;   // D^2 var, exact
+        const unsigned long long r = isqrt_variant((unsigned long long)V, c.variant);        // D * std
+        const long long F = r ? (long long)((1ull << 40) / r) : 0;
+        int* yr = reinterpret_cast<int*>(y + row * D);
+#pragma unroll
+        for (int k = 0; k < NW; ++k) {
+            const int wi = lane + 32 * k;
+            if (wi < words) {
+                int4 gg, bb;
+                if (KEEP) { gg = g[k]; bb = b[k]; }
+                else {
+                    gg = __ldg(reinterpret_cast<const int4*>(gamma_q) + wi);
+                    bb = __ldg(reinterpret_cast<const int4*>(beta_q) + wi);
+                }
+                const int gv[4] = {gg.x, gg.y, gg.z, gg.w};
+                const int bv[4] = {bb.x, bb.y, bb.z, bb.w};
+                int o[4];
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    int xv = (int)(int8_t)(w[k] >> (8 * t));
+                    if (PTF) xv <<= ((sh[k] >> (8 * t)) & 3);
+                    const int u = D * xv - s1;                                   // D (x - mean)
+                    const int nq = (int)(((long long)u * F) >> 30);              // (x - mean) / std, Q10
+                    o[t] = requant_full(nq * gv[t] + bv[t], c.out);
+                }
+                __stcs(yr + wi, (int)pack4_s8(o[0], o[1], o[2], o[3]));
+            }
+        }
+    }
+}
+
+template <int NW>
+static int launch_ln(const int8_t* x, int8_t* y, int64_t rows, const int32_t* gq, const int32_t* bq,
+                     const uint8_t* ptf, const LnDev& c, cudaStream_t st)
+{
+    const int threads = 256;
+    const int64_t want = (rows + 7) / 8;
+    const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 8);
+    if (c.variant == IPTQ_LN_PTF) layernorm_rows_kernel<NW, true><<<grid, threads, 0, st>>>(x, y, rows, gq, bq, ptf, c);
+    else                          layernorm_rows_kernel<NW, false><<<grid, threads, 0, st>>>(x, y, rows, gq, bq, ptf, c);
+    note_launch();
+    return last_launch_status();
+}
+
+// Used by the encoder block as well.
+int layernorm_launch(const int8_t* x, int8_t* y, int64_t rows, int dim, const int32_t* gq, const int32_t* bq,
+                     const uint8_t* ptf, const iptq_ln_consts* consts, cudaStream_t st)
+{
+    if (!consts) return IPTQ_ERR_NULL;
+    if (rows < 0 || dim != consts->dim || dim < 2 || dim > 4096 || (dim & 3)) return IPTQ_ERR_SHAPE;
+    if (rows == 0) return IPTQ_OK;
+    if (!x || !y || !gq || !bq) return IPTQ_ERR_NULL;
+    if (consts->variant < 0 || consts->variant > 2) return IPTQ_ERR_VARIANT;
+    if (consts->variant == IPTQ_LN_PTF && !ptf) return IPTQ_ERR_NULL;
+    if (!aligned16(x) || !aligned16(y) || !aligned16(gq) || !aligned16(bq) ||
+        (ptf && (reinterpret_cast<uintptr_t>(ptf) & 3u)))
+        return IPTQ_ERR_ALIGN;
+    int rc = check_requant(&consts->out);
+    if (rc != IPTQ_OK) return rc;
+    if (rows == 0) return IPTQ_OK;
+    LnDev c;
+    c.variant = consts->variant; c.dim = dim; c.out = to_dev(consts->out);
+    const int nw = (dim / 4 + 31) / 32;
+    switch (nw) {
+        case 1: return launch_ln<1>(x, y, rows, gq, bq, ptf, c, st);
+        case 2: return launch_ln<2>(x, y, rows, gq, bq, ptf, c, st);
+        case 3: return launch_ln<3>(x, y, rows, gq, bq, ptf, c, st);
+        case 4: return launch_ln<4>(x, y, rows, gq, bq, ptf, c, st);
+        case 5: case 6: return launch_ln<6>(x, y, rows, gq, bq, ptf, c, st);
+        case 7: case 8: return launch_ln<8>(x, y, rows, gq, bq, ptf, c, st);
+        default:
+            if (nw <= 12) return launch_ln<12>(x, y, rows, gq, bq, ptf, c, st);
+            if (nw <= 16) return launch_ln<16>(x, y, rows, gq, bq, ptf, c, st);
+            return launch_ln<32>(x, y, rows, gq, bq, ptf, c, st);
+    }
+}
+
+}  // namespace iptq
+
+using namespace iptq;
+
+extern "C" {
+
+int iptq_softmax(const int32_t* scores, uint8_t* probs, int64_t rows, int row_len, const int32_t* bias,
+                 int64_t bias_period, const iptq_softmax_consts* consts, iptq_stream_t stream)
+{
+    if (!consts) return IPTQ_ERR_NULL;
+    if (rows < 0 || row_len < 1 || row_len > 1024 || row_len != consts->row_len) return IPTQ_ERR_SHAPE;
+    if (rows == 0) return IPTQ_OK;                      // empty input: nothing to read or write
+    if (!scores || !probs) return IPTQ_ERR_NULL;
+    if (bias && bias_period < 1) return IPTQ_ERR_SHAPE;
+    if (!aligned16(scores) || !aligned16(probs) || (bias && !aligned16(bias))) return IPTQ_ERR_ALIGN;
+    if (consts->out_bits < 4 || consts->out_bits > 8) return IPTQ_ERR_BITS;
+    if (consts->x0 < 8 || consts->M < 31 || consts->M > 40) return IPTQ_ERR_SCALE_RANGE;
+    if (rows == 0) return IPTQ_OK;
+    SoftmaxDev c;
+    c.ex = to_dev_exp(*consts);
+    c.M = consts->M; c.f_shl = consts->f_shl; c.p_shr = consts->p_shr;
+    switch (consts->variant) {
+        case IPTQ_SM_BITEXP: return launch_softmax1<IPTQ_SM_BITEXP>(scores, probs, rows, row_len, bias, bias_period, c, stream);
+        case IPTQ_SM_SHIFTMAX: return launch_softmax1<IPTQ_SM_SHIFTMAX>(scores, probs, rows, row_len, bias, bias_period, c, stream);
+        case IPTQ_SM_POLY: return launch_softmax1<IPTQ_SM_POLY>(scores, probs, rows, row_len, bias, bias_period, c, stream);
+        default: return IPTQ_ERR_VARIANT;
+    }
+}
+
+int iptq_gelu(const int32_t* x, int8_t* y, int64_t n, const iptq_gelu_consts* consts, iptq_stream_t stream)
+{
+    if (!consts) return IPTQ_ERR_NULL;
+    if (n < 0) return IPTQ_ERR_SHAPE;
+    if (n == 0) return IPTQ_OK;
+    if (!x || !y) return IPTQ_ERR_NULL;
+    if (!aligned16(x) || !aligned16(y)) return IPTQ_ERR_ALIGN;
+    if (consts->in_bits < 8 || consts->in_bits > 16) return IPTQ_ERR_BITS;
+    int rc = check_requant(&consts->out);
+    if (rc != IPTQ_OK) return rc;
+    if (n == 0) return IPTQ_OK;
+    const GeluDev c = to_dev(*consts);
+    const int threads = 256;
+    const int64_t groups = (n + 3) / 4;
+    const int grid = (int)std::min<int64_t>((groups + threads - 1) / threads, (int64_t)sm_count() * 16);
+    switch (consts->variant) {
+        case IPTQ_GELU_POLY4: gelu_kernel<IPTQ_GELU_POLY4><<<grid, threads, 0, stream>>>(x, y, n, c); break;
+        case IPTQ_GELU_POLY2: gelu_kernel<IPTQ_GELU_POLY2><<<grid, threads, 0, stream>>>(x, y, n, c); break;
+        case IPTQ_GELU_SHIFT: gelu_kernel<IPTQ_GELU_SHIFT><<<grid, threads, 0, stream>>>(x, y, n, c); break;
+        default: return IPTQ_ERR_VARIANT;
+    }
+    note_launch();
+    return last_launch_status();
+}
+
+int iptq_layernorm(const int8_t* x, int8_t* y, int64_t rows, int dim, const int32_t* gamma_q,
+                   const int32_t* beta_q, const uint8_t* ptf_shift, const iptq_ln_consts* consts,
+                   iptq_stream_t stream)
+{
+    return layernorm_launch(x, y, rows, dim, gamma_q, beta_q, ptf_shift, consts, stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,191 @@
+"""GPU parity of the tensor-core paths (INT8 GEMM carrier, fused MLP, fused attention, encoder block):
+bit-exact against the CPU oracle on the same seeded inputs, through the C-ABI."""
+import numpy as np
+import pytest
+
+from paper_2511_15369_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def api():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2511_15369_b200 import api as _api
+    _api.lib()
+    return _api
+
+
+def _cu(a):
+    import torch
+    return None if a is None else torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _mismatch(got, want):
+    bad = np.argwhere(got != want)
+    return "%d of %d differ; first at %s: got %s want %s" % (
+        len(bad), got.size, bad[:3].tolist(), got[tuple(bad[0])] if len(bad) else None,
+        want[tuple(bad[0])] if len(bad) else None)
+
+
+def _linear_case(rng, M, N, K, w_bits=8):
+    x = rng.integers(-128, 128, size=(M, K)).astype(np.int8)
+    lim = 8 if w_bits == 4 else 128
+    w = rng.integers(-lim, lim, size=(N, K)).astype(np.int8)
+    bias = rng.integers(-3000, 3000, size=N).astype(np.int32)
+    ratios = 2.0 ** rng.uniform(-12, -7, size=N) * (16 if w_bits == 4 else 1)
+    return x, w, bias, ratios
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (197, 384, 384), (300, 1152, 384), (1000, 384, 1536),
+                                   (77, 96, 96), (130, 288, 96), (256, 16, 16), (5, 144, 272)])
+def test_linear_parity(api, orc, M, N, K):
+    rng = np.random.default_rng(M + N + K)
+    x, w, bias, ratios = _linear_case(rng, M, N, K)
+    mo, so = [], []
+    for r in ratios:
+        q = orc.requant_prepare(r)
+        mo.append(q.mult)
+        so.append(q.shift)
+    mo, so = np.array(mo, np.int32), np.array(so, np.int8)
+    ma, sa = api.channel_requant_prepare(ratios)
+    assert (ma == mo).all() and (sa == so).all()
+    ws = api.Workspace(api.linear_workspace_bytes(M, N, K))
+    want = orc.linear(x, w, bias, mo, so, out_zp=3)
+    got = api.linear(_cu(x), _cu(w), _cu(bias), _cu(ma), _cu(sa), ws, out_zp=3).cpu().numpy()
+    ws.check()
+    assert (got == want).all(), _mismatch(got, want)
+    # residual branch, no bias
+    res = rng.integers(-128, 128, size=(M, N)).astype(np.int8)
+    rro = orc.requant_prepare(0.9 / 65536, zp=-4)
+    rra = api.requant_prepare(0.9 / 65536, zp=-4)
+    want = orc.linear(x, w, None, mo, so, out_zp=-2, residual=res, residual_rq=rro)
+    got = api.linear(_cu(x), _cu(w), None, _cu(ma), _cu(sa), ws, out_zp=-2, residual=_cu(res), residual_rq=rra).cpu().numpy()
+    ws.check()
+    assert (got == want).all(), _mismatch(got, want)
+
+
+def test_linear_w4(api, orc):
+    rng = np.random.default_rng(44)
+    M, N, K = 200, 256, 384
+    x, w, bias, ratios = _linear_case(rng, M, N, K, 4)
+    wp = synth.pack_int4(w)
+    ma, sa = api.channel_requant_prepare(ratios)
+    ws = api.Workspace(api.linear_workspace_bytes(M, N, K, 4))
+    want = orc.linear(x, wp, bias, ma, sa, w_bits=4)
+    got = api.linear(_cu(x), _cu(wp), _cu(bias), _cu(ma), _cu(sa), ws, w_bits=4).cpu().numpy()
+    ws.check()
+    assert (got == want).all(), _mismatch(got, want)
+    assert (want == orc.linear(x, w, bias, ma, sa)).all()
+
+
+def test_linear_errors(api):
+    import torch
+    ws = api.Workspace(256)
+    x = torch.zeros((8, 24), dtype=torch.int8, device="cuda")
+    w = torch.zeros((16, 24), dtype=torch.int8, device="cuda")
+    m = torch.full((16,), 1 << 30, dtype=torch.int32, device="cuda")
+    s = torch.ones((16,), dtype=torch.int8, device="cuda")
+    with pytest.raises(api.IptqError) as e:
+        api.linear(x, w, None, m, s, ws)          # K not a multiple of 16
+    assert e.value.status == api.ERR_SHAPE
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("M,D,Dh", [(197, 192, 768), (333, 384, 1536), (64, 96, 384)])
+def test_mlp_parity(api, orc, variant, M, D, Dh):
+    rng = np.random.default_rng(M + variant)
+    x = rng.integers(-128, 128, size=(M, D)).astype(np.int8)
+    w1 = rng.integers(-128, 128, size=(Dh, D)).astype(np.int8)
+    b1 = rng.integers(-2000, 2000, size=Dh).astype(np.int32)
+    in_bits = 12
+    # accumulator std ~ 74*74*sqrt(D); bring 4 sigma to the in_bits range
+    acc_std = 74.0 * 74.0 * np.sqrt(D)
+    r1 = (2047 / (4 * acc_std)) * 2.0 ** rng.uniform(-0.3, 0.3, size=Dh)
+    m1, s1 = api.channel_requant_prepare(r1)
+    S_in = 4.0 / 2047                                   # the GELU sees roughly N(0, 1)
+    go = orc.gelu_prepare(S_in, in_bits, 0.03, -100, 8, variant)
+    ga = api.gelu_prepare(S_in, in_bits, 0.03, -100, 8, variant)
+    w2 = rng.integers(-128, 128, size=(D, Dh)).astype(np.int8)
+    b2 = rng.integers(-2000, 2000, size=D).astype(np.int32)
+    m2, s2 = api.channel_requant_prepare(2.0 ** rng.uniform(-13, -11, size=D))
+    res = rng.integers(-128, 128, size=(M, D)).astype(np.int8)
+    rro, rra = orc.requant_prepare(0.5 / 65536), api.requant_prepare(0.5 / 65536)
+    ws = api.Workspace(api.mlp_workspace_bytes(M, D, Dh))
+    # stop after GELU
+    want_h = orc.mlp_block(x, w1, b1, m1, s1, go)
+    got_h = api.mlp_block(_cu(x), _cu(w1), _cu(b1), _cu(m1), _cu(s1), ga, ws).cpu().numpy()
+    ws.check()
+    assert len(np.unique(want_h)) > 50
+    assert (got_h == want_h).all(), _mismatch(got_h, want_h)
+    # full MLP with residual
+    want = orc.mlp_block(x, w1, b1, m1, s1, go, w2, b2, m2, s2, 1, res, rro)
+    got = api.mlp_block(_cu(x), _cu(w1), _cu(b1), _cu(m1), _cu(s1), ga, ws, _cu(w2), _cu(b2), _cu(m2), _cu(s2), 1,
+                        _cu(res), rra).cpu().numpy()
+    ws.check()
+    assert (got == want).all(), _mismatch(got, want)
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("B,H,N,dh,use_bias,use_mask", [
+    (2, 3, 197, 64, False, False), (3, 2, 49, 32, True, False), (4, 3, 49, 32, True, True),
+    (1, 1, 1, 64, False, False), (2, 2, 128, 64, False, False), (1, 2, 129, 32, False, False),
+    (1, 1, 256, 64, True, False), (2, 1, 80, 32, False, True), (5, 6, 197, 64, False, False)])
+def test_attention_parity(api, orc, variant, B, H, N, dh, use_bias, use_mask):
+    rng = np.random.default_rng(B * 1000 + N + dh + variant)
+    q, k, v = (np.clip(np.round(rng.normal(0, 40, size=(B, H, N, dh))), -128, 127).astype(np.int8) for _ in range(3))
+    # logit scale: q.k has std ~ 1600 * sqrt(dh); put the logits on N(0, 3^2)
+    S = 3.0 / (1600.0 * np.sqrt(dh))
+    bias = np.round(rng.normal(0, 1, size=(H, N, N)) / S).astype(np.int32) if use_bias else None
+    mask_id = rng.integers(0, 3, size=(B, N)).astype(np.uint8) if use_mask else None
+    so, sa = orc.softmax_prepare(S, N, 8, variant), api.softmax_prepare(S, N, 8, variant)
+    ro, ra = orc.requant_prepare(0.011, zp=1), api.requant_prepare(0.011, zp=1)
+    want = orc.attention_block(q, k, v, so, ro, bias, mask_id)
+    ws = api.Workspace(api.attention_workspace_bytes(B, H, N, dh))
+    got = api.attention_block(_cu(q), _cu(k), _cu(v), sa, ra, ws, _cu(bias), _cu(mask_id)).cpu().numpy()
+    ws.check()
+    assert len(np.unique(want)) > 10 or N == 1
+    assert (got == want).all(), _mismatch(got, want)
+
+
+def _oracle_block(orc, spec, table):
+    sm_v, gelu_v, ln1_v, ln2_v = table
+    sh = spec.shape
+    d = dict(B=sh.B, N=sh.N, D=sh.D, H=sh.H, dh=sh.dh, Dh=sh.Dh, w_bits=spec.w_bits)
+    for name, lnspec, var in (("ln1", spec.ln1, ln1_v), ("ln2", spec.ln2, ln2_v)):
+        gq, bq, c = orc.layernorm_prepare(lnspec["gamma"], lnspec["beta"], lnspec["out_scale"], lnspec["out_zp"], 8, var)
+        d[name + "_gamma"], d[name + "_beta"], d[name] = gq, bq, c
+        d[name + "_ptf"] = lnspec.get("ptf")
+    for name, ls in (("qkv", spec.qkv), ("proj", spec.proj), ("fc1", spec.fc1), ("fc2", spec.fc2)):
+        rq = [orc.requant_prepare(float(r)) for r in ls.ratio]
+        d["w_" + name], d["b_" + name] = ls.w_packed, ls.bias
+        d["m_" + name] = np.array([r.mult for r in rq], np.int32)
+        d["s_" + name] = np.array([r.shift for r in rq], np.int8)
+    d["sm"] = orc.softmax_prepare(spec.softmax_scale, sh.N, 8, sm_v)
+    d["pv_rq"] = orc.requant_prepare(spec.pv_ratio)
+    d["attn_bias"], d["mask_id"] = spec.attn_bias, spec.mask_id
+    d["res1_rq"] = orc.requant_prepare(spec.proj.res_ratio / 65536, zp=spec.proj.res_zp)
+    d["res2_rq"] = orc.requant_prepare(spec.fc2.res_ratio / 65536, zp=spec.fc2.res_zp)
+    gl = spec.gelu
+    d["gelu"] = orc.gelu_prepare(gl["in_scale"], gl["in_bits"], gl["out_scale"], gl["out_zp"], 8, gelu_v)
+    d["proj_zp"], d["fc2_zp"] = spec.proj.out_zp, spec.fc2.out_zp
+    return orc.encoder_block(spec.x, d)
+
+
+@pytest.mark.parametrize("shape,w_bits,table", [
+    (synth.CONFIGS["cfg0"], 8, (0, 0, 0, 0)),
+    (synth.BlockShape("DeiT-S b3", 3, 197, 384, 6, 64, 1536), 8, (0, 0, 0, 0)),
+    (synth.BlockShape("DeiT-S b2 alt", 2, 197, 384, 6, 64, 1536), 8, (1, 1, 1, 1)),
+    (synth.BlockShape("ViT-B b1 W4", 1, 197, 768, 12, 64, 3072), 4, (2, 2, 1, 0)),
+    (synth.BlockShape("Swin-T 8 windows", 8, 49, 96, 3, 32, 384, True), 8, (0, 0, 0, 0)),
+])
+def test_encoder_block_parity(api, orc, shape, w_bits, table):
+    spec = synth.make_block(shape, seed=1, w_bits=w_bits, gelu_in_bits=14 if table[1] == 2 else 16)
+    want = _oracle_block(orc, spec, table)
+    blk = api.EncoderBlock(spec, table)
+    got = blk(_cu(spec.x)).cpu().numpy()
+    blk.ws.check()
+    assert len(np.unique(want)) > 30
+    assert (got == want).all(), _mismatch(got, want)

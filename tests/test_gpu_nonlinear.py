@@ -1,0 +1,153 @@
+"""GPU parity of the stand-alone integer Softmax / GELU / LayerNorm kernels: bit-exact against the
+CPU oracle on the same seeded inputs, through the C-ABI."""
+import numpy as np
+import pytest
+
+from paper_2511_15369_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def api():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2511_15369_b200 import api as _api
+    _api.lib()
+    return _api
+
+
+def _cu(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def test_prepared_constants_agree_with_the_oracle(api, orc):
+    for S in (3e-4, 12 / 127, 1 / 777.7):
+        for n in (1, 49, 197, 1024):
+            for var in (0, 1, 2):
+                a, b = api.softmax_prepare(S, n, 8, var), orc.softmax_prepare(S, n, 8, var)
+                for f, _ in b._fields_:
+                    assert getattr(a, f) == getattr(b, f), (f, S, n, var)
+    for S, bits in ((1.3e-4, 16), (2e-3, 12), (0.05, 8)):
+        for var in (0, 1, 2):
+            a, b = api.gelu_prepare(S, bits, 0.02, -100, 8, var), orc.gelu_prepare(S, bits, 0.02, -100, 8, var)
+            for f, _ in b._fields_[:-1]:
+                assert getattr(a, f) == getattr(b, f), (f, S, bits, var)
+            for f in ("mult", "shift", "zp", "qmin", "qmax"):
+                assert getattr(a.out, f) == getattr(b.out, f)
+    rng = np.random.default_rng(0)
+    for r in 2.0 ** rng.uniform(-32, -2.001, size=200):
+        a, b = api.requant_prepare(r), orc.requant_prepare(r)
+        assert (a.mult, a.shift) == (b.mult, b.shift)
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("rows,n", [(591, 197), (1000, 49), (33, 1), (17, 2), (40, 208), (9, 1000), (5, 64)])
+@pytest.mark.parametrize("scale", [synth.SOFTMAX_SCALE_ACC, synth.SOFTMAX_SCALE_8BIT])
+def test_softmax_parity(api, orc, variant, rows, n, scale):
+    s = synth.quantize_scores(synth.softmax_logits(rows, n, seed=rows + n), scale)
+    want = orc.softmax(s, orc.softmax_prepare(scale, n, 8, variant))
+    got = api.softmax(_cu(s), api.softmax_prepare(scale, n, 8, variant)).cpu().numpy()
+    assert (got == want).all()
+
+
+def test_softmax_edge_rows_and_bias(api, orc):
+    n = 197
+    rng = np.random.default_rng(3)
+    s = rng.integers(-50000, 50000, size=(64, n)).astype(np.int32)
+    s[0] = 7                                   # all-equal row
+    s[1] = -(1 << 30) + 1
+    s[1, 5] = (1 << 30) - 1                    # one huge outlier, extreme magnitudes
+    s[2] = (1 << 30) - 1
+    s[3, :] = np.arange(n) * 1000
+    bias = rng.integers(-20000, 20000, size=(3, n)).astype(np.int32)
+    for variant in (0, 1, 2):
+        for bits in (8, 6, 4):
+            co = orc.softmax_prepare(3e-4, n, bits, variant)
+            ca = api.softmax_prepare(3e-4, n, bits, variant)
+            assert (api.softmax(_cu(s), ca).cpu().numpy() == orc.softmax(s, co)).all()
+            got = api.softmax(_cu(s), ca, bias=_cu(bias)).cpu().numpy()
+            assert (got == orc.softmax(s, co, bias=bias, bias_period=3)).all()
+    # large x0 (N = 0, M capped)
+    S = 1.0 / ((1 << 20) - 2.5)
+    s2 = rng.integers(-(1 << 26), 1 << 26, size=(32, 49)).astype(np.int32)
+    assert (api.softmax(_cu(s2), api.softmax_prepare(S, 49)).cpu().numpy() == orc.softmax(s2, orc.softmax_prepare(S, 49))).all()
+
+
+def test_softmax_empty_and_errors(api):
+    import torch
+    c = api.softmax_prepare(3e-4, 197)
+    out = api.softmax(torch.empty((0, 197), dtype=torch.int32, device="cuda"), c)
+    assert out.shape == (0, 197)
+    with pytest.raises(api.IptqError) as e:
+        api.softmax(torch.zeros((4, 49), dtype=torch.int32, device="cuda"), c)      # row_len mismatch
+    assert e.value.status == api.ERR_SHAPE
+    with pytest.raises(api.IptqError) as e:
+        api.softmax_prepare(0.5, 197)
+    assert e.value.status == api.ERR_SCALE_RANGE
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("n", [151296, 4099, 3, 1 << 20])
+def test_gelu_parity(api, orc, variant, n):
+    bits = 16 if variant != 2 else 12
+    x, S = synth.quantize_sym(synth.gelu_values(n, seed=n), bits)
+    ref = synth.gelu_ref(x[:4096] * S)
+    So, zp = synth.affine_out_quant(ref)
+    want = orc.gelu(x, orc.gelu_prepare(S, bits, So, zp, 8, variant))
+    got = api.gelu(_cu(x), api.gelu_prepare(S, bits, So, zp, 8, variant)).cpu().numpy()
+    assert (got == want).all()
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("bits,S", [(8, 8.0 / 127), (12, 0.003), (16, 1.3e-4)])
+def test_gelu_exhaustive_inputs(api, orc, variant, bits, S):
+    if variant == 2 and bits == 16:
+        S = 1.0 / 9000                     # the shift exponential needs floor(1/S) < 2^14
+    x = np.arange(-(1 << 17), 1 << 17, dtype=np.int32)       # covers every in_bits value and the clamp
+    for out_bits in (8, 5):
+        want = orc.gelu(x, orc.gelu_prepare(S, bits, 0.03, -7, out_bits, variant))
+        got = api.gelu(_cu(x), api.gelu_prepare(S, bits, 0.03, -7, out_bits, variant)).cpu().numpy()
+        assert (got == want).all()
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("rows,dim", [(197, 192), (300, 384), (100, 768), (513, 96), (7, 1536), (3, 4096), (5, 8)])
+def test_layernorm_parity(api, orc, variant, rows, dim):
+    xf, gamma, beta, _ = synth.ln_values(rows, dim, seed=dim)
+    xq, _ = synth.quantize_sym(xf, 8, np.int8)
+    ptf = synth.ptf_shifts(xq) if variant == 2 else None
+    ref = synth.layernorm_ref(xq[:64].astype(np.float64), gamma, beta)
+    So, zp = synth.affine_out_quant(ref)
+    gq, bq, co = orc.layernorm_prepare(gamma, beta, So, zp, 8, variant)
+    gq2, bq2, ca = api.layernorm_prepare(gamma, beta, So, zp, 8, variant)
+    assert (gq == gq2).all() and (bq == bq2).all()
+    assert (ca.out.mult, ca.out.shift, ca.out.zp) == (co.out.mult, co.out.shift, co.out.zp)
+    want = orc.layernorm(xq, gq, bq, co, ptf)
+    got = api.layernorm(_cu(xq), _cu(gq2), _cu(bq2), ca, None if ptf is None else _cu(ptf)).cpu().numpy()
+    assert (got == want).all()
+
+
+def test_layernorm_degenerate_rows(api, orc):
+    dim = 192
+    rng = np.random.default_rng(5)
+    x = rng.integers(-128, 128, size=(40, dim)).astype(np.int8)
+    x[0] = 0
+    x[1] = 127                                  # zero variance
+    x[2] = -128
+    x[3] = 0
+    x[3, 17] = 1                                # smallest non-zero variance
+    x[4, ::2] = 127
+    x[4, 1::2] = -128                           # largest variance
+    # rows whose D^2 var + 1 is a perfect square make the fixed-step square root stop one above
+    x[5] = 0
+    x[5, :3] = [1, 1, 1]
+    gamma = rng.normal(1, 0.1, dim).astype(np.float32)
+    beta = rng.normal(0, 0.1, dim).astype(np.float32)
+    for variant in (0, 1):
+        gq, bq, co = orc.layernorm_prepare(gamma, beta, 0.02, 3, 8, variant)
+        _, _, ca = api.layernorm_prepare(gamma, beta, 0.02, 3, 8, variant)
+        got = api.layernorm(_cu(x), _cu(gq), _cu(bq), ca).cpu().numpy()
+        assert (got == orc.layernorm(x, gq, bq, co)).all()
