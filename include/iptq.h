@@ -146,7 +146,7 @@ typedef struct {
 
 /* host.  gamma/beta: host float [dim]; gamma_q/beta_q: host int32 [dim] outputs
  * (gamma_q = round(gamma / S_g), S_g = max|gamma| / 32767; beta_q = round(beta / (2^-10 S_g))).
- * 2 <= dim <= 4096, dim % 4 == 0. */
+ * 2 <= dim <= 3072 (n_c gamma_q + beta_q must stay below 2^31), dim % 4 == 0. */
 int iptq_layernorm_prepare(int dim, const float* gamma, const float* beta, double out_scale, int out_zp,
                            int out_bits, iptq_ln_variant variant, int32_t* gamma_q, int32_t* beta_q,
                            iptq_ln_consts* out /*host*/);
@@ -223,6 +223,15 @@ size_t iptq_encoder_block_workspace_bytes(const iptq_block_params* p /*host*/);
 /* x, y: dev int8 [B*N, D]. */
 int iptq_encoder_block(const int8_t* x, int8_t* y, const iptq_block_params* p /*host*/, void* ws, size_t ws_bytes,
                        iptq_stream_t stream);
+
+/* The same block with a stage boundary recorded into caller-owned events, for per-kernel timing:
+ * events (host array of IPTQ_BLOCK_STAGES + 1 cudaEvent_t handles created with timing enabled) --
+ * events[0] is recorded before the first launch and events[i] after stage i, in the order
+ * LN1, QKV, attention, proj, LN2, FC1+GELU, FC2 (the int4 unpack launches of w_bits = 4 fall into stage 1).
+ * The kernels and their results are those of iptq_encoder_block(). */
+#define IPTQ_BLOCK_STAGES 7
+int iptq_encoder_block_profiled(const int8_t* x, int8_t* y, const iptq_block_params* p /*host*/, void* ws,
+                                size_t ws_bytes, iptq_stream_t stream, void* const* events /*host*/, int n_events);
 
 /* ------------------------------------------------------------------ status
  * iptq_workspace_init: zero the status block (enqueued on the stream); call once per workspace.

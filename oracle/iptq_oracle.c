@@ -311,7 +311,7 @@ int oracle_layernorm_prepare(int dim, const float* gamma, const float* beta, dou
                              int out_bits, int variant, int32_t* gamma_q, int32_t* beta_q, oracle_ln_consts_t* out)
 {
     if (!gamma || !beta || !gamma_q || !beta_q || !out) return ORACLE_ERR_ARG;
-    if (dim < 2 || dim > 4096 || out_bits < 4 || out_bits > 8) return ORACLE_ERR_ARG;
+    if (dim < 2 || dim > 3072 || out_bits < 4 || out_bits > 8) return ORACLE_ERR_ARG;
     if (variant < 0 || variant > 2) return ORACLE_ERR_ARG;
     if (!(out_scale > 0.0)) return ORACLE_ERR_RANGE;
     double gmax = 0.0;

@@ -19,6 +19,8 @@ SM_BITEXP, SM_SHIFTMAX, SM_POLY = 0, 1, 2
 GELU_POLY4, GELU_POLY2, GELU_SHIFT = 0, 1, 2
 LN_SHIFT, LN_NEWTON, LN_PTF = 0, 1, 2
 
+BLOCK_STAGES = ("ln1", "qkv", "attention", "proj", "ln2", "fc1_gelu", "fc2")
+
 OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_BITS, ERR_SCALE_RANGE, ERR_VARIANT, ERR_WORKSPACE, ERR_TIMEOUT, ERR_CUDA = range(10)
 
 
@@ -114,6 +116,8 @@ def lib():
         L.iptq_encoder_block_workspace_bytes.restype = C.c_size_t
         L.iptq_encoder_block_workspace_bytes.argtypes = [C.POINTER(BlockParams)]
         L.iptq_encoder_block.argtypes = [_vp, _vp, C.POINTER(BlockParams), _vp, C.c_size_t, _vp]
+        L.iptq_encoder_block_profiled.argtypes = [_vp, _vp, C.POINTER(BlockParams), _vp, C.c_size_t, _vp,
+                                                  C.POINTER(C.c_void_p), C.c_int]
         L.iptq_workspace_init.argtypes = [_vp, C.c_size_t, _vp]
         L.iptq_check.argtypes = [_vp, _vp]
         _lib = L
@@ -126,7 +130,7 @@ def exported_symbols():
             "iptq_gelu_prepare", "iptq_gelu", "iptq_layernorm_prepare", "iptq_layernorm",
             "iptq_linear_workspace_bytes", "iptq_linear", "iptq_attention_workspace_bytes", "iptq_attention_block",
             "iptq_mlp_workspace_bytes", "iptq_mlp_block", "iptq_encoder_block_workspace_bytes",
-            "iptq_encoder_block", "iptq_workspace_init", "iptq_check", "iptq_strerror", "iptq_launch_count"]
+            "iptq_encoder_block", "iptq_encoder_block_profiled", "iptq_workspace_init", "iptq_check", "iptq_strerror", "iptq_launch_count"]
 
 
 def _chk(rc, what):
@@ -339,3 +343,20 @@ class EncoderBlock:
         _chk(lib().iptq_encoder_block(_dp(x), _dp(out), C.byref(self.params), self.ws.ptr, self.ws.nbytes,
                                       _stream()), "iptq_encoder_block")
         return out
+
+    def profiled(self, x, out, events):
+        """Same launches as ``__call__`` with ``events[0]`` recorded before the first kernel and ``events[i]``
+        after stage i of ``BLOCK_STAGES`` (``torch.cuda.Event(enable_timing=True)``, each recorded once before)."""
+        assert len(events) == len(BLOCK_STAGES) + 1
+        arr = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
+        _chk(lib().iptq_encoder_block_profiled(_dp(x), _dp(out), C.byref(self.params), self.ws.ptr, self.ws.nbytes,
+                                               _stream(), arr, len(events)), "iptq_encoder_block_profiled")
+        return out
+
+    def run_host(self, x_host, y_host, x_dev, y_dev):
+        """One step from HOST buffers: pinned ``x_host`` -> device, the block, device -> pinned ``y_host``;
+        all three are enqueued on the current stream (the caller synchronises)."""
+        x_dev.copy_(x_host, non_blocking=True)
+        self(x_dev, y_dev)
+        y_host.copy_(y_dev, non_blocking=True)
+        return y_host

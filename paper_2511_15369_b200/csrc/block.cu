@@ -86,8 +86,8 @@ size_t iptq_encoder_block_workspace_bytes(const iptq_block_params* p)
     return block_layout(p).total;
 }
 
-int iptq_encoder_block(const int8_t* x, int8_t* y, const iptq_block_params* p, void* ws, size_t ws_bytes,
-                       iptq_stream_t stream)
+static int encoder_block_run(const int8_t* x, int8_t* y, const iptq_block_params* p, void* ws, size_t ws_bytes,
+                             cudaStream_t stream, cudaEvent_t* ev)
 {
     int rc = check_block(p);
     if (rc != IPTQ_OK) return rc;
@@ -107,6 +107,12 @@ int iptq_encoder_block(const int8_t* x, int8_t* y, const iptq_block_params* p, v
     int8_t* hid = reinterpret_cast<int8_t*>(base + l.hid);
     const int64_t T = p->B * p->N;
     const int D = p->D, Dh = p->Dh;
+    int stage = 0;
+    auto mark = [&]() -> int {                     // stage boundary: record the caller's event, if any
+        if (!ev) return IPTQ_OK;
+        return cuda_status(cudaEventRecord(ev[stage++], stream));
+    };
+    if ((rc = mark()) != IPTQ_OK) return rc;
 
     const int8_t *wq = static_cast<const int8_t*>(p->w_qkv), *wp = static_cast<const int8_t*>(p->w_proj),
                  *w1 = static_cast<const int8_t*>(p->w_fc1), *w2 = static_cast<const int8_t*>(p->w_fc2);
@@ -122,19 +128,44 @@ int iptq_encoder_block(const int8_t* x, int8_t* y, const iptq_block_params* p, v
     }
 
     if ((rc = layernorm_launch(x, h1, T, D, p->ln1_gamma, p->ln1_beta, p->ln1_ptf, p->ln1, stream)) != IPTQ_OK) return rc;
+    if ((rc = mark()) != IPTQ_OK) return rc;
     LinearArgs lq{h1, wq, p->b_qkv, p->m_qkv, p->s_qkv, 0, nullptr, nullptr, nullptr, qkv, T, 3 * D, D, status};
     if ((rc = linear_launch(lq, stream)) != IPTQ_OK) return rc;
+    if ((rc = mark()) != IPTQ_OK) return rc;
     // a row of qkv is [q | k | v]; head h occupies columns h*dh .. of each third
     AttnArgs aa{qkv, qkv + D, qkv + 2 * D, (int64_t)3 * D, (int64_t)p->dh, (int64_t)p->N * 3 * D, att, p->B, p->H, p->N,
                 p->dh, p->attn_bias, p->mask_id, p->sm, p->pv_rq, status};
     if ((rc = attention_launch(aa, stream)) != IPTQ_OK) return rc;
+    if ((rc = mark()) != IPTQ_OK) return rc;
     LinearArgs lp{att, wp, p->b_proj, p->m_proj, p->s_proj, p->proj_zp, x, p->res1_rq, nullptr, x1, T, D, D, status};
     if ((rc = linear_launch(lp, stream)) != IPTQ_OK) return rc;
+    if ((rc = mark()) != IPTQ_OK) return rc;
     if ((rc = layernorm_launch(x1, h2, T, D, p->ln2_gamma, p->ln2_beta, p->ln2_ptf, p->ln2, stream)) != IPTQ_OK) return rc;
+    if ((rc = mark()) != IPTQ_OK) return rc;
     LinearArgs l1{h2, w1, p->b_fc1, p->m_fc1, p->s_fc1, 0, nullptr, nullptr, p->gelu, hid, T, Dh, D, status};
     if ((rc = linear_launch(l1, stream)) != IPTQ_OK) return rc;
+    if ((rc = mark()) != IPTQ_OK) return rc;
     LinearArgs l2{hid, w2, p->b_fc2, p->m_fc2, p->s_fc2, p->fc2_zp, x1, p->res2_rq, nullptr, y, T, D, Dh, status};
-    return linear_launch(l2, stream);
+    if ((rc = linear_launch(l2, stream)) != IPTQ_OK) return rc;
+    return mark();
+}
+
+int iptq_encoder_block(const int8_t* x, int8_t* y, const iptq_block_params* p, void* ws, size_t ws_bytes,
+                       iptq_stream_t stream)
+{
+    return encoder_block_run(x, y, p, ws, ws_bytes, stream, nullptr);
+}
+
+int iptq_encoder_block_profiled(const int8_t* x, int8_t* y, const iptq_block_params* p, void* ws, size_t ws_bytes,
+                                iptq_stream_t stream, void* const* events, int n_events)
+{
+    if (!events) return IPTQ_ERR_NULL;
+    if (n_events != IPTQ_BLOCK_STAGES + 1) return IPTQ_ERR_SHAPE;
+    for (int i = 0; i < n_events; ++i)
+        if (!events[i]) return IPTQ_ERR_NULL;
+    cudaEvent_t ev[IPTQ_BLOCK_STAGES + 1];
+    for (int i = 0; i < n_events; ++i) ev[i] = static_cast<cudaEvent_t>(events[i]);
+    return encoder_block_run(x, y, p, ws, ws_bytes, stream, ev);
 }
 
 }  // extern "C"

@@ -214,7 +214,7 @@ int iptq_layernorm_prepare(int dim, const float* gamma, const float* beta, doubl
                            iptq_ln_consts* out)
 {
     if (!gamma || !beta || !gamma_q || !beta_q || !out) return IPTQ_ERR_NULL;
-    if (dim < 2 || dim > 4096 || (dim & 3)) return IPTQ_ERR_SHAPE;
+    if (dim < 2 || dim > 3072 || (dim & 3)) return IPTQ_ERR_SHAPE;
     if (out_bits < 4 || out_bits > 8) return IPTQ_ERR_BITS;
     if (variant != IPTQ_LN_SHIFT && variant != IPTQ_LN_NEWTON && variant != IPTQ_LN_PTF) return IPTQ_ERR_VARIANT;
     if (!(out_scale > 0.0)) return IPTQ_ERR_SCALE_RANGE;

@@ -267,7 +267,7 @@ int layernorm_launch(const int8_t* x, int8_t* y, int64_t rows, int dim, const in
                      const uint8_t* ptf, const iptq_ln_consts* consts, cudaStream_t st)
 {
     if (!consts) return IPTQ_ERR_NULL;
-    if (rows < 0 || dim != consts->dim || dim < 2 || dim > 4096 || (dim & 3)) return IPTQ_ERR_SHAPE;
+    if (rows < 0 || dim != consts->dim || dim < 2 || dim > 3072 || (dim & 3)) return IPTQ_ERR_SHAPE;
     if (rows == 0) return IPTQ_OK;
     if (!x || !y || !gq || !bq) return IPTQ_ERR_NULL;
     if (consts->variant < 0 || consts->variant > 2) return IPTQ_ERR_VARIANT;

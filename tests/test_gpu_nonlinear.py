@@ -93,8 +93,10 @@ def test_softmax_empty_and_errors(api):
 @pytest.mark.parametrize("n", [151296, 4099, 3, 1 << 20])
 def test_gelu_parity(api, orc, variant, n):
     bits = 16 if variant != 2 else 12
-    x, S = synth.quantize_sym(synth.gelu_values(n, seed=n), bits)
-    ref = synth.gelu_ref(x[:4096] * S)
+    # scales are calibrated on at least 4096 draws so that the ragged n = 3 case keeps a realistic output range
+    xall, S = synth.quantize_sym(synth.gelu_values(max(n, 4096), seed=n), bits)
+    x = np.ascontiguousarray(xall[:n])
+    ref = synth.gelu_ref(xall[:4096] * S)
     So, zp = synth.affine_out_quant(ref)
     want = orc.gelu(x, orc.gelu_prepare(S, bits, So, zp, 8, variant))
     got = api.gelu(_cu(x), api.gelu_prepare(S, bits, So, zp, 8, variant)).cpu().numpy()
@@ -114,7 +116,7 @@ def test_gelu_exhaustive_inputs(api, orc, variant, bits, S):
 
 
 @pytest.mark.parametrize("variant", [0, 1, 2])
-@pytest.mark.parametrize("rows,dim", [(197, 192), (300, 384), (100, 768), (513, 96), (7, 1536), (3, 4096), (5, 8)])
+@pytest.mark.parametrize("rows,dim", [(197, 192), (300, 384), (100, 768), (513, 96), (7, 1536), (3, 3072), (5, 8)])
 def test_layernorm_parity(api, orc, variant, rows, dim):
     xf, gamma, beta, _ = synth.ln_values(rows, dim, seed=dim)
     xq, _ = synth.quantize_sym(xf, 8, np.int8)
