@@ -205,6 +205,28 @@ class ClockSampler:
                 "samples": len(inside), "power_w_max": max(pw) if pw else None, "note": note}
 
 
+# ---------------------------------------------------------------------------------------------- ranks
+def shard_seed(rank):
+    """Seed of the batch shard a rank owns: shards are independent draws of the same distribution."""
+    return int(rank)
+
+
+def rank_max(v, world, device=None):
+    """Max over ranks of a per-rank scalar (the timed region of a multi-GPU run is as long as its slowest rank)."""
+    if world == 1:
+        return float(v)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([v], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tops(ops_per_rank_step, steps, world, total_ms_max):
+    """Whole-job throughput: every rank did `steps` passes over its own shard within the slowest rank's time."""
+    return ops_per_rank_step * steps * world / (total_ms_max * 1e-3) / 1e12
+
+
 # ---------------------------------------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
@@ -228,14 +250,10 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     def max_over_ranks(v):
-        if world == 1:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return rank_max(v, world, dev)
 
     shape = synth.CONFIGS["cfg1"]
-    spec = synth.make_block(shape, seed=rank)          # each rank owns its own batch shard (weak scaling)
+    spec = synth.make_block(shape, seed=shard_seed(rank))   # each rank owns its own batch shard (weak scaling)
     blk = api.EncoderBlock(spec, TABLE, device=dev)
     x = torch.from_numpy(spec.x).to(dev)
     y = torch.empty_like(x)
@@ -269,7 +287,7 @@ def run_ours(args):
     launches = api.launch_count() - launches0
     blk.ws.check()
     total_ms = max_over_ranks(sum(ms))
-    value = ops * K * world / (total_ms * 1e-3) / 1e12
+    value = job_tops(ops, K, world, total_ms)
 
     # ---- per-stage times from the same kernels with events at the stage boundaries
     nst = len(api.BLOCK_STAGES)
@@ -295,7 +313,7 @@ def run_ours(args):
         blk.run_host(xh, yh, x, y)
     ms_e2e = timed_loop(lambda: blk.run_host(xh, yh, x, y), K)
     total_e2e = max_over_ranks(sum(ms_e2e))
-    e2e_value = ops * K * world / (total_e2e * 1e-3) / 1e12
+    e2e_value = job_tops(ops, K, world, total_e2e)
     got_full = yh.numpy().copy()
 
     # ---- stand-alone non-linear kernels on tensors larger than L2
