@@ -171,6 +171,39 @@ int iptq_linear(const int8_t* x, const void* w, int w_bits, const int32_t* bias,
                 const int8_t* shift, int32_t out_zp, const int8_t* residual, const iptq_requant* residual_rq,
                 int8_t* y, int64_t M, int N, int K, void* ws, size_t ws_bytes, iptq_stream_t stream);
 
+/* ------------------------------------------------------------------ 4-bit-weight GEMM without any allocation
+ * (No counterpart in the paper: this is a packaging variant of iptq_linear(w_bits = 4) for callers that
+ * cannot provide a workspace.)
+ *
+ * Who needs it: code that is not allowed to allocate device memory at the point where it runs the layer --
+ * an inference loop that must never reach cudaMalloc/cudaFree (both may synchronise the whole device and
+ * their latency is unbounded), a plug-in running inside a host application that handed it a fixed set of
+ * buffers, or a process whose memory pool is owned by another component.  Such a caller has the layer's
+ * inputs and outputs but nowhere to put the N*K bytes of sign-extended weights that the tensor-core kernel
+ * reads, so the library keeps that scratch itself: one file-scope device array of
+ * 256 + IPTQ_STATIC_SCRATCH_BYTES bytes, present on every GPU that loads the library until the process ends.
+ *
+ * Same arithmetic, arguments and result as iptq_linear(..., w_bits = 4, ...), minus the workspace:
+ *   - N * K must not exceed IPTQ_STATIC_SCRATCH_BYTES (4 MiB; ViT-Base FC1/FC2 need 2.25 MiB);
+ *     larger weights return IPTQ_ERR_WORKSPACE before anything is launched.
+ *   - status: nullable dev pointer to a caller-owned 256-byte, 256-byte-aligned status block (as at the start
+ *     of a workspace; read it with iptq_check).  With NULL the array's own status block is used and cleared
+ *     on the stream at the start of the call; a bounded wait that gives up then still ends the kernel but
+ *     cannot be queried.
+ *   - The call allocates nothing (no cudaMalloc/cudaFree, no allocating library routine); it enqueues the
+ *     unpack kernel, the GEMM kernel and, with status == NULL, one 256-byte memset on `stream`.
+ *   - The first call on each device looks up the array's device address (a one-time set-up done with that
+ *     device current); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents: every byte a call
+ *     reads is rewritten by that call first, but two calls whose GPU work overlaps (different streams, or
+ *     several host threads) race on it.  Serialise them on one stream or with events.
+ */
+#define IPTQ_STATIC_SCRATCH_BYTES (4u << 20)
+int iptq_linear_w4_static(const int8_t* x, const void* w_packed, const int32_t* bias, const int32_t* mult,
+                          const int8_t* shift, int32_t out_zp, const int8_t* residual,
+                          const iptq_requant* residual_rq, int8_t* y, int64_t M, int N, int K,
+                          void* status /*nullable dev*/, iptq_stream_t stream);
+
 /* ------------------------------------------------------------------ fused attention
  * QK^T (INT8 -> int32, kept on chip) -> (+ bias) -> integer Softmax of Sec. 3.4 -> uint8 P -> P.V
  * (INT8 -> int32) -> R(out_rq) -> int8, heads re-interleaved.  No int32 intermediate reaches HBM.

@@ -104,6 +104,8 @@ def lib():
         L.iptq_linear_workspace_bytes.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
         L.iptq_linear.argtypes = [_vp, _vp, C.c_int, _vp, _vp, _vp, C.c_int32, _vp, C.POINTER(Requant), _vp,
                                   C.c_int64, C.c_int, C.c_int, _vp, C.c_size_t, _vp]
+        L.iptq_linear_w4_static.argtypes = [_vp, _vp, _vp, _vp, _vp, C.c_int32, _vp, C.POINTER(Requant), _vp,
+                                            C.c_int64, C.c_int, C.c_int, _vp, _vp]
         L.iptq_attention_workspace_bytes.restype = C.c_size_t
         L.iptq_attention_workspace_bytes.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
         L.iptq_attention_block.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, C.c_int, C.c_int, C.c_int, _vp, _vp,
@@ -128,7 +130,7 @@ def exported_symbols():
     """Names declared in include/iptq.h (used by the CPU-side load test)."""
     return ["iptq_requant_prepare", "iptq_channel_requant_prepare", "iptq_softmax_prepare", "iptq_softmax",
             "iptq_gelu_prepare", "iptq_gelu", "iptq_layernorm_prepare", "iptq_layernorm",
-            "iptq_linear_workspace_bytes", "iptq_linear", "iptq_attention_workspace_bytes", "iptq_attention_block",
+            "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_w4_static", "iptq_attention_workspace_bytes", "iptq_attention_block",
             "iptq_mlp_workspace_bytes", "iptq_mlp_block", "iptq_encoder_block_workspace_bytes",
             "iptq_encoder_block", "iptq_encoder_block_profiled", "iptq_workspace_init", "iptq_check", "iptq_strerror", "iptq_launch_count"]
 
@@ -255,6 +257,24 @@ def linear(x, w, bias, mult, shift, ws: Workspace, out_zp=0, residual=None, resi
         out = torch.empty((M, N), dtype=torch.int8, device=x.device)
     _chk(lib().iptq_linear(_dp(x), _dp(w), w_bits, _dp(bias), _dp(mult), _dp(shift), out_zp, _dp(residual),
                            _ref(residual_rq), _dp(out), M, N, K, ws.ptr, ws.nbytes, _stream()), "iptq_linear")
+    return out
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def linear_w4_static(x, w_packed, bias, mult, shift, out_zp=0, residual=None, residual_rq=None, status=None, out=None):
+    """``linear(..., w_bits=4)`` for callers that cannot hand over a workspace: the unpacked weights go to a
+    device array the library owns (N*K <= STATIC_SCRATCH_BYTES).  Nothing is allocated by the call itself, so
+    ``out`` should be passed in by such callers; it is created here only as a convenience.  Calls on one
+    device share the array: keep them on one stream."""
+    M, K = x.shape
+    N = w_packed.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.int8, device=x.device)
+    _chk(lib().iptq_linear_w4_static(_dp(x), _dp(w_packed), _dp(bias), _dp(mult), _dp(shift), out_zp, _dp(residual),
+                                     _ref(residual_rq), _dp(out), M, N, K, status, _stream()),
+         "iptq_linear_w4_static")
     return out
 
 

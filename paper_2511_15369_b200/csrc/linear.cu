@@ -380,6 +380,28 @@ int linear_launch(const LinearArgs& a, cudaStream_t st)
 
 static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 
+// ---------------------------------------------------------------- library-owned scratch (no-allocation entry point)
+// [status block | unpacked int8 weights].  Every GPU that loads the library holds this array until the
+// process exits.  In host code the name below is only a stand-in for the symbol: the device address comes from
+// cudaGetSymbolAddress(), asked once per device with that device current.
+static __device__ __align__(256) uint8_t g_static_scratch[kStatusBytes + IPTQ_STATIC_SCRATCH_BYTES];
+
+static int static_scratch_ptr(uint8_t** out)
+{
+    static std::mutex mu;
+    static uint8_t* per_device[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return IPTQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!per_device[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return IPTQ_ERR_CUDA;
+        per_device[dev] = static_cast<uint8_t*>(ptr);
+    }
+    *out = per_device[dev];
+    return IPTQ_OK;
+}
+
 }  // namespace iptq
 
 using namespace iptq;
@@ -414,6 +436,30 @@ int iptq_linear(const int8_t* x, const void* w, int w_bits, const int32_t* bias,
     }
     LinearArgs a{x, w8, bias, mult, shift, out_zp, residual, residual_rq, nullptr, y, M, N, K,
                  static_cast<StatusBlock*>(ws)};
+    return linear_launch(a, stream);
+}
+
+int iptq_linear_w4_static(const int8_t* x, const void* w_packed, const int32_t* bias, const int32_t* mult,
+                          const int8_t* shift, int32_t out_zp, const int8_t* residual,
+                          const iptq_requant* residual_rq, int8_t* y, int64_t M, int N, int K, void* status,
+                          iptq_stream_t stream)
+{
+    if (!w_packed) return IPTQ_ERR_NULL;
+    if (N < 1 || K < 1 || (K & 1)) return IPTQ_ERR_SHAPE;
+    if ((size_t)N * (size_t)K > (size_t)IPTQ_STATIC_SCRATCH_BYTES) return IPTQ_ERR_WORKSPACE;
+    if (status && (reinterpret_cast<uintptr_t>(status) & 255u)) return IPTQ_ERR_ALIGN;
+    uint8_t* base = nullptr;
+    int rc = static_scratch_ptr(&base);            // first call on this device: looks the array's address up
+    if (rc != IPTQ_OK) return rc;
+    StatusBlock* st = static_cast<StatusBlock*>(status);
+    if (!st) {
+        // the built-in status block keeps the previous call's contents: it must start at zero
+        st = reinterpret_cast<StatusBlock*>(base);
+        if (cudaMemsetAsync(st, 0, kStatusBytes, stream) != cudaSuccess) return IPTQ_ERR_CUDA;
+    }
+    int8_t* w8 = reinterpret_cast<int8_t*>(base + kStatusBytes);
+    if ((rc = unpack_int4_launch(w_packed, w8, (int64_t)N * K, stream)) != IPTQ_OK) return rc;
+    LinearArgs a{x, w8, bias, mult, shift, out_zp, residual, residual_rq, nullptr, y, M, N, K, st};
     return linear_launch(a, stream);
 }
 
