@@ -29,10 +29,55 @@ constexpr size_t kStatusBytes = 256;
 // ---------------------------------------------------------------- device arithmetic
 #ifdef __CUDACC__
 
+// The integer pipes of sm_100a issue one simple 32-bit instruction (add, shift, min/max, logic, byte pack,
+// IMAD) per clock per SM sub-partition; IMAD.HI costs about 1.5 issue slots and 64-bit results about 2.5.
+// The helpers below pin the instruction selection where the compiler's choice matters.
+
+// hi32(a * b) + c in one instruction (IMAD.HI with addend).
+__device__ __forceinline__ int mad_hi(int a, int b, int c)
+{
+    int d;
+    asm("mad.hi.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+// Logical right shift that yields 0 for shift amounts >= 32 (PTX shr clamps the amount).
+__device__ __forceinline__ unsigned shr_clamp(unsigned v, unsigned n)
+{
+    unsigned d;
+    asm("shr.u32 %0, %1, %2;" : "=r"(d) : "r"(v), "r"(n));
+    return d;
+}
+// Two int32 saturated to int8 / uint8 into the low half of a word, `hi16` supplying the upper half:
+// pack4 = pack2(c, d, 0) then pack2(a, b, that) -- two instructions for four values, clamp included.
+__device__ __forceinline__ unsigned pack4_sat_s8(int a, int b, int c, int d)
+{
+    unsigned t, r;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(d), "r"(c), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(b), "r"(a), "r"(t));
+    return r;
+}
+__device__ __forceinline__ unsigned pack4_sat_u8(int a, int b, int c, int d)
+{
+    unsigned t, r;
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(d), "r"(c), "r"(0));
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(b), "r"(a), "r"(t));
+    return r;
+}
+
+// Byte `idx` (compile-time 0..3) of a word, sign-extended to 32 bits: one PRMT whose upper three selector
+// nibbles replicate the sign of the selected byte.
+template <int IDX>
+__device__ __forceinline__ int sext_byte(unsigned w)
+{
+    int d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(w), "r"(0u), "r"(0x8880u | (unsigned)(IDX * 0x1111)));
+    return d;
+}
+
 // R without zero point / clamp: (hi32(y * mult) + rnd) >> shift, rnd = 2^(shift-1).
 __device__ __forceinline__ int requant_core(int y, int mult, int rnd, int shift)
 {
-    return (__mulhi(y, mult) + rnd) >> shift;    // >> on int is arithmetic (floor)
+    return mad_hi(y, mult, rnd) >> shift;        // >> on int is arithmetic (floor)
 }
 
 struct RequantDev {
@@ -44,6 +89,11 @@ __device__ __forceinline__ int requant_full(int y, const RequantDev& r)
     int v = requant_core(y, r.mult, r.rnd, r.shift) + r.zp;
     return max(r.qmin, min(r.qmax, v));
 }
+// Same without the clamp, for callers that saturate to 8 bits while packing (qmin/qmax = -128/127).
+__device__ __forceinline__ int requant_nosat(int y, const RequantDev& r)
+{
+    return requant_core(y, r.mult, r.rnd, r.shift) + r.zp;
+}
 
 // Constants of the integer exponential (Eqs. (7)-(10), (13)-(14)) as the kernels use them.
 struct ExpDev {
@@ -52,29 +102,32 @@ struct ExpDev {
     int qln2, qb, qc, norm_l, norm_r;    // polynomial candidate
 };
 
-// Integer exponential of a clamped distance d = min(max - s, dcap) >= 0.
+// Integer exponential of nd = -min(max - s, dcap), i.e. Q_delta of Eq. (6) clamped to [-dcap, 0].
 template <int VARIANT>
-__device__ __forceinline__ unsigned exp_core(unsigned d, const ExpDev& c)
+__device__ __forceinline__ unsigned exp_core_nd(int nd, const ExpDev& c)
 {
     if (VARIANT == IPTQ_SM_POLY) {
+        const unsigned d = (unsigned)(-nd);
         unsigned z = __umulhi(d, c.div_mul) >> c.div_shift;          // octave: floor(d / qln2)
-        int p = -(int)(d - z * (unsigned)c.qln2);                      // in (-qln2, 0]
-        int t = p + c.qb;
+        int t = (int)(z * (unsigned)c.qln2) - (int)d + c.qb;           // p + qb, p in (-qln2, 0]
         unsigned poly = (unsigned)(t * t + c.qc);
         unsigned e = (poly << c.norm_l) >> c.norm_r;
-        return z > 31u ? 0u : (e >> z);
+        return shr_clamp(e, z);
     } else {
-        int nd = -(int)d;                                              // Q_delta
-        int Qp = nd + (nd >> 1) - (nd >> 4);                           // Eq. (7)
-        unsigned P = (unsigned)(-Qp);
-        unsigned q = __umulhi(P, c.div_mul) >> c.div_shift;            // Eq. (8): floor(P / x0)
-        int u = -(int)(P - q * (unsigned)c.x0);                        // -r
+        const int a = nd >> 1, b = nd >> 4;
+        const unsigned P = (unsigned)(b - a - nd);                     // -Q_p, Eq. (7)
+        const unsigned q = __umulhi(P, c.div_mul) >> c.div_shift;      // Eq. (8): floor(P / x0)
+        const int u = (int)(q * (unsigned)c.x0) - (int)P;              // -r
         int base;
         if (VARIANT == IPTQ_SM_BITEXP) base = (u >> 1) + (u >> 3) + (u >> 4) + c.x0;   // Eqs. (13)-(14)
         else                           base = (u >> 1) + c.x0;                         // Eq. (10)
-        unsigned b = (unsigned)base << c.nsh;
-        return q > 31u ? 0u : (b >> q);                                // Eq. (9)
+        return shr_clamp((unsigned)base << c.nsh, q);                  // Eq. (9); 0 once q >= 32
     }
+}
+template <int VARIANT>
+__device__ __forceinline__ unsigned exp_core(unsigned d, const ExpDev& c)
+{
+    return exp_core_nd<VARIANT>(-(int)d, c);
 }
 
 // floor(2^M / sum) for 0 < sum < 2^31, M <= 40: the fp64 quotient cannot round across an integer
@@ -93,11 +146,14 @@ struct GeluDev {
 };
 
 // Pre-requant GELU value: x * (G >> gs)  (Eqs. (3), (5)), or x * sigmoid_q(1.702 x).
+// Polynomial variants: with t = max(Bq - |x|, 0) (zero outside the clip range of Eq. (3)) and
+// t2 = (t t) >> sh2, G = 2C - t2^2 for x >= 0 and t2^2 for x < 0 (second order: t2 instead of t2^2).
+// x = 0 gives 0 whatever G is, so the sign(0) = 0 case of Eq. (3) needs no branch.
 template <int VARIANT>
 __device__ __forceinline__ int gelu_core(int x, const GeluDev& c)
 {
-    x = max(c.lo, min(c.hi, x));
     if (VARIANT == IPTQ_GELU_SHIFT) {
+        x = max(c.lo, min(c.hi, x));
         int xp = x + (x >> 1) + (x >> 3) + (x >> 4);
         unsigned d = min((unsigned)abs(xp), (unsigned)c.ex.dcap);
         unsigned e = exp_core<IPTQ_SM_SHIFTMAX>(d, c.ex);
@@ -107,12 +163,13 @@ __device__ __forceinline__ int gelu_core(int x, const GeluDev& c)
         int sig = (int)((f * num) >> 16);            // Q15; f * num <= 2^31
         return x * sig;
     } else {
-        int m = min(abs(x), c.Bq);
-        int t = c.Bq - m;
-        int t2 = (t * t) >> c.sh2;
-        int pw = (VARIANT == IPTQ_GELU_POLY4) ? t2 * t2 : t2;
-        int E = c.C - pw;
-        int G = x > 0 ? c.C + E : (x < 0 ? c.C - E : c.C);
+        x = max(c.lo, min(c.hi, x));                 // one 3-input min/max instruction
+        const int t = max(min(c.Bq - x, c.Bq + x), 0);
+        const int t2 = (t * t) >> c.sh2;
+        const bool pos = x >= 0;
+        int G;
+        if (VARIANT == IPTQ_GELU_POLY4) G = t2 * (pos ? -t2 : t2) + (pos ? 2 * c.C : 0);
+        else                            G = pos ? 2 * c.C - t2 : t2;
         return x * (G >> c.gs);
     }
 }

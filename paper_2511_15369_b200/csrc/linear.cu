@@ -59,67 +59,80 @@ int make_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint6
 enum { EPI_REQUANT = 0, EPI_RESIDUAL = 1, EPI_GELU = 2 };
 
 constexpr int BM = 128;          // rows per tile = TMEM lanes
+constexpr int BN = 128;          // columns per tile
 constexpr int BK = 128;          // bytes of K per stage = one 128-byte swizzle row = 4 MMA k-steps
 constexpr int STAGES = 4;
-constexpr int EPI_WARPS = 8;
+constexpr int EPI_PARTS = 2;     // epilogue warps per TMEM lane quadrant; each owns BN / EPI_PARTS columns
+constexpr int EPI_WARPS = 4 * EPI_PARTS;
+constexpr int COLS = BN / EPI_PARTS;                 // 64: bytes per output row per warp, one 64-byte swizzle row
 constexpr int GEMM_THREADS = 32 * (2 + EPI_WARPS);
+static_assert(COLS == 64, "staging addresses below assume 64-byte rows (64-byte TMA swizzle)");
 
 struct GemmParams {
     int M, N, K;
     int num_m_tiles, num_n_tiles;
     const int32_t* bias; const int32_t* mult; const int8_t* shift;
     int out_zp;
-    const int8_t* residual;
-    int res_mult, res_rnd, res_shift, res_zp;
-    int8_t* y;
+    int res_mult, res_rnd, res_shift, res_off;        // residual branch: ((res << 16) - res_off) through R
     GeluDev gelu;
     StatusBlock* status;
 };
 
-template <int BN>
 struct GemmSmem {
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_BYTES = BN * BK;
-    static constexpr int COLS_PER_WARP = BN / 2;
+    static constexpr int WARP_TILE = 32 * COLS;                                   // bytes of one warp's output block
     static constexpr int OFF_A = 0;
     static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
-    static constexpr int OFF_CP = OFF_B + STAGES * B_BYTES;                      // [EPI_WARPS][COLS_PER_WARP] int4
-    static constexpr int OFF_BAR = OFF_CP + EPI_WARPS * COLS_PER_WARP * 16;
-    static constexpr int OFF_END = OFF_BAR + (2 * STAGES + 4) * 8 + 16;
+    static constexpr int OFF_OUT = OFF_B + STAGES * B_BYTES;                     // [EPI_WARPS][32 rows][COLS] int8
+    static constexpr int OFF_RES = OFF_OUT + EPI_WARPS * WARP_TILE;              // same shape, residual tiles
+    static constexpr int OFF_CP = OFF_RES + EPI_WARPS * WARP_TILE;               // [EPI_WARPS][COLS] int4
+    static constexpr int OFF_BAR = OFF_CP + EPI_WARPS * COLS * 16;
+    static constexpr int NUM_BARS = 2 * STAGES + 4 + EPI_WARPS;
+    static constexpr int OFF_END = OFF_BAR + NUM_BARS * 8 + 16;
     static constexpr int TOTAL = OFF_END + 1024;                                 // slack for 1024-byte alignment
 };
 
-template <int BN, int EPI, int GELU_VARIANT>
+// Byte offset of 16-byte chunk `chunk` of row `row` inside a [32][64]-byte block written/read by TMA with the
+// 64-byte swizzle (chunk index XOR bits 7-8 of the address); also makes the per-row 16-byte accesses of a
+// warp conflict-free.
+__device__ __forceinline__ uint32_t swz64(int row, int chunk) { return (uint32_t)(row * 64 + ((chunk ^ ((row >> 1) & 3)) << 4)); }
+
+template <int EPI, int GELU_VARIANT, bool SAT8>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_res,
                const GemmParams p)
 {
-    using L = GemmSmem<BN>;
+    using L = GemmSmem;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sA = smem + L::OFF_A;
     uint8_t* sB = smem + L::OFF_B;
-    int4* sCP = reinterpret_cast<int4*>(smem + L::OFF_CP);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
     uint64_t* empty_bar = full_bar + STAGES;
     uint64_t* acc_full = empty_bar + STAGES;      // [2]
     uint64_t* acc_empty = acc_full + 2;           // [2]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    uint64_t* res_bar = acc_empty + 2;            // [EPI_WARPS]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(res_bar + EPI_WARPS);
     CtaControl* ctl = reinterpret_cast<CtaControl*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int num_tiles = p.num_m_tiles * p.num_n_tiles;
     const int kblocks = (p.K + BK - 1) / BK;
-    constexpr uint32_t TMEM_COLS = 2 * BN;        // two accumulator buffers (power of two for BN in {64, 128})
+    constexpr uint32_t TMEM_COLS = 2 * BN;        // two accumulator buffers
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EPI_WARPS); }
+        for (int w = 0; w < EPI_WARPS; ++w) mbar_init(&res_bar[w], 1);
         ctl->abort = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_a);
         prefetch_tensormap(&map_b);
+        prefetch_tensormap(&map_y);
+        if (EPI == EPI_RESIDUAL) prefetch_tensormap(&map_res);
     }
     if (warp == 1) {
         tmem_alloc(tmem_slot, TMEM_COLS);
@@ -135,8 +148,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (elect_one()) {
             int s = 0; uint32_t ph = 0;
             for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
-                const int m0 = (t / p.num_n_tiles) * BM;
-                const int n0 = (t % p.num_n_tiles) * BN;
+                const int m0 = (t % p.num_m_tiles) * BM;
+                const int n0 = (t / p.num_m_tiles) * BN;
                 bool ok = true;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(&empty_bar[s], ph ^ 1u, ctl, p.status, 1)) { ok = false; break; }
@@ -182,20 +195,34 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else {
         // ------------------------------------------------------------ epilogue warps
-        const int ew = warp - 2;                              // 0..7
-        const int quad = warp & 3;                            // TMEM lane quadrant this warp may access
-        const int half = ew >> 2;                             // which half of the tile's columns
-        int4* cp = sCP + ew * L::COLS_PER_WARP;
+        // Warp (quad, part) owns TMEM lanes 32*quad.. (the only ones it may touch) and columns part*COLS.. of
+        // every tile: it turns them into a [32 rows][COLS] int8 block in shared memory and stores that block
+        // with one TMA copy; nothing in the epilogue synchronises across warps.
+        const int ew = warp - 2;
+        const int quad = warp & 3;
+        const int part = ew >> 2;
+        int4* cp = reinterpret_cast<int4*>(smem + L::OFF_CP) + ew * COLS;
+        const uint32_t out_blk = smem_u32(smem + L::OFF_OUT + ew * L::WARP_TILE);
+        uint8_t* res_ptr = smem + L::OFF_RES + ew * L::WARP_TILE;
+        const uint32_t res_blk = smem_u32(res_ptr);
+        uint32_t res_ph = 0;
         int it = 0;
         for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
             const int ab = it & 1;
             const uint32_t abph = (uint32_t)(it >> 1) & 1u;
-            const int m0 = (t / p.num_n_tiles) * BM;
-            const int n0 = (t % p.num_n_tiles) * BN + half * L::COLS_PER_WARP;
-            // per-column constants of this warp's columns: (bias, mult, 2^(shift-1), shift)
+            const int row0 = (t % p.num_m_tiles) * BM + quad * 32;
+            const int col0 = (t / p.num_m_tiles) * BN + part * COLS;
+            const bool active = row0 < p.M && col0 < p.N;     // warp-uniform
+            // the previous tile's store must have read the staging block before it is rewritten
+            if (lane == 0) bulk_wait_read_all();
             __syncwarp();
-            for (int c = lane; c < L::COLS_PER_WARP; c += 32) {
-                const int n = n0 + c;
+            if (EPI == EPI_RESIDUAL && active && lane == 0) {
+                mbar_expect_tx(&res_bar[ew], L::WARP_TILE);
+                tma_load_2d(res_ptr, &map_res, &res_bar[ew], col0, row0);
+            }
+            // per-column constants of this warp's columns: (bias, mult, 2^(shift-1), shift)
+            for (int c = lane; c < COLS; c += 32) {
+                const int n = col0 + c;
                 int4 v = make_int4(0, 1 << 30, 1, 1);
                 if (n < p.N) {
                     const int sh = (int)__ldg(p.shift + n);
@@ -206,48 +233,59 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             __syncwarp();
             if (!mbar_wait(&acc_full[ab], abph, ctl, p.status, 4)) break;
             tc_fence_after_sync();
-            const int row = m0 + quad * 32 + lane;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * BN + half * L::COLS_PER_WARP);
-#pragma unroll 1
-            for (int c0 = 0; c0 < L::COLS_PER_WARP; c0 += 16) {
-                uint32_t r[16];
-                tmem_ld16(taddr + c0, r);
-                tmem_wait_ld();
-                if (n0 + c0 >= p.N) continue;                 // N is a multiple of 16: whole chunk in or out
-                int o[16];
-                int4 resv = make_int4(0, 0, 0, 0);
-                if (EPI == EPI_RESIDUAL && row < p.M)
-                    resv = __ldg(reinterpret_cast<const int4*>(p.residual + (size_t)row * p.N + n0 + c0));
-                const int resw[4] = {resv.x, resv.y, resv.z, resv.w};
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int4 k4 = cp[c0 + j];
-                    int v = requant_core((int)r[j] + k4.x, k4.y, k4.z, k4.w);
-                    if (EPI == EPI_GELU) {
-                        v = gelu_core<GELU_VARIANT>(v, p.gelu);               // clamps to in_bits first
-                        v = requant_full(v, p.gelu.out);
-                    } else {
-                        if (EPI == EPI_RESIDUAL) {
-                            const int rb = (int)(int8_t)(resw[j >> 2] >> (8 * (j & 3)));
-                            v += requant_core((rb - p.res_zp) << 16, p.res_mult, p.res_rnd, p.res_shift);
-                        }
-                        v += p.out_zp;
-                    }
-                    o[j] = v;
+            if (active) {
+                if (EPI == EPI_RESIDUAL) {
+                    if (!mbar_wait(&res_bar[ew], res_ph, ctl, p.status, 5)) break;
+                    res_ph ^= 1u;
                 }
-                if (row < p.M) {
-                    int4 pk;
-                    pk.x = (int)pack4_sat_s8(o[0], o[1], o[2], o[3]);
-                    pk.y = (int)pack4_sat_s8(o[4], o[5], o[6], o[7]);
-                    pk.z = (int)pack4_sat_s8(o[8], o[9], o[10], o[11]);
-                    pk.w = (int)pack4_sat_s8(o[12], o[13], o[14], o[15]);
-                    *reinterpret_cast<int4*>(p.y + (size_t)row * p.N + n0 + c0) = pk;
+                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * BN + part * COLS);
+                uint32_t r[2][16];
+                tmem_ld16(taddr, r[0]);
+#pragma unroll
+                for (int ch = 0; ch < COLS / 16; ++ch) {
+                    tmem_wait_ld();
+                    if (ch + 1 < COLS / 16) tmem_ld16(taddr + (ch + 1) * 16, r[(ch + 1) & 1]);   // overlaps the math below
+                    const uint32_t* acc = r[ch & 1];
+                    uint4 resv = make_uint4(0, 0, 0, 0);
+                    if (EPI == EPI_RESIDUAL) resv = ld_shared_v4(res_blk + swz64(lane, ch));
+                    const uint32_t resw[4] = {resv.x, resv.y, resv.z, resv.w};
+                    int o[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int4 k4 = cp[ch * 16 + j];
+                        int v = requant_core((int)acc[j] + k4.x, k4.y, k4.z, k4.w);
+                        if (EPI == EPI_GELU) {
+                            v = gelu_core<GELU_VARIANT>(v, p.gelu);
+                            v = requant_nosat(v, p.gelu.out);
+                            if (!SAT8) v = max(p.gelu.out.qmin, min(p.gelu.out.qmax, v));
+                        } else if (EPI == EPI_RESIDUAL) {
+                            // byte j of the residual word, sign-extended, widened by 2^16 and requantised
+                            const int rb = (j & 3) == 0 ? sext_byte<0>(resw[j >> 2]) : (j & 3) == 1 ? sext_byte<1>(resw[j >> 2])
+                                         : (j & 3) == 2 ? sext_byte<2>(resw[j >> 2]) : sext_byte<3>(resw[j >> 2]);
+                            v += requant_core(rb * 65536 - p.res_off, p.res_mult, p.res_rnd, p.res_shift) + p.out_zp;
+                        } else {
+                            v += p.out_zp;
+                        }
+                        o[j] = v;
+                    }
+                    st_shared_v4(out_blk + swz64(lane, ch), pack4_sat_s8(o[0], o[1], o[2], o[3]),
+                                 pack4_sat_s8(o[4], o[5], o[6], o[7]), pack4_sat_s8(o[8], o[9], o[10], o[11]),
+                                 pack4_sat_s8(o[12], o[13], o[14], o[15]));
                 }
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[ab]);
+            if (lane == 0) mbar_arrive(&acc_empty[ab]);       // the MMA warp may refill this accumulator
+            if (active) {
+                fence_proxy_async_smem();                     // this lane's st.shared -> visible to the TMA engine
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(&map_y, smem + L::OFF_OUT + ew * L::WARP_TILE, col0, row0);   // clipped at M and N
+                    bulk_commit();
+                }
+            }
         }
+        if (lane == 0) bulk_wait_all();                       // stores complete before shared memory goes away
     }
 
     // ------------------------------------------------------------ teardown (also reached after an abort)
@@ -300,20 +338,23 @@ struct LinearArgs {
     StatusBlock* status;
 };
 
-template <int BN, int EPI, int GV>
-static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, cudaStream_t st)
+template <int EPI, int GV, bool SAT8>
+static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& my, const CUtensorMap& mr,
+                       const GemmParams& p, cudaStream_t st)
 {
-    using L = GemmSmem<BN>;
-    auto kern = gemm_i8_kernel<BN, EPI, GV>;
-    static bool configured = false;           // one attribute call per instantiation is enough per process/device
-    if (!configured) {
+    using L = GemmSmem;
+    auto kern = gemm_i8_kernel<EPI, GV, SAT8>;
+    static bool configured[64];               // one attribute call per instantiation and device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return IPTQ_ERR_CUDA;
+    if (!configured[dev]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) != cudaSuccess)
             return IPTQ_ERR_CUDA;
-        configured = true;
+        configured[dev] = true;
     }
     const int tiles = p.num_m_tiles * p.num_n_tiles;
     const int grid = std::min(tiles, sm_count());
-    kern<<<grid, GEMM_THREADS, L::TOTAL, st>>>(ma, mb, p);
+    kern<<<grid, GEMM_THREADS, L::TOTAL, st>>>(ma, mb, my, mr, p);
     note_launch();
     return last_launch_status();
 }
@@ -335,47 +376,55 @@ int linear_launch(const LinearArgs& a, cudaStream_t st)
     if (!a.status) return IPTQ_ERR_WORKSPACE;
     if (a.M == 0) return IPTQ_OK;
 
-    constexpr int BN = 128;
     GemmParams p;
     p.M = (int)a.M; p.N = a.N; p.K = a.K;
     p.num_m_tiles = (int)((a.M + BM - 1) / BM);
     p.num_n_tiles = (a.N + BN - 1) / BN;
     p.bias = a.bias; p.mult = a.mult; p.shift = a.shift; p.out_zp = a.out_zp;
-    p.residual = a.residual;
-    p.res_mult = p.res_rnd = p.res_shift = p.res_zp = 0;
+    p.res_mult = p.res_rnd = p.res_shift = p.res_off = 0;
     if (a.residual) {
         p.res_mult = a.residual_rq->mult; p.res_shift = a.residual_rq->shift;
-        p.res_rnd = 1 << (a.residual_rq->shift - 1); p.res_zp = a.residual_rq->zp;
+        p.res_rnd = 1 << (a.residual_rq->shift - 1); p.res_off = a.residual_rq->zp * 65536;
     }
-    p.y = a.y;
     p.status = a.status;
     if (a.gelu) p.gelu = to_dev(*a.gelu);
     else { iptq_gelu_consts z{}; z.in_bits = 8; z.out.shift = 1; p.gelu = to_dev(z); }
 
-    CUtensorMap ma, mb;
+    CUtensorMap ma, mb, my, mr;
+    int rc;
     {
         const uint64_t dims[2] = {(uint64_t)a.K, (uint64_t)a.M};
         const uint64_t str[1] = {(uint64_t)a.K};
         const uint32_t box[2] = {BK, BM};
-        int rc = make_tensor_map_u8(&ma, a.x, 2, dims, str, box, 128);
-        if (rc != IPTQ_OK) return rc;
+        if ((rc = make_tensor_map_u8(&ma, a.x, 2, dims, str, box, 128)) != IPTQ_OK) return rc;
     }
     {
         const uint64_t dims[2] = {(uint64_t)a.K, (uint64_t)a.N};
         const uint64_t str[1] = {(uint64_t)a.K};
         const uint32_t box[2] = {BK, BN};
-        int rc = make_tensor_map_u8(&mb, a.w, 2, dims, str, box, 128);
-        if (rc != IPTQ_OK) return rc;
+        if ((rc = make_tensor_map_u8(&mb, a.w, 2, dims, str, box, 128)) != IPTQ_OK) return rc;
+    }
+    {
+        // output and residual: one [32 rows][COLS] block per epilogue warp, clipped at M and N by the copy engine
+        const uint64_t dims[2] = {(uint64_t)a.N, (uint64_t)a.M};
+        const uint64_t str[1] = {(uint64_t)a.N};
+        const uint32_t box[2] = {COLS, 32};
+        if ((rc = make_tensor_map_u8(&my, a.y, 2, dims, str, box, 64)) != IPTQ_OK) return rc;
+        if ((rc = make_tensor_map_u8(&mr, a.residual ? a.residual : a.y, 2, dims, str, box, 64)) != IPTQ_OK) return rc;
     }
     if (a.gelu) {
+        const bool sat8 = a.gelu->out.qmin == -128 && a.gelu->out.qmax == 127;
+#define IPTQ_GEMM_GELU(V) (sat8 ? launch_gemm<EPI_GELU, V, true>(ma, mb, my, mr, p, st) \
+                                : launch_gemm<EPI_GELU, V, false>(ma, mb, my, mr, p, st))
         switch (a.gelu->variant) {
-            case IPTQ_GELU_POLY4: return launch_gemm<BN, EPI_GELU, IPTQ_GELU_POLY4>(ma, mb, p, st);
-            case IPTQ_GELU_POLY2: return launch_gemm<BN, EPI_GELU, IPTQ_GELU_POLY2>(ma, mb, p, st);
-            default: return launch_gemm<BN, EPI_GELU, IPTQ_GELU_SHIFT>(ma, mb, p, st);
+            case IPTQ_GELU_POLY4: return IPTQ_GEMM_GELU(IPTQ_GELU_POLY4);
+            case IPTQ_GELU_POLY2: return IPTQ_GEMM_GELU(IPTQ_GELU_POLY2);
+            default: return IPTQ_GEMM_GELU(IPTQ_GELU_SHIFT);
         }
+#undef IPTQ_GEMM_GELU
     }
-    if (a.residual) return launch_gemm<BN, EPI_RESIDUAL, 0>(ma, mb, p, st);
-    return launch_gemm<BN, EPI_REQUANT, 0>(ma, mb, p, st);
+    if (a.residual) return launch_gemm<EPI_RESIDUAL, 0, true>(ma, mb, my, mr, p, st);
+    return launch_gemm<EPI_REQUANT, 0, true>(ma, mb, my, mr, p, st);
 }
 
 static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }

@@ -1,5 +1,6 @@
 // Stand-alone integer Softmax / GELU / LayerNorm kernels (row- and element-wise, HBM/ALU bound).
 #include <climits>
+#include <type_traits>
 
 #include "iptq_common.cuh"
 
@@ -16,7 +17,10 @@ struct SoftmaxDev {
     int M, f_shl, p_shr;
 };
 
-template <int VARIANT, int NITER, bool HAS_BIAS>
+// Lanes past the row end carry a score so low that the clamp at -dcap applies and the exponential is 0.
+constexpr int kPadScore = -(1 << 30);
+
+template <int VARIANT, int NITER, bool HAS_BIAS, bool PSHR>
 __global__ void __launch_bounds__(256)
 softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ probs, int64_t rows, int n,
                     const int32_t* __restrict__ bias, int64_t bias_period, const SoftmaxDev c)
@@ -24,6 +28,7 @@ softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ pr
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int ndmin = -c.ex.dcap;
     for (int64_t row = warp; row < rows; row += nwarps) {
         const int32_t* sr = scores + row * n;
         const int32_t* br = HAS_BIAS ? bias + (row % bias_period) * n : nullptr;
@@ -32,25 +37,21 @@ softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ pr
 #pragma unroll
         for (int k = 0; k < NITER; ++k) {
             const int j = lane + 32 * k;
+            int s = kPadScore;
             if (j < n) {
-                int s = __ldg(sr + j);
+                s = __ldcs(sr + j);
                 if (HAS_BIAS) s += __ldg(br + j);
-                v[k] = s;
-                mx = max(mx, s);
-            } else {
-                v[k] = 0;
             }
+            v[k] = s;
+            mx = max(mx, s);
         }
         mx = __reduce_max_sync(kFull, mx);                      // Eq. (6)
-        unsigned e[NITER];
         unsigned sum = 0;
 #pragma unroll
         for (int k = 0; k < NITER; ++k) {
-            const int j = lane + 32 * k;
-            unsigned d = min((unsigned)(mx - v[k]), (unsigned)c.ex.dcap);
-            unsigned ev = exp_core<VARIANT>(d, c.ex);
-            e[k] = j < n ? ev : 0u;
-            sum += e[k];
+            const unsigned e = exp_core_nd<VARIANT>(max(v[k] - mx, ndmin), c.ex);
+            v[k] = (int)e;
+            sum += e;
         }
         sum = __reduce_add_sync(kFull, sum);
         const unsigned f = intdiv_factor(sum, c.M) << c.f_shl;  // Eq. (15)
@@ -58,7 +59,9 @@ softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ pr
 #pragma unroll
         for (int k = 0; k < NITER; ++k) {
             const int j = lane + 32 * k;
-            if (j < n) pr[j] = (uint8_t)(__umulhi(f, e[k]) >> c.p_shr);
+            unsigned pv = __umulhi(f, (unsigned)v[k]);
+            if (PSHR) pv >>= c.p_shr;
+            if (j < n) __stcs(pr + j, (uint8_t)pv);
         }
     }
 }
@@ -70,8 +73,13 @@ static int launch_softmax2(const int32_t* s, uint8_t* p, int64_t rows, int n, co
     const int threads = 256;
     const int64_t want = (rows + 7) / 8;
     const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 8);
-    if (bias) softmax_rows_kernel<VARIANT, NITER, true><<<grid, threads, 0, st>>>(s, p, rows, n, bias, period, c);
-    else      softmax_rows_kernel<VARIANT, NITER, false><<<grid, threads, 0, st>>>(s, p, rows, n, bias, period, c);
+    if (bias) {
+        if (c.p_shr) softmax_rows_kernel<VARIANT, NITER, true, true><<<grid, threads, 0, st>>>(s, p, rows, n, bias, period, c);
+        else         softmax_rows_kernel<VARIANT, NITER, true, false><<<grid, threads, 0, st>>>(s, p, rows, n, bias, period, c);
+    } else {
+        if (c.p_shr) softmax_rows_kernel<VARIANT, NITER, false, true><<<grid, threads, 0, st>>>(s, p, rows, n, bias, period, c);
+        else         softmax_rows_kernel<VARIANT, NITER, false, false><<<grid, threads, 0, st>>>(s, p, rows, n, bias, period, c);
+    }
     note_launch();
     return last_launch_status();
 }
@@ -100,13 +108,17 @@ static int launch_softmax1(const int32_t* s, uint8_t* p, int64_t rows, int n, co
 // GELU: element-wise; each warp iteration covers 512 elements with four coalesced 16-byte loads per
 // lane and four coalesced 4-byte stores.
 // ------------------------------------------------------------------------------------------------
-template <int VARIANT>
-__device__ __forceinline__ int gelu_elem(int x, const GeluDev& c)
+template <int VARIANT, bool SAT8>
+__device__ __forceinline__ unsigned gelu4(int4 a, const GeluDev& c)
 {
-    return requant_full(gelu_core<VARIANT>(x, c), c.out);
+    if (SAT8)
+        return pack4_sat_s8(requant_nosat(gelu_core<VARIANT>(a.x, c), c.out), requant_nosat(gelu_core<VARIANT>(a.y, c), c.out),
+                            requant_nosat(gelu_core<VARIANT>(a.z, c), c.out), requant_nosat(gelu_core<VARIANT>(a.w, c), c.out));
+    return pack4_s8(requant_full(gelu_core<VARIANT>(a.x, c), c.out), requant_full(gelu_core<VARIANT>(a.y, c), c.out),
+                    requant_full(gelu_core<VARIANT>(a.z, c), c.out), requant_full(gelu_core<VARIANT>(a.w, c), c.out));
 }
 
-template <int VARIANT>
+template <int VARIANT, bool SAT8>
 __global__ void __launch_bounds__(256)
 gelu_kernel(const int32_t* __restrict__ x, int8_t* __restrict__ y, int64_t n, const GeluDev c)
 {
@@ -121,20 +133,12 @@ gelu_kernel(const int32_t* __restrict__ x, int8_t* __restrict__ y, int64_t n, co
 #pragma unroll
         for (int u = 0; u < 4; ++u) a[u] = __ldcs(xv + i + u * stride);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            unsigned o = pack4_s8(gelu_elem<VARIANT>(a[u].x, c), gelu_elem<VARIANT>(a[u].y, c),
-                                  gelu_elem<VARIANT>(a[u].z, c), gelu_elem<VARIANT>(a[u].w, c));
-            __stcs(yv + i + u * stride, o);
-        }
+        for (int u = 0; u < 4; ++u) __stcs(yv + i + u * stride, gelu4<VARIANT, SAT8>(a[u], c));
     }
-    for (; i < nvec; i += stride) {
-        int4 a = __ldcs(xv + i);
-        yv[i] = pack4_s8(gelu_elem<VARIANT>(a.x, c), gelu_elem<VARIANT>(a.y, c), gelu_elem<VARIANT>(a.z, c),
-                         gelu_elem<VARIANT>(a.w, c));
-    }
+    for (; i < nvec; i += stride) yv[i] = gelu4<VARIANT, SAT8>(__ldcs(xv + i), c);
     // ragged tail (n % 4 elements)
     const int64_t t = (nvec << 2) + (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t < n) y[t] = (int8_t)gelu_elem<VARIANT>(x[t], c);
+    if (t < n) y[t] = (int8_t)requant_full(gelu_core<VARIANT>(x[t], c), c.out);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -154,21 +158,30 @@ __device__ __forceinline__ unsigned long long isqrt_floor(unsigned long long V)
     return r;
 }
 
+// floor(a / b) for integers 0 <= a < 2^53, 1 <= b with a / b * b <= 2^53: the correctly rounded fp64 quotient of
+// a non-integer a / b lies at least 1 / b below the next integer, i.e. 2^-53 relatively away whenever the
+// quotient times b stays below 2^53, so truncation gives the exact floor.
+__device__ __forceinline__ double floor_div_f64(double a, double b) { return floor(a / b); }
+
 __device__ __forceinline__ unsigned long long isqrt_variant(unsigned long long V, int variant)
 {
     if (V == 0) return 0;
-    if (variant == IPTQ_LN_SHIFT) {
-        // fixed 10 steps of r <- (r + V / r) >> 1 from 2^ceil(bitlen(V) / 2); no convergence test
-        const int w = 64 - __clzll((long long)V);
-        unsigned long long r = 1ull << ((w + 1) >> 1);
+    const unsigned long long s = isqrt_floor(V);
+    if (variant != IPTQ_LN_SHIFT) return s;
+    // Fixed 10 steps of r <- (r + V / r) >> 1 from 2^ceil(bitlen(V) / 2), no convergence test.  From a start
+    // within a factor 2 of sqrt(V) the recurrence reaches floor(sqrt V) in at most 7 steps and then stays there,
+    // except when V + 1 is a perfect square, where it alternates between s and s + 1: only then is the
+    // recurrence actually run (in fp64, every intermediate is an exact integer below 2^53).
+    if ((s + 1) * (s + 1) != V + 1) return s;
+    const int w = 64 - __clzll((long long)V);
+    double r = (double)(1ull << ((w + 1) >> 1));
+    const double Vd = (double)V;
 #pragma unroll 1
-        for (int it = 0; it < 10; ++it) r = (r + V / r) >> 1;
-        return r;
-    }
-    return isqrt_floor(V);
+    for (int it = 0; it < 10; ++it) r = floor((r + floor_div_f64(Vd, r)) * 0.5);
+    return (unsigned long long)r;
 }
 
-template <int NW, bool PTF>
+template <int NW, bool PTF, bool SAT8>
 __global__ void __launch_bounds__(256)
 layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int64_t rows,
                       const int32_t* __restrict__ gamma_q, const int32_t* __restrict__ beta_q,
@@ -220,32 +233,41 @@ layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int6
         s2 = __reduce_add_sync(kFull, s2);
         const long long V = (long long)D * (long long)s2 - (long long)s1 * (long long)s1;   // D^2 var, exact
         const unsigned long long r = isqrt_variant((unsigned long long)V, c.variant);        // D * std
-        const long long F = r ? (long long)((1ull << 40) / r) : 0;
+        const long long F = r ? (long long)floor_div_f64(1099511627776.0, (double)r) : 0;   // floor(2^40 / r)
+        // (u F) >> 30 = hi32(u * 4F) when 4F fits in 32 bits (rows whose D * std exceeds 2^11: all but near-constant rows)
+        const bool narrow = F < (1ll << 29);
+        const int F4 = (int)(F << 2);
         int* yr = reinterpret_cast<int*>(y + row * D);
+        auto emit = [&](auto narrow_c) {
+            constexpr bool NARROW = decltype(narrow_c)::value;
 #pragma unroll
-        for (int k = 0; k < NW; ++k) {
-            const int wi = lane + 32 * k;
-            if (wi < words) {
-                int4 gg, bb;
-                if (KEEP) { gg = g[k]; bb = b[k]; }
-                else {
-                    gg = __ldg(reinterpret_cast<const int4*>(gamma_q) + wi);
-                    bb = __ldg(reinterpret_cast<const int4*>(beta_q) + wi);
-                }
-                const int gv[4] = {gg.x, gg.y, gg.z, gg.w};
-                const int bv[4] = {bb.x, bb.y, bb.z, bb.w};
-                int o[4];
+            for (int k = 0; k < NW; ++k) {
+                const int wi = lane + 32 * k;
+                if (wi < words) {
+                    int4 gg, bb;
+                    if (KEEP) { gg = g[k]; bb = b[k]; }
+                    else {
+                        gg = __ldg(reinterpret_cast<const int4*>(gamma_q) + wi);
+                        bb = __ldg(reinterpret_cast<const int4*>(beta_q) + wi);
+                    }
+                    const int gv[4] = {gg.x, gg.y, gg.z, gg.w};
+                    const int bv[4] = {bb.x, bb.y, bb.z, bb.w};
+                    int o[4];
 #pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    int xv = (int)(int8_t)(w[k] >> (8 * t));
-                    if (PTF) xv <<= ((sh[k] >> (8 * t)) & 3);
-                    const int u = D * xv - s1;                                   // D (x - mean)
-                    const int nq = (int)(((long long)u * F) >> 30);              // (x - mean) / std, Q10
-                    o[t] = requant_full(nq * gv[t] + bv[t], c.out);
+                    for (int t = 0; t < 4; ++t) {
+                        int xv = (int)(int8_t)(w[k] >> (8 * t));
+                        if (PTF) xv <<= ((sh[k] >> (8 * t)) & 3);
+                        const int u = D * xv - s1;                               // D (x - mean)
+                        const int nq = NARROW ? __mulhi(u, F4) : (int)(((long long)u * F) >> 30);   // (x - mean) / std, Q10
+                        o[t] = requant_nosat(nq * gv[t] + bv[t], c.out);
+                        if (!SAT8) o[t] = max(c.out.qmin, min(c.out.qmax, o[t]));
+                    }
+                    __stcs(yr + wi, SAT8 ? (int)pack4_sat_s8(o[0], o[1], o[2], o[3]) : (int)pack4_s8(o[0], o[1], o[2], o[3]));
                 }
-                __stcs(yr + wi, (int)pack4_s8(o[0], o[1], o[2], o[3]));
             }
-        }
+        };
+        if (narrow) emit(std::true_type{});
+        else        emit(std::false_type{});
     }
 }
 
@@ -256,8 +278,14 @@ static int launch_ln(const int8_t* x, int8_t* y, int64_t rows, const int32_t* gq
     const int threads = 256;
     const int64_t want = (rows + 7) / 8;
     const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 8);
-    if (c.variant == IPTQ_LN_PTF) layernorm_rows_kernel<NW, true><<<grid, threads, 0, st>>>(x, y, rows, gq, bq, ptf, c);
-    else                          layernorm_rows_kernel<NW, false><<<grid, threads, 0, st>>>(x, y, rows, gq, bq, ptf, c);
+    const bool sat8 = c.out.qmin == -128 && c.out.qmax == 127;
+    if (c.variant == IPTQ_LN_PTF) {
+        if (sat8) layernorm_rows_kernel<NW, true, true><<<grid, threads, 0, st>>>(x, y, rows, gq, bq, ptf, c);
+        else      layernorm_rows_kernel<NW, true, false><<<grid, threads, 0, st>>>(x, y, rows, gq, bq, ptf, c);
+    } else {
+        if (sat8) layernorm_rows_kernel<NW, false, true><<<grid, threads, 0, st>>>(x, y, rows, gq, bq, ptf, c);
+        else      layernorm_rows_kernel<NW, false, false><<<grid, threads, 0, st>>>(x, y, rows, gq, bq, ptf, c);
+    }
     note_launch();
     return last_launch_status();
 }
@@ -339,12 +367,19 @@ int iptq_gelu(const int32_t* x, int8_t* y, int64_t n, const iptq_gelu_consts* co
     const int threads = 256;
     const int64_t groups = (n + 3) / 4;
     const int grid = (int)std::min<int64_t>((groups + threads - 1) / threads, (int64_t)sm_count() * 16);
+    const bool sat8 = consts->out.qmin == -128 && consts->out.qmax == 127;
+#define IPTQ_GELU_LAUNCH(V)                                                               \
+    do {                                                                                  \
+        if (sat8) gelu_kernel<V, true><<<grid, threads, 0, stream>>>(x, y, n, c);         \
+        else      gelu_kernel<V, false><<<grid, threads, 0, stream>>>(x, y, n, c);        \
+    } while (0)
     switch (consts->variant) {
-        case IPTQ_GELU_POLY4: gelu_kernel<IPTQ_GELU_POLY4><<<grid, threads, 0, stream>>>(x, y, n, c); break;
-        case IPTQ_GELU_POLY2: gelu_kernel<IPTQ_GELU_POLY2><<<grid, threads, 0, stream>>>(x, y, n, c); break;
-        case IPTQ_GELU_SHIFT: gelu_kernel<IPTQ_GELU_SHIFT><<<grid, threads, 0, stream>>>(x, y, n, c); break;
+        case IPTQ_GELU_POLY4: IPTQ_GELU_LAUNCH(IPTQ_GELU_POLY4); break;
+        case IPTQ_GELU_POLY2: IPTQ_GELU_LAUNCH(IPTQ_GELU_POLY2); break;
+        case IPTQ_GELU_SHIFT: IPTQ_GELU_LAUNCH(IPTQ_GELU_SHIFT); break;
         default: return IPTQ_ERR_VARIANT;
     }
+#undef IPTQ_GELU_LAUNCH
     note_launch();
     return last_launch_status();
 }
