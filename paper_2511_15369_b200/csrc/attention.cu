@@ -1,31 +1,35 @@
 // Fused integer attention: S = Q K^T (tcgen05 INT8 -> int32 in TMEM) -> (+bias, mask) -> integer Softmax of
-// Sec. 3.4 (Eqs. (6)-(15)) computed straight out of TMEM, one thread per query row -> uint8 P written to
-// shared memory in the tensor-core operand layout -> O = P V (u8 x s8 -> int32 in TMEM) -> dyadic requant ->
-// int8, heads re-interleaved.  Neither S nor P ever reaches HBM.
+// Sec. 3.4 (Eqs. (6)-(15)) computed straight out of TMEM -> uint8 P written to shared memory in the tensor-core
+// operand layout -> O = P V (u8 x s8 -> int32 in TMEM) -> dyadic requant -> int8, heads re-interleaved.
+// Neither S nor P ever reaches HBM.
 //
 // The integer Softmax cannot be computed "online" (flash style): the floor in Eq. (9) depends on the final row
 // maximum and P depends on floor(2^M / sum) before it multiplies V, so the whole score row stays in TMEM
 // (<= 256 columns) and is swept three times (max; exponentials + sum, written back to TMEM; probabilities).
 //
-// Work item = (batch, head, 128-row query tile).  6 warps per CTA: warp 0 = TMA producer (2-stage ring of
-// Q/K/V tiles), warp 1 = MMA issuer, warps 2..5 = softmax + output epilogue (warp w owns TMEM lanes 32*(w%4)..).
-// Two CTAs fit on an SM so that one CTA's tensor-core / copy latency hides behind the other's integer ALU work.
+// Work item = (batch, head, 128-row query tile), handed out dynamically (full tiles first) through a counter in
+// the workspace status block.  10 warps per CTA: warp 0 = TMA producer (2-stage ring of Q/K/V tiles), warp 1 = MMA
+// issuer, warps 2..9 = softmax + output.  A query row is shared by two threads (one per half of the columns; a warp
+// may only touch TMEM lanes 32*(warp%4)..), which exchange their partial max / sum through shared memory.
+// Two CTAs fit on an SM so that one CTA's tensor-core / copy latency hides behind the other's integer work.
 #include <algorithm>
 
 #include "tc_common.cuh"
 
 namespace iptq {
 
-constexpr int ATT_THREADS = 192;
+constexpr int ATT_THREADS = 320;
 constexpr int ATT_STAGES = 2;
+constexpr int kPadScore = -(1 << 30);     // a score this low has exponential 0 for every row maximum below 2^30
 
 struct AttnParams {
     int B, H, N, dh;
     int mtiles;            // ceil(N / 128)
+    int items, full_items; // all work items; those of them that are full 128-row tiles (handed out first)
     int npad_s;            // N rounded up to 16: UMMA N of QK^T, TMEM columns of S
     int kpad;              // N rounded up to 32: UMMA K extent of P V
     int q_bytes, k_bytes, v_bytes, stage_bytes;
-    int p_off, bar_off;
+    int p_off, xch_off, bar_off;
     uint32_t tmem_cols;
     const int32_t* bias;   // [H, N, N] or null
     const uint8_t* mask_id;// [B, N] or null
@@ -35,7 +39,15 @@ struct AttnParams {
     StatusBlock* status;
 };
 
-template <int DH, int VARIANT, bool HAS_BIAS, bool HAS_MASK>
+// item index -> (batch*head, row tile): full tiles first, then the ragged last tiles
+__device__ __forceinline__ void decode_item(const AttnParams& p, int it, int& bh, int& mt)
+{
+    const int full_per = p.N >> 7;                        // full 128-row tiles per (batch, head)
+    if (it < p.full_items) { bh = it / full_per; mt = it - bh * full_per; }
+    else                   { bh = it - p.full_items; mt = full_per; }
+}
+
+template <int DH, int VARIANT, bool HAS_BIAS, bool HAS_MASK, bool PSHR>
 __global__ void __launch_bounds__(ATT_THREADS, 2)
 attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, const AttnParams p)
@@ -43,25 +55,27 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sP = smem + p.p_off;
+    int* xch_max = reinterpret_cast<int*>(smem + p.xch_off);              // [2 parts][128 rows]
+    unsigned* xch_sum = reinterpret_cast<unsigned*>(xch_max + 256);       // [2 parts][128 rows]
     uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + p.bar_off);   // [ATT_STAGES]
     uint64_t* kv_empty = kv_full + ATT_STAGES;                            // [ATT_STAGES]
     uint64_t* s_full = kv_empty + ATT_STAGES;
     uint64_t* p_ready = s_full + 1;
     uint64_t* o_full = p_ready + 1;
     uint64_t* t_empty = o_full + 1;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(t_empty + 1);
+    volatile int* item_of = reinterpret_cast<volatile int*>(t_empty + 1); // [ATT_STAGES] item held by a stage, -1 = stop
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(item_of) + ATT_STAGES);
     CtaControl* ctl = reinterpret_cast<CtaControl*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int items = p.B * p.H * p.mtiles;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < ATT_STAGES; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
         mbar_init(s_full, 1);
-        mbar_init(p_ready, 128);
+        mbar_init(p_ready, 256);
         mbar_init(o_full, 1);
-        mbar_init(t_empty, 128);
+        mbar_init(t_empty, 256);
         ctl->abort = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_q);
@@ -78,20 +92,34 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------ TMA producer + work distribution
         if (elect_one()) {
             int s = 0; uint32_t ph = 0;
-            for (int it = blockIdx.x; it < items; it += gridDim.x) {
-                const int mt = it % p.mtiles;
-                const int bh = it / p.mtiles;
-                const int h = bh % p.H, b = bh / p.H;
+            for (;;) {
                 if (!mbar_wait(&kv_empty[s], ph ^ 1u, ctl, p.status, 11)) break;
+                const int it = atomicAdd(&p.status->work_next, 1);
+                if (it >= p.items) {
+                    item_of[s] = -1;
+                    mbar_arrive(&kv_full[s]);                  // release: the consumers see the stop mark
+                    break;
+                }
+                int bh, mt;
+                decode_item(p, it, bh, mt);
+                const int h = bh % p.H, b = bh / p.H;
+                item_of[s] = it;
                 uint8_t* st = smem + s * p.stage_bytes;
                 mbar_expect_tx(&kv_full[s], (uint32_t)((128 + p.npad_s + p.kpad) * DH));   // bytes of the three full boxes
                 tma_load_4d(st, &map_q, &kv_full[s], 0, mt * 128, h, b);
                 tma_load_4d(st + p.q_bytes, &map_k, &kv_full[s], 0, 0, h, b);
                 tma_load_4d(st + p.q_bytes + p.k_bytes, &map_v, &kv_full[s], 0, 0, h, b);
                 if (++s == ATT_STAGES) { s = 0; ph ^= 1u; }
+            }
+            // the last CTA to finish re-arms the counters for the next launch that uses this workspace
+            __threadfence();
+            if (atomicAdd(&p.status->work_done, 1) == (int)gridDim.x - 1) {
+                p.status->work_next = 0;
+                p.status->work_done = 0;
+                __threadfence();
             }
         }
     } else if (warp == 1) {
@@ -101,9 +129,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const uint32_t idesc_o = umma_idesc_i8(128, DH, false, true, false, true);     // u8 P (K-major) x s8 V (MN-major)
             int s = 0; uint32_t ph = 0;
             uint32_t iph = 0;                                  // parity of the per-item barriers
-            for (int it = blockIdx.x; it < items; it += gridDim.x, iph ^= 1u) {
+            for (;; iph ^= 1u) {
                 if (!mbar_wait(t_empty, iph ^ 1u, ctl, p.status, 12)) break;     // previous O has been read
                 if (!mbar_wait(&kv_full[s], ph, ctl, p.status, 13)) break;
+                if (item_of[s] < 0) break;
                 tc_fence_after_sync();
                 const uint32_t q_addr = smem_u32(smem + s * p.stage_bytes);
                 const uint32_t k_addr = q_addr + p.q_bytes;
@@ -132,105 +161,171 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
         }
     } else {
-        // ------------------------------------------------------------ softmax + output warps (thread = query row)
-        const int quad = warp & 3;
+        // ------------------------------------------------------------ softmax + output warps
+        const int quad = warp & 3;                             // TMEM lane quadrant this warp may touch
+        const int part = (warp - 2) >> 2;                      // which half of the columns
         const int rloc = quad * 32 + lane;                     // row inside the 128-row tile
         const uint32_t trow = tmem_base + ((uint32_t)(quad * 32) << 16);
         const uint32_t p_row = smem_u32(sP) + (uint32_t)((rloc >> 3) * 1024 + (rloc & 7) * 128);
         const int HD = p.H * DH;
+        const int chunks = p.npad_s >> 4;
+        const int c_half = (chunks + 1) >> 1;
+        const int cb = part ? c_half : 0, ce = part ? chunks : c_half;   // this thread's 16-column chunks
+        const bool sat8 = p.orq.qmin == -128 && p.orq.qmax == 127;
+        int s = 0; uint32_t ph = 0;
         uint32_t iph = 0;
-        for (int it = blockIdx.x; it < items; it += gridDim.x, iph ^= 1u) {
-            const int mt = it % p.mtiles;
-            const int bh = it / p.mtiles;
+
+        auto sweep_single = [&](auto&& body) {      // for the arithmetic-heavy sweep: one buffer, fewer live registers
+            uint32_t ra[16];
+#pragma unroll 1
+            for (int c = cb; c < ce; ++c) {
+                tmem_ld16(trow + c * 16, ra);
+                tmem_wait_ld();
+                body(ra, c);
+            }
+        };
+        // Runs `body(values, chunk)` over this thread's chunks with the TMEM load of the next chunk in flight.
+        auto sweep = [&](auto&& body) {
+            uint32_t ra[16], rb[16];
+            if (cb < ce) tmem_ld16(trow + cb * 16, ra);
+#pragma unroll 1
+            for (int c = cb; c < ce; c += 2) {
+                tmem_wait_ld();
+                if (c + 1 < ce) tmem_ld16(trow + (c + 1) * 16, rb);
+                body(ra, c);
+                if (c + 1 < ce) {
+                    tmem_wait_ld();
+                    if (c + 2 < ce) tmem_ld16(trow + (c + 2) * 16, ra);
+                    body(rb, c + 1);
+                }
+            }
+        };
+
+        for (;; iph ^= 1u) {
+            // the partner warp of this quadrant meets this one at two named barriers per item: a warp that gives up
+            // before them arrives without waiting, so that a bounded wait running out can never strand the partner
+            if (!mbar_wait(&kv_full[s], ph, ctl, p.status, 17)) {   // acquire: the item number is visible
+                named_barrier_arrive(1 + quad, 64); named_barrier_arrive(1 + quad, 64);
+                break;
+            }
+            const int it = item_of[s];
+            if (it < 0) break;
+            if (++s == ATT_STAGES) { s = 0; ph ^= 1u; }
+            int bh, mt;
+            decode_item(p, it, bh, mt);
             const int h = bh % p.H, b = bh / p.H;
             const int row = mt * 128 + rloc;
             const bool valid = row < p.N;
+            const bool warp_rows = mt * 128 + quad * 32 < p.N;            // warp-uniform: any valid row in this warp
             const int32_t* brow = HAS_BIAS ? p.bias + ((size_t)h * p.N + (valid ? row : 0)) * p.N : nullptr;
             const uint8_t* mrow = HAS_MASK ? p.mask_id + (size_t)b * p.N : nullptr;
-            const unsigned my_id = (HAS_MASK && valid) ? mrow[row] : 0u;
+            const unsigned my_id = HAS_MASK ? mrow[valid ? row : 0] : 0u;
 
-            if (!mbar_wait(s_full, iph, ctl, p.status, 15)) break;
+            if (!mbar_wait(s_full, iph, ctl, p.status, 15)) {
+                named_barrier_arrive(1 + quad, 64); named_barrier_arrive(1 + quad, 64);
+                break;
+            }
             tc_fence_after_sync();
-            // ---- sweep 1: row maximum over the real, unmasked columns (Eq. (6))
-            int mx = INT_MIN;
-#pragma unroll 1
-            for (int c0 = 0; c0 < p.npad_s; c0 += 16) {
-                uint32_t r[16];
-                tmem_ld16(trow + c0, r);
-                tmem_wait_ld();
+            if (warp_rows) {
+                // ---- sweep 1: row maximum over the real, unmasked columns (Eq. (6)).  Chunks that hold padding,
+                //      masked pairs or a bias are rewritten in TMEM (pad / masked -> kPadScore, score + bias) so
+                //      that the next sweep needs no per-element case analysis.
+                int mx = INT_MIN;
+                sweep([&](uint32_t (&v)[16], int c) {
+                    const int c0 = c * 16;
+                    if (HAS_BIAS || HAS_MASK || c0 + 16 > p.N) {              // warp-uniform
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int col = c0 + j;
-                    int s = (int)r[j];
-                    if (HAS_BIAS && col < p.N) s += __ldg(brow + col);
-                    bool use = col < p.N;
-                    if (HAS_MASK && use && valid) use = (mrow[col] == my_id);
-                    if (use) mx = max(mx, s);
-                }
+                        for (int j = 0; j < 16; ++j) {
+                            const int col = c0 + j;
+                            int sc = (int)v[j];
+                            bool use = col < p.N;
+                            if (HAS_BIAS && use) sc += __ldg(brow + col);
+                            if (HAS_MASK && use) use = (mrow[col] == my_id);
+                            v[j] = (uint32_t)(use ? sc : kPadScore);
+                        }
+                        tmem_st16(trow + c0, v);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) mx = max(mx, (int)v[j]);
+                });
+                xch_max[part * 128 + rloc] = mx;
+                tmem_wait_st();
+                named_barrier(1 + quad, 64);
+                mx = max(xch_max[rloc], xch_max[128 + rloc]);
+                // ---- sweep 2: integer exponentials (Eqs. (7)-(14)) and their sum; e goes back to TMEM
+                unsigned sum = 0;
+                sweep_single([&](uint32_t (&v)[16], int c) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const unsigned e = exp_core_nd<VARIANT>((int)v[j] - mx, p.ex);
+                        sum += e;
+                        v[j] = e;
+                    }
+                    tmem_st16(trow + c * 16, v);
+                });
+                xch_sum[part * 128 + rloc] = sum;
+                tmem_wait_st();
+                named_barrier(1 + quad, 64);
+                sum = xch_sum[rloc] + xch_sum[128 + rloc];
+                // ---- sweep 3: IntDiv (Eq. (15)) -> uint8 probabilities in the UMMA A-operand layout
+                const unsigned f = intdiv_factor(sum, p.M) << p.f_shl;
+                sweep([&](uint32_t (&v)[16], int c) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        int pv[4];
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            unsigned x = __umulhi(f, v[q4 * 4 + t]);
+                            if (PSHR) x >>= p.p_shr;
+                            pv[t] = (int)x;
+                        }
+                        w[q4] = pack4_sat_u8(pv[0], pv[1], pv[2], pv[3]);          // values are <= 2^(b-1): nothing saturates
+                    }
+                    const int c0 = c * 16;
+                    const int chunk = (c0 & 127) >> 4;
+                    st_shared_v4(p_row + (uint32_t)((c0 >> 7) * 16384 + ((chunk ^ (rloc & 7)) << 4)), w[0], w[1], w[2], w[3]);
+                });
+            } else {
+                named_barrier_arrive(1 + quad, 64); named_barrier_arrive(1 + quad, 64);   // keeps the barrier generations aligned
             }
-            // ---- sweep 2: integer exponentials (Eqs. (7)-(14)) and their sum; e goes back to TMEM
-            unsigned sum = 0;
-#pragma unroll 1
-            for (int c0 = 0; c0 < p.npad_s; c0 += 16) {
-                uint32_t r[16];
-                tmem_ld16(trow + c0, r);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int col = c0 + j;
-                    int s = (int)r[j];
-                    if (HAS_BIAS && col < p.N) s += __ldg(brow + col);
-                    bool use = col < p.N;
-                    if (HAS_MASK && use && valid) use = (mrow[col] == my_id);
-                    const unsigned d = min((unsigned)(mx - s), (unsigned)p.ex.dcap);
-                    const unsigned e = use ? exp_core<VARIANT>(d, p.ex) : 0u;
-                    sum += e;
-                    r[j] = e;
-                }
-                tmem_st16(trow + c0, r);
-            }
-            tmem_wait_st();
-            // ---- sweep 3: IntDiv (Eq. (15)) -> uint8 probabilities in the UMMA A-operand layout
-            const unsigned f = intdiv_factor(sum, p.M) << p.f_shl;
-#pragma unroll 1
-            for (int c0 = 0; c0 < p.npad_s; c0 += 16) {
-                uint32_t r[16];
-                tmem_ld16(trow + c0, r);
-                tmem_wait_ld();
-                uint32_t w[4];
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    uint32_t acc = 0;
-#pragma unroll
-                    for (int t = 0; t < 4; ++t) acc |= ((__umulhi(f, r[q4 * 4 + t]) >> p.p_shr) & 255u) << (8 * t);
-                    w[q4] = acc;
-                }
+            // key columns between npad_s and kpad (at most one 16-column chunk) meet zero rows of V, but the bytes
+            // the tensor core reads there must be defined
+            if (part == 1 && p.kpad > p.npad_s) {
+                const int c0 = p.npad_s;
                 const int chunk = (c0 & 127) >> 4;
-                st_shared_v4(p_row + (uint32_t)((c0 >> 7) * 16384 + ((chunk ^ (rloc & 7)) << 4)), w[0], w[1], w[2], w[3]);
+                st_shared_v4(p_row + (uint32_t)((c0 >> 7) * 16384 + ((chunk ^ (rloc & 7)) << 4)), 0u, 0u, 0u, 0u);
             }
             fence_proxy_async_smem();            // generic-proxy stores -> visible to the tensor core's reads
             tc_fence_before_sync();
             mbar_arrive(p_ready);
 
-            // ---- output: O = P V from TMEM -> requant -> int8
+            // ---- output: O = P V from TMEM -> requant -> int8 (each half of the threads takes half of the columns)
             if (!mbar_wait(o_full, iph, ctl, p.status, 16)) break;
             tc_fence_after_sync();
-            int8_t* orow = p.out + ((size_t)b * p.N + (valid ? row : 0)) * HD + h * DH;
+            if (warp_rows) {
+                int8_t* orow = p.out + ((size_t)b * p.N + (valid ? row : 0)) * HD + h * DH;
+                constexpr int OC = DH / 32;                    // 16-column chunks per thread
 #pragma unroll
-            for (int c0 = 0; c0 < DH; c0 += 16) {
-                uint32_t r[16];
-                tmem_ld16(trow + c0, r);
-                tmem_wait_ld();
-                int o[16];
+                for (int cc = 0; cc < OC; ++cc) {
+                    const int c0 = (part * OC + cc) * 16;
+                    uint32_t r[16];
+                    tmem_ld16(trow + c0, r);
+                    tmem_wait_ld();
+                    int o[16];
 #pragma unroll
-                for (int j = 0; j < 16; ++j) o[j] = requant_full((int)r[j], p.orq);
-                if (valid) {
-                    int4 pk;
-                    pk.x = (int)pack4_s8(o[0], o[1], o[2], o[3]);
-                    pk.y = (int)pack4_s8(o[4], o[5], o[6], o[7]);
-                    pk.z = (int)pack4_s8(o[8], o[9], o[10], o[11]);
-                    pk.w = (int)pack4_s8(o[12], o[13], o[14], o[15]);
-                    *reinterpret_cast<int4*>(orow + c0) = pk;
+                    for (int j = 0; j < 16; ++j) {
+                        o[j] = requant_nosat((int)r[j], p.orq);
+                        if (!sat8) o[j] = max(p.orq.qmin, min(p.orq.qmax, o[j]));
+                    }
+                    if (valid) {
+                        int4 pk;
+                        pk.x = (int)pack4_sat_s8(o[0], o[1], o[2], o[3]);
+                        pk.y = (int)pack4_sat_s8(o[4], o[5], o[6], o[7]);
+                        pk.z = (int)pack4_sat_s8(o[8], o[9], o[10], o[11]);
+                        pk.w = (int)pack4_sat_s8(o[12], o[13], o[14], o[15]);
+                        *reinterpret_cast<int4*>(orow + c0) = pk;
+                    }
                 }
             }
             tc_fence_before_sync();
@@ -268,20 +363,30 @@ template <int DH, int VARIANT>
 static int launch_attn(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const AttnParams& p,
                        int smem_bytes, cudaStream_t st)
 {
-    const int items = p.B * p.H * p.mtiles;
-    const int grid = std::min(items, 2 * sm_count());
+    const int grid = std::min(p.items, 2 * sm_count());
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return IPTQ_ERR_CUDA;
+#define IPTQ_ATT_LAUNCH2(HB, HM, PS)                                                                              \
+    do {                                                                                                          \
+        auto kern = attention_kernel<DH, VARIANT, HB, HM, PS>;                                                    \
+        static int configured[64];          /* largest dynamic shared memory size set so far, per device */     \
+        if (configured[dev] < smem_bytes) {                                                                       \
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) \
+                return IPTQ_ERR_CUDA;                                                                             \
+            configured[dev] = smem_bytes;                                                                         \
+        }                                                                                                         \
+        kern<<<grid, ATT_THREADS, smem_bytes, st>>>(mq, mk, mv, p);                                               \
+    } while (0)
 #define IPTQ_ATT_LAUNCH(HB, HM)                                                                                   \
     do {                                                                                                          \
-        auto kern = attention_kernel<DH, VARIANT, HB, HM>;                                                        \
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)  \
-            return IPTQ_ERR_CUDA;                                                                                 \
-        kern<<<grid, ATT_THREADS, smem_bytes, st>>>(mq, mk, mv, p);                                               \
+        if (p.p_shr) IPTQ_ATT_LAUNCH2(HB, HM, true); else IPTQ_ATT_LAUNCH2(HB, HM, false);                        \
     } while (0)
     if (p.bias && p.mask_id) IPTQ_ATT_LAUNCH(true, true);
     else if (p.bias) IPTQ_ATT_LAUNCH(true, false);
     else if (p.mask_id) IPTQ_ATT_LAUNCH(false, true);
     else IPTQ_ATT_LAUNCH(false, false);
 #undef IPTQ_ATT_LAUNCH
+#undef IPTQ_ATT_LAUNCH2
     note_launch();
     return last_launch_status();
 }
@@ -320,6 +425,8 @@ int attention_launch(const AttnArgs& a, cudaStream_t st)
     AttnParams p;
     p.B = (int)a.B; p.H = a.H; p.N = a.N; p.dh = a.dh;
     p.mtiles = (a.N + 127) / 128;
+    p.items = p.B * p.H * p.mtiles;
+    p.full_items = p.B * p.H * (a.N / 128);
     p.npad_s = (a.N + 15) & ~15;
     p.kpad = (a.N + 31) & ~31;
     auto up1k = [](int v) { return (v + 1023) & ~1023; };
@@ -329,7 +436,8 @@ int attention_launch(const AttnArgs& a, cudaStream_t st)
     p.stage_bytes = p.q_bytes + p.k_bytes + p.v_bytes;
     p.p_off = ATT_STAGES * p.stage_bytes;
     const int p_bytes = ((p.kpad + 127) / 128) * 16384;
-    p.bar_off = p.p_off + p_bytes;
+    p.xch_off = p.p_off + p_bytes;
+    p.bar_off = p.xch_off + 2 * 2 * 128 * 4;
     const int smem_bytes = p.bar_off + 128 + 1024;
     p.tmem_cols = 32;
     while ((int)p.tmem_cols < std::max(p.npad_s, a.dh)) p.tmem_cols <<= 1;

@@ -21,7 +21,9 @@ struct StatusBlock {
     int32_t timeout_flag;     // non-zero once any bounded wait has given up
     int32_t where;            // id of the wait that gave up first (kernel-specific)
     int32_t block;            // blockIdx.x of the CTA that gave up
-    int32_t pad[61];
+    int32_t work_next;        // next work item of a kernel that hands out items dynamically (0 between launches)
+    int32_t work_done;        // CTAs of that kernel that have finished (0 between launches)
+    int32_t pad[59];
 };
 static_assert(sizeof(StatusBlock) == 256, "status block is 256 bytes");
 constexpr size_t kStatusBytes = 256;
@@ -102,7 +104,10 @@ struct ExpDev {
     int qln2, qb, qc, norm_l, norm_r;    // polynomial candidate
 };
 
-// Integer exponential of nd = -min(max - s, dcap), i.e. Q_delta of Eq. (6) clamped to [-dcap, 0].
+// Integer exponential of nd = s - max <= 0, i.e. Q_delta of Eq. (6).  The clamp of max - s at dcap = 34 x0 needs no
+// instruction: for any nd > -2^31 the magnitude -Q_p stays below 2^32, and from the clamp point on the octave count
+// q is at least 48 (the multiply-high quotient of an operand >= 2^31 is >= 127), so the shift of Eq. (9) returns 0
+// exactly as the clamped value would.
 template <int VARIANT>
 __device__ __forceinline__ unsigned exp_core_nd(int nd, const ExpDev& c)
 {
@@ -115,7 +120,7 @@ __device__ __forceinline__ unsigned exp_core_nd(int nd, const ExpDev& c)
         return shr_clamp(e, z);
     } else {
         const int a = nd >> 1, b = nd >> 4;
-        const unsigned P = (unsigned)(b - a - nd);                     // -Q_p, Eq. (7)
+        const unsigned P = (unsigned)b - (unsigned)a - (unsigned)nd;   // -Q_p, Eq. (7); < 2^32 for nd > -2^31
         const unsigned q = __umulhi(P, c.div_mul) >> c.div_shift;      // Eq. (8): floor(P / x0)
         const int u = (int)(q * (unsigned)c.x0) - (int)P;              // -r
         int base;

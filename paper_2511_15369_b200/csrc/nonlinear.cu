@@ -28,7 +28,6 @@ softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ pr
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    const int ndmin = -c.ex.dcap;
     for (int64_t row = warp; row < rows; row += nwarps) {
         const int32_t* sr = scores + row * n;
         const int32_t* br = HAS_BIAS ? bias + (row % bias_period) * n : nullptr;
@@ -49,7 +48,7 @@ softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ pr
         unsigned sum = 0;
 #pragma unroll
         for (int k = 0; k < NITER; ++k) {
-            const unsigned e = exp_core_nd<VARIANT>(max(v[k] - mx, ndmin), c.ex);
+            const unsigned e = exp_core_nd<VARIANT>(v[k] - mx, c.ex);
             v[k] = (int)e;
             sum += e;
         }

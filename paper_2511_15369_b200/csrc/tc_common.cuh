@@ -213,6 +213,10 @@ __device__ __forceinline__ bool elect_one()
     return pred != 0;
 }
 
+__device__ __forceinline__ void named_barrier_arrive(int id, int threads)
+{
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 // Named barrier among a subset of the CTA's warps.
 __device__ __forceinline__ void named_barrier(int id, int threads)
 {
