@@ -4,9 +4,12 @@
 //   - FC1: requantise to the GELU input scale, integer GELU (Sec. 3.3, Eqs. (3), (5)), requantise to int8.
 // No int32 intermediate is written to HBM.
 //
-// One persistent CTA per SM, 10 warps: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM),
-// warps 2..9 = epilogue (two warps per TMEM lane quadrant, each taking half of the tile's columns).
+// One persistent CTA per SM, 14 warps: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM),
+// warps 2..13 = epilogue (three warps per TMEM lane quadrant, each taking a third of the tile's columns).
 // The accumulator is double-buffered in TMEM so that the epilogue of tile i overlaps the mainloop of tile i+1.
+// Per-column requantisation constants live in TMEM beside the accumulators (shared-memory reads of them would
+// cost one load per output and saturate the load/store pipe); the bias is written into each accumulator before
+// the MMAs start, which then always accumulate.
 #include <algorithm>
 #include <mutex>
 
@@ -59,14 +62,17 @@ int make_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint6
 enum { EPI_REQUANT = 0, EPI_RESIDUAL = 1, EPI_GELU = 2 };
 
 constexpr int BM = 128;          // rows per tile = TMEM lanes
-constexpr int BN = 128;          // columns per tile
+constexpr int BN = 96;           // columns per tile: two accumulators + three per-column constant rows fit 512 TMEM columns
 constexpr int BK = 128;          // bytes of K per stage = one 128-byte swizzle row = 4 MMA k-steps
-constexpr int STAGES = 4;
-constexpr int EPI_PARTS = 2;     // epilogue warps per TMEM lane quadrant; each owns BN / EPI_PARTS columns
+constexpr int STAGES = 5;
+constexpr int EPI_PARTS = 3;     // epilogue warps per TMEM lane quadrant; each owns BN / EPI_PARTS columns
 constexpr int EPI_WARPS = 4 * EPI_PARTS;
-constexpr int COLS = BN / EPI_PARTS;                 // 64: bytes per output row per warp, one 64-byte swizzle row
+constexpr int COLS = BN / EPI_PARTS;                 // 32: bytes per output row per warp, one 32-byte swizzle row
 constexpr int GEMM_THREADS = 32 * (2 + EPI_WARPS);
-static_assert(COLS == 64, "staging addresses below assume 64-byte rows (64-byte TMA swizzle)");
+static_assert(COLS == 32, "staging addresses below assume 32-byte rows (32-byte TMA swizzle)");
+// TMEM columns: [0, 2 BN) accumulators, then mult, rounding constant, shift -- one row of BN words each,
+// replicated over the 128 lanes so that a thread reads them with the same instruction as its accumulators.
+constexpr uint32_t TM_MULT = 2 * BN, TM_RND = 3 * BN, TM_SHIFT = 4 * BN, TMEM_COLS = 512;
 
 struct GemmParams {
     int M, N, K;
@@ -86,18 +92,21 @@ struct GemmSmem {
     static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
     static constexpr int OFF_OUT = OFF_B + STAGES * B_BYTES;                     // [EPI_WARPS][32 rows][COLS] int8
     static constexpr int OFF_RES = OFF_OUT + EPI_WARPS * WARP_TILE;              // same shape, residual tiles
-    static constexpr int OFF_CP = OFF_RES + EPI_WARPS * WARP_TILE;               // [EPI_WARPS][COLS] int4
-    static constexpr int OFF_BAR = OFF_CP + EPI_WARPS * COLS * 16;
+    static constexpr int OFF_BIAS = OFF_RES + EPI_WARPS * WARP_TILE;             // [EPI_WARPS][COLS] int32
+    static constexpr int OFF_BAR = OFF_BIAS + EPI_WARPS * COLS * 4;
     static constexpr int NUM_BARS = 2 * STAGES + 4 + EPI_WARPS;
     static constexpr int OFF_END = OFF_BAR + NUM_BARS * 8 + 16;
     static constexpr int TOTAL = OFF_END + 1024;                                 // slack for 1024-byte alignment
 };
 
-// Byte offset of 16-byte chunk `chunk` of row `row` inside a [32][64]-byte block written/read by TMA with the
-// 64-byte swizzle (chunk index XOR bits 7-8 of the address); also makes the per-row 16-byte accesses of a
-// warp conflict-free.
-__device__ __forceinline__ uint32_t swz64(int row, int chunk) { return (uint32_t)(row * 64 + ((chunk ^ ((row >> 1) & 3)) << 4)); }
+// Byte offset of 16-byte chunk `chunk` (0/1) of row `row` inside a [32][32]-byte block written/read by TMA with
+// the 32-byte swizzle (chunk bit XOR bit 7 of the address); also keeps a warp's per-row 16-byte accesses
+// conflict-free.
+__device__ __forceinline__ uint32_t swz32(int row, int chunk) { return (uint32_t)(row * 32 + ((chunk ^ ((row >> 2) & 1)) << 4)); }
 
+// One CTA works on ONE column tile (blockIdx.x % num_n_tiles) and walks down its row tiles, so the per-column
+// constants are set up once per CTA: mult / rounding / shift in TMEM, the bias in shared memory, from where the
+// epilogue writes it back into each accumulator it has just drained (the MMAs then always accumulate).
 template <int EPI, int GELU_VARIANT, bool SAT8>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -119,9 +128,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int num_tiles = p.num_m_tiles * p.num_n_tiles;
     const int kblocks = (p.K + BK - 1) / BK;
-    constexpr uint32_t TMEM_COLS = 2 * BN;        // two accumulator buffers
+    const int n0 = (int)(blockIdx.x % (unsigned)p.num_n_tiles) * BN;
+    const int mt0 = (int)(blockIdx.x / (unsigned)p.num_n_tiles);
+    const int mt_step = (int)(gridDim.x / (unsigned)p.num_n_tiles);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
@@ -147,14 +157,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ------------------------------------------------------------ TMA producer
         if (elect_one()) {
             int s = 0; uint32_t ph = 0;
-            for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
-                const int m0 = (t % p.num_m_tiles) * BM;
-                const int n0 = (t / p.num_m_tiles) * BN;
+            for (int mt = mt0; mt < p.num_m_tiles; mt += mt_step) {
                 bool ok = true;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(&empty_bar[s], ph ^ 1u, ctl, p.status, 1)) { ok = false; break; }
                     mbar_expect_tx(&full_bar[s], L::A_BYTES + L::B_BYTES);
-                    tma_load_2d(sA + s * L::A_BYTES, &map_a, &full_bar[s], kb * BK, m0);
+                    tma_load_2d(sA + s * L::A_BYTES, &map_a, &full_bar[s], kb * BK, mt * BM);
                     tma_load_2d(sB + s * L::B_BYTES, &map_b, &full_bar[s], kb * BK, n0);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -167,10 +175,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             constexpr uint32_t idesc = umma_idesc_i8(BM, BN, true, true, false, false);
             int s = 0; uint32_t ph = 0;
             int it = 0;
-            for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+            for (int mt = mt0; mt < p.num_m_tiles; mt += mt_step, ++it) {
                 const int ab = it & 1;
-                const uint32_t abph = (uint32_t)(it >> 1) & 1u;
-                if (!mbar_wait(&acc_empty[ab], abph ^ 1u, ctl, p.status, 2)) break;
+                // the accumulator holds the bias, written by the epilogue warps (first at start-up, then after each drain)
+                if (!mbar_wait(&acc_empty[ab], (uint32_t)(it >> 1) & 1u, ctl, p.status, 2)) break;
                 tc_fence_after_sync();
                 const uint32_t tacc = tmem_base + (uint32_t)(ab * BN);
                 bool ok = true;
@@ -184,7 +192,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart; a k-step is 32 bytes
                         const uint64_t da = umma_smem_desc(a_addr + k * 32, 16, 1024, 128);
                         const uint64_t db = umma_smem_desc(b_addr + k * 32, 16, 1024, 128);
-                        umma_i8(tacc, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+                        umma_i8(tacc, da, db, idesc, 1u);
                     }
                     umma_commit(&empty_bar[s]);               // frees the stage once these MMAs have read it
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
@@ -201,17 +209,53 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int ew = warp - 2;
         const int quad = warp & 3;
         const int part = ew >> 2;
-        int4* cp = reinterpret_cast<int4*>(smem + L::OFF_CP) + ew * COLS;
+        int* sbias = reinterpret_cast<int*>(smem + L::OFF_BIAS) + ew * COLS;
+        const uint32_t bias_addr = smem_u32(sbias);
         const uint32_t out_blk = smem_u32(smem + L::OFF_OUT + ew * L::WARP_TILE);
         uint8_t* res_ptr = smem + L::OFF_RES + ew * L::WARP_TILE;
         const uint32_t res_blk = smem_u32(res_ptr);
+        const int col0 = n0 + part * COLS;
+        const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(part * COLS);
         uint32_t res_ph = 0;
+        {
+            // ---- once per CTA: this warp's per-column constants (lane = column)
+            const int n = col0 + lane;
+            int cb = 0, cm = 1 << 30, cr = 1, cs = 1;
+            if (n < p.N) {
+                cs = (int)__ldg(p.shift + n);
+                cb = p.bias ? __ldg(p.bias + n) : 0;
+                cm = __ldg(p.mult + n);
+                cr = 1 << (cs - 1);
+            }
+            sbias[lane] = cb;
+            __syncwarp();
+            uint32_t v[16];
+#pragma unroll
+            for (int ch = 0; ch < COLS / 16; ++ch) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = (uint32_t)__shfl_sync(0xffffffffu, cm, ch * 16 + j);
+                tmem_st16(tlane + TM_MULT + ch * 16, v);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = (uint32_t)__shfl_sync(0xffffffffu, cr, ch * 16 + j);
+                tmem_st16(tlane + TM_RND + ch * 16, v);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = (uint32_t)__shfl_sync(0xffffffffu, cs, ch * 16 + j);
+                tmem_st16(tlane + TM_SHIFT + ch * 16, v);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = (uint32_t)__shfl_sync(0xffffffffu, cb, ch * 16 + j);
+                tmem_st16(tlane + ch * 16, v);                // both accumulators start from the bias
+                tmem_st16(tlane + BN + ch * 16, v);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(&acc_empty[0]); mbar_arrive(&acc_empty[1]); }
+        }
         int it = 0;
-        for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+        for (int mt = mt0; mt < p.num_m_tiles; mt += mt_step, ++it) {
             const int ab = it & 1;
             const uint32_t abph = (uint32_t)(it >> 1) & 1u;
-            const int row0 = (t % p.num_m_tiles) * BM + quad * 32;
-            const int col0 = (t / p.num_m_tiles) * BN + part * COLS;
+            const int row0 = mt * BM + quad * 32;
             const bool active = row0 < p.M && col0 < p.N;     // warp-uniform
             // the previous tile's store must have read the staging block before it is rewritten
             if (lane == 0) bulk_wait_read_all();
@@ -220,59 +264,55 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 mbar_expect_tx(&res_bar[ew], L::WARP_TILE);
                 tma_load_2d(res_ptr, &map_res, &res_bar[ew], col0, row0);
             }
-            // per-column constants of this warp's columns: (bias, mult, 2^(shift-1), shift)
-            for (int c = lane; c < COLS; c += 32) {
-                const int n = col0 + c;
-                int4 v = make_int4(0, 1 << 30, 1, 1);
-                if (n < p.N) {
-                    const int sh = (int)__ldg(p.shift + n);
-                    v = make_int4(p.bias ? __ldg(p.bias + n) : 0, __ldg(p.mult + n), 1 << (sh - 1), sh);
-                }
-                cp[c] = v;
-            }
-            __syncwarp();
             if (!mbar_wait(&acc_full[ab], abph, ctl, p.status, 4)) break;
             tc_fence_after_sync();
-            if (active) {
-                if (EPI == EPI_RESIDUAL) {
-                    if (!mbar_wait(&res_bar[ew], res_ph, ctl, p.status, 5)) break;
-                    res_ph ^= 1u;
-                }
-                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * BN + part * COLS);
-                uint32_t r[2][16];
-                tmem_ld16(taddr, r[0]);
-#pragma unroll
-                for (int ch = 0; ch < COLS / 16; ++ch) {
-                    tmem_wait_ld();
-                    if (ch + 1 < COLS / 16) tmem_ld16(taddr + (ch + 1) * 16, r[(ch + 1) & 1]);   // overlaps the math below
-                    const uint32_t* acc = r[ch & 1];
-                    uint4 resv = make_uint4(0, 0, 0, 0);
-                    if (EPI == EPI_RESIDUAL) resv = ld_shared_v4(res_blk + swz64(lane, ch));
-                    const uint32_t resw[4] = {resv.x, resv.y, resv.z, resv.w};
-                    int o[16];
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int4 k4 = cp[ch * 16 + j];
-                        int v = requant_core((int)acc[j] + k4.x, k4.y, k4.z, k4.w);
-                        if (EPI == EPI_GELU) {
-                            v = gelu_core<GELU_VARIANT>(v, p.gelu);
-                            v = requant_nosat(v, p.gelu.out);
-                            if (!SAT8) v = max(p.gelu.out.qmin, min(p.gelu.out.qmax, v));
-                        } else if (EPI == EPI_RESIDUAL) {
-                            // byte j of the residual word, sign-extended, widened by 2^16 and requantised
-                            const int rb = (j & 3) == 0 ? sext_byte<0>(resw[j >> 2]) : (j & 3) == 1 ? sext_byte<1>(resw[j >> 2])
-                                         : (j & 3) == 2 ? sext_byte<2>(resw[j >> 2]) : sext_byte<3>(resw[j >> 2]);
-                            v += requant_core(rb * 65536 - p.res_off, p.res_mult, p.res_rnd, p.res_shift) + p.out_zp;
-                        } else {
-                            v += p.out_zp;
-                        }
-                        o[j] = v;
-                    }
-                    st_shared_v4(out_blk + swz64(lane, ch), pack4_sat_s8(o[0], o[1], o[2], o[3]),
-                                 pack4_sat_s8(o[4], o[5], o[6], o[7]), pack4_sat_s8(o[8], o[9], o[10], o[11]),
-                                 pack4_sat_s8(o[12], o[13], o[14], o[15]));
-                }
+            if (EPI == EPI_RESIDUAL && active) {
+                if (!mbar_wait(&res_bar[ew], res_ph, ctl, p.status, 5)) break;
+                res_ph ^= 1u;
             }
+            const uint32_t tacc = tlane + (uint32_t)(ab * BN);
+#pragma unroll
+            for (int ch = 0; ch < COLS / 16; ++ch) {
+                uint32_t acc[16], cm[16], cr[16], cs[16];
+                tmem_ld16(tacc + ch * 16, acc);
+                tmem_ld16(tlane + TM_MULT + ch * 16, cm);
+                tmem_ld16(tlane + TM_RND + ch * 16, cr);
+                tmem_ld16(tlane + TM_SHIFT + ch * 16, cs);
+                uint32_t bv[16];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint4 t = ld_shared_v4(bias_addr + ch * 64 + q * 16);
+                    bv[4 * q] = t.x; bv[4 * q + 1] = t.y; bv[4 * q + 2] = t.z; bv[4 * q + 3] = t.w;
+                }
+                tmem_wait_ld();
+                tmem_st16(tacc + ch * 16, bv);                // re-arm this accumulator with the bias
+                if (!active) continue;
+                uint4 resv = make_uint4(0, 0, 0, 0);
+                if (EPI == EPI_RESIDUAL) resv = ld_shared_v4(res_blk + swz32(lane, ch));
+                const uint32_t resw[4] = {resv.x, resv.y, resv.z, resv.w};
+                int o[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    int v = requant_core((int)acc[j], (int)cm[j], (int)cr[j], (int)cs[j]);
+                    if (EPI == EPI_GELU) {
+                        v = gelu_core<GELU_VARIANT>(v, p.gelu);
+                        v = requant_nosat(v, p.gelu.out);
+                        if (!SAT8) v = max(p.gelu.out.qmin, min(p.gelu.out.qmax, v));
+                    } else if (EPI == EPI_RESIDUAL) {
+                        // byte j of the residual word, sign-extended, widened by 2^16 and requantised
+                        const int rb = (j & 3) == 0 ? sext_byte<0>(resw[j >> 2]) : (j & 3) == 1 ? sext_byte<1>(resw[j >> 2])
+                                     : (j & 3) == 2 ? sext_byte<2>(resw[j >> 2]) : sext_byte<3>(resw[j >> 2]);
+                        v += requant_core(rb * 65536 - p.res_off, p.res_mult, p.res_rnd, p.res_shift) + p.out_zp;
+                    } else {
+                        v += p.out_zp;
+                    }
+                    o[j] = v;
+                }
+                st_shared_v4(out_blk + swz32(lane, ch), pack4_sat_s8(o[0], o[1], o[2], o[3]),
+                             pack4_sat_s8(o[4], o[5], o[6], o[7]), pack4_sat_s8(o[8], o[9], o[10], o[11]),
+                             pack4_sat_s8(o[12], o[13], o[14], o[15]));
+            }
+            tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[ab]);       // the MMA warp may refill this accumulator
@@ -352,8 +392,9 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUten
             return IPTQ_ERR_CUDA;
         configured[dev] = true;
     }
-    const int tiles = p.num_m_tiles * p.num_n_tiles;
-    const int grid = std::min(tiles, sm_count());
+    // every CTA serves one column tile; the SMs are split evenly among the column tiles
+    const int per_n = std::max(1, std::min(sm_count() / p.num_n_tiles, p.num_m_tiles));
+    const int grid = p.num_n_tiles * per_n;
     kern<<<grid, GEMM_THREADS, L::TOTAL, st>>>(ma, mb, my, mr, p);
     note_launch();
     return last_launch_status();
@@ -409,8 +450,8 @@ int linear_launch(const LinearArgs& a, cudaStream_t st)
         const uint64_t dims[2] = {(uint64_t)a.N, (uint64_t)a.M};
         const uint64_t str[1] = {(uint64_t)a.N};
         const uint32_t box[2] = {COLS, 32};
-        if ((rc = make_tensor_map_u8(&my, a.y, 2, dims, str, box, 64)) != IPTQ_OK) return rc;
-        if ((rc = make_tensor_map_u8(&mr, a.residual ? a.residual : a.y, 2, dims, str, box, 64)) != IPTQ_OK) return rc;
+        if ((rc = make_tensor_map_u8(&my, a.y, 2, dims, str, box, 32)) != IPTQ_OK) return rc;
+        if ((rc = make_tensor_map_u8(&mr, a.residual ? a.residual : a.y, 2, dims, str, box, 32)) != IPTQ_OK) return rc;
     }
     if (a.gelu) {
         const bool sat8 = a.gelu->out.qmin == -128 && a.gelu->out.qmax == 127;
