@@ -90,10 +90,12 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    grid_dep_launch();
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer + work distribution
         if (elect_one()) {
+            grid_dep_wait();                                   // q/k/v come from the previous kernel
             int s = 0; uint32_t ph = 0;
             for (;;) {
                 if (!mbar_wait(&kv_empty[s], ph ^ 1u, ctl, p.status, 11)) break;
@@ -174,6 +176,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const bool sat8 = p.orq.qmin == -128 && p.orq.qmax == 127;
         int s = 0; uint32_t ph = 0;
         uint32_t iph = 0;
+        grid_dep_wait();                                       // output rows are written only after this
 
         auto sweep_single = [&](auto&& body) {      // for the arithmetic-heavy sweep: one buffer, fewer live registers
             uint32_t ra[16];
@@ -375,7 +378,7 @@ static int launch_attn(const CUtensorMap& mq, const CUtensorMap& mk, const CUten
                 return IPTQ_ERR_CUDA;                                                                             \
             configured[dev] = smem_bytes;                                                                         \
         }                                                                                                         \
-        kern<<<grid, ATT_THREADS, smem_bytes, st>>>(mq, mk, mv, p);                                               \
+        launch_kernel(kern, grid, ATT_THREADS, smem_bytes, st, mq, mk, mv, p);                                               \
     } while (0)
 #define IPTQ_ATT_LAUNCH(HB, HM)                                                                                   \
     do {                                                                                                          \

@@ -28,6 +28,32 @@ struct StatusBlock {
 static_assert(sizeof(StatusBlock) == 256, "status block is 256 bytes");
 constexpr size_t kStatusBytes = 256;
 
+// ---------------------------------------------------------------- launches
+#ifdef __CUDACC__
+
+// Every kernel of the library is launched with programmatic stream serialisation: its CTAs may become resident and
+// run their set-up (barrier init, TMEM allocation, constant tables) while the kernel before it on the stream is
+// still draining.  In exchange every kernel calls grid_dep_wait() before it reads or writes anything another
+// kernel may touch; grid_dep_launch() lets the kernel after it start its own set-up early.
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                        Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+// Blocks until the kernels this one depends on have completed and their writes are visible.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Allows the next kernel on the stream to be scheduled once every CTA of this grid has passed this point.
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+#endif  // __CUDACC__
+
 // ---------------------------------------------------------------- device arithmetic
 #ifdef __CUDACC__
 

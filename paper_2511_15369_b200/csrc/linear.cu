@@ -152,10 +152,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    grid_dep_launch();
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (elect_one()) {
+            grid_dep_wait();                                   // the activations come from the previous kernel
             int s = 0; uint32_t ph = 0;
             for (int mt = mt0; mt < p.num_m_tiles; mt += mt_step) {
                 bool ok = true;
@@ -251,6 +253,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             __syncwarp();
             if (lane == 0) { mbar_arrive(&acc_empty[0]); mbar_arrive(&acc_empty[1]); }
         }
+        grid_dep_wait();                                       // residual reads and output writes come after this
         int it = 0;
         for (int mt = mt0; mt < p.num_m_tiles; mt += mt_step, ++it) {
             const int ab = it & 1;
@@ -347,6 +350,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 __global__ void unpack_int4_kernel(const uint8_t* __restrict__ packed, int8_t* __restrict__ out, int64_t nbytes)
 {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    grid_dep_launch();
+    grid_dep_wait();                                // the scratch may still be read by the previous kernel
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nbytes; i += stride) {
         const unsigned b = packed[i];
         const int lo = (int)(b & 15u), hi = (int)(b >> 4);
@@ -361,7 +366,7 @@ int unpack_int4_launch(const void* packed, int8_t* out, int64_t n_elems, cudaStr
 {
     const int64_t nbytes = n_elems / 2;
     const int grid = (int)std::min<int64_t>((nbytes + 255) / 256, (int64_t)sm_count() * 8);
-    unpack_int4_kernel<<<grid, 256, 0, st>>>(static_cast<const uint8_t*>(packed), out, nbytes);
+    launch_kernel(unpack_int4_kernel, grid, 256, 0, st, static_cast<const uint8_t*>(packed), out, nbytes);
     note_launch();
     return last_launch_status();
 }
@@ -395,7 +400,7 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUten
     // every CTA serves one column tile; the SMs are split evenly among the column tiles
     const int per_n = std::max(1, std::min(sm_count() / p.num_n_tiles, p.num_m_tiles));
     const int grid = p.num_n_tiles * per_n;
-    kern<<<grid, GEMM_THREADS, L::TOTAL, st>>>(ma, mb, my, mr, p);
+    launch_kernel(kern, grid, GEMM_THREADS, L::TOTAL, st, ma, mb, my, mr, p);
     note_launch();
     return last_launch_status();
 }

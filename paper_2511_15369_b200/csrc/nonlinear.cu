@@ -28,6 +28,8 @@ softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ pr
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    grid_dep_launch();
+    grid_dep_wait();
     for (int64_t row = warp; row < rows; row += nwarps) {
         const int32_t* sr = scores + row * n;
         const int32_t* br = HAS_BIAS ? bias + (row % bias_period) * n : nullptr;
@@ -73,11 +75,11 @@ static int launch_softmax2(const int32_t* s, uint8_t* p, int64_t rows, int n, co
     const int64_t want = (rows + 7) / 8;
     const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 8);
     if (bias) {
-        if (c.p_shr) softmax_rows_kernel<VARIANT, NITER, true, true><<<grid, threads, 0, st>>>(s, p, rows, n, bias, period, c);
-        else         softmax_rows_kernel<VARIANT, NITER, true, false><<<grid, threads, 0, st>>>(s, p, rows, n, bias, period, c);
+        if (c.p_shr) launch_kernel(softmax_rows_kernel<VARIANT, NITER, true, true>, grid, threads, 0, st, s, p, rows, n, bias, period, c);
+        else         launch_kernel(softmax_rows_kernel<VARIANT, NITER, true, false>, grid, threads, 0, st, s, p, rows, n, bias, period, c);
     } else {
-        if (c.p_shr) softmax_rows_kernel<VARIANT, NITER, false, true><<<grid, threads, 0, st>>>(s, p, rows, n, bias, period, c);
-        else         softmax_rows_kernel<VARIANT, NITER, false, false><<<grid, threads, 0, st>>>(s, p, rows, n, bias, period, c);
+        if (c.p_shr) launch_kernel(softmax_rows_kernel<VARIANT, NITER, false, true>, grid, threads, 0, st, s, p, rows, n, bias, period, c);
+        else         launch_kernel(softmax_rows_kernel<VARIANT, NITER, false, false>, grid, threads, 0, st, s, p, rows, n, bias, period, c);
     }
     note_launch();
     return last_launch_status();
@@ -121,6 +123,8 @@ template <int VARIANT, bool SAT8>
 __global__ void __launch_bounds__(256)
 gelu_kernel(const int32_t* __restrict__ x, int8_t* __restrict__ y, int64_t n, const GeluDev c)
 {
+    grid_dep_launch();
+    grid_dep_wait();
     const int64_t nvec = n >> 2;                                 // int4 / 4-byte groups
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     const int4* xv = reinterpret_cast<const int4*>(x);
@@ -188,6 +192,7 @@ layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int6
 {
     const int lane = threadIdx.x & 31;
     const int D = c.dim;
+    grid_dep_launch();
     const int words = D >> 2;
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
@@ -207,6 +212,7 @@ layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int6
             if (PTF) sh[k] = __ldg(reinterpret_cast<const unsigned*>(ptf) + wi);
         }
     }
+    grid_dep_wait();                                // gamma / beta above are static; the rows come from the previous kernel
     for (int64_t row = warp; row < rows; row += nwarps) {
         const int* xr = reinterpret_cast<const int*>(x + row * D);
         int w[NW];
@@ -279,11 +285,11 @@ static int launch_ln(const int8_t* x, int8_t* y, int64_t rows, const int32_t* gq
     const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 8);
     const bool sat8 = c.out.qmin == -128 && c.out.qmax == 127;
     if (c.variant == IPTQ_LN_PTF) {
-        if (sat8) layernorm_rows_kernel<NW, true, true><<<grid, threads, 0, st>>>(x, y, rows, gq, bq, ptf, c);
-        else      layernorm_rows_kernel<NW, true, false><<<grid, threads, 0, st>>>(x, y, rows, gq, bq, ptf, c);
+        if (sat8) launch_kernel(layernorm_rows_kernel<NW, true, true>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
+        else      launch_kernel(layernorm_rows_kernel<NW, true, false>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
     } else {
-        if (sat8) layernorm_rows_kernel<NW, false, true><<<grid, threads, 0, st>>>(x, y, rows, gq, bq, ptf, c);
-        else      layernorm_rows_kernel<NW, false, false><<<grid, threads, 0, st>>>(x, y, rows, gq, bq, ptf, c);
+        if (sat8) launch_kernel(layernorm_rows_kernel<NW, false, true>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
+        else      launch_kernel(layernorm_rows_kernel<NW, false, false>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
     }
     note_launch();
     return last_launch_status();
@@ -369,8 +375,8 @@ int iptq_gelu(const int32_t* x, int8_t* y, int64_t n, const iptq_gelu_consts* co
     const bool sat8 = consts->out.qmin == -128 && consts->out.qmax == 127;
 #define IPTQ_GELU_LAUNCH(V)                                                               \
     do {                                                                                  \
-        if (sat8) gelu_kernel<V, true><<<grid, threads, 0, stream>>>(x, y, n, c);         \
-        else      gelu_kernel<V, false><<<grid, threads, 0, stream>>>(x, y, n, c);        \
+        if (sat8) launch_kernel(gelu_kernel<V, true>, grid, threads, 0, stream, x, y, n, c);         \
+        else      launch_kernel(gelu_kernel<V, false>, grid, threads, 0, stream, x, y, n, c);        \
     } while (0)
     switch (consts->variant) {
         case IPTQ_GELU_POLY4: IPTQ_GELU_LAUNCH(IPTQ_GELU_POLY4); break;
