@@ -62,17 +62,23 @@ int make_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint6
 enum { EPI_REQUANT = 0, EPI_RESIDUAL = 1, EPI_GELU = 2 };
 
 constexpr int BM = 128;          // rows per tile = TMEM lanes
-constexpr int BN = 96;           // columns per tile: two accumulators + three per-column constant rows fit 512 TMEM columns
 constexpr int BK = 128;          // bytes of K per stage = one 128-byte swizzle row = 4 MMA k-steps
-constexpr int STAGES = 5;
-constexpr int EPI_PARTS = 3;     // epilogue warps per TMEM lane quadrant; each owns BN / EPI_PARTS columns
-constexpr int EPI_WARPS = 4 * EPI_PARTS;
-constexpr int COLS = BN / EPI_PARTS;                 // 32: bytes per output row per warp, one 32-byte swizzle row
-constexpr int GEMM_THREADS = 32 * (2 + EPI_WARPS);
-static_assert(COLS == 32, "staging addresses below assume 32-byte rows (32-byte TMA swizzle)");
-// TMEM columns: [0, 2 BN) accumulators, then mult, rounding constant, shift -- one row of BN words each,
-// replicated over the 128 lanes so that a thread reads them with the same instruction as its accumulators.
-constexpr uint32_t TM_MULT = 2 * BN, TM_RND = 3 * BN, TM_SHIFT = 4 * BN, TMEM_COLS = 512;
+constexpr int COLS = 32;         // columns per epilogue warp: bytes per output row, one 32-byte swizzle row
+constexpr uint32_t TMEM_COLS = 512;
+
+// Tile width BN is 96 or 128.  TMEM holds two accumulators plus per-column constant rows (one row = BN words,
+// replicated over the 128 lanes so that a thread reads them with the same instruction as its accumulators):
+//   BN =  96: mult, rounding constant, shift           (5 x 96 = 480 columns)
+//   BN = 128: mult, shift - 1; the rounding constant 2^(shift-1) is rebuilt with one shift  (4 x 128 = 512 columns)
+template <int BN>
+struct GemmCfg {
+    static constexpr int STAGES = BN == 96 ? 5 : 4;
+    static constexpr int EPI_PARTS = BN / COLS;          // epilogue warps per TMEM lane quadrant
+    static constexpr int EPI_WARPS = 4 * EPI_PARTS;
+    static constexpr int THREADS = 32 * (2 + EPI_WARPS);
+    static constexpr uint32_t TM_MULT = 2 * BN, TM_RND = 3 * BN, TM_SHIFT = BN == 96 ? 4 * BN : 3 * BN;
+    static constexpr bool HAS_RND = BN == 96;
+};
 
 struct GemmParams {
     int M, N, K;
@@ -84,7 +90,10 @@ struct GemmParams {
     StatusBlock* status;
 };
 
+template <int BN>
 struct GemmSmem {
+    static constexpr int STAGES = GemmCfg<BN>::STAGES;
+    static constexpr int EPI_WARPS = GemmCfg<BN>::EPI_WARPS;
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_BYTES = BN * BK;
     static constexpr int WARP_TILE = 32 * COLS;                                   // bytes of one warp's output block
@@ -107,13 +116,16 @@ __device__ __forceinline__ uint32_t swz32(int row, int chunk) { return (uint32_t
 // One CTA works on ONE column tile (blockIdx.x % num_n_tiles) and walks down its row tiles, so the per-column
 // constants are set up once per CTA: mult / rounding / shift in TMEM, the bias in shared memory, from where the
 // epilogue writes it back into each accumulator it has just drained (the MMAs then always accumulate).
-template <int EPI, int GELU_VARIANT, bool SAT8>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+template <int BN, int EPI, int GELU_VARIANT, bool SAT8>
+__global__ void __launch_bounds__(GemmCfg<BN>::THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_res,
                const GemmParams p)
 {
-    using L = GemmSmem;
+    using L = GemmSmem<BN>;
+    using G = GemmCfg<BN>;
+    constexpr int STAGES = G::STAGES, EPI_WARPS = G::EPI_WARPS;
+    constexpr uint32_t TM_MULT = G::TM_MULT, TM_RND = G::TM_RND, TM_SHIFT = G::TM_SHIFT;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sA = smem + L::OFF_A;
@@ -229,6 +241,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 cm = __ldg(p.mult + n);
                 cr = 1 << (cs - 1);
             }
+            if (!G::HAS_RND) cs -= 1;                         // the shift row holds shift - 1
             sbias[lane] = cb;
             __syncwarp();
             uint32_t v[16];
@@ -237,9 +250,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                 for (int j = 0; j < 16; ++j) v[j] = (uint32_t)__shfl_sync(0xffffffffu, cm, ch * 16 + j);
                 tmem_st16(tlane + TM_MULT + ch * 16, v);
+                if (G::HAS_RND) {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] = (uint32_t)__shfl_sync(0xffffffffu, cr, ch * 16 + j);
-                tmem_st16(tlane + TM_RND + ch * 16, v);
+                    for (int j = 0; j < 16; ++j) v[j] = (uint32_t)__shfl_sync(0xffffffffu, cr, ch * 16 + j);
+                    tmem_st16(tlane + TM_RND + ch * 16, v);
+                }
 #pragma unroll
                 for (int j = 0; j < 16; ++j) v[j] = (uint32_t)__shfl_sync(0xffffffffu, cs, ch * 16 + j);
                 tmem_st16(tlane + TM_SHIFT + ch * 16, v);
@@ -276,10 +291,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t tacc = tlane + (uint32_t)(ab * BN);
 #pragma unroll
             for (int ch = 0; ch < COLS / 16; ++ch) {
-                uint32_t acc[16], cm[16], cr[16], cs[16];
+                uint32_t acc[16], cm[16], cr[G::HAS_RND ? 16 : 1], cs[16];
                 tmem_ld16(tacc + ch * 16, acc);
                 tmem_ld16(tlane + TM_MULT + ch * 16, cm);
-                tmem_ld16(tlane + TM_RND + ch * 16, cr);
+                if constexpr (G::HAS_RND) tmem_ld16(tlane + TM_RND + ch * 16, cr);
                 tmem_ld16(tlane + TM_SHIFT + ch * 16, cs);
                 uint32_t bv[16];
 #pragma unroll
@@ -296,7 +311,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 int o[16];
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
-                    int v = requant_core((int)acc[j], (int)cm[j], (int)cr[j], (int)cs[j]);
+                    int v;
+                    if constexpr (G::HAS_RND) v = requant_core((int)acc[j], (int)cm[j], (int)cr[j], (int)cs[j]);
+                    else v = (mad_hi((int)acc[j], (int)cm[j], 1 << cs[j]) >> cs[j]) >> 1;   // cs = shift - 1
                     if (EPI == EPI_GELU) {
                         v = gelu_core<GELU_VARIANT>(v, p.gelu);
                         v = requant_nosat(v, p.gelu.out);
@@ -383,12 +400,12 @@ struct LinearArgs {
     StatusBlock* status;
 };
 
-template <int EPI, int GV, bool SAT8>
+template <int BN, int EPI, int GV, bool SAT8>
 static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& my, const CUtensorMap& mr,
                        const GemmParams& p, cudaStream_t st)
 {
-    using L = GemmSmem;
-    auto kern = gemm_i8_kernel<EPI, GV, SAT8>;
+    using L = GemmSmem<BN>;
+    auto kern = gemm_i8_kernel<BN, EPI, GV, SAT8>;
     static bool configured[64];               // one attribute call per instantiation and device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return IPTQ_ERR_CUDA;
@@ -400,10 +417,13 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUten
     // every CTA serves one column tile; the SMs are split evenly among the column tiles
     const int per_n = std::max(1, std::min(sm_count() / p.num_n_tiles, p.num_m_tiles));
     const int grid = p.num_n_tiles * per_n;
-    launch_kernel(kern, grid, GEMM_THREADS, L::TOTAL, st, ma, mb, my, mr, p);
+    launch_kernel(kern, grid, GemmCfg<BN>::THREADS, L::TOTAL, st, ma, mb, my, mr, p);
     note_launch();
     return last_launch_status();
 }
+
+template <int BN>
+static int linear_launch_bn(const LinearArgs& a, cudaStream_t st);
 
 int linear_launch(const LinearArgs& a, cudaStream_t st)
 {
@@ -421,7 +441,15 @@ int linear_launch(const LinearArgs& a, cudaStream_t st)
     }
     if (!a.status) return IPTQ_ERR_WORKSPACE;
     if (a.M == 0) return IPTQ_OK;
+    // 128-wide tiles use the tensor core fully and re-read the activations less often, but rebuild the rounding
+    // constant per output (two more instructions); measured, they win only for the plain epilogue at small K
+    const bool wide = a.N % 128 == 0 && (a.N % 96 != 0 || (!a.gelu && !a.residual && a.K <= 768));
+    return wide ? linear_launch_bn<128>(a, st) : linear_launch_bn<96>(a, st);
+}
 
+template <int BN>
+static int linear_launch_bn(const LinearArgs& a, cudaStream_t st)
+{
     GemmParams p;
     p.M = (int)a.M; p.N = a.N; p.K = a.K;
     p.num_m_tiles = (int)((a.M + BM - 1) / BM);
@@ -460,8 +488,8 @@ int linear_launch(const LinearArgs& a, cudaStream_t st)
     }
     if (a.gelu) {
         const bool sat8 = a.gelu->out.qmin == -128 && a.gelu->out.qmax == 127;
-#define IPTQ_GEMM_GELU(V) (sat8 ? launch_gemm<EPI_GELU, V, true>(ma, mb, my, mr, p, st) \
-                                : launch_gemm<EPI_GELU, V, false>(ma, mb, my, mr, p, st))
+#define IPTQ_GEMM_GELU(V) (sat8 ? launch_gemm<BN, EPI_GELU, V, true>(ma, mb, my, mr, p, st) \
+                                : launch_gemm<BN, EPI_GELU, V, false>(ma, mb, my, mr, p, st))
         switch (a.gelu->variant) {
             case IPTQ_GELU_POLY4: return IPTQ_GEMM_GELU(IPTQ_GELU_POLY4);
             case IPTQ_GELU_POLY2: return IPTQ_GEMM_GELU(IPTQ_GELU_POLY2);
@@ -469,8 +497,8 @@ int linear_launch(const LinearArgs& a, cudaStream_t st)
         }
 #undef IPTQ_GEMM_GELU
     }
-    if (a.residual) return launch_gemm<EPI_RESIDUAL, 0, true>(ma, mb, my, mr, p, st);
-    return launch_gemm<EPI_REQUANT, 0, true>(ma, mb, my, mr, p, st);
+    if (a.residual) return launch_gemm<BN, EPI_RESIDUAL, 0, true>(ma, mb, my, mr, p, st);
+    return launch_gemm<BN, EPI_REQUANT, 0, true>(ma, mb, my, mr, p, st);
 }
 
 static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }

@@ -145,7 +145,7 @@ gelu_kernel(const int32_t* __restrict__ x, int8_t* __restrict__ y, int64_t n, co
 }
 
 // ------------------------------------------------------------------------------------------------
-// LayerNorm: one warp per row; the row lives in registers as packed int8 words (NW per lane).
+// LayerNorm: a warp takes a few rows at a time; the rows live in registers as packed int8 words (NW per lane).
 // ------------------------------------------------------------------------------------------------
 struct LnDev {
     int variant, dim;
@@ -154,11 +154,16 @@ struct LnDev {
 
 __device__ __forceinline__ unsigned long long isqrt_floor(unsigned long long V)
 {
-    // V < 2^53: start from the fp64 square root and fix the last unit
-    unsigned long long r = (unsigned long long)sqrt((double)V);
-    while (r * r > V) --r;
-    while ((r + 1) * (r + 1) <= V) ++r;
-    return r;
+    // V >= 1.  Estimate from the hardware reciprocal square root (about 22 good bits), then walk to the exact
+    // floor with the remainder e = V - s^2: one or two steps for the 44-bit values of this kernel.
+    const double vd = (double)(long long)V;
+    double y;
+    asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(vd));
+    long long s = (long long)(vd * y);
+    long long e = (long long)V - s * s;
+    while (e < 0) { --s; e += 2 * s + 1; }
+    while (e > 2 * s) { e -= 2 * s + 1; ++s; }
+    return (unsigned long long)s;
 }
 
 // floor(a / b) for integers 0 <= a < 2^53, 1 <= b with a / b * b <= 2^53: the correctly rounded fp64 quotient of
@@ -184,7 +189,9 @@ __device__ __forceinline__ unsigned long long isqrt_variant(unsigned long long V
     return (unsigned long long)r;
 }
 
-template <int NW, bool PTF, bool SAT8>
+// One warp handles RW rows at a time.  The per-row scalar work (variance, integer square root, reciprocal) is the
+// long dependent chain of this kernel; lane r of the warp runs it for row r, so its cost is shared by RW rows.
+template <int NW, int RW, bool PTF, bool SAT8>
 __global__ void __launch_bounds__(256)
 layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int64_t rows,
                       const int32_t* __restrict__ gamma_q, const int32_t* __restrict__ beta_q,
@@ -196,6 +203,7 @@ layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int6
     const int words = D >> 2;
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t groups = (rows + RW - 1) / RW;
     // per-lane channel parameters stay in registers across rows when they fit
     constexpr bool KEEP = NW <= 8;
     int4 g[KEEP ? NW : 1], b[KEEP ? NW : 1];
@@ -213,66 +221,92 @@ layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int6
         }
     }
     grid_dep_wait();                                // gamma / beta above are static; the rows come from the previous kernel
-    for (int64_t row = warp; row < rows; row += nwarps) {
-        const int* xr = reinterpret_cast<const int*>(x + row * D);
-        int w[NW];
-        int s1 = 0;
-        unsigned s2 = 0;
+    for (int64_t grp = warp; grp < groups; grp += nwarps) {
+        const int64_t row0 = grp * RW;
+        int w[RW][NW];
+        int my_s1 = 0;
+        unsigned my_s2 = 0;
 #pragma unroll
-        for (int k = 0; k < NW; ++k) {
-            const int wi = lane + 32 * k;
-            w[k] = wi < words ? __ldcs(xr + wi) : 0;
-            if (!PTF) {
-                s1 = __dp4a(w[k], 0x01010101, s1);
-                s2 = (unsigned)__dp4a(w[k], w[k], (int)s2);
-            } else {
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    const int xv = ((int)(int8_t)(w[k] >> (8 * t))) << ((sh[k] >> (8 * t)) & 3);
-                    s1 += xv;
-                    s2 += (unsigned)(xv * xv);
-                }
-            }
-        }
-        s1 = __reduce_add_sync(kFull, s1);
-        s2 = __reduce_add_sync(kFull, s2);
-        const long long V = (long long)D * (long long)s2 - (long long)s1 * (long long)s1;   // D^2 var, exact
-        const unsigned long long r = isqrt_variant((unsigned long long)V, c.variant);        // D * std
-        const long long F = r ? (long long)floor_div_f64(1099511627776.0, (double)r) : 0;   // floor(2^40 / r)
-        // (u F) >> 30 = hi32(u * 4F) when 4F fits in 32 bits (rows whose D * std exceeds 2^11: all but near-constant rows)
-        const bool narrow = F < (1ll << 29);
-        const int F4 = (int)(F << 2);
-        int* yr = reinterpret_cast<int*>(y + row * D);
-        auto emit = [&](auto narrow_c) {
-            constexpr bool NARROW = decltype(narrow_c)::value;
+        for (int r = 0; r < RW; ++r) {
+            const bool live = row0 + r < rows;
+            const int* xr = reinterpret_cast<const int*>(x + (row0 + (live ? r : 0)) * D);
 #pragma unroll
             for (int k = 0; k < NW; ++k) {
                 const int wi = lane + 32 * k;
-                if (wi < words) {
-                    int4 gg, bb;
-                    if (KEEP) { gg = g[k]; bb = b[k]; }
-                    else {
-                        gg = __ldg(reinterpret_cast<const int4*>(gamma_q) + wi);
-                        bb = __ldg(reinterpret_cast<const int4*>(beta_q) + wi);
-                    }
-                    const int gv[4] = {gg.x, gg.y, gg.z, gg.w};
-                    const int bv[4] = {bb.x, bb.y, bb.z, bb.w};
-                    int o[4];
+                w[r][k] = (live && wi < words) ? __ldcs(xr + wi) : 0;
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < RW; ++r) {
+            int s1 = 0;
+            unsigned s2 = 0;
+#pragma unroll
+            for (int k = 0; k < NW; ++k) {
+                if (!PTF) {
+                    s1 = __dp4a(w[r][k], 0x01010101, s1);
+                    s2 = (unsigned)__dp4a(w[r][k], w[r][k], (int)s2);
+                } else {
 #pragma unroll
                     for (int t = 0; t < 4; ++t) {
-                        int xv = (int)(int8_t)(w[k] >> (8 * t));
-                        if (PTF) xv <<= ((sh[k] >> (8 * t)) & 3);
-                        const int u = D * xv - s1;                               // D (x - mean)
-                        const int nq = NARROW ? __mulhi(u, F4) : (int)(((long long)u * F) >> 30);   // (x - mean) / std, Q10
-                        o[t] = requant_nosat(nq * gv[t] + bv[t], c.out);
-                        if (!SAT8) o[t] = max(c.out.qmin, min(c.out.qmax, o[t]));
+                        const int xv = ((int)(int8_t)(w[r][k] >> (8 * t))) << ((sh[k] >> (8 * t)) & 3);
+                        s1 += xv;
+                        s2 += (unsigned)(xv * xv);
                     }
-                    __stcs(yr + wi, SAT8 ? (int)pack4_sat_s8(o[0], o[1], o[2], o[3]) : (int)pack4_s8(o[0], o[1], o[2], o[3]));
                 }
             }
-        };
-        if (narrow) emit(std::true_type{});
-        else        emit(std::false_type{});
+            s1 = __reduce_add_sync(kFull, s1);
+            s2 = __reduce_add_sync(kFull, s2);
+            if (lane == r) { my_s1 = s1; my_s2 = s2; }
+        }
+        // lane r: statistics of row r (the other lanes run the same instructions on zeros)
+        const long long V = (long long)D * (long long)my_s2 - (long long)my_s1 * (long long)my_s1;   // D^2 var, exact
+        const unsigned long long rt = isqrt_variant((unsigned long long)V, c.variant);                // D * std
+        const long long F = rt ? (long long)floor_div_f64(1099511627776.0, (double)rt) : 0;          // floor(2^40 / rt)
+        // (u F) >> 30 = hi32(u * 4F) when 4F fits in 32 bits (rows whose D * std exceeds 2^11: all but near-constant rows)
+        const int my_narrow = F < (1ll << 29);
+        const int my_F4 = (int)(F << 2);
+#pragma unroll
+        for (int r = 0; r < RW; ++r) {
+            if (row0 + r >= rows) break;                                        // warp-uniform
+            const int s1 = __shfl_sync(kFull, my_s1, r);
+            const int F4 = __shfl_sync(kFull, my_F4, r);
+            const bool narrow = __shfl_sync(kFull, my_narrow, r) != 0;
+            const long long Fr = narrow ? 0 : (((long long)__shfl_sync(kFull, (int)(F >> 32), r) << 32) |
+                                               (unsigned)__shfl_sync(kFull, (int)(unsigned)F, r));
+            int* yr = reinterpret_cast<int*>(y + (row0 + r) * D);
+            auto emit = [&](auto narrow_c) {
+                constexpr bool NARROW = decltype(narrow_c)::value;
+#pragma unroll
+                for (int k = 0; k < NW; ++k) {
+                    const int wi = lane + 32 * k;
+                    if (wi < words) {
+                        int4 gg, bb;
+                        if (KEEP) { gg = g[k]; bb = b[k]; }
+                        else {
+                            gg = __ldg(reinterpret_cast<const int4*>(gamma_q) + wi);
+                            bb = __ldg(reinterpret_cast<const int4*>(beta_q) + wi);
+                        }
+                        const int gv[4] = {gg.x, gg.y, gg.z, gg.w};
+                        const int bv[4] = {bb.x, bb.y, bb.z, bb.w};
+                        const unsigned wk = (unsigned)w[r][k];
+                        int xs[4] = {sext_byte<0>(wk), sext_byte<1>(wk), sext_byte<2>(wk), sext_byte<3>(wk)};
+                        int o[4];
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            int xv = xs[t];
+                            if (PTF) xv <<= ((sh[k] >> (8 * t)) & 3);
+                            const int u = D * xv - s1;                           // D (x - mean)
+                            const int nq = NARROW ? __mulhi(u, F4) : (int)(((long long)u * Fr) >> 30);   // (x - mean) / std, Q10
+                            o[t] = requant_nosat(nq * gv[t] + bv[t], c.out);
+                            if (!SAT8) o[t] = max(c.out.qmin, min(c.out.qmax, o[t]));
+                        }
+                        __stcs(yr + wi, SAT8 ? (int)pack4_sat_s8(o[0], o[1], o[2], o[3]) : (int)pack4_s8(o[0], o[1], o[2], o[3]));
+                    }
+                }
+            };
+            if (narrow) emit(std::true_type{});
+            else        emit(std::false_type{});
+        }
     }
 }
 
@@ -280,16 +314,17 @@ template <int NW>
 static int launch_ln(const int8_t* x, int8_t* y, int64_t rows, const int32_t* gq, const int32_t* bq,
                      const uint8_t* ptf, const LnDev& c, cudaStream_t st)
 {
+    constexpr int RW = NW <= 4 ? 4 : NW <= 8 ? 2 : 1;
     const int threads = 256;
-    const int64_t want = (rows + 7) / 8;
+    const int64_t want = ((rows + RW - 1) / RW + 7) / 8;
     const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 8);
     const bool sat8 = c.out.qmin == -128 && c.out.qmax == 127;
     if (c.variant == IPTQ_LN_PTF) {
-        if (sat8) launch_kernel(layernorm_rows_kernel<NW, true, true>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
-        else      launch_kernel(layernorm_rows_kernel<NW, true, false>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
+        if (sat8) launch_kernel(layernorm_rows_kernel<NW, RW, true, true>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
+        else      launch_kernel(layernorm_rows_kernel<NW, RW, true, false>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
     } else {
-        if (sat8) launch_kernel(layernorm_rows_kernel<NW, false, true>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
-        else      launch_kernel(layernorm_rows_kernel<NW, false, false>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
+        if (sat8) launch_kernel(layernorm_rows_kernel<NW, RW, false, true>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
+        else      launch_kernel(layernorm_rows_kernel<NW, RW, false, false>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
     }
     note_launch();
     return last_launch_status();
