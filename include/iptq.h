@@ -231,6 +231,15 @@ int iptq_mlp_block(const int8_t* x, const void* w1, const int32_t* b1, const int
                    int8_t* y, int64_t M, int D, int Dh, int w_bits, void* ws, size_t ws_bytes,
                    iptq_stream_t stream);
 
+/* ------------------------------------------------------------------ token re-ordering
+ * The Swin models of Sec. 4 run the block on 7x7 windows of a token grid (with a cyclic shift in every other
+ * block) and merge 2x2 patches between stages; the paper does not describe either, so the layout is the usual
+ * one and is expressed as a row gather: dst row i = concatenation over p < parts of src row index[i*parts + p]
+ * (each row_bytes long; index < 0 -> zeros).  src: dev int8 [n_src, row_bytes]; dst: dev int8
+ * [n_dst, parts*row_bytes]; index: dev int32 [n_dst, parts], built on the host; row_bytes % 16 == 0. */
+int iptq_gather_rows(const int8_t* src, int8_t* dst, const int32_t* index, int64_t n_dst, int parts,
+                     int row_bytes, iptq_stream_t stream);
+
 /* ------------------------------------------------------------------ one encoder block
  * LN1 -> QKV GEMM -> fused attention -> proj GEMM (+ residual x) -> LN2 -> fused MLP (+ residual),
  * each layer running the variant its consts name (the per-layer table of Sec. 3.2).

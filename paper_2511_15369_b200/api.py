@@ -106,6 +106,7 @@ def lib():
                                   C.c_int64, C.c_int, C.c_int, _vp, C.c_size_t, _vp]
         L.iptq_linear_w4_static.argtypes = [_vp, _vp, _vp, _vp, _vp, C.c_int32, _vp, C.POINTER(Requant), _vp,
                                             C.c_int64, C.c_int, C.c_int, _vp, _vp]
+        L.iptq_gather_rows.argtypes = [_vp, _vp, _vp, C.c_int64, C.c_int, C.c_int, _vp]
         L.iptq_attention_workspace_bytes.restype = C.c_size_t
         L.iptq_attention_workspace_bytes.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
         L.iptq_attention_block.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, C.c_int, C.c_int, C.c_int, _vp, _vp,
@@ -130,7 +131,7 @@ def exported_symbols():
     """Names declared in include/iptq.h (used by the CPU-side load test)."""
     return ["iptq_requant_prepare", "iptq_channel_requant_prepare", "iptq_softmax_prepare", "iptq_softmax",
             "iptq_gelu_prepare", "iptq_gelu", "iptq_layernorm_prepare", "iptq_layernorm",
-            "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_w4_static", "iptq_attention_workspace_bytes", "iptq_attention_block",
+            "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_attention_workspace_bytes", "iptq_attention_block",
             "iptq_mlp_workspace_bytes", "iptq_mlp_block", "iptq_encoder_block_workspace_bytes",
             "iptq_encoder_block", "iptq_encoder_block_profiled", "iptq_workspace_init", "iptq_check", "iptq_strerror", "iptq_launch_count"]
 
@@ -275,6 +276,16 @@ def linear_w4_static(x, w_packed, bias, mult, shift, out_zp=0, residual=None, re
     _chk(lib().iptq_linear_w4_static(_dp(x), _dp(w_packed), _dp(bias), _dp(mult), _dp(shift), out_zp, _dp(residual),
                                      _ref(residual_rq), _dp(out), M, N, K, status, _stream()),
          "iptq_linear_w4_static")
+    return out
+
+
+def gather_rows(src, index, out=None):
+    """dst row i = concatenation of the src rows index[i, :] (negative -> zeros); src [n_src, C] int8, index [n_dst, parts] int32."""
+    n_dst, parts = index.shape
+    C_ = src.shape[1]
+    if out is None:
+        out = torch.empty((n_dst, parts * C_), dtype=torch.int8, device=src.device)
+    _chk(lib().iptq_gather_rows(_dp(src), _dp(out), _dp(index), n_dst, parts, C_, _stream()), "iptq_gather_rows")
     return out
 
 

@@ -1,0 +1,49 @@
+// Token re-ordering for windowed attention (Swin-style blocks): window partition with cyclic shift and padding,
+// its inverse, and the 2x2 patch merge are all "destination row i = concatenation of some source rows", with the
+// source row numbers in a table built once on the host.  Pure data movement, 16 bytes per thread per step.
+#include <algorithm>
+
+#include "iptq_common.cuh"
+
+namespace iptq {
+
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const int4* __restrict__ src, int4* __restrict__ dst, const int32_t* __restrict__ index,
+                   int64_t n_dst, int parts, int vec_per_part)
+{
+    grid_dep_launch();
+    grid_dep_wait();
+    const int vec_per_row = parts * vec_per_part;
+    const int64_t total = n_dst * vec_per_row;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int64_t row = i / vec_per_row;
+        const int v = (int)(i - row * vec_per_row);
+        const int part = v / vec_per_part;
+        const int s = __ldg(index + row * parts + part);
+        int4 val = make_int4(0, 0, 0, 0);
+        if (s >= 0) val = __ldg(src + (int64_t)s * vec_per_part + (v - part * vec_per_part));
+        dst[i] = val;
+    }
+}
+
+}  // namespace iptq
+
+using namespace iptq;
+
+extern "C" int iptq_gather_rows(const int8_t* src, int8_t* dst, const int32_t* index, int64_t n_dst, int parts,
+                                int row_bytes, iptq_stream_t stream)
+{
+    if (n_dst < 0 || parts < 1 || row_bytes < 16 || (row_bytes & 15)) return IPTQ_ERR_SHAPE;
+    if (n_dst == 0) return IPTQ_OK;
+    if (!src || !dst || !index) return IPTQ_ERR_NULL;
+    if (!aligned16(src) || !aligned16(dst) || (reinterpret_cast<uintptr_t>(index) & 3u)) return IPTQ_ERR_ALIGN;
+    const int vec_per_part = row_bytes / 16;
+    const int64_t total = n_dst * parts * vec_per_part;
+    const int grid = (int)std::min<int64_t>((total + 255) / 256, (int64_t)sm_count() * 16);
+    if (launch_kernel(gather_rows_kernel, grid, 256, 0, stream, reinterpret_cast<const int4*>(src),
+                      reinterpret_cast<int4*>(dst), index, n_dst, parts, vec_per_part) != cudaSuccess)
+        return IPTQ_ERR_CUDA;
+    note_launch();
+    return last_launch_status();
+}

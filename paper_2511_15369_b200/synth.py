@@ -327,3 +327,127 @@ def swin_mask_ids(window: int = 7, shift: int = 3) -> np.ndarray:
         for ew in (0, 1):
             out.append((lab(eh)[:, None] * 2 + lab(ew)[None, :]).reshape(-1))
     return np.stack(out).astype(np.uint8)
+
+
+# ------------------------------------------------------------------ Swin backbone layout (config 4)
+# The tables below are pure index arithmetic (which token goes where); both the CUDA library and the oracle-side
+# composition in the tests consume them.  Conventions (the paper describes none of this): the token grid is padded
+# at the bottom/right to multiples of the window; shifted blocks roll the padded grid by -shift before the
+# partition and back afterwards; tokens of one window attend to each other only if they carry the same label --
+# the 3 x 3 region labels of the rolled grid for shifted blocks, 0 otherwise; padding tokens are zero rows that
+# carry label 255, so no real token ever attends to them.
+
+PAD_LABEL = 255
+
+
+def swin_window_tables(B: int, Hh: int, Ww: int, shift: int, window: int = 7):
+    """Returns (fwd, mask_id, rev, n_windows):
+    fwd     int32 [B*nW*window^2]  source token row of every window-layout row (-1 = padding),
+    mask_id uint8 [B*nW, window^2] attention labels,
+    rev     int32 [B*Hh*Ww]        window-layout row holding every token's result."""
+    Hp = -(-Hh // window) * window
+    Wp = -(-Ww // window) * window
+    nh, nw = Hp // window, Wp // window
+    ii, jj = np.meshgrid(np.arange(Hp), np.arange(Wp), indexing="ij")      # positions in the rolled, padded grid
+    si, sj = (ii + shift) % Hp, (jj + shift) % Wp                          # where each of them comes from
+    real = (si < Hh) & (sj < Ww)
+    src = np.where(real, si * Ww + sj, -1)
+
+    def region(n, size):
+        r = np.zeros(n, dtype=np.int64)
+        if shift:
+            r[size - window:size - shift] = 1
+            r[size - shift:] = 2
+        return r
+    label = region(Hp, Hp)[:, None] * 3 + region(Wp, Wp)[None, :]
+    label = np.where(real, label, PAD_LABEL)
+
+    def to_windows(a):
+        return a.reshape(nh, window, nw, window).transpose(0, 2, 1, 3).reshape(nh * nw, window * window)
+    src_w, lab_w = to_windows(src), to_windows(label)
+    nW = nh * nw
+    fwd = np.empty((B, nW, window * window), dtype=np.int32)
+    for b in range(B):
+        fwd[b] = np.where(src_w >= 0, src_w + b * Hh * Ww, -1)
+    mask_id = np.broadcast_to(lab_w.astype(np.uint8), (B, nW, window * window)).reshape(B * nW, window * window)
+    rev = np.full(B * Hh * Ww, -1, dtype=np.int32)
+    flat = fwd.reshape(-1)
+    rows = np.nonzero(flat >= 0)[0]
+    rev[flat[rows]] = rows.astype(np.int32)
+    assert (rev >= 0).all()
+    return fwd.reshape(-1), mask_id.copy(), rev, nW
+
+
+def swin_merge_table(B: int, Hh: int, Ww: int) -> np.ndarray:
+    """int32 [B*(Hh/2)*(Ww/2), 4]: the four tokens (even/even, odd/even, even/odd, odd/odd rows/columns of a
+    2 x 2 patch) whose channels are concatenated by the patch merge; -1 where an odd grid has no token."""
+    H2, W2 = -(-Hh // 2), -(-Ww // 2)
+    i2, j2 = np.meshgrid(np.arange(H2), np.arange(W2), indexing="ij")
+    out = np.empty((B, H2 * W2, 4), dtype=np.int32)
+    for p, (di, dj) in enumerate(((0, 0), (1, 0), (0, 1), (1, 1))):
+        i, j = 2 * i2 + di, 2 * j2 + dj
+        ok = (i < Hh) & (j < Ww)
+        t = np.where(ok, i * Ww + j, -1).reshape(-1)
+        for b in range(B):
+            out[b, :, p] = np.where(t >= 0, t + b * Hh * Ww, -1)
+    return out.reshape(-1, 4)
+
+
+@dataclass
+class MergeSpec:
+    gamma: np.ndarray       # float32 [4C]
+    beta: np.ndarray        # float32 [4C]
+    ln_out_scale: float
+    w: np.ndarray           # int8 [2C, 4C]
+    ratio: np.ndarray       # fp64 [2C]
+
+
+def make_merge(C: int, seed: int) -> MergeSpec:
+    """Patch-merge layer 4C -> 2C: LayerNorm(4C) then a bias-free linear, scales from an fp64 shadow pass."""
+    g = _rng(seed, 4)
+    xin, _, _, _ = ln_values(256, 4 * C, seed)
+    xq, _ = quantize_sym(xin, 8, np.int8)
+    gamma = g.normal(1.0, 0.1, size=4 * C).astype(np.float32)
+    beta = g.normal(0.0, 0.1, size=4 * C).astype(np.float32)
+    h = layernorm_ref(xq.astype(np.float64), gamma, beta)
+    S_h = float(np.abs(h).max()) / 127.0
+    h = np.clip(np.round(h / S_h), -128, 127) * S_h
+    wf = g.normal(0.0, 0.02, size=(2 * C, 4 * C))
+    wq, Sw = quantize_weight(wf, 8)
+    o = h @ (wq * Sw[:, None]).T
+    S_o = float(np.abs(o).max()) / 127.0
+    return MergeSpec(gamma, beta, S_h, wq, S_h * Sw / S_o)
+
+
+@dataclass
+class SwinSpec:
+    B: int
+    stages: list            # per stage: dict(dim, heads, grid, blocks=[(BlockSpec, shift, fwd, rev, n_rows)], merge=(MergeSpec, table) or None)
+    x: np.ndarray           # int8 [B*H0*W0, C0]
+
+
+def make_swin(B: int = 2, stages=None, seed: int = 0, window: int = 7) -> SwinSpec:
+    """Swin-Tiny-shaped backbone on a B x grid token field: per stage `depth` blocks (odd ones shifted by
+    window // 2) followed, except after the last stage, by a patch merge.  Every block draws its own weights and
+    calibrates its scales on its own synthetic input (see make_block)."""
+    stages = SWIN_T_STAGES if stages is None else stages
+    out = []
+    for si, st in enumerate(stages):
+        Hh, Ww = st["grid"]
+        C, H = st["dim"], st["heads"]
+        blocks = []
+        for d in range(st["depth"]):
+            shift = (window // 2) if d % 2 else 0
+            fwd, mask_id, rev, nW = swin_window_tables(B, Hh, Ww, shift, window)
+            shape = BlockShape("swin s%d b%d" % (si, d), B * nW, window * window, C, H, C // H, 4 * C, True)
+            spec = make_block(shape, seed=seed + 100 * si + d, mask_id=mask_id, calib_images=4)
+            spec.x = None                                   # the block's input comes from the layer before it
+            blocks.append((spec, shift, fwd, rev))
+        merge = None
+        if si + 1 < len(stages):
+            merge = (make_merge(C, seed + 100 * si + 50), swin_merge_table(B, Hh, Ww))
+        out.append(dict(dim=C, heads=H, grid=(Hh, Ww), blocks=blocks, merge=merge))
+    Hh, Ww = stages[0]["grid"]
+    xin, _, _, _ = ln_values(B * Hh * Ww, stages[0]["dim"], seed)
+    x, _ = quantize_sym(xin, 8, np.int8)
+    return SwinSpec(B, out, x)
