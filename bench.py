@@ -322,16 +322,52 @@ def run_ours(args):
     windows.append((t0, time.perf_counter()))
     stage_ms = [statistics.mean(evs[i].elapsed_time(evs[i + 1]) for evs in sets) for i in range(nst)]
 
-    # ---- end to end from pinned host buffers
+    # ---- end to end from pinned host buffers: every step copies its input host -> device, runs the block and copies
+    #      the result device -> host.  Steps are independent, so they are pipelined over three streams with two
+    #      buffer sets: the copies of neighbouring steps overlap the block of the current one.
     xh = torch.from_numpy(spec.x).pin_memory()
-    yh = torch.empty_like(xh).pin_memory()
-    e2e_graph = capture(lambda: blk.run_host(xh, yh, x, y))
-    for _ in range(W):
-        e2e_graph.replay()
-    ms_e2e = timed_loop(e2e_graph.replay, K)
-    total_e2e = max_over_ranks(sum(ms_e2e))
+    yh = [torch.empty_like(xh).pin_memory() for _ in range(2)]
+    xd = [torch.empty_like(x) for _ in range(2)]
+    yd = [torch.empty_like(x) for _ in range(2)]
+    graphs = [capture(lambda i=i: blk(xd[i], yd[i])) for i in range(2)]
+    s_in, s_run, s_out = (torch.cuda.Stream(device=dev) for _ in range(3))
+
+    def e2e_steps(n):
+        ev_in = [None, None]; ev_run = [None, None]; ev_out = [None, None]
+        for k in range(n):
+            i = k & 1
+            with torch.cuda.stream(s_in):
+                if ev_run[i] is not None:
+                    s_in.wait_event(ev_run[i])              # the block two steps back has consumed this input buffer
+                xd[i].copy_(xh, non_blocking=True)
+                ev_in[i] = s_in.record_event()
+            with torch.cuda.stream(s_run):
+                s_run.wait_event(ev_in[i])
+                if ev_out[i] is not None:
+                    s_run.wait_event(ev_out[i])             # ... and its result has left the output buffer
+                graphs[i].replay()
+                ev_run[i] = s_run.record_event()
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_run[i])
+                yh[i].copy_(yd[i], non_blocking=True)
+                ev_out[i] = s_out.record_event()
+        for st_ in (s_in, s_run, s_out):
+            torch.cuda.current_stream().wait_stream(st_)
+
+    e2e_steps(W)
+    barrier()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for st_ in (s_in, s_run, s_out):
+        st_.wait_event(e0)
+    e2e_steps(K)
+    e1.record()
+    barrier()
+    windows.append((t0, time.perf_counter()))
+    total_e2e = max_over_ranks(e0.elapsed_time(e1))
     e2e_value = job_tops(ops, K, world, total_e2e)
-    got_full = yh.numpy().copy()
+    got_full = yh[(K - 1) & 1].numpy().copy()
 
     # ---- stand-alone non-linear kernels on tensors larger than L2
     peaks, peak_kind = measured_peaks()
@@ -393,8 +429,8 @@ def run_ours(args):
                    "variants": "SM_BITEXP, GELU_POLY4, LN_SHIFT", "parallelism": "replicas, batch-sharded, no collective",
                    "cache": "L2 flushed (256 MiB write) before every timed step, outside the event pairs",
                    "launch": "each step is one CUDA-graph replay of the launches iptq_encoder_block() enqueues"},
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(xh.numel()), "d2h_bytes_per_step": int(yh.numel()),
-                "ms_per_step": total_e2e / K},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(xh.numel()), "d2h_bytes_per_step": int(yh[0].numel()),
+                "ms_per_step": total_e2e / K, "pipelining": "input copy, block and output copy of neighbouring steps overlap (3 streams, 2 buffer sets)"},
         "gpu_launches": int(launches),
         "clocks": clocks.summary(windows),
         "roofline": roofline,

@@ -38,14 +38,17 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// One try: the thread may be suspended by the hardware for up to `kSuspendNs` and is woken as soon as the phase
+// completes, so a waiting warp costs a handful of issue slots per wait instead of spinning beside the working warps.
+constexpr uint32_t kSuspendNs = 20000;
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendNs) : "memory");
     return ok != 0;
 }
 
@@ -54,7 +57,7 @@ struct CtaControl {
     volatile int abort;
 };
 
-constexpr uint32_t kWaitSpins = 1u << 22;      // each try_wait already blocks for a hardware time slice
+constexpr uint32_t kWaitSpins = 1u << 18;      // tries; each may block for up to kSuspendNs (seconds in total)
 
 // Bounded wait.  Returns false when the wait ran out or another role already aborted; the first
 // waiter to give up records (where, blockIdx) in the status block.
@@ -63,7 +66,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, CtaCon
 {
     for (uint32_t spin = 0; spin < kWaitSpins; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 255u) == 255u && ctl->abort) return false;
+        if ((spin & 15u) == 15u && ctl->abort) return false;
     }
     ctl->abort = 1;
     if (status && atomicExch(&status->timeout_flag, 1) == 0) {
