@@ -397,10 +397,13 @@ def run_ours(args):
             s["gbs"] = stage_bytes[name] / (t * 1e-3) / 1e9
             s["frac_hbm"] = s["gbs"] / peaks["hbm_gbs"]
         stages.append(s)
+    # DRAM bytes per launch of the kernels of this workload, from the ncu capture summarised in
+    # profiles/encoder_block_kernels_cfg1.md (dram__bytes_read.sum + dram__bytes_write.sum); valid for that kernel version
+    traffic = {"attention": 14.57e6}
     top = max(stages, key=lambda s: s["us"])
     if "tops" in top:
         roofline = {"kernel": top["kernel"], "bound": "tensor", "achieved": top["tops"], "peak": int8_peak,
-                    "unit": "TOP/s", "frac": top["tops"] / int8_peak, "traffic": None,
+                    "unit": "TOP/s", "frac": top["tops"] / int8_peak, "traffic": traffic.get(top["kernel"]),
                     "peak_source": "%s bf16 burst GEMM x %.0f (nominal dense INT8 : bf16 ratio)" % (peak_kind, INT8_OVER_BF16),
                     "ops_per_launch": stage_ops[top["kernel"]], "us_per_launch": top["us"]}
     else:
