@@ -191,7 +191,10 @@ __device__ __forceinline__ unsigned long long isqrt_variant(unsigned long long V
 
 // One warp handles RW rows at a time.  The per-row scalar work (variance, integer square root, reciprocal) is the
 // long dependent chain of this kernel; lane r of the warp runs it for row r, so its cost is shared by RW rows.
-template <int NW, int RW, bool PTF, bool SAT8>
+// EXACT: the row is exactly 32 * NW words, so no lane ever needs a bounds predicate.  ZPF: the output zero point is
+// folded into the rounding constant (c.out.rnd already holds rnd + (zp << shift), c.out.zp is 0).  PREFETCH: the rows
+// of a warp's next group are loaded before the current group is processed (pays off once a warp has several groups).
+template <int NW, int RW, bool PTF, bool SAT8, bool EXACT, bool ZPF, bool PREFETCH>
 __global__ void __launch_bounds__(256)
 layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int64_t rows,
                       const int32_t* __restrict__ gamma_q, const int32_t* __restrict__ beta_q,
@@ -212,7 +215,7 @@ layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int6
     for (int k = 0; k < NW; ++k) {
         const int wi = lane + 32 * k;
         sh[k] = 0;
-        if (wi < words) {
+        if (EXACT || wi < words) {
             if (KEEP) {
                 g[k] = __ldg(reinterpret_cast<const int4*>(gamma_q) + wi);
                 b[k] = __ldg(reinterpret_cast<const int4*>(beta_q) + wi);
@@ -221,21 +224,36 @@ layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int6
         }
     }
     grid_dep_wait();                                // gamma / beta above are static; the rows come from the previous kernel
-    for (int64_t grp = warp; grp < groups; grp += nwarps) {
+    // the rows of the next group are fetched while the current group is processed
+    auto fetch = [&](int64_t grp, int (&dst)[RW][NW]) {
         const int64_t row0 = grp * RW;
-        int w[RW][NW];
-        int my_s1 = 0;
-        unsigned my_s2 = 0;
 #pragma unroll
         for (int r = 0; r < RW; ++r) {
-            const bool live = row0 + r < rows;
-            const int* xr = reinterpret_cast<const int*>(x + (row0 + (live ? r : 0)) * D);
+            const bool live = grp < groups && row0 + r < rows;
+            const int* xr = reinterpret_cast<const int*>(x + (live ? row0 + r : 0) * D);
 #pragma unroll
             for (int k = 0; k < NW; ++k) {
                 const int wi = lane + 32 * k;
-                w[r][k] = (live && wi < words) ? __ldcs(xr + wi) : 0;
+                dst[r][k] = (live && (EXACT || wi < words)) ? __ldcs(xr + wi) : 0;
             }
         }
+    };
+    int wn[PREFETCH ? RW : 1][PREFETCH ? NW : 1];
+    if constexpr (PREFETCH) fetch(warp, wn);
+    for (int64_t grp = warp; grp < groups; grp += nwarps) {
+        const int64_t row0 = grp * RW;
+        int w[RW][NW];
+        if constexpr (PREFETCH) {
+#pragma unroll
+            for (int r = 0; r < RW; ++r)
+#pragma unroll
+                for (int k = 0; k < NW; ++k) w[r][k] = wn[r][k];
+            fetch(grp + nwarps, wn);
+        } else {
+            fetch(grp, w);
+        }
+        int my_s1 = 0;
+        unsigned my_s2 = 0;
 #pragma unroll
         for (int r = 0; r < RW; ++r) {
             int s1 = 0;
@@ -274,33 +292,34 @@ layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int6
             const long long Fr = narrow ? 0 : (((long long)__shfl_sync(kFull, (int)(F >> 32), r) << 32) |
                                                (unsigned)__shfl_sync(kFull, (int)(unsigned)F, r));
             int* yr = reinterpret_cast<int*>(y + (row0 + r) * D);
+            const int om = c.out.mult, ornd = c.out.rnd, osh = c.out.shift, ozp = c.out.zp;
             auto emit = [&](auto narrow_c) {
                 constexpr bool NARROW = decltype(narrow_c)::value;
+                auto elem = [&](int xv, unsigned shw, int t, int gg, int bb) -> int {
+                    if (PTF) xv <<= ((shw >> (8 * t)) & 3);
+                    const int u = D * xv - s1;                                   // D (x - mean)
+                    const int nq = NARROW ? __mulhi(u, F4) : (int)(((long long)u * Fr) >> 30);   // (x - mean) / std, Q10
+                    int o = mad_hi(nq * gg + bb, om, ornd) >> osh;
+                    if (!ZPF) o += ozp;
+                    if (!SAT8) o = max(c.out.qmin, min(c.out.qmax, o));
+                    return o;
+                };
 #pragma unroll
                 for (int k = 0; k < NW; ++k) {
                     const int wi = lane + 32 * k;
-                    if (wi < words) {
+                    if (EXACT || wi < words) {
                         int4 gg, bb;
                         if (KEEP) { gg = g[k]; bb = b[k]; }
                         else {
                             gg = __ldg(reinterpret_cast<const int4*>(gamma_q) + wi);
                             bb = __ldg(reinterpret_cast<const int4*>(beta_q) + wi);
                         }
-                        const int gv[4] = {gg.x, gg.y, gg.z, gg.w};
-                        const int bv[4] = {bb.x, bb.y, bb.z, bb.w};
                         const unsigned wk = (unsigned)w[r][k];
-                        int xs[4] = {sext_byte<0>(wk), sext_byte<1>(wk), sext_byte<2>(wk), sext_byte<3>(wk)};
-                        int o[4];
-#pragma unroll
-                        for (int t = 0; t < 4; ++t) {
-                            int xv = xs[t];
-                            if (PTF) xv <<= ((sh[k] >> (8 * t)) & 3);
-                            const int u = D * xv - s1;                           // D (x - mean)
-                            const int nq = NARROW ? __mulhi(u, F4) : (int)(((long long)u * Fr) >> 30);   // (x - mean) / std, Q10
-                            o[t] = requant_nosat(nq * gv[t] + bv[t], c.out);
-                            if (!SAT8) o[t] = max(c.out.qmin, min(c.out.qmax, o[t]));
-                        }
-                        __stcs(yr + wi, SAT8 ? (int)pack4_sat_s8(o[0], o[1], o[2], o[3]) : (int)pack4_s8(o[0], o[1], o[2], o[3]));
+                        const int o0 = elem(sext_byte<0>(wk), sh[k], 0, gg.x, bb.x);
+                        const int o1 = elem(sext_byte<1>(wk), sh[k], 1, gg.y, bb.y);
+                        const int o2 = elem(sext_byte<2>(wk), sh[k], 2, gg.z, bb.z);
+                        const int o3 = elem(sext_byte<3>(wk), sh[k], 3, gg.w, bb.w);
+                        __stcs(yr + wi, SAT8 ? (int)pack4_sat_s8(o0, o1, o2, o3) : (int)pack4_s8(o0, o1, o2, o3));
                     }
                 }
             };
@@ -312,20 +331,34 @@ layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int6
 
 template <int NW>
 static int launch_ln(const int8_t* x, int8_t* y, int64_t rows, const int32_t* gq, const int32_t* bq,
-                     const uint8_t* ptf, const LnDev& c, cudaStream_t st)
+                     const uint8_t* ptf_in, const LnDev& c, cudaStream_t st)
 {
     constexpr int RW = NW <= 4 ? 4 : NW <= 8 ? 2 : 1;
     const int threads = 256;
     const int64_t want = ((rows + RW - 1) / RW + 7) / 8;
     const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 8);
     const bool sat8 = c.out.qmin == -128 && c.out.qmax == 127;
-    if (c.variant == IPTQ_LN_PTF) {
-        if (sat8) launch_kernel(layernorm_rows_kernel<NW, RW, true, true>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
-        else      launch_kernel(layernorm_rows_kernel<NW, RW, true, false>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
-    } else {
-        if (sat8) launch_kernel(layernorm_rows_kernel<NW, RW, false, true>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
-        else      launch_kernel(layernorm_rows_kernel<NW, RW, false, false>, grid, threads, 0, st, x, y, rows, gq, bq, ptf, c);
-    }
+    const bool exact = c.dim == 128 * NW;
+    // fold the zero point into the rounding constant when the sum stays clear of 32-bit overflow (|hi32| < 2^30)
+    LnDev cc = c;
+    const long long rz = (long long)c.out.rnd + ((long long)c.out.zp << c.out.shift);
+    const bool zpf = rz > -(1ll << 30) && rz < (1ll << 30);
+    if (zpf) { cc.out.rnd = (int)rz; cc.out.zp = 0; }
+    const bool ptf = c.variant == IPTQ_LN_PTF;
+    const bool pf = (rows + RW - 1) / RW >= (int64_t)4 * grid * (threads / 32);     // several groups per warp
+#define IPTQ_LN_GO(P, S8, EX, ZF)                                                                                        \
+    do {                                                                                                                 \
+        if (pf) launch_kernel(layernorm_rows_kernel<NW, RW, P, S8, EX, ZF, true>, grid, threads, 0, st, x, y, rows, gq, bq, ptf_ptr, cc);  \
+        else    launch_kernel(layernorm_rows_kernel<NW, RW, P, S8, EX, ZF, false>, grid, threads, 0, st, x, y, rows, gq, bq, ptf_ptr, cc); \
+    } while (0)
+    const uint8_t* ptf_ptr = ptf_in;
+    if (ptf)                      { if (sat8) IPTQ_LN_GO(true, true, false, false); else IPTQ_LN_GO(true, false, false, false); }
+    else if (!sat8)               { IPTQ_LN_GO(false, false, false, false); }
+    else if (exact && zpf)        { IPTQ_LN_GO(false, true, true, true); }
+    else if (exact)               { IPTQ_LN_GO(false, true, true, false); }
+    else if (zpf)                 { IPTQ_LN_GO(false, true, false, true); }
+    else                          { IPTQ_LN_GO(false, true, false, false); }
+#undef IPTQ_LN_GO
     note_launch();
     return last_launch_status();
 }
