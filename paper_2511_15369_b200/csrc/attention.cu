@@ -1,25 +1,28 @@
 // Fused integer attention: S = Q K^T (tcgen05 INT8 -> int32 in TMEM) -> (+bias, mask) -> integer Softmax of
-// Sec. 3.4 (Eqs. (6)-(15)) computed straight out of TMEM -> uint8 P written to shared memory in the tensor-core
-// operand layout -> O = P V (u8 x s8 -> int32 in TMEM) -> dyadic requant -> int8, heads re-interleaved.
+// Sec. 3.4 (Eqs. (6)-(15)) -> uint8 P written to shared memory in the tensor-core operand layout ->
+// O = P V (u8 x s8 -> int32 in TMEM) -> dyadic requant -> int8, heads re-interleaved.
 // Neither S nor P ever reaches HBM.
 //
 // The integer Softmax cannot be computed "online" (flash style): the floor in Eq. (9) depends on the final row
-// maximum and P depends on floor(2^M / sum) before it multiplies V, so the whole score row stays in TMEM
-// (<= 256 columns) and is swept three times (max; exponentials + sum, written back to TMEM; probabilities).
+// maximum and P depends on floor(2^M / sum) before it multiplies V, so the whole score row is needed at once.
+// A query row (<= 256 scores) is shared by four threads; each pulls its quarter (<= 64 scores) out of TMEM with one
+// batch of loads and keeps it in registers through the three steps (max; exponentials + sum; probabilities), the
+// four exchanging their partial max / sum through shared memory.  S leaves TMEM right after the load, so the MMA
+// warp computes the next item's scores while the Softmax of the current one runs.
 //
 // Work item = (batch, head, 128-row query tile), handed out dynamically (full tiles first) through a counter in
-// the workspace status block.  10 warps per CTA: warp 0 = TMA producer (2-stage ring of Q/K/V tiles), warp 1 = MMA
-// issuer, warps 2..9 = softmax + output.  A query row is shared by two threads (one per half of the columns; a warp
-// may only touch TMEM lanes 32*(warp%4)..), which exchange their partial max / sum through shared memory.
-// Two CTAs fit on an SM so that one CTA's tensor-core / copy latency hides behind the other's integer work.
+// the workspace status block.  One CTA per SM, 18 warps: warp 0 = TMA producer (3-stage ring of Q/K/V tiles),
+// warp 1 = MMA issuer, warps 2..17 = Softmax + output (warp w may only touch TMEM lanes 32*(w%4)..).
+// The output of item k is requantised after the Softmax of item k+1, when its P V product is certainly done.
 #include <algorithm>
 
 #include "tc_common.cuh"
 
 namespace iptq {
 
-constexpr int ATT_THREADS = 320;
-constexpr int ATT_STAGES = 2;
+constexpr int ATT_THREADS = 576;
+constexpr int ATT_SOFTMAX_THREADS = 512;
+constexpr int ATT_STAGES = 3;              // upper bound of the Q/K/V ring depth
 constexpr int kPadScore = -(1 << 30);     // a score this low has exponential 0 for every row maximum below 2^30
 
 struct AttnParams {
@@ -28,8 +31,11 @@ struct AttnParams {
     int items, full_items; // all work items; those of them that are full 128-row tiles (handed out first)
     int npad_s;            // N rounded up to 16: UMMA N of QK^T, TMEM columns of S
     int kpad;              // N rounded up to 32: UMMA K extent of P V
+    int o_col;             // first TMEM column of O
     int q_bytes, k_bytes, v_bytes, stage_bytes;
-    int p_off, xch_off, bar_off;
+    int p_off, p_bytes, xch_off, bar_off;
+    int stages;            // Q/K/V ring depth (3, or 2 when the exponential table needs the room)
+    int lut_off, lut_n;    // exponential table: e(d) for d < lut_n, 0 beyond (lut_n = 0: no table)
     uint32_t tmem_cols;
     const int32_t* bias;   // [H, N, N] or null
     const uint8_t* mask_id;// [B, N] or null
@@ -47,35 +53,41 @@ __device__ __forceinline__ void decode_item(const AttnParams& p, int it, int& bh
     else                   { bh = it - p.full_items; mt = full_per; }
 }
 
-template <int DH, int VARIANT, bool HAS_BIAS, bool HAS_MASK, bool PSHR>
-__global__ void __launch_bounds__(ATT_THREADS, 2)
+// USE_LUT: the integer exponential of Eqs. (7)-(14) depends only on d = max - s, is below 2^16 and vanishes for
+// d >= lut_n (a few times x0); each CTA tabulates it once in shared memory with the same arithmetic and the
+// Softmax step then costs one table read per score instead of some sixteen dependent integer instructions.
+template <int DH, int VARIANT, bool HAS_BIAS, bool HAS_MASK, bool PSHR, bool USE_LUT>
+__global__ void __launch_bounds__(ATT_THREADS, 1)
 attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, const AttnParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* sP = smem + p.p_off;
-    int* xch_max = reinterpret_cast<int*>(smem + p.xch_off);              // [2 parts][128 rows]
-    unsigned* xch_sum = reinterpret_cast<unsigned*>(xch_max + 256);       // [2 parts][128 rows]
+    uint8_t* sP = smem + p.p_off;                                         // two P buffers
+    int* xch_max = reinterpret_cast<int*>(smem + p.xch_off);              // [4 parts][128 rows]
+    unsigned* xch_sum = reinterpret_cast<unsigned*>(xch_max + 512);       // [4 parts][128 rows]
     uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + p.bar_off);   // [ATT_STAGES]
     uint64_t* kv_empty = kv_full + ATT_STAGES;                            // [ATT_STAGES]
     uint64_t* s_full = kv_empty + ATT_STAGES;
-    uint64_t* p_ready = s_full + 1;
-    uint64_t* o_full = p_ready + 1;
-    uint64_t* t_empty = o_full + 1;
-    volatile int* item_of = reinterpret_cast<volatile int*>(t_empty + 1); // [ATT_STAGES] item held by a stage, -1 = stop
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(item_of) + ATT_STAGES);
+    uint64_t* s_empty = s_full + 1;
+    uint64_t* p_ready = s_empty + 1;                                      // [2]
+    uint64_t* o_full = p_ready + 2;
+    uint64_t* o_empty = o_full + 1;
+    volatile int* item_of = reinterpret_cast<volatile int*>(o_empty + 1); // [ATT_STAGES] item held by a stage, -1 = stop
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(item_of) + ATT_STAGES + 1);
     CtaControl* ctl = reinterpret_cast<CtaControl*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < ATT_STAGES; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
+        for (int s = 0; s < p.stages; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
         mbar_init(s_full, 1);
-        mbar_init(p_ready, 256);
+        mbar_init(s_empty, ATT_SOFTMAX_THREADS);
+        mbar_init(&p_ready[0], ATT_SOFTMAX_THREADS);
+        mbar_init(&p_ready[1], ATT_SOFTMAX_THREADS);
         mbar_init(o_full, 1);
-        mbar_init(t_empty, 256);
+        mbar_init(o_empty, ATT_SOFTMAX_THREADS);
         ctl->abort = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_q);
@@ -114,7 +126,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 tma_load_4d(st, &map_q, &kv_full[s], 0, mt * 128, h, b);
                 tma_load_4d(st + p.q_bytes, &map_k, &kv_full[s], 0, 0, h, b);
                 tma_load_4d(st + p.q_bytes + p.k_bytes, &map_v, &kv_full[s], 0, 0, h, b);
-                if (++s == ATT_STAGES) { s = 0; ph ^= 1u; }
+                if (++s == p.stages) { s = 0; ph ^= 1u; }
             }
             // the last CTA to finish re-arms the counters for the next launch that uses this workspace
             __threadfence();
@@ -125,95 +137,121 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------ MMA issuer: S(k), then P V of item k-1
         if (elect_one()) {
             const uint32_t idesc_s = umma_idesc_i8(128, p.npad_s, true, true, false, false);
             const uint32_t idesc_o = umma_idesc_i8(128, DH, false, true, false, true);     // u8 P (K-major) x s8 V (MN-major)
+            const uint32_t tmem_o = tmem_base + (uint32_t)p.o_col;
             int s = 0; uint32_t ph = 0;
-            uint32_t iph = 0;                                  // parity of the per-item barriers
-            for (;; iph ^= 1u) {
-                if (!mbar_wait(t_empty, iph ^ 1u, ctl, p.status, 12)) break;     // previous O has been read
-                if (!mbar_wait(&kv_full[s], ph, ctl, p.status, 13)) break;
-                if (item_of[s] < 0) break;
+            int s_prev = 0;
+            auto issue_pv = [&](int k) -> bool {                // k = item count index of the item whose P is ready
+                if (!mbar_wait(&p_ready[k & 1], (uint32_t)(k >> 1) & 1u, ctl, p.status, 14)) return false;
+                if (!mbar_wait(o_empty, ((uint32_t)k & 1u) ^ 1u, ctl, p.status, 12)) return false;   // previous O has been read
                 tc_fence_after_sync();
-                const uint32_t q_addr = smem_u32(smem + s * p.stage_bytes);
-                const uint32_t k_addr = q_addr + p.q_bytes;
-                const uint32_t v_addr = k_addr + p.k_bytes;
-                // S = Q K^T: both operands K-major with DH-byte rows (DH-byte swizzle, 8-row groups 8*DH apart)
-#pragma unroll
-                for (int k = 0; k < DH / 32; ++k) {
-                    const uint64_t da = umma_smem_desc(q_addr + k * 32, 16, 8 * DH, DH);
-                    const uint64_t db = umma_smem_desc(k_addr + k * 32, 16, 8 * DH, DH);
-                    umma_i8(tmem_base, da, db, idesc_s, k != 0 ? 1u : 0u);
-                }
-                umma_commit(s_full);
-                if (!mbar_wait(p_ready, iph, ctl, p.status, 14)) break;          // P is in shared memory, S is dead
-                tc_fence_after_sync();
-                const uint32_t p_addr = smem_u32(sP);
+                const uint32_t p_addr = smem_u32(sP + (k & 1) * p.p_bytes);
+                const uint32_t v_addr = smem_u32(smem + s_prev * p.stage_bytes) + p.q_bytes + p.k_bytes;
                 for (int ks = 0; ks < p.kpad / 32; ++ks) {
                     // A = P: K-major, 128-byte swizzle, column blocks of 128 keys are 16 KB apart
                     const uint64_t da = umma_smem_desc(p_addr + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, 128);
                     // B = V [keys, DH]: MN-major (DH contiguous), DH-byte swizzle, 8-key groups 8*DH apart
                     const uint64_t db = umma_smem_desc(v_addr + ks * 32 * DH, 8 * DH, 8 * DH, DH);
-                    umma_i8(tmem_base, da, db, idesc_o, ks != 0 ? 1u : 0u);
+                    umma_i8(tmem_o, da, db, idesc_o, ks != 0 ? 1u : 0u);
                 }
-                umma_commit(&kv_empty[s]);                     // the stage may be refilled
+                umma_commit(&kv_empty[s_prev]);                // the stage may be refilled
                 umma_commit(o_full);
-                if (++s == ATT_STAGES) { s = 0; ph ^= 1u; }
+                return true;
+            };
+            int k = 0;
+            for (;; ++k) {
+                if (!mbar_wait(&kv_full[s], ph, ctl, p.status, 13)) break;
+                const bool stop = item_of[s] < 0;
+                if (!stop) {
+                    if (!mbar_wait(s_empty, ((uint32_t)k & 1u) ^ 1u, ctl, p.status, 18)) break;   // S(k-1) is in registers
+                    tc_fence_after_sync();
+                    const uint32_t q_addr = smem_u32(smem + s * p.stage_bytes);
+                    const uint32_t k_addr = q_addr + p.q_bytes;
+                    // S = Q K^T: both operands K-major with DH-byte rows (DH-byte swizzle, 8-row groups 8*DH apart)
+#pragma unroll
+                    for (int kk = 0; kk < DH / 32; ++kk) {
+                        const uint64_t da = umma_smem_desc(q_addr + kk * 32, 16, 8 * DH, DH);
+                        const uint64_t db = umma_smem_desc(k_addr + kk * 32, 16, 8 * DH, DH);
+                        umma_i8(tmem_base, da, db, idesc_s, kk != 0 ? 1u : 0u);
+                    }
+                    umma_commit(s_full);
+                }
+                if (k > 0 && !issue_pv(k - 1)) break;
+                if (stop) break;
+                s_prev = s;
+                if (++s == p.stages) { s = 0; ph ^= 1u; }
             }
         }
     } else {
         // ------------------------------------------------------------ softmax + output warps
         const int quad = warp & 3;                             // TMEM lane quadrant this warp may touch
-        const int part = (warp - 2) >> 2;                      // which half of the columns
+        const int part = (warp - 2) >> 2;                      // which quarter of the columns
         const int rloc = quad * 32 + lane;                     // row inside the 128-row tile
         const uint32_t trow = tmem_base + ((uint32_t)(quad * 32) << 16);
-        const uint32_t p_row = smem_u32(sP) + (uint32_t)((rloc >> 3) * 1024 + (rloc & 7) * 128);
+        const uint32_t p_row0 = smem_u32(sP) + (uint32_t)((rloc >> 3) * 1024 + (rloc & 7) * 128);
         const int HD = p.H * DH;
-        const int chunks = p.npad_s >> 4;
-        const int c_half = (chunks + 1) >> 1;
-        const int cb = part ? c_half : 0, ce = part ? chunks : c_half;   // this thread's 16-column chunks
+        const int chunks = p.npad_s >> 4;                      // 16-column chunks of a row (<= 16)
+        const int cbase = chunks >> 2, crem = chunks & 3;
+        const int nch = cbase + (part < crem ? 1 : 0);         // this thread's chunks (<= 4) ...
+        const int c_begin = part * cbase + min(part, crem);    // ... starting here
         const bool sat8 = p.orq.qmin == -128 && p.orq.qmax == 127;
         int s = 0; uint32_t ph = 0;
-        uint32_t iph = 0;
+        uint16_t* lut = reinterpret_cast<uint16_t*>(smem + p.lut_off);
+        const uint32_t lut_addr = smem_u32(lut);
+        if (USE_LUT) {
+            for (int d = (int)threadIdx.x - 64; d <= p.lut_n; d += ATT_SOFTMAX_THREADS)
+                lut[d] = d < p.lut_n ? (uint16_t)exp_core_nd<VARIANT>(-d, p.ex) : (uint16_t)0;
+            named_barrier(5, ATT_SOFTMAX_THREADS);              // the table is complete before anyone reads it
+        }
         grid_dep_wait();                                       // output rows are written only after this
 
-        auto sweep_single = [&](auto&& body) {      // for the arithmetic-heavy sweep: one buffer, fewer live registers
-            uint32_t ra[16];
-#pragma unroll 1
-            for (int c = cb; c < ce; ++c) {
-                tmem_ld16(trow + c * 16, ra);
+        // requantises and stores this thread's share of the output tile of item (b, h, mt), count index k
+        auto epilogue = [&](int k, int b, int h, int mt) -> bool {
+            if (!mbar_wait(o_full, (uint32_t)k & 1u, ctl, p.status, 16)) return false;
+            tc_fence_after_sync();
+            const int row = mt * 128 + rloc;
+            constexpr int OPARTS = DH / 16;                    // threads of a row that hold 16 output columns each
+            if (mt * 128 + quad * 32 < p.N && part < OPARTS) {
+                uint32_t r[16];
+                tmem_ld16(trow + (uint32_t)(p.o_col + part * 16), r);
                 tmem_wait_ld();
-                body(ra, c);
-            }
-        };
-        // Runs `body(values, chunk)` over this thread's chunks with the TMEM load of the next chunk in flight.
-        auto sweep = [&](auto&& body) {
-            uint32_t ra[16], rb[16];
-            if (cb < ce) tmem_ld16(trow + cb * 16, ra);
-#pragma unroll 1
-            for (int c = cb; c < ce; c += 2) {
-                tmem_wait_ld();
-                if (c + 1 < ce) tmem_ld16(trow + (c + 1) * 16, rb);
-                body(ra, c);
-                if (c + 1 < ce) {
-                    tmem_wait_ld();
-                    if (c + 2 < ce) tmem_ld16(trow + (c + 2) * 16, ra);
-                    body(rb, c + 1);
+                int o[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    o[j] = requant_nosat((int)r[j], p.orq);
+                    if (!sat8) o[j] = max(p.orq.qmin, min(p.orq.qmax, o[j]));
+                }
+                if (row < p.N) {
+                    int4 pk;
+                    pk.x = (int)pack4_sat_s8(o[0], o[1], o[2], o[3]);
+                    pk.y = (int)pack4_sat_s8(o[4], o[5], o[6], o[7]);
+                    pk.z = (int)pack4_sat_s8(o[8], o[9], o[10], o[11]);
+                    pk.w = (int)pack4_sat_s8(o[12], o[13], o[14], o[15]);
+                    *reinterpret_cast<int4*>(p.out + ((size_t)b * p.N + row) * HD + h * DH + part * 16) = pk;
                 }
             }
+            tc_fence_before_sync();
+            mbar_arrive(o_empty);
+            return true;
         };
 
-        for (;; iph ^= 1u) {
-            // the partner warp of this quadrant meets this one at two named barriers per item: a warp that gives up
-            // before them arrives without waiting, so that a bounded wait running out can never strand the partner
+        int k = 0;
+        int pb = 0, phd = 0, pmt = 0;                          // item whose output is still to be written
+        bool ok = true;
+        for (;; ++k) {
+            // the four warps of a quadrant meet at two named barriers per item: a warp that gives up before them
+            // arrives without waiting, so that a bounded wait running out can never strand the others
             if (!mbar_wait(&kv_full[s], ph, ctl, p.status, 17)) {   // acquire: the item number is visible
-                named_barrier_arrive(1 + quad, 64); named_barrier_arrive(1 + quad, 64);
+                named_barrier_arrive(1 + quad, 128); named_barrier_arrive(1 + quad, 128);
+                ok = false;
                 break;
             }
             const int it = item_of[s];
             if (it < 0) break;
-            if (++s == ATT_STAGES) { s = 0; ph ^= 1u; }
+            if (++s == p.stages) { s = 0; ph ^= 1u; }
             int bh, mt;
             decode_item(p, it, bh, mt);
             const int h = bh % p.H, b = bh / p.H;
@@ -223,117 +261,109 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const int32_t* brow = HAS_BIAS ? p.bias + ((size_t)h * p.N + (valid ? row : 0)) * p.N : nullptr;
             const uint8_t* mrow = HAS_MASK ? p.mask_id + (size_t)b * p.N : nullptr;
             const unsigned my_id = HAS_MASK ? mrow[valid ? row : 0] : 0u;
+            const uint32_t p_row = p_row0 + (uint32_t)((k & 1) * p.p_bytes);
 
-            if (!mbar_wait(s_full, iph, ctl, p.status, 15)) {
-                named_barrier_arrive(1 + quad, 64); named_barrier_arrive(1 + quad, 64);
+            if (!mbar_wait(s_full, (uint32_t)k & 1u, ctl, p.status, 15)) {
+                named_barrier_arrive(1 + quad, 128); named_barrier_arrive(1 + quad, 128);
+                ok = false;
                 break;
             }
             tc_fence_after_sync();
+            // ---- this thread's quarter of the score row, TMEM -> registers, in one batch
+            uint32_t v[4][16];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (warp_rows && i < nch) tmem_ld16(trow + (uint32_t)((c_begin + i) * 16), v[i]);
+            tmem_wait_ld();
+            tc_fence_before_sync();
+            mbar_arrive(s_empty);                              // the MMA warp may overwrite S with the next item's scores
             if (warp_rows) {
-                // ---- sweep 1: row maximum over the real, unmasked columns (Eq. (6)).  Chunks that hold padding,
-                //      masked pairs or a bias are rewritten in TMEM (pad / masked -> kPadScore, score + bias) so
-                //      that the next sweep needs no per-element case analysis.
+                // ---- row maximum over the real, unmasked columns (Eq. (6)); padding and masked pairs become
+                //      kPadScore, a bias is added in place, so that the next step needs no case analysis
                 int mx = INT_MIN;
-                sweep([&](uint32_t (&v)[16], int c) {
-                    const int c0 = c * 16;
-                    if (HAS_BIAS || HAS_MASK || c0 + 16 > p.N) {              // warp-uniform
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (i < nch) {
+                        const int c0 = (c_begin + i) * 16;
+                        if (HAS_BIAS || HAS_MASK || c0 + 16 > p.N) {          // warp-uniform
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const int col = c0 + j;
+                                int sc = (int)v[i][j];
+                                bool use = col < p.N;
+                                if (HAS_BIAS && use) sc += __ldg(brow + col);
+                                if (HAS_MASK && use) use = (mrow[col] == my_id);
+                                v[i][j] = (uint32_t)(use ? sc : kPadScore);
+                            }
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) mx = max(mx, (int)v[i][j]);
+                    }
+                }
+                xch_max[part * 128 + rloc] = mx;
+                named_barrier(1 + quad, 128);
+                mx = max(max(xch_max[rloc], xch_max[128 + rloc]), max(xch_max[256 + rloc], xch_max[384 + rloc]));
+                // ---- integer exponentials (Eqs. (7)-(14)), in place, and their sum
+                unsigned sum = 0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (i < nch) {
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
-                            const int col = c0 + j;
-                            int sc = (int)v[j];
-                            bool use = col < p.N;
-                            if (HAS_BIAS && use) sc += __ldg(brow + col);
-                            if (HAS_MASK && use) use = (mrow[col] == my_id);
-                            v[j] = (uint32_t)(use ? sc : kPadScore);
+                            unsigned e;
+                            if (USE_LUT) {
+                                const unsigned d = min((unsigned)(mx - (int)v[i][j]), (unsigned)p.lut_n);
+                                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(e) : "r"(lut_addr + 2u * d));
+                            } else {
+                                e = exp_core_nd<VARIANT>((int)v[i][j] - mx, p.ex);
+                            }
+                            sum += e;
+                            v[i][j] = e;
                         }
-                        tmem_st16(trow + c0, v);
                     }
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) mx = max(mx, (int)v[j]);
-                });
-                xch_max[part * 128 + rloc] = mx;
-                tmem_wait_st();
-                named_barrier(1 + quad, 64);
-                mx = max(xch_max[rloc], xch_max[128 + rloc]);
-                // ---- sweep 2: integer exponentials (Eqs. (7)-(14)) and their sum; e goes back to TMEM
-                unsigned sum = 0;
-                sweep_single([&](uint32_t (&v)[16], int c) {
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const unsigned e = exp_core_nd<VARIANT>((int)v[j] - mx, p.ex);
-                        sum += e;
-                        v[j] = e;
-                    }
-                    tmem_st16(trow + c * 16, v);
-                });
+                }
                 xch_sum[part * 128 + rloc] = sum;
-                tmem_wait_st();
-                named_barrier(1 + quad, 64);
-                sum = xch_sum[rloc] + xch_sum[128 + rloc];
-                // ---- sweep 3: IntDiv (Eq. (15)) -> uint8 probabilities in the UMMA A-operand layout
+                named_barrier(1 + quad, 128);
+                sum = (xch_sum[rloc] + xch_sum[128 + rloc]) + (xch_sum[256 + rloc] + xch_sum[384 + rloc]);
+                // ---- IntDiv (Eq. (15)) -> uint8 probabilities in the UMMA A-operand layout
                 const unsigned f = intdiv_factor(sum, p.M) << p.f_shl;
-                sweep([&](uint32_t (&v)[16], int c) {
-                    uint32_t w[4];
 #pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        int pv[4];
+                for (int i = 0; i < 4; ++i) {
+                    if (i < nch) {
+                        uint32_t w[4];
 #pragma unroll
-                        for (int t = 0; t < 4; ++t) {
-                            unsigned x = __umulhi(f, v[q4 * 4 + t]);
-                            if (PSHR) x >>= p.p_shr;
-                            pv[t] = (int)x;
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            int pv[4];
+#pragma unroll
+                            for (int t = 0; t < 4; ++t) {
+                                unsigned x = __umulhi(f, v[i][q4 * 4 + t]);
+                                if (PSHR) x >>= p.p_shr;
+                                pv[t] = (int)x;
+                            }
+                            w[q4] = pack4_sat_u8(pv[0], pv[1], pv[2], pv[3]);      // values are <= 2^(b-1): nothing saturates
                         }
-                        w[q4] = pack4_sat_u8(pv[0], pv[1], pv[2], pv[3]);          // values are <= 2^(b-1): nothing saturates
+                        const int c0 = (c_begin + i) * 16;
+                        const int chunk = (c0 & 127) >> 4;
+                        st_shared_v4(p_row + (uint32_t)((c0 >> 7) * 16384 + ((chunk ^ (rloc & 7)) << 4)), w[0], w[1], w[2], w[3]);
                     }
-                    const int c0 = c * 16;
-                    const int chunk = (c0 & 127) >> 4;
-                    st_shared_v4(p_row + (uint32_t)((c0 >> 7) * 16384 + ((chunk ^ (rloc & 7)) << 4)), w[0], w[1], w[2], w[3]);
-                });
+                }
             } else {
-                named_barrier_arrive(1 + quad, 64); named_barrier_arrive(1 + quad, 64);   // keeps the barrier generations aligned
+                named_barrier_arrive(1 + quad, 128); named_barrier_arrive(1 + quad, 128);   // keeps the barrier generations aligned
             }
             // key columns between npad_s and kpad (at most one 16-column chunk) meet zero rows of V, but the bytes
             // the tensor core reads there must be defined
-            if (part == 1 && p.kpad > p.npad_s) {
+            if (part == 3 && p.kpad > p.npad_s) {
                 const int c0 = p.npad_s;
                 const int chunk = (c0 & 127) >> 4;
                 st_shared_v4(p_row + (uint32_t)((c0 >> 7) * 16384 + ((chunk ^ (rloc & 7)) << 4)), 0u, 0u, 0u, 0u);
             }
             fence_proxy_async_smem();            // generic-proxy stores -> visible to the tensor core's reads
-            tc_fence_before_sync();
-            mbar_arrive(p_ready);
-
-            // ---- output: O = P V from TMEM -> requant -> int8 (each half of the threads takes half of the columns)
-            if (!mbar_wait(o_full, iph, ctl, p.status, 16)) break;
-            tc_fence_after_sync();
-            if (warp_rows) {
-                int8_t* orow = p.out + ((size_t)b * p.N + (valid ? row : 0)) * HD + h * DH;
-                constexpr int OC = DH / 32;                    // 16-column chunks per thread
-#pragma unroll
-                for (int cc = 0; cc < OC; ++cc) {
-                    const int c0 = (part * OC + cc) * 16;
-                    uint32_t r[16];
-                    tmem_ld16(trow + c0, r);
-                    tmem_wait_ld();
-                    int o[16];
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        o[j] = requant_nosat((int)r[j], p.orq);
-                        if (!sat8) o[j] = max(p.orq.qmin, min(p.orq.qmax, o[j]));
-                    }
-                    if (valid) {
-                        int4 pk;
-                        pk.x = (int)pack4_sat_s8(o[0], o[1], o[2], o[3]);
-                        pk.y = (int)pack4_sat_s8(o[4], o[5], o[6], o[7]);
-                        pk.z = (int)pack4_sat_s8(o[8], o[9], o[10], o[11]);
-                        pk.w = (int)pack4_sat_s8(o[12], o[13], o[14], o[15]);
-                        *reinterpret_cast<int4*>(orow + c0) = pk;
-                    }
-                }
-            }
-            tc_fence_before_sync();
-            mbar_arrive(t_empty);
+            mbar_arrive(&p_ready[k & 1]);
+            // ---- output of the previous item: its P V product was issued right after that item's Softmax
+            if (k > 0 && !epilogue(k - 1, pb, phd, pmt)) { ok = false; break; }
+            pb = b; phd = h; pmt = mt;
         }
+        if (ok && k > 0) epilogue(k - 1, pb, phd, pmt);
     }
 
     // ------------------------------------------------------------ teardown (also reached after an abort)
@@ -366,12 +396,12 @@ template <int DH, int VARIANT>
 static int launch_attn(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const AttnParams& p,
                        int smem_bytes, cudaStream_t st)
 {
-    const int grid = std::min(p.items, 2 * sm_count());
+    const int grid = std::min(p.items, sm_count());
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return IPTQ_ERR_CUDA;
-#define IPTQ_ATT_LAUNCH2(HB, HM, PS)                                                                              \
+#define IPTQ_ATT_LAUNCH3(HB, HM, PS, LT)                                                                          \
     do {                                                                                                          \
-        auto kern = attention_kernel<DH, VARIANT, HB, HM, PS>;                                                    \
+        auto kern = attention_kernel<DH, VARIANT, HB, HM, PS, LT>;                                                \
         static int configured[64];          /* largest dynamic shared memory size set so far, per device */     \
         if (configured[dev] < smem_bytes) {                                                                       \
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) \
@@ -379,6 +409,10 @@ static int launch_attn(const CUtensorMap& mq, const CUtensorMap& mk, const CUten
             configured[dev] = smem_bytes;                                                                         \
         }                                                                                                         \
         launch_kernel(kern, grid, ATT_THREADS, smem_bytes, st, mq, mk, mv, p);                                               \
+    } while (0)
+#define IPTQ_ATT_LAUNCH2(HB, HM, PS)                                                                              \
+    do {                                                                                                          \
+        if (p.lut_n) IPTQ_ATT_LAUNCH3(HB, HM, PS, true); else IPTQ_ATT_LAUNCH3(HB, HM, PS, false);                \
     } while (0)
 #define IPTQ_ATT_LAUNCH(HB, HM)                                                                                   \
     do {                                                                                                          \
@@ -390,6 +424,7 @@ static int launch_attn(const CUtensorMap& mq, const CUtensorMap& mk, const CUten
     else IPTQ_ATT_LAUNCH(false, false);
 #undef IPTQ_ATT_LAUNCH
 #undef IPTQ_ATT_LAUNCH2
+#undef IPTQ_ATT_LAUNCH3
     note_launch();
     return last_launch_status();
 }
@@ -437,13 +472,31 @@ int attention_launch(const AttnArgs& a, cudaStream_t st)
     p.k_bytes = up1k(p.npad_s * a.dh);
     p.v_bytes = up1k(p.kpad * a.dh);
     p.stage_bytes = p.q_bytes + p.k_bytes + p.v_bytes;
-    p.p_off = ATT_STAGES * p.stage_bytes;
-    const int p_bytes = ((p.kpad + 127) / 128) * 16384;
-    p.xch_off = p.p_off + p_bytes;
-    p.bar_off = p.xch_off + 2 * 2 * 128 * 4;
-    const int smem_bytes = p.bar_off + 128 + 1024;
+    p.p_bytes = ((p.kpad + 127) / 128) * 16384;
+    // Exponential table (shift-based variants with values below 2^16): e(d) = 0 once -Q_p >= qz * x0, where qz is the
+    // bit length of the largest value x0 << nsh; -Q_p >= 23 (d >> 4) puts that at d >= 16 qz x0 / 23 + 15.
+    p.lut_n = 0;
+    p.stages = ATT_STAGES;
+    const int fixed = 2 * p.p_bytes + 2 * 4 * 128 * 4 + 256 + 1024;
+    if (a.sm->variant != IPTQ_SM_POLY) {
+        int qz = 0;
+        for (int64_t u = (int64_t)a.sm->x0 << a.sm->nsh; u; u >>= 1) ++qz;
+        const int64_t n = (16 * (int64_t)qz * a.sm->x0) / 23 + 32;
+        const int64_t bytes = (2 * (n + 1) + 255) & ~(int64_t)255;
+        if (qz <= 16) {
+            if (fixed + 3 * p.stage_bytes + bytes <= 227 * 1024) { p.lut_n = (int)n; }
+            else if (fixed + 2 * p.stage_bytes + bytes <= 227 * 1024) { p.lut_n = (int)n; p.stages = 2; }
+        }
+    }
+    const int lut_bytes = p.lut_n ? (int)((2 * ((int64_t)p.lut_n + 1) + 255) & ~255) : 0;
+    p.p_off = p.stages * p.stage_bytes;
+    p.xch_off = p.p_off + 2 * p.p_bytes;
+    p.lut_off = p.xch_off + 2 * 4 * 128 * 4;
+    p.bar_off = p.lut_off + lut_bytes;
+    const int smem_bytes = p.bar_off + 256 + 1024;
+    p.o_col = (p.npad_s + 31) & ~31;                     // O sits behind S in TMEM
     p.tmem_cols = 32;
-    while ((int)p.tmem_cols < std::max(p.npad_s, a.dh)) p.tmem_cols <<= 1;
+    while ((int)p.tmem_cols < p.o_col + a.dh) p.tmem_cols <<= 1;
     p.bias = a.bias; p.mask_id = a.mask_id; p.out = a.out;
     p.ex = to_dev_exp(*a.sm);
     p.M = a.sm->M; p.f_shl = a.sm->f_shl; p.p_shr = a.sm->p_shr;
