@@ -30,31 +30,22 @@ softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ pr
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
     grid_dep_launch();
     grid_dep_wait();
-    const bool tight = n > 32 * (NITER - 1);        // every 32-column step but the last is full (uniform)
-    // the scores of the warp's next row are fetched while the current row is processed
-    auto fetch = [&](int64_t row, int (&dst)[NITER]) {
-        const bool live = row < rows;
-        const int32_t* sr = scores + (live ? row : 0) * n;
-        const int32_t* br = HAS_BIAS ? bias + ((live ? row : 0) % bias_period) * n : nullptr;
+    for (int64_t row = warp; row < rows; row += nwarps) {
+        const int32_t* sr = scores + row * n;
+        const int32_t* br = HAS_BIAS ? bias + (row % bias_period) * n : nullptr;
+        int v[NITER];
+        int mx = INT_MIN;
 #pragma unroll
         for (int k = 0; k < NITER; ++k) {
             const int j = lane + 32 * k;
             int s = kPadScore;
-            if (live && ((tight && k + 1 < NITER) || j < n)) {   // only the last 32-column step can be ragged
+            if (j < n) {
                 s = __ldcs(sr + j);
                 if (HAS_BIAS) s += __ldg(br + j);
             }
-            dst[k] = s;
+            v[k] = s;
+            mx = max(mx, s);
         }
-    };
-    int vn[NITER];
-    fetch(warp, vn);
-    for (int64_t row = warp; row < rows; row += nwarps) {
-        int v[NITER];
-        int mx = INT_MIN;
-#pragma unroll
-        for (int k = 0; k < NITER; ++k) { v[k] = vn[k]; mx = max(mx, v[k]); }
-        fetch(row + nwarps, vn);
         mx = __reduce_max_sync(kFull, mx);                      // Eq. (6)
         unsigned sum = 0;
 #pragma unroll
@@ -71,7 +62,7 @@ softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ pr
             const int j = lane + 32 * k;
             unsigned pv = __umulhi(f, (unsigned)v[k]);
             if (PSHR) pv >>= c.p_shr;
-            if ((tight && k + 1 < NITER) || j < n) __stcs(pr + j, (uint8_t)pv);
+            if (j < n) __stcs(pr + j, (uint8_t)pv);
         }
     }
 }
