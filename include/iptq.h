@@ -125,7 +125,17 @@ typedef struct {
     int32_t x0, nsh, dcap;                   /* IPTQ_GELU_SHIFT only */
     uint32_t div_mul; int32_t div_shift;     /* IPTQ_GELU_SHIFT only: division by x0 */
     iptq_requant out;
+    const int8_t* table;                     /* optional: dev, IPTQ_GELU_TABLE_SIZE bytes from iptq_gelu_table(); NULL = none */
 } iptq_gelu_consts;
+
+/* The integer GELU maps an in_bits-bit input (<= 16 bits) to 8 bits, so the whole function fits a 64 KB table:
+ * table[x + 32768] = the value iptq_gelu() returns for x (x below/above the in_bits range is clamped first, as
+ * in the kernel).  iptq_gelu_table() fills such a table with the same arithmetic; when consts->table points to it,
+ * the FC1 epilogue of iptq_mlp_block() / iptq_encoder_block() keeps a copy in shared memory and replaces the
+ * polynomial by one read per output.  The results are identical with and without the table.
+ * table: dev int8 [IPTQ_GELU_TABLE_SIZE], 16-byte aligned, caller-owned; consts: host (its own `table` is ignored). */
+#define IPTQ_GELU_TABLE_SIZE 65536
+int iptq_gelu_table(const iptq_gelu_consts* consts, int8_t* table, iptq_stream_t stream);
 
 /* host.  in_bits in [8, 16], out_bits in [4, 8]; floor(|b| / S') must be in [1, 2^15). */
 int iptq_gelu_prepare(double in_scale, int in_bits, double out_scale, int out_zp, int out_bits,

@@ -36,7 +36,7 @@ class SoftmaxConsts(C.Structure):
 
 class GeluConsts(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("variant", "in_bits", "Bq", "sh2", "C", "gs", "x0", "nsh", "dcap")] + \
-               [("div_mul", C.c_uint32), ("div_shift", C.c_int32), ("out", Requant)]
+               [("div_mul", C.c_uint32), ("div_shift", C.c_int32), ("out", Requant), ("table", C.c_void_p)]
 
 
 class LnConsts(C.Structure):
@@ -97,6 +97,7 @@ def lib():
         L.iptq_gelu_prepare.argtypes = [C.c_double, C.c_int, C.c_double, C.c_int, C.c_int, C.c_int,
                                         C.POINTER(GeluConsts)]
         L.iptq_gelu.argtypes = [_vp, _vp, C.c_int64, C.POINTER(GeluConsts), _vp]
+        L.iptq_gelu_table.argtypes = [C.POINTER(GeluConsts), _vp, _vp]
         L.iptq_layernorm_prepare.argtypes = [C.c_int, _vp, _vp, C.c_double, C.c_int, C.c_int, C.c_int, _vp, _vp,
                                              C.POINTER(LnConsts)]
         L.iptq_layernorm.argtypes = [_vp, _vp, C.c_int64, C.c_int, _vp, _vp, _vp, C.POINTER(LnConsts), _vp]
@@ -130,7 +131,7 @@ def lib():
 def exported_symbols():
     """Names declared in include/iptq.h (used by the CPU-side load test)."""
     return ["iptq_requant_prepare", "iptq_channel_requant_prepare", "iptq_softmax_prepare", "iptq_softmax",
-            "iptq_gelu_prepare", "iptq_gelu", "iptq_layernorm_prepare", "iptq_layernorm",
+            "iptq_gelu_prepare", "iptq_gelu", "iptq_gelu_table", "iptq_layernorm_prepare", "iptq_layernorm",
             "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_attention_workspace_bytes", "iptq_attention_block",
             "iptq_mlp_workspace_bytes", "iptq_mlp_block", "iptq_encoder_block_workspace_bytes",
             "iptq_encoder_block", "iptq_encoder_block_profiled", "iptq_workspace_init", "iptq_check", "iptq_strerror", "iptq_launch_count"]
@@ -238,6 +239,19 @@ def gelu(x, consts: GeluConsts, out=None):
     return out
 
 
+GELU_TABLE_SIZE = 65536
+
+
+def gelu_table(consts: GeluConsts, device="cuda"):
+    """Tabulates the integer GELU of ``consts`` over all 16-bit inputs on the device and attaches the table to
+    ``consts`` (the FC1 epilogue then reads it instead of evaluating the polynomial).  Returns the table tensor,
+    which the caller must keep alive as long as ``consts`` is used."""
+    t = torch.empty(GELU_TABLE_SIZE, dtype=torch.int8, device=device)
+    _chk(lib().iptq_gelu_table(C.byref(consts), _dp(t), _stream()), "iptq_gelu_table")
+    consts.table = t.data_ptr()
+    return t
+
+
 def layernorm(x, gamma_q, beta_q, consts: LnConsts, ptf_shift=None, out=None):
     rows, dim = x.shape
     if out is None:
@@ -323,7 +337,7 @@ class EncoderBlock:
     """Device-resident parameters of one integer encoder block, prepared from a ``synth.BlockSpec``
     (or any object with the same fields) with the library's own ``*_prepare`` functions."""
 
-    def __init__(self, spec, table=(SM_BITEXP, GELU_POLY4, LN_SHIFT, LN_SHIFT), device="cuda"):
+    def __init__(self, spec, table=(SM_BITEXP, GELU_POLY4, LN_SHIFT, LN_SHIFT), device="cuda", gelu_table_on=True):
         sh = spec.shape
         self.shape = sh
         self.keep = []          # host structs and device tensors referenced by raw pointers
@@ -363,7 +377,10 @@ class EncoderBlock:
         p.res1_rq = host(requant_prepare(spec.proj.res_ratio / 65536.0, zp=spec.proj.res_zp))
         p.res2_rq = host(requant_prepare(spec.fc2.res_ratio / 65536.0, zp=spec.fc2.res_zp))
         gl = spec.gelu
-        p.gelu = host(gelu_prepare(gl["in_scale"], gl["in_bits"], gl["out_scale"], gl["out_zp"], 8, gelu_v))
+        gc = gelu_prepare(gl["in_scale"], gl["in_bits"], gl["out_scale"], gl["out_zp"], 8, gelu_v)
+        if gelu_table_on:
+            self.keep.append(gelu_table(gc, device))
+        p.gelu = host(gc)
         self.params = p
         self.ws = Workspace(int(lib().iptq_encoder_block_workspace_bytes(C.byref(p))), device)
 

@@ -70,9 +70,10 @@ constexpr uint32_t TMEM_COLS = 512;
 // replicated over the 128 lanes so that a thread reads them with the same instruction as its accumulators):
 //   BN =  96: mult, rounding constant, shift           (5 x 96 = 480 columns)
 //   BN = 128: mult, shift - 1; the rounding constant 2^(shift-1) is rebuilt with one shift  (4 x 128 = 512 columns)
-template <int BN>
+// GTAB: the FC1 epilogue reads the integer GELU from a 64 KB table in shared memory (one ring stage fewer).
+template <int BN, bool GTAB = false>
 struct GemmCfg {
-    static constexpr int STAGES = BN == 96 ? 5 : 4;
+    static constexpr int STAGES = (BN == 96 ? 5 : 4) - (GTAB ? 1 : 0);
     static constexpr int EPI_PARTS = BN / COLS;          // epilogue warps per TMEM lane quadrant
     static constexpr int EPI_WARPS = 4 * EPI_PARTS;
     static constexpr int THREADS = 32 * (2 + EPI_WARPS);
@@ -87,13 +88,14 @@ struct GemmParams {
     int out_zp;
     int res_mult, res_rnd, res_shift, res_off;        // residual branch: ((res << 16) - res_off) through R
     GeluDev gelu;
+    const int8_t* gelu_tab;                           // device table of the integer GELU, or null
     StatusBlock* status;
 };
 
-template <int BN>
+template <int BN, bool GTAB = false>
 struct GemmSmem {
-    static constexpr int STAGES = GemmCfg<BN>::STAGES;
-    static constexpr int EPI_WARPS = GemmCfg<BN>::EPI_WARPS;
+    static constexpr int STAGES = GemmCfg<BN, GTAB>::STAGES;
+    static constexpr int EPI_WARPS = GemmCfg<BN, GTAB>::EPI_WARPS;
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_BYTES = BN * BK;
     static constexpr int WARP_TILE = 32 * COLS;                                   // bytes of one warp's output block
@@ -102,7 +104,8 @@ struct GemmSmem {
     static constexpr int OFF_OUT = OFF_B + STAGES * B_BYTES;                     // [EPI_WARPS][32 rows][COLS] int8
     static constexpr int OFF_RES = OFF_OUT + EPI_WARPS * WARP_TILE;              // same shape, residual tiles
     static constexpr int OFF_BIAS = OFF_RES + EPI_WARPS * WARP_TILE;             // [EPI_WARPS][COLS] int32
-    static constexpr int OFF_BAR = OFF_BIAS + EPI_WARPS * COLS * 4;
+    static constexpr int OFF_TAB = OFF_BIAS + EPI_WARPS * COLS * 4;              // GELU table (GTAB only)
+    static constexpr int OFF_BAR = OFF_TAB + (GTAB ? IPTQ_GELU_TABLE_SIZE : 0);
     static constexpr int NUM_BARS = 2 * STAGES + 4 + EPI_WARPS;
     static constexpr int OFF_END = OFF_BAR + NUM_BARS * 8 + 16;
     static constexpr int TOTAL = OFF_END + 1024;                                 // slack for 1024-byte alignment
@@ -116,14 +119,14 @@ __device__ __forceinline__ uint32_t swz32(int row, int chunk) { return (uint32_t
 // One CTA works on ONE column tile (blockIdx.x % num_n_tiles) and walks down its row tiles, so the per-column
 // constants are set up once per CTA: mult / rounding / shift in TMEM, the bias in shared memory, from where the
 // epilogue writes it back into each accumulator it has just drained (the MMAs then always accumulate).
-template <int BN, int EPI, int GELU_VARIANT, bool SAT8>
+template <int BN, int EPI, int GELU_VARIANT, bool SAT8, bool GTAB>
 __global__ void __launch_bounds__(GemmCfg<BN>::THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_res,
                const GemmParams p)
 {
-    using L = GemmSmem<BN>;
-    using G = GemmCfg<BN>;
+    using L = GemmSmem<BN, GTAB>;
+    using G = GemmCfg<BN, GTAB>;
     constexpr int STAGES = G::STAGES, EPI_WARPS = G::EPI_WARPS;
     constexpr uint32_t TM_MULT = G::TM_MULT, TM_RND = G::TM_RND, TM_SHIFT = G::TM_SHIFT;
     extern __shared__ uint8_t smem_raw[];
@@ -268,6 +271,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             __syncwarp();
             if (lane == 0) { mbar_arrive(&acc_empty[0]); mbar_arrive(&acc_empty[1]); }
         }
+        const uint32_t tab_mid = smem_u32(smem + L::OFF_TAB) + 32768u;      // address of table[0 + 32768]
+        if (GTAB) {
+            // the GELU table is static data: copy it while the previous kernel may still be running
+            const int4* src = reinterpret_cast<const int4*>(p.gelu_tab);
+            int4* dst = reinterpret_cast<int4*>(smem + L::OFF_TAB);
+            for (int i = ew * 32 + lane; i < IPTQ_GELU_TABLE_SIZE / 16; i += EPI_WARPS * 32) dst[i] = __ldg(src + i);
+            named_barrier(1, EPI_WARPS * 32);
+        }
         grid_dep_wait();                                       // residual reads and output writes come after this
         int it = 0;
         for (int mt = mt0; mt < p.num_m_tiles; mt += mt_step, ++it) {
@@ -314,7 +325,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     int v;
                     if constexpr (G::HAS_RND) v = requant_core((int)acc[j], (int)cm[j], (int)cr[j], (int)cs[j]);
                     else v = (mad_hi((int)acc[j], (int)cm[j], 1 << cs[j]) >> cs[j]) >> 1;   // cs = shift - 1
-                    if (EPI == EPI_GELU) {
+                    if (EPI == EPI_GELU && GTAB) {
+                        v = max(-32768, min(32767, v));
+                        asm volatile("ld.shared.s8 %0, [%1];" : "=r"(v) : "r"(tab_mid + (uint32_t)v));
+                    } else if (EPI == EPI_GELU) {
                         v = gelu_core<GELU_VARIANT>(v, p.gelu);
                         v = requant_nosat(v, p.gelu.out);
                         if (!SAT8) v = max(p.gelu.out.qmin, min(p.gelu.out.qmax, v));
@@ -400,12 +414,12 @@ struct LinearArgs {
     StatusBlock* status;
 };
 
-template <int BN, int EPI, int GV, bool SAT8>
+template <int BN, int EPI, int GV, bool SAT8, bool GTAB = false>
 static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& my, const CUtensorMap& mr,
                        const GemmParams& p, cudaStream_t st)
 {
-    using L = GemmSmem<BN>;
-    auto kern = gemm_i8_kernel<BN, EPI, GV, SAT8>;
+    using L = GemmSmem<BN, GTAB>;
+    auto kern = gemm_i8_kernel<BN, EPI, GV, SAT8, GTAB>;
     static bool configured[64];               // one attribute call per instantiation and device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return IPTQ_ERR_CUDA;
@@ -485,6 +499,11 @@ static int linear_launch_bn(const LinearArgs& a, cudaStream_t st)
         const uint32_t box[2] = {COLS, 32};
         if ((rc = make_tensor_map_u8(&my, a.y, 2, dims, str, box, 32)) != IPTQ_OK) return rc;
         if ((rc = make_tensor_map_u8(&mr, a.residual ? a.residual : a.y, 2, dims, str, box, 32)) != IPTQ_OK) return rc;
+    }
+    p.gelu_tab = a.gelu ? a.gelu->table : nullptr;
+    if (a.gelu && a.gelu->table) {
+        if (!aligned16(a.gelu->table)) return IPTQ_ERR_ALIGN;
+        return launch_gemm<BN, EPI_GELU, 0, true, true>(ma, mb, my, mr, p, st);    // the variant is in the table
     }
     if (a.gelu) {
         const bool sat8 = a.gelu->out.qmin == -128 && a.gelu->out.qmax == 127;

@@ -144,6 +144,17 @@ gelu_kernel(const int32_t* __restrict__ x, int8_t* __restrict__ y, int64_t n, co
     if (t < n) y[t] = (int8_t)requant_full(gelu_core<VARIANT>(x[t], c), c.out);
 }
 
+// table[x + 32768] = integer GELU of x for every 16-bit x (the input clamp to in_bits is part of gelu_core)
+template <int VARIANT>
+__global__ void __launch_bounds__(256)
+gelu_table_kernel(int8_t* __restrict__ table, const GeluDev c)
+{
+    grid_dep_launch();
+    grid_dep_wait();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    table[i] = (int8_t)requant_full(gelu_core<VARIANT>(i - 32768, c), c.out);
+}
+
 // ------------------------------------------------------------------------------------------------
 // LayerNorm: a warp takes a few rows at a time; the rows live in registers as packed int8 words (NW per lane).
 // ------------------------------------------------------------------------------------------------
@@ -453,6 +464,25 @@ int iptq_gelu(const int32_t* x, int8_t* y, int64_t n, const iptq_gelu_consts* co
         default: return IPTQ_ERR_VARIANT;
     }
 #undef IPTQ_GELU_LAUNCH
+    note_launch();
+    return last_launch_status();
+}
+
+int iptq_gelu_table(const iptq_gelu_consts* consts, int8_t* table, iptq_stream_t stream)
+{
+    if (!consts || !table) return IPTQ_ERR_NULL;
+    if (!aligned16(table)) return IPTQ_ERR_ALIGN;
+    if (consts->in_bits < 8 || consts->in_bits > 16) return IPTQ_ERR_BITS;
+    int rc = check_requant(&consts->out);
+    if (rc != IPTQ_OK) return rc;
+    const GeluDev c = to_dev(*consts);
+    const int threads = 256, grid = IPTQ_GELU_TABLE_SIZE / threads;
+    switch (consts->variant) {
+        case IPTQ_GELU_POLY4: launch_kernel(gelu_table_kernel<IPTQ_GELU_POLY4>, grid, threads, 0, stream, table, c); break;
+        case IPTQ_GELU_POLY2: launch_kernel(gelu_table_kernel<IPTQ_GELU_POLY2>, grid, threads, 0, stream, table, c); break;
+        case IPTQ_GELU_SHIFT: launch_kernel(gelu_table_kernel<IPTQ_GELU_SHIFT>, grid, threads, 0, stream, table, c); break;
+        default: return IPTQ_ERR_VARIANT;
+    }
     note_launch();
     return last_launch_status();
 }

@@ -120,6 +120,14 @@ def test_mlp_parity(api, orc, variant, M, D, Dh):
     ws.check()
     assert len(np.unique(want_h)) > 50
     assert (got_h == want_h).all(), _mismatch(got_h, want_h)
+    # the same epilogue reading the tabulated GELU instead of evaluating it
+    gt = api.gelu_prepare(S_in, in_bits, 0.03, -100, 8, variant)
+    tab = api.gelu_table(gt)
+    got_t = api.mlp_block(_cu(x), _cu(w1), _cu(b1), _cu(m1), _cu(s1), gt, ws).cpu().numpy()
+    ws.check()
+    assert (got_t == want_h).all(), _mismatch(got_t, want_h)
+    xs = np.arange(-32768, 32768, dtype=np.int32)
+    assert (tab.cpu().numpy() == orc.gelu(xs, go)).all()         # the table itself is the oracle's GELU on every input
     # full MLP with residual
     want = orc.mlp_block(x, w1, b1, m1, s1, go, w2, b2, m2, s2, 1, res, rro)
     got = api.mlp_block(_cu(x), _cu(w1), _cu(b1), _cu(m1), _cu(s1), ga, ws, _cu(w2), _cu(b2), _cu(m2), _cu(s2), 1,
@@ -189,3 +197,8 @@ def test_encoder_block_parity(api, orc, shape, w_bits, table):
     blk.ws.check()
     assert len(np.unique(want)) > 30
     assert (got == want).all(), _mismatch(got, want)
+    # FC1 epilogue evaluating the polynomial instead of reading the table
+    blk2 = api.EncoderBlock(spec, table, gelu_table_on=False)
+    got2 = blk2(_cu(spec.x)).cpu().numpy()
+    blk2.ws.check()
+    assert (got2 == want).all(), _mismatch(got2, want)
