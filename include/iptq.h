@@ -100,12 +100,26 @@ typedef struct {
     /* derived, for the kernels: floor(v / x0) == umulhi(v, div_mul) >> div_shift for 0 <= v < 2^31 */
     uint32_t div_mul; int32_t div_shift;
     int32_t f_shl, p_shr;                    /* p = umulhi(f << f_shl, e) >> p_shr */
+    const uint16_t* table;                   /* optional: dev, from iptq_softmax_table(); NULL = none */
+    int32_t table_n;                         /* entries e(0) .. e(table_n - 1) of that table */
 } iptq_softmax_consts;
 
 /* host.  in_scale: scale of the scores (1/sqrt(d_head) folded in); needs 8 <= floor(1/in_scale) < 2^24
  * and row_len * (x0 << nsh) < 2^31 (IPTQ_ERR_SCALE_RANGE); out_bits in [4, 8]; 1 <= row_len <= 1024. */
 int iptq_softmax_prepare(double in_scale, int row_len, int out_bits, iptq_softmax_variant variant,
                          iptq_softmax_consts* out /*host*/);
+/* The shift-based exponentials (IPTQ_SM_BITEXP, IPTQ_SM_SHIFTMAX) of Eq. (9) are 0 from some d = max - s on (a
+ * few x0) and, where x0 << nsh < 2^16, fit 16 bits, so the whole function is a short table.  iptq_softmax() and
+ * the attention kernel build that table per CTA in shared memory; iptq_softmax_table() writes it once to device
+ * memory with the same arithmetic -- e(0) .. e(n - 1), then zeros up to the next multiple of 8 entries -- and
+ * stores the pointer and n in consts, after which the kernels copy it instead.  Results are identical either way.
+ * *consts: host, updated (table = NULL, table_n = 0 and nothing written where this variant or scale has no such
+ * table).  table: dev uint16 [capacity], 16-byte aligned, caller-owned, must outlive every use of consts;
+ * IPTQ_ERR_SHAPE when capacity is too small (IPTQ_SOFTMAX_TABLE_MAX entries always suffice: larger tables are
+ * not used by the kernels and count as "no table").  Work submitted to the stream after this call sees the
+ * complete table. */
+#define IPTQ_SOFTMAX_TABLE_MAX 51200
+int iptq_softmax_table(iptq_softmax_consts* consts, uint16_t* table, int32_t capacity, iptq_stream_t stream);
 /* scores: dev int32 [rows, row_len], |score| < 2^30.  probs: dev uint8 [rows, row_len].
  * bias: nullable dev int32 [bias_period, row_len] at the score scale; row i adds bias row (i % bias_period).
  * consts: host.  No workspace. */
@@ -133,7 +147,8 @@ typedef struct {
  * in the kernel).  iptq_gelu_table() fills such a table with the same arithmetic; when consts->table points to it,
  * the FC1 epilogue of iptq_mlp_block() / iptq_encoder_block() keeps a copy in shared memory and replaces the
  * polynomial by one read per output.  The results are identical with and without the table.
- * table: dev int8 [IPTQ_GELU_TABLE_SIZE], 16-byte aligned, caller-owned; consts: host (its own `table` is ignored). */
+ * table: dev int8 [IPTQ_GELU_TABLE_SIZE], 16-byte aligned, caller-owned; consts: host (its own `table` is ignored).
+ * Work submitted to the stream after this call sees the complete table. */
 #define IPTQ_GELU_TABLE_SIZE 65536
 int iptq_gelu_table(const iptq_gelu_consts* consts, int8_t* table, iptq_stream_t stream);
 

@@ -31,7 +31,8 @@ class Requant(C.Structure):
 class SoftmaxConsts(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("variant", "out_bits", "row_len", "x0", "nsh", "M", "dcap",
                                          "qln2", "qb", "qc", "norm_l", "norm_r")] + \
-               [("div_mul", C.c_uint32), ("div_shift", C.c_int32), ("f_shl", C.c_int32), ("p_shr", C.c_int32)]
+               [("div_mul", C.c_uint32), ("div_shift", C.c_int32), ("f_shl", C.c_int32), ("p_shr", C.c_int32),
+                ("table", C.c_void_p), ("table_n", C.c_int32)]
 
 
 class GeluConsts(C.Structure):
@@ -94,6 +95,7 @@ def lib():
         L.iptq_channel_requant_prepare.argtypes = [_vp, C.c_int, _vp, _vp]
         L.iptq_softmax_prepare.argtypes = [C.c_double, C.c_int, C.c_int, C.c_int, C.POINTER(SoftmaxConsts)]
         L.iptq_softmax.argtypes = [_vp, _vp, C.c_int64, C.c_int, _vp, C.c_int64, C.POINTER(SoftmaxConsts), _vp]
+        L.iptq_softmax_table.argtypes = [C.POINTER(SoftmaxConsts), _vp, C.c_int32, _vp]
         L.iptq_gelu_prepare.argtypes = [C.c_double, C.c_int, C.c_double, C.c_int, C.c_int, C.c_int,
                                         C.POINTER(GeluConsts)]
         L.iptq_gelu.argtypes = [_vp, _vp, C.c_int64, C.POINTER(GeluConsts), _vp]
@@ -130,7 +132,7 @@ def lib():
 
 def exported_symbols():
     """Names declared in include/iptq.h (used by the CPU-side load test)."""
-    return ["iptq_requant_prepare", "iptq_channel_requant_prepare", "iptq_softmax_prepare", "iptq_softmax",
+    return ["iptq_requant_prepare", "iptq_channel_requant_prepare", "iptq_softmax_prepare", "iptq_softmax", "iptq_softmax_table",
             "iptq_gelu_prepare", "iptq_gelu", "iptq_gelu_table", "iptq_layernorm_prepare", "iptq_layernorm",
             "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_attention_workspace_bytes", "iptq_attention_block",
             "iptq_mlp_workspace_bytes", "iptq_mlp_block", "iptq_encoder_block_workspace_bytes",
@@ -230,6 +232,21 @@ def softmax(scores, consts: SoftmaxConsts, bias=None, out=None):
     _chk(lib().iptq_softmax(_dp(scores), _dp(out), rows, n, _dp(bias), period, C.byref(consts), _stream()),
          "iptq_softmax")
     return out
+
+
+SOFTMAX_TABLE_MAX = 51200
+
+
+def softmax_table(consts: SoftmaxConsts, device="cuda"):
+    """Writes the exponential table of ``consts`` to device memory once and attaches it to ``consts`` (the Softmax
+    and attention kernels then copy it to shared memory instead of rebuilding it in every CTA).  Returns the table
+    tensor, which the caller must keep alive as long as ``consts`` is used, or None where the variant or scale has
+    no table."""
+    t = torch.empty(SOFTMAX_TABLE_MAX, dtype=torch.int16, device=device)
+    _chk(lib().iptq_softmax_table(C.byref(consts), _dp(t), SOFTMAX_TABLE_MAX, _stream()), "iptq_softmax_table")
+    if not consts.table:
+        return None
+    return t
 
 
 def gelu(x, consts: GeluConsts, out=None):
@@ -337,7 +354,8 @@ class EncoderBlock:
     """Device-resident parameters of one integer encoder block, prepared from a ``synth.BlockSpec``
     (or any object with the same fields) with the library's own ``*_prepare`` functions."""
 
-    def __init__(self, spec, table=(SM_BITEXP, GELU_POLY4, LN_SHIFT, LN_SHIFT), device="cuda", gelu_table_on=True):
+    def __init__(self, spec, table=(SM_BITEXP, GELU_POLY4, LN_SHIFT, LN_SHIFT), device="cuda", gelu_table_on=True,
+                 softmax_table_on=True):
         sh = spec.shape
         self.shape = sh
         self.keep = []          # host structs and device tensors referenced by raw pointers
@@ -371,7 +389,10 @@ class EncoderBlock:
             setattr(p, "s_" + name, dev(s))
         p.attn_bias = dev(spec.attn_bias)
         p.mask_id = dev(spec.mask_id)
-        p.sm = host(softmax_prepare(spec.softmax_scale, sh.N, 8, sm_v))
+        sc = softmax_prepare(spec.softmax_scale, sh.N, 8, sm_v)
+        if softmax_table_on:
+            self.keep.append(softmax_table(sc, device))
+        p.sm = host(sc)
         p.pv_rq = host(requant_prepare(spec.pv_ratio))
         p.proj_zp, p.fc2_zp = spec.proj.out_zp, spec.fc2.out_zp
         p.res1_rq = host(requant_prepare(spec.proj.res_ratio / 65536.0, zp=spec.proj.res_zp))

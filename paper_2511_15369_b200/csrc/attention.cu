@@ -36,6 +36,7 @@ struct AttnParams {
     int p_off, p_bytes, xch_off, bar_off;
     int stages;            // Q/K/V ring depth (3, or 2 when the exponential table needs the room)
     int lut_off, lut_n;    // exponential table: e(d) for d < lut_n, 0 beyond (lut_n = 0: no table)
+    const uint16_t* lut_src;   // the same table in device memory (copied), or null (built by each CTA)
     uint32_t tmem_cols;
     const int32_t* bias;   // [H, N, N] or null
     const uint8_t* mask_id;// [B, N] or null
@@ -202,8 +203,15 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         uint16_t* lut = reinterpret_cast<uint16_t*>(smem + p.lut_off);
         const uint32_t lut_addr = smem_u32(lut);
         if (USE_LUT) {
-            for (int d = (int)threadIdx.x - 64; d <= p.lut_n; d += ATT_SOFTMAX_THREADS)
-                lut[d] = d < p.lut_n ? (uint16_t)exp_core_nd<VARIANT>(-d, p.ex) : (uint16_t)0;
+            if (p.lut_src) {
+                // written and fenced by iptq_softmax_table(): safe to read ahead of the dependency wait
+                const int4* src = reinterpret_cast<const int4*>(p.lut_src);
+                int4* dst = reinterpret_cast<int4*>(lut);
+                for (int i = (int)threadIdx.x - 64; i < (p.lut_n + 8) / 8; i += ATT_SOFTMAX_THREADS) dst[i] = __ldg(src + i);
+            } else {
+                for (int d = (int)threadIdx.x - 64; d <= p.lut_n; d += ATT_SOFTMAX_THREADS)
+                    lut[d] = d < p.lut_n ? (uint16_t)exp_core_nd<VARIANT>(-d, p.ex) : (uint16_t)0;
+            }
             named_barrier(5, ATT_SOFTMAX_THREADS);              // the table is complete before anyone reads it
         }
         grid_dep_wait();                                       // output rows are written only after this
@@ -473,21 +481,16 @@ int attention_launch(const AttnArgs& a, cudaStream_t st)
     p.v_bytes = up1k(p.kpad * a.dh);
     p.stage_bytes = p.q_bytes + p.k_bytes + p.v_bytes;
     p.p_bytes = ((p.kpad + 127) / 128) * 16384;
-    // Exponential table (shift-based variants with values below 2^16): e(d) = 0 once -Q_p >= qz * x0, where qz is the
-    // bit length of the largest value x0 << nsh; -Q_p >= 23 (d >> 4) puts that at d >= 16 qz x0 / 23 + 15.
+    // Exponential table (shift-based variants with values below 2^16), where it fits beside 3 or 2 operand stages.
     p.lut_n = 0;
     p.stages = ATT_STAGES;
     const int fixed = 2 * p.p_bytes + 2 * 4 * 128 * 4 + 256 + 1024;
-    if (a.sm->variant != IPTQ_SM_POLY) {
-        int qz = 0;
-        for (int64_t u = (int64_t)a.sm->x0 << a.sm->nsh; u; u >>= 1) ++qz;
-        const int64_t n = (16 * (int64_t)qz * a.sm->x0) / 23 + 32;
+    if (const int64_t n = exp_table_entries(*a.sm)) {
         const int64_t bytes = (2 * (n + 1) + 255) & ~(int64_t)255;
-        if (qz <= 16) {
-            if (fixed + 3 * p.stage_bytes + bytes <= 227 * 1024) { p.lut_n = (int)n; }
-            else if (fixed + 2 * p.stage_bytes + bytes <= 227 * 1024) { p.lut_n = (int)n; p.stages = 2; }
-        }
+        if (fixed + 3 * p.stage_bytes + bytes <= 227 * 1024) { p.lut_n = (int)n; }
+        else if (fixed + 2 * p.stage_bytes + bytes <= 227 * 1024) { p.lut_n = (int)n; p.stages = 2; }
     }
+    p.lut_src = (p.lut_n && a.sm->table && a.sm->table_n == p.lut_n) ? a.sm->table : nullptr;
     const int lut_bytes = p.lut_n ? (int)((2 * ((int64_t)p.lut_n + 1) + 255) & ~255) : 0;
     p.p_off = p.stages * p.stage_bytes;
     p.xch_off = p.p_off + 2 * p.p_bytes;

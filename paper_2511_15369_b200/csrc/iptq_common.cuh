@@ -161,6 +161,19 @@ __device__ __forceinline__ unsigned exp_core(unsigned d, const ExpDev& c)
     return exp_core_nd<VARIANT>(-(int)d, c);
 }
 
+// Length of the exponential table for the shift-based variants: e(d) = 0 once the octave count q of Eq. (8)
+// reaches qz, the bit length of the largest value x0 << nsh; -Q_p >= 23 (d >> 4) puts that at
+// d >= 16 qz x0 / 23 + 15.  Returns 0 where no 16-bit table exists (polynomial variant, values of 2^16 and more).
+inline int exp_table_entries(const iptq_softmax_consts& sm)
+{
+    if (sm.variant == IPTQ_SM_POLY) return 0;
+    int qz = 0;
+    for (int64_t u = (int64_t)sm.x0 << sm.nsh; u; u >>= 1) ++qz;
+    if (qz > 16) return 0;
+    const int64_t n = (16 * (int64_t)qz * sm.x0) / 23 + 32;
+    return n > (1 << 20) ? 0 : (int)n;
+}
+
 // floor(2^M / sum) for 0 < sum < 2^31, M <= 40: the fp64 quotient cannot round across an integer
 // (a non-integer quotient is at least 2^-M away, relatively, from the next integer).
 __device__ __forceinline__ unsigned intdiv_factor(unsigned sum, int M)

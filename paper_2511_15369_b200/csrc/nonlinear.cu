@@ -15,6 +15,8 @@ constexpr unsigned kFull = 0xffffffffu;
 struct SoftmaxDev {
     ExpDev ex;
     int M, f_shl, p_shr;
+    int tab_n;                 // entries of the exponential table, 0: evaluate
+    const uint16_t* tab_src;   // the table in device memory, or null: each CTA builds it
 };
 
 // Lanes past the row end carry a score so low that the clamp at -dcap applies and the exponential is 0.
@@ -67,10 +69,108 @@ softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ pr
     }
 }
 
+// Tabulated form for the shift-based variants: the exponential of Eq. (9) is 0 beyond a few multiples of x0 and
+// below 2^16, so each CTA keeps it as a table in shared memory (copied from the one iptq_softmax_table() wrote, or
+// built here with the same arithmetic) and a score costs one 16-bit shared-memory load instead of the evaluation.
+// Two CTAs of 1024 threads per SM: 32 registers per thread, 64 warps to cover the load latency.
+constexpr int kSmTabThreads = 1024;
+constexpr int kSmTabMaxBytes = 2 * IPTQ_SOFTMAX_TABLE_MAX;
+// Smallest inputs for which the table pays for its set-up (copied from device memory / built by every CTA).
+constexpr int64_t kSmTabMinElemsCopy = 1 << 20, kSmTabMinElemsBuild = 16 << 20;
+
+template <int VARIANT, int NITER, bool HAS_BIAS, bool PSHR>
+__global__ void __launch_bounds__(kSmTabThreads, 2)
+softmax_rows_tab_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ probs, int64_t rows, int n,
+                        const int32_t* __restrict__ bias, int64_t bias_period, const SoftmaxDev c, int tab_n,
+                        const uint16_t* __restrict__ tab_src)
+{
+    constexpr int TPB = kSmTabThreads;
+    extern __shared__ __align__(16) uint16_t exp_tab[];
+    if (tab_src) {
+        // Written by iptq_softmax_table() and fenced there, so it may be read ahead of the dependency wait.
+        const int4* src = reinterpret_cast<const int4*>(tab_src);
+        int4* dst = reinterpret_cast<int4*>(exp_tab);
+        for (int i = threadIdx.x; i < (tab_n + 8) / 8; i += TPB) dst[i] = __ldg(src + i);
+    } else {
+        for (int d = threadIdx.x; d <= tab_n; d += TPB)
+            exp_tab[d] = d < tab_n ? (uint16_t)exp_core_nd<VARIANT>(-d, c.ex) : (uint16_t)0;
+    }
+    __syncthreads();
+    const uint32_t tab_addr = (uint32_t)__cvta_generic_to_shared(exp_tab);
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = (int64_t)blockIdx.x * (TPB >> 5) + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * (TPB >> 5);
+    grid_dep_launch();
+    grid_dep_wait();
+    // Only the last 32-column step of a row can pass the row end.
+    const bool tail_ok = lane + 32 * (NITER - 1) < n;
+    auto load_row = [&](int64_t row, int (&v)[NITER]) {
+        const int32_t* sr = scores + row * n + lane;
+        const int32_t* br = HAS_BIAS ? bias + (row % bias_period) * n + lane : nullptr;
+#pragma unroll
+        for (int k = 0; k < NITER; ++k) {
+            int s = kPadScore;
+            if (k < NITER - 1 || tail_ok) {
+                s = __ldcs(sr + 32 * k);
+                if (HAS_BIAS) s += __ldg(br + 32 * k);
+            }
+            v[k] = s;
+        }
+    };
+    auto finish_row = [&](int64_t row, int (&v)[NITER]) {
+        int mx = INT_MIN;
+#pragma unroll
+        for (int k = 0; k < NITER; ++k) mx = max(mx, v[k]);
+        mx = __reduce_max_sync(kFull, mx);                      // Eq. (6)
+        unsigned sum = 0;
+#pragma unroll
+        for (int k = 0; k < NITER; ++k) {
+            const unsigned d = min((unsigned)mx - (unsigned)v[k], (unsigned)tab_n);   // exact for any int32 pair
+            unsigned e;
+            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(e) : "r"(tab_addr + 2u * d));
+            v[k] = (int)e;
+            sum += e;
+        }
+        sum = __reduce_add_sync(kFull, sum);
+        const unsigned f = intdiv_factor(sum, c.M) << c.f_shl;  // Eq. (15)
+        uint8_t* pr = probs + row * n + lane;
+#pragma unroll
+        for (int k = 0; k < NITER; ++k) {
+            unsigned pv = __umulhi(f, (unsigned)v[k]);
+            if (PSHR) pv >>= c.p_shr;
+            if (k < NITER - 1 || tail_ok) __stcs(pr + 32 * k, (uint8_t)pv);
+        }
+    };
+    int v[NITER];
+    for (int64_t row = warp; row < rows; row += nwarps) {
+        load_row(row, v);
+        finish_row(row, v);
+    }
+}
+
 template <int VARIANT, int NITER>
 static int launch_softmax2(const int32_t* s, uint8_t* p, int64_t rows, int n, const int32_t* bias, int64_t period,
                            const SoftmaxDev& c, cudaStream_t st)
 {
+    if constexpr (VARIANT != IPTQ_SM_POLY && NITER <= 8)
+    if (c.tab_n > 0 && ((c.tab_n + 8) & ~7) <= IPTQ_SOFTMAX_TABLE_MAX &&
+        rows * n >= (c.tab_src ? kSmTabMinElemsCopy : kSmTabMinElemsBuild)) {
+        // Tabulated exponential: worth the per-CTA table set-up once every warp has several rows.
+        const size_t smem = (2 * ((size_t)c.tab_n + 1) + 15) & ~(size_t)15;
+        const int wpc = kSmTabThreads / 32;
+        const int grid = (int)std::min<int64_t>((rows + wpc - 1) / wpc, (int64_t)sm_count() * 2);
+#define IPTQ_SM_TAB(HB, PS)                                                                                         \
+        do {                                                                                                        \
+            auto kern = softmax_rows_tab_kernel<VARIANT, NITER, HB, PS>;                                            \
+            cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmTabMaxBytes);              \
+            launch_kernel(kern, grid, kSmTabThreads, smem, st, s, p, rows, n, bias, period, c, c.tab_n, c.tab_src); \
+        } while (0)
+        if (bias) { if (c.p_shr) IPTQ_SM_TAB(true, true); else IPTQ_SM_TAB(true, false); }
+        else      { if (c.p_shr) IPTQ_SM_TAB(false, true); else IPTQ_SM_TAB(false, false); }
+#undef IPTQ_SM_TAB
+        note_launch();
+        return last_launch_status();
+    }
     const int threads = 256;
     const int64_t want = (rows + 7) / 8;
     const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 8);
@@ -149,11 +249,24 @@ template <int VARIANT>
 __global__ void __launch_bounds__(256)
 gelu_table_kernel(int8_t* __restrict__ table, const GeluDev c)
 {
-    grid_dep_launch();
     grid_dep_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     table[i] = (int8_t)requant_full(gelu_core<VARIANT>(i - 32768, c), c.out);
 }
+
+// table[d] = integer exponential of -d for d < n, 0 for n <= d < n_pad
+template <int VARIANT>
+__global__ void __launch_bounds__(256)
+softmax_table_kernel(uint16_t* __restrict__ table, int n, int n_pad, const ExpDev ex)
+{
+    grid_dep_wait();
+    const int d = blockIdx.x * blockDim.x + threadIdx.x;
+    if (d < n_pad) table[d] = d < n ? (uint16_t)exp_core_nd<VARIANT>(-d, ex) : (uint16_t)0;
+}
+
+// Launched without programmatic serialisation behind a table kernel: it starts only once the table is complete
+// and visible, so a later kernel that reads the table ahead of its own dependency wait cannot overtake the writer.
+__global__ void stream_fence_kernel() {}
 
 // ------------------------------------------------------------------------------------------------
 // LayerNorm: a warp takes a few rows at a time; the rows live in registers as packed int8 words (NW per lane).
@@ -428,6 +541,8 @@ int iptq_softmax(const int32_t* scores, uint8_t* probs, int64_t rows, int row_le
     SoftmaxDev c;
     c.ex = to_dev_exp(*consts);
     c.M = consts->M; c.f_shl = consts->f_shl; c.p_shr = consts->p_shr;
+    c.tab_n = exp_table_entries(*consts);
+    c.tab_src = (consts->table && consts->table_n == c.tab_n) ? consts->table : nullptr;
     switch (consts->variant) {
         case IPTQ_SM_BITEXP: return launch_softmax1<IPTQ_SM_BITEXP>(scores, probs, rows, row_len, bias, bias_period, c, stream);
         case IPTQ_SM_SHIFTMAX: return launch_softmax1<IPTQ_SM_SHIFTMAX>(scores, probs, rows, row_len, bias, bias_period, c, stream);
@@ -483,8 +598,31 @@ int iptq_gelu_table(const iptq_gelu_consts* consts, int8_t* table, iptq_stream_t
         case IPTQ_GELU_SHIFT: launch_kernel(gelu_table_kernel<IPTQ_GELU_SHIFT>, grid, threads, 0, stream, table, c); break;
         default: return IPTQ_ERR_VARIANT;
     }
+    stream_fence_kernel<<<1, 32, 0, stream>>>();
     note_launch();
     return last_launch_status();
+}
+
+int iptq_softmax_table(iptq_softmax_consts* consts, uint16_t* table, int32_t capacity, iptq_stream_t stream)
+{
+    if (!consts) return IPTQ_ERR_NULL;
+    consts->table = nullptr;
+    consts->table_n = 0;
+    const int n = exp_table_entries(*consts);
+    const int n_pad = (n + 8) & ~7;                     // at least one zero behind the last entry
+    if (n == 0 || n_pad > IPTQ_SOFTMAX_TABLE_MAX) return IPTQ_OK;
+    if (!table) return IPTQ_ERR_NULL;
+    if (!aligned16(table)) return IPTQ_ERR_ALIGN;
+    if (capacity < n_pad) return IPTQ_ERR_SHAPE;
+    const ExpDev ex = to_dev_exp(*consts);
+    const int threads = 256, grid = (n_pad + threads - 1) / threads;
+    if (consts->variant == IPTQ_SM_BITEXP) launch_kernel(softmax_table_kernel<IPTQ_SM_BITEXP>, grid, threads, 0, stream, table, n, n_pad, ex);
+    else                                   launch_kernel(softmax_table_kernel<IPTQ_SM_SHIFTMAX>, grid, threads, 0, stream, table, n, n_pad, ex);
+    stream_fence_kernel<<<1, 32, 0, stream>>>();
+    note_launch();
+    const int rc = last_launch_status();
+    if (rc == IPTQ_OK) { consts->table = table; consts->table_n = n; }
+    return rc;
 }
 
 int iptq_layernorm(const int8_t* x, int8_t* y, int64_t rows, int dim, const int32_t* gamma_q,

@@ -53,6 +53,65 @@ def test_softmax_parity(api, orc, variant, rows, n, scale):
     assert (got == want).all()
 
 
+@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("scale", [synth.SOFTMAX_SCALE_ACC, synth.SOFTMAX_SCALE_8BIT])
+@pytest.mark.parametrize("rows,n,use_table", [(6001, 197, True), (86017, 197, False), (86017, 197, True),
+                                              (40003, 49, True), (9000, 208, True)])
+def test_softmax_tabulated_parity(api, orc, variant, scale, rows, n, use_table):
+    """Inputs large enough for the kernel that reads the exponential from a shared-memory table, with the table
+    copied from device memory (iptq_softmax_table) or built by every CTA."""
+    base = 4096
+    s0 = synth.quantize_scores(synth.softmax_logits(base, n, seed=rows + n), scale)
+    s0[7] = -(1 << 30) + 1
+    s0[7, n // 2] = (1 << 30) - 1                  # largest admissible distance to the row maximum
+    s0[8] = 12345                                  # all-equal row
+    reps = (rows + base - 1) // base
+    s = np.ascontiguousarray(np.tile(s0, (reps, 1))[:rows])
+    bias = np.random.default_rng(5).integers(-3000, 3000, size=(3, n)).astype(np.int32)
+    co = orc.softmax_prepare(scale, n, 8, variant)
+    ca = api.softmax_prepare(scale, n, 8, variant)
+    keep = api.softmax_table(ca) if use_table else None
+    assert (keep is not None) == use_table and bool(ca.table) == use_table
+    want0 = orc.softmax(s0, co)
+    got = api.softmax(_cu(s), ca).cpu().numpy()
+    assert (got == np.tile(want0, (reps, 1))[:rows]).all()
+    sub = slice(rows - 1500, rows)                 # rows whose bias row differs from their position in the block
+    want_b = orc.softmax(np.ascontiguousarray(s[sub]), co,
+                         bias=np.ascontiguousarray(np.roll(bias, -((rows - 1500) % 3), axis=0)), bias_period=3)
+    got_b = api.softmax(_cu(s), ca, bias=_cu(bias)).cpu().numpy()
+    assert (got_b[sub] == want_b).all()
+
+
+@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("scale,n", [(synth.SOFTMAX_SCALE_ACC, 197), (synth.SOFTMAX_SCALE_8BIT, 197), (1.0 / 700, 49)])
+def test_softmax_table_contents(api, orc, variant, scale, n):
+    """The device table holds the oracle's exponential for every tabulated distance, and the oracle's
+    exponential is 0 at every distance the table leaves out (up to the clamp of Eq. (6))."""
+    co = orc.softmax_prepare(scale, n, 8, variant)
+    ca = api.softmax_prepare(scale, n, 8, variant)
+    t = api.softmax_table(ca)
+    assert t is not None and 0 < ca.table_n < api.SOFTMAX_TABLE_MAX
+    tab = t.cpu().numpy().view(np.uint16)
+    want = np.array([orc.softmax_exp(d, co) for d in range(ca.table_n)])
+    assert (tab[:ca.table_n] == want).all()
+    assert tab[ca.table_n] == 0
+    assert tab[0] == co.x0 << co.nsh
+    for d in list(range(ca.table_n, min(co.dcap, ca.table_n + 5000))) + list(range(ca.table_n, co.dcap + 1, 97)) + [co.dcap]:
+        assert orc.softmax_exp(d, co) == 0, d
+
+
+def test_softmax_table_absent(api):
+    import torch
+    c = api.softmax_prepare(synth.SOFTMAX_SCALE_ACC, 197, 8, 2)       # polynomial exponential: no table
+    assert api.softmax_table(c) is None and not c.table and c.table_n == 0
+    c = api.softmax_prepare(1.0 / ((1 << 20) - 2.5), 49)               # x0 too large for a shared-memory table
+    assert api.softmax_table(c) is None and not c.table
+    c = api.softmax_prepare(synth.SOFTMAX_SCALE_ACC, 197)
+    small = torch.empty(64, dtype=torch.int16, device="cuda")
+    rc = api.lib().iptq_softmax_table(api.C.byref(c), small.data_ptr(), 64, None)
+    assert rc == api.ERR_SHAPE and not c.table
+
+
 def test_softmax_edge_rows_and_bias(api, orc):
     n = 197
     rng = np.random.default_rng(3)
