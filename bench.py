@@ -399,7 +399,7 @@ def run_ours(args):
         stages.append(s)
     # DRAM bytes per launch of the kernels of this workload, from the ncu capture summarised in
     # profiles/encoder_block_kernels_cfg1.md (dram__bytes_read.sum + dram__bytes_write.sum); valid for that kernel version
-    traffic = {"attention": 14.58e6}
+    traffic = {"attention": 14.61e6}
     top = max(stages, key=lambda s: s["us"])
     if "tops" in top:
         roofline = {"kernel": top["kernel"], "bound": "tensor", "achieved": top["tops"], "peak": int8_peak,
