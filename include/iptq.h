@@ -300,6 +300,50 @@ int iptq_encoder_block(const int8_t* x, int8_t* y, const iptq_block_params* p /*
 int iptq_encoder_block_profiled(const int8_t* x, int8_t* y, const iptq_block_params* p /*host*/, void* ws,
                                 size_t ws_bytes, iptq_stream_t stream, void* const* events /*host*/, int n_events);
 
+/* ------------------------------------------------------------------ Unified Metric
+ * Sec. 3.5 ("Unified Metric for Approximation Function Assignment"), Eqs. (16)-(20): every non-linear layer is
+ * run with each candidate function and scored by
+ *     term = 3 / ( 1/N(Q) + N(P) + N(C) ),   N(v) = log(1 + exp(v))                       Eqs. (16), (17)
+ *     Q = 10 log10( E[X^2] / E[(X - Qd)^2] )  (dB; the worked example beside Eq. (18) fixes 10 log10)
+ *     P = || X - Qd ||_2^2                                                                   Eq. (19)
+ *     C = integer operation count of the layer                                             Eq. (20)
+ * where X is the float layer and Qd the de-quantised output of the integer candidate; the layer takes the candidate
+ * with the largest term (stage 2 of the pipeline).
+ *
+ * Device part: after the candidate's own kernel (iptq_softmax / iptq_gelu / iptq_layernorm) has produced the
+ * integer output, iptq_metric_*() evaluate X in fp64 on the de-quantised integer input and reduce
+ *     sums[0] = sum X^2,   sums[1] = sum (X - Qd)^2
+ * over the whole tensor with a fixed summation order (the same device and sizes give the same bits).
+ *   Softmax:   X = softmax(in_scale * scores) per row;  Qd = probs * 2^-(out_bits-1)
+ *   GELU:      X = v/2 (1 + erf(v / sqrt 2)), v = in_scale * x;  Qd = (y - out_zp) * out_scale
+ *   LayerNorm: X = (v - mean)/std * gamma + beta per row, v = x << ptf_shift[channel] (biased variance, no
+ *              epsilon; a constant row gives beta);  Qd = (y - out_zp) * out_scale
+ * sums: dev double [2], 16-byte aligned, written by the call.  work: dev scratch of IPTQ_METRIC_WORK_BYTES,
+ * 16-byte aligned, caller-owned, free for reuse once the call has completed on the stream.  gamma / beta: dev
+ * float [dim] (the float parameters handed to iptq_layernorm_prepare); ptf_shift nullable.  row_len <= 1024,
+ * dim % 4 == 0 and dim <= 3072 as for the kernels measured.  Empty tensors give sums of 0. */
+#define IPTQ_METRIC_WORK_BYTES 32768
+int iptq_metric_softmax(const int32_t* scores, const uint8_t* probs, int64_t rows, int row_len, double in_scale,
+                        int out_bits, double* sums, void* work, iptq_stream_t stream);
+int iptq_metric_gelu(const int32_t* x, const int8_t* y, int64_t n, double in_scale, double out_scale, int out_zp,
+                     double* sums, void* work, iptq_stream_t stream);
+int iptq_metric_layernorm(const int8_t* x, const int8_t* y, int64_t rows, int dim, const float* gamma,
+                          const float* beta, const uint8_t* ptf_shift, double out_scale, int out_zp, double* sums,
+                          void* work, iptq_stream_t stream);
+
+/* Host part.  iptq_sqnr_db returns +inf for sum_err2 == 0.  iptq_metric_term: op_count is divided by c_unit before
+ * N() (the paper gives no unit; raw counts of 1e7 and more would leave N(C) as the only term that matters).
+ * iptq_op_count: integer operations of one layer on [rows, row_len] (GELU: rows * row_len elements) counted from
+ * this library's integer definitions, one per add / subtract / multiply / shift / compare / divide; returns a
+ * negative value for an unknown kind or variant.  iptq_metric_select: index of the largest term, the first of
+ * equals; -1 for n < 1. */
+typedef enum { IPTQ_LAYER_SOFTMAX = 0, IPTQ_LAYER_GELU = 1, IPTQ_LAYER_LAYERNORM = 2 } iptq_layer_kind;
+double iptq_softplus(double v);
+double iptq_sqnr_db(double sum_x2, double sum_err2);
+double iptq_metric_term(double sqnr_db, double perturbation, double op_count, double c_unit);
+double iptq_op_count(int layer_kind, int variant, int64_t rows, int row_len);
+int iptq_metric_select(const double* terms /*host*/, int n);
+
 /* ------------------------------------------------------------------ status
  * iptq_workspace_init: zero the status block (enqueued on the stream); call once per workspace.
  * iptq_check: synchronise the stream and return IPTQ_ERR_TIMEOUT if any kernel that used `ws`

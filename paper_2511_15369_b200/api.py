@@ -126,6 +126,17 @@ def lib():
                                                   C.POINTER(C.c_void_p), C.c_int]
         L.iptq_workspace_init.argtypes = [_vp, C.c_size_t, _vp]
         L.iptq_check.argtypes = [_vp, _vp]
+        L.iptq_metric_softmax.argtypes = [_vp, _vp, C.c_int64, C.c_int, C.c_double, C.c_int, _vp, _vp, _vp]
+        L.iptq_metric_gelu.argtypes = [_vp, _vp, C.c_int64, C.c_double, C.c_double, C.c_int, _vp, _vp, _vp]
+        L.iptq_metric_layernorm.argtypes = [_vp, _vp, C.c_int64, C.c_int, _vp, _vp, _vp, C.c_double, C.c_int, _vp,
+                                            _vp, _vp]
+        for f in (L.iptq_softplus, L.iptq_sqnr_db, L.iptq_metric_term, L.iptq_op_count):
+            f.restype = C.c_double
+        L.iptq_softplus.argtypes = [C.c_double]
+        L.iptq_sqnr_db.argtypes = [C.c_double, C.c_double]
+        L.iptq_metric_term.argtypes = [C.c_double, C.c_double, C.c_double, C.c_double]
+        L.iptq_op_count.argtypes = [C.c_int, C.c_int, C.c_int64, C.c_int]
+        L.iptq_metric_select.argtypes = [C.POINTER(C.c_double), C.c_int]
         _lib = L
     return _lib
 
@@ -136,7 +147,9 @@ def exported_symbols():
             "iptq_gelu_prepare", "iptq_gelu", "iptq_gelu_table", "iptq_layernorm_prepare", "iptq_layernorm",
             "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_attention_workspace_bytes", "iptq_attention_block",
             "iptq_mlp_workspace_bytes", "iptq_mlp_block", "iptq_encoder_block_workspace_bytes",
-            "iptq_encoder_block", "iptq_encoder_block_profiled", "iptq_workspace_init", "iptq_check", "iptq_strerror", "iptq_launch_count"]
+            "iptq_encoder_block", "iptq_encoder_block_profiled", "iptq_workspace_init", "iptq_check", "iptq_strerror", "iptq_launch_count",
+            "iptq_metric_softmax", "iptq_metric_gelu", "iptq_metric_layernorm", "iptq_softplus", "iptq_sqnr_db",
+            "iptq_metric_term", "iptq_op_count", "iptq_metric_select"]
 
 
 def _chk(rc, what):
@@ -267,6 +280,67 @@ def gelu_table(consts: GeluConsts, device="cuda"):
     _chk(lib().iptq_gelu_table(C.byref(consts), _dp(t), _stream()), "iptq_gelu_table")
     consts.table = t.data_ptr()
     return t
+
+
+# ------------------------------------------------------------------ Unified Metric (Sec. 3.5)
+
+LAYER_SOFTMAX, LAYER_GELU, LAYER_LAYERNORM = 0, 1, 2
+METRIC_WORK_BYTES = 32768
+
+
+class MetricScratch:
+    """Device scratch of the metric reductions: the partial sums and the [sum X^2, sum (X - Q)^2] result."""
+
+    def __init__(self, device="cuda"):
+        self.work = torch.empty(METRIC_WORK_BYTES // 8, dtype=torch.float64, device=device)
+        self.sums = torch.empty(2, dtype=torch.float64, device=device)
+
+
+def metric_softmax(scores, probs, in_scale, out_bits=8, scratch: MetricScratch | None = None):
+    """Enqueues the reduction; returns the device tensor [sum X^2, sum (X - Q)^2] (scratch.sums)."""
+    sc = scratch or MetricScratch(scores.device)
+    rows, n = scores.shape
+    _chk(lib().iptq_metric_softmax(_dp(scores), _dp(probs), rows, n, float(in_scale), out_bits, _dp(sc.sums),
+                                   _dp(sc.work), _stream()), "iptq_metric_softmax")
+    return sc.sums
+
+
+def metric_gelu(x, y, in_scale, out_scale, out_zp, scratch: MetricScratch | None = None):
+    sc = scratch or MetricScratch(x.device)
+    _chk(lib().iptq_metric_gelu(_dp(x), _dp(y), x.numel(), float(in_scale), float(out_scale), int(out_zp),
+                                _dp(sc.sums), _dp(sc.work), _stream()), "iptq_metric_gelu")
+    return sc.sums
+
+
+def metric_layernorm(x, y, gamma, beta, out_scale, out_zp, ptf_shift=None, scratch: MetricScratch | None = None):
+    """gamma, beta: device float32 [dim] (the float parameters, not the quantised ones)."""
+    sc = scratch or MetricScratch(x.device)
+    rows, dim = x.shape
+    _chk(lib().iptq_metric_layernorm(_dp(x), _dp(y), rows, dim, _dp(gamma), _dp(beta), _dp(ptf_shift),
+                                     float(out_scale), int(out_zp), _dp(sc.sums), _dp(sc.work), _stream()),
+         "iptq_metric_layernorm")
+    return sc.sums
+
+
+def softplus(v):
+    return float(lib().iptq_softplus(float(v)))
+
+
+def sqnr_db(sum_x2, sum_err2):
+    return float(lib().iptq_sqnr_db(float(sum_x2), float(sum_err2)))
+
+
+def metric_term(q_db, p, c_ops, c_unit=1.0e6):
+    return float(lib().iptq_metric_term(float(q_db), float(p), float(c_ops), float(c_unit)))
+
+
+def op_count(kind, variant, rows, row_len):
+    return float(lib().iptq_op_count(int(kind), int(variant), int(rows), int(row_len)))
+
+
+def metric_select(terms):
+    arr = (C.c_double * len(terms))(*[float(t) for t in terms])
+    return int(lib().iptq_metric_select(arr, len(terms)))
 
 
 def layernorm(x, gamma_q, beta_q, consts: LnConsts, ptf_shift=None, out=None):

@@ -136,6 +136,30 @@ def affine_out_quant(y: np.ndarray, bits: int = 8):
     return scale, zp
 
 
+def calibration_layers(D: int, H: int, N: int, Dh: int, depth: int, batch: int, seed: int = 0):
+    """Seeded calibration activations for every non-linear layer of a ViT encoder, in execution order: per block
+    LN1, Softmax, LN2, GELU, then the final LayerNorm (4 * depth + 1 layers; ViT-Base: 49).  Each layer draws from
+    the distribution of its kind (``ln_values`` / ``softmax_logits`` / ``gelu_values``) with its own seed and is
+    quantised the way the block generator does it.  Yields (name, kind, dict of host arrays and scales), one layer
+    at a time so that only one layer's activations are alive."""
+    def ln(name, k):
+        xf, gamma, beta, _ = ln_values(batch * N, D, seed=seed * 1000 + k)
+        xq, S = quantize_sym(xf, 8, np.int8)
+        So, zp = affine_out_quant(layernorm_ref(xq[:256].astype(np.float64), gamma, beta))
+        return name, "layernorm", dict(x=xq, in_scale=S, gamma=gamma, beta=beta, out_scale=So, out_zp=zp,
+                                       ptf=ptf_shifts(xq))
+    k = 0
+    for i in range(depth):
+        yield ln("blk%d.ln1" % i, k); k += 1
+        s = quantize_scores(softmax_logits(batch * H * N, N, seed=seed * 1000 + k), SOFTMAX_SCALE_ACC); k += 1
+        yield "blk%d.softmax" % i, "softmax", dict(scores=s, in_scale=SOFTMAX_SCALE_ACC)
+        yield ln("blk%d.ln2" % i, k); k += 1
+        xg, S = quantize_sym(gelu_values(batch * N * Dh, seed=seed * 1000 + k), 16); k += 1
+        So, zp = affine_out_quant(gelu_ref(xg[:4096] * S))
+        yield "blk%d.gelu" % i, "gelu", dict(x=xg, in_scale=S, in_bits=16, out_scale=So, out_zp=zp)
+    yield ln("final.ln", k)
+
+
 # ------------------------------------------------------------------ fp64 references (for calibration / error reports)
 
 def gelu_ref(x):
