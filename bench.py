@@ -10,6 +10,8 @@ One step = one pass of the whole block over one batch of seeded synthetic input.
   stages       every kernel of the step with its share of the step;
   nonlinear    the stand-alone integer Softmax / GELU / LayerNorm kernels on tensors larger than L2, as
                Gelem/s and fraction of the measured HBM copy bandwidth;
+  assignment   the Unified-Metric analysis (every candidate of every non-linear layer of the encoder scored and
+               selected on the device) as evaluations/s, with the oracle's scores of the first block beside it;
   cpu_baseline the CPU oracle timed on the host cores on a bounded sample of the same workload, and the
                element-by-element comparison of the GPU output with it.
 `--impl reference` times the CPU oracle alone (rank 0 only).  Multi-GPU runs are independent replicas of the
@@ -375,6 +377,7 @@ def run_ours(args):
     if rank == 0:
         nonlinear = bench_nonlinear(api, torch, dev, peaks, peak_kind)
     clocks.stop()
+    assignment = bench_assignment(api, torch, dev) if rank == 0 else None
 
     if rank != 0:
         if world > 1:
@@ -439,6 +442,7 @@ def run_ours(args):
         "roofline": roofline,
         "stages": stages,
         "nonlinear": nonlinear,
+        "assignment": assignment,
         "cpu_baseline": cpu,
     }))
     if world > 1:
@@ -503,6 +507,81 @@ def bench_nonlinear(api, torch, dev, peaks, peak_kind):
     record("iptq_layernorm", rows * dim, 2 * rows * dim, time_kernel(lambda: api.layernorm(xl, gqd, bqd, lc, out=yl)),
            "int8 [201728, 768] -> int8 (155 MB in)")
     return out
+
+
+def bench_assignment(api, torch, dev):
+    """Stages 1-2 of the assignment pipeline (Sec. 3.5) for the 49 non-linear layers of the DeiT-Small encoder on
+    seeded calibration activations of 8 images, resident in HBM: every candidate kernel, its fp64 reference and
+    error reduction, scoring and selection.  Also runs the oracle on the first block and compares."""
+    from paper_2511_15369_b200 import assign
+    from oracle import metric as om
+    import oracle
+    D, H, N, Dh, depth, batch = 384, 6, 197, 1536, 12, 8
+    host_layers = list(synth.calibration_layers(D, H, N, Dh, depth, batch, seed=0))
+    dev_layers = []
+    for name, kind, d in host_layers:
+        dev_layers.append((name, kind, {k: (torch.from_numpy(np.ascontiguousarray(v)).to(dev)
+                                            if isinstance(v, np.ndarray) and k in ("scores", "x", "ptf") else v)
+                                        for k, v in d.items()}))
+
+    def run():
+        an = assign.Analyzer(dev)
+        for name, kind, d in dev_layers:
+            if kind == "softmax":
+                an.softmax_layer(name, d["scores"], d["in_scale"])
+            elif kind == "gelu":
+                an.gelu_layer(name, d["x"], d["in_scale"], d["in_bits"], d["out_scale"], d["out_zp"])
+            else:
+                an.layernorm_layer(name, d["x"], d["gamma"], d["beta"], d["out_scale"], d["out_zp"], ptf_shift=d["ptf"])
+        layers, omega = an.finish()
+        return layers, omega, an.n_eval
+
+    run()
+    times = []
+    for _ in range(3):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        layers, omega, n_eval = run()
+        times.append(time.perf_counter() - t0)
+    t = statistics.median(times)
+    names = {api.LAYER_SOFTMAX: ("bit", "shiftmax", "poly"), api.LAYER_GELU: ("poly4", "poly2", "shift"),
+             api.LAYER_LAYERNORM: ("shift", "newton", "ptf")}
+    kinds = {api.LAYER_SOFTMAX: "softmax", api.LAYER_GELU: "gelu", api.LAYER_LAYERNORM: "layernorm"}
+    chosen = {}
+    for l in layers:
+        key = kinds[l.kind] + ":" + names[l.kind][l.choice]
+        chosen[key] = chosen.get(key, 0) + 1
+    # oracle on the first block (4 layers), same inputs
+    t0 = time.perf_counter()
+    agree, compared = 0, 0
+    for (name, kind, d), l in list(zip(host_layers, layers))[:4]:
+        terms = []
+        for c in l.candidates:
+            v = c.variant
+            if kind == "softmax":
+                q = om.softmax_deq(oracle.softmax(d["scores"], oracle.softmax_prepare(d["in_scale"], N, 8, v)), 8)
+                x = om.softmax_float(d["scores"], d["in_scale"])
+                ops = om.op_count(om.SOFTMAX, v, d["scores"].shape[0], N)
+            elif kind == "gelu":
+                gc = oracle.gelu_prepare(d["in_scale"], d["in_bits"], d["out_scale"], d["out_zp"], 8, v)
+                q = om.affine_deq(oracle.gelu(d["x"], gc), d["out_scale"], d["out_zp"])
+                x = om.gelu_float(d["x"], d["in_scale"])
+                ops = om.op_count(om.GELU, v, d["x"].size, 1)
+            else:
+                ptf = d["ptf"] if v == 2 else None
+                gq, bq, lc = oracle.layernorm_prepare(d["gamma"], d["beta"], d["out_scale"], d["out_zp"], 8, v)
+                q = om.affine_deq(oracle.layernorm(d["x"], gq, bq, lc, ptf), d["out_scale"], d["out_zp"])
+                x = om.layernorm_float(d["x"], d["gamma"], d["beta"], ptf)
+                ops = om.op_count(om.LAYERNORM, v, d["x"].shape[0], D)
+            qdb, pp, term = om.evaluate(x, q, ops)
+            compared += 1
+            agree += int(abs(term - c.term) <= 1e-9 * term and abs(pp - c.perturbation) <= 1e-9 * pp)
+            terms.append(term)
+    t_cpu = time.perf_counter() - t0
+    return {"workload": "DeiT-Small encoder, 49 non-linear layers, calibration batch 8 (synthetic), 3 candidates each",
+            "layers": len(layers), "evaluations": int(n_eval), "ms": 1e3 * t, "evaluations_per_s": n_eval / t,
+            "omega": omega, "selected": chosen,
+            "oracle_first_block": {"evaluations": compared, "agree_within_1e-9": agree, "seconds": t_cpu}}
 
 
 def main():
