@@ -404,7 +404,25 @@ def run_ours(args):
     # profiles/encoder_block_kernels_cfg1.md (dram__bytes_read.sum + dram__bytes_write.sum); valid for that kernel version
     traffic = {"attention": 14.61e6}
     top = max(stages, key=lambda s: s["us"])
-    if "tops" in top:
+    clock_summary = clocks.summary(windows)
+    if top["kernel"] == "attention":
+        # The fused attention is bound by the integer pipes, not by the contraction: a score costs 2 * 2 * dh tensor
+        # operations but the 21 integer operations of Eqs. (6)-(15) (the count iptq_op_count() gives the variant).
+        # Ceiling: every SM sub-partition issues one 32-lane integer instruction per clock.
+        props = torch.cuda.get_device_properties(dev)
+        sm_mhz = clock_summary.get("sm_max_mhz") or 1965.0
+        alu_peak = props.multi_processor_count * 4 * 32 * sm_mhz * 1e6 / 1e12
+        alu_ops = api.op_count(api.LAYER_SOFTMAX, TABLE[0], B * H * N, N)
+        achieved = alu_ops / (top["us"] * 1e-6) / 1e12
+        roofline = {"kernel": "attention", "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "Tint-op/s",
+                    "frac": achieved / alu_peak, "traffic": traffic.get("attention"),
+                    "peak_source": "%d SMs x 4 sub-partitions x 32 lanes x %.0f MHz (clocks.max.sm), one integer "
+                                   "instruction per lane per clock" % (props.multi_processor_count, sm_mhz),
+                    "ops_per_launch": alu_ops, "us_per_launch": top["us"],
+                    "tensor": {"achieved": top["tops"], "peak": int8_peak, "unit": "TOP/s", "frac": top["tops"] / int8_peak,
+                               "ops_per_launch": stage_ops["attention"],
+                               "peak_source": "%s bf16 burst GEMM x %.0f (nominal dense INT8 : bf16 ratio)" % (peak_kind, INT8_OVER_BF16)}}
+    elif "tops" in top:
         roofline = {"kernel": top["kernel"], "bound": "tensor", "achieved": top["tops"], "peak": int8_peak,
                     "unit": "TOP/s", "frac": top["tops"] / int8_peak, "traffic": traffic.get(top["kernel"]),
                     "peak_source": "%s bf16 burst GEMM x %.0f (nominal dense INT8 : bf16 ratio)" % (peak_kind, INT8_OVER_BF16),
@@ -438,7 +456,7 @@ def run_ours(args):
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(xh.numel()), "d2h_bytes_per_step": int(yh[0].numel()),
                 "ms_per_step": total_e2e / K, "pipelining": "input copy, block and output copy of neighbouring steps overlap (3 streams, 2 buffer sets)"},
         "gpu_launches": int(launches),
-        "clocks": clocks.summary(windows),
+        "clocks": clock_summary,
         "roofline": roofline,
         "stages": stages,
         "nonlinear": nonlinear,

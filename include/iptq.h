@@ -265,6 +265,12 @@ int iptq_mlp_block(const int8_t* x, const void* w1, const int32_t* b1, const int
 int iptq_gather_rows(const int8_t* src, int8_t* dst, const int32_t* index, int64_t n_dst, int parts,
                      int row_bytes, iptq_stream_t stream);
 
+/* Patch embedding front end of the ViT / DeiT models of Sec. 4 (the paper does not describe it; the usual one):
+ * the P x P, stride-P convolution is an INT8 linear layer on patch rows, and this call lays the rows out:
+ * out[(b, py, px), (c, dy, dx)] = img[b, c, py*P + dy, px*P + dx].
+ * img: dev int8 [B, C, H, W]; out: dev int8 [B * (H/P) * (W/P), C*P*P]; P % 16 == 0, H % P == W % P == 0. */
+int iptq_patchify(const int8_t* img, int8_t* out, int64_t B, int C, int H, int W, int P, iptq_stream_t stream);
+
 /* ------------------------------------------------------------------ one encoder block
  * LN1 -> QKV GEMM -> fused attention -> proj GEMM (+ residual x) -> LN2 -> fused MLP (+ residual),
  * each layer running the variant its consts name (the per-layer table of Sec. 3.2).

@@ -110,6 +110,7 @@ def lib():
         L.iptq_linear_w4_static.argtypes = [_vp, _vp, _vp, _vp, _vp, C.c_int32, _vp, C.POINTER(Requant), _vp,
                                             C.c_int64, C.c_int, C.c_int, _vp, _vp]
         L.iptq_gather_rows.argtypes = [_vp, _vp, _vp, C.c_int64, C.c_int, C.c_int, _vp]
+        L.iptq_patchify.argtypes = [_vp, _vp, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, _vp]
         L.iptq_attention_workspace_bytes.restype = C.c_size_t
         L.iptq_attention_workspace_bytes.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
         L.iptq_attention_block.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, C.c_int, C.c_int, C.c_int, _vp, _vp,
@@ -145,7 +146,7 @@ def exported_symbols():
     """Names declared in include/iptq.h (used by the CPU-side load test)."""
     return ["iptq_requant_prepare", "iptq_channel_requant_prepare", "iptq_softmax_prepare", "iptq_softmax", "iptq_softmax_table",
             "iptq_gelu_prepare", "iptq_gelu", "iptq_gelu_table", "iptq_layernorm_prepare", "iptq_layernorm",
-            "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_attention_workspace_bytes", "iptq_attention_block",
+            "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_patchify", "iptq_attention_workspace_bytes", "iptq_attention_block",
             "iptq_mlp_workspace_bytes", "iptq_mlp_block", "iptq_encoder_block_workspace_bytes",
             "iptq_encoder_block", "iptq_encoder_block_profiled", "iptq_workspace_init", "iptq_check", "iptq_strerror", "iptq_launch_count",
             "iptq_metric_softmax", "iptq_metric_gelu", "iptq_metric_layernorm", "iptq_softplus", "iptq_sqnr_db",
@@ -391,6 +392,15 @@ def gather_rows(src, index, out=None):
     if out is None:
         out = torch.empty((n_dst, parts * C_), dtype=torch.int8, device=src.device)
     _chk(lib().iptq_gather_rows(_dp(src), _dp(out), _dp(index), n_dst, parts, C_, _stream()), "iptq_gather_rows")
+    return out
+
+
+def patchify(img, patch=16, out=None):
+    """img: int8 [B, C, H, W] -> patch rows int8 [B * (H/patch) * (W/patch), C * patch * patch]."""
+    B, C_, H, W = img.shape
+    if out is None:
+        out = torch.empty((B * (H // patch) * (W // patch), C_ * patch * patch), dtype=torch.int8, device=img.device)
+    _chk(lib().iptq_patchify(_dp(img), _dp(out), B, C_, H, W, patch, _stream()), "iptq_patchify")
     return out
 
 

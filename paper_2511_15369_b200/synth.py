@@ -475,3 +475,91 @@ def make_swin(B: int = 2, stages=None, seed: int = 0, window: int = 7) -> SwinSp
     xin, _, _, _ = ln_values(B * Hh * Ww, stages[0]["dim"], seed)
     x, _ = quantize_sym(xin, 8, np.int8)
     return SwinSpec(B, out, x)
+
+
+# ------------------------------------------------------------------ whole ViT / DeiT models (Sec. 4, latency table)
+
+VIT_MODELS = {
+    "DeiT-T": dict(D=192, H=3, depth=12),
+    "DeiT-S": dict(D=384, H=6, depth=12),
+    "DeiT-B": dict(D=768, H=12, depth=12),
+}
+
+
+@dataclass
+class VitSpec:
+    name: str
+    B: int
+    D: int
+    H: int
+    depth: int
+    img_size: int
+    patch: int
+    classes: int
+    image: np.ndarray           # int8 [B, 3, img, img]
+    embed: LinearSpec           # patch rows [B*P, 3*patch*patch] -> [B*P, D]; residual = position rows
+    pos: np.ndarray             # int8 [P, D] position embedding of the patch tokens (residual branch)
+    cls_row: np.ndarray         # int8 [D]: class token + its position embedding, at the token scale
+    blocks: list                # BlockSpec per encoder block (x = None: the input comes from the layer before)
+    final_ln: dict              # gamma, beta, out_scale, out_zp
+    head: LinearSpec            # [B, D] -> [B, classes]
+
+    @property
+    def N(self) -> int:
+        return (self.img_size // self.patch) ** 2 + 1
+
+    def gemm_ops(self) -> int:
+        P = self.N - 1
+        ops = 2 * self.B * P * self.D * 3 * self.patch * self.patch + 2 * self.B * self.D * self.classes
+        return ops + sum(b.shape.gemm_ops() for b in self.blocks)
+
+
+def make_vit(name: str = "DeiT-S", B: int = 8, seed: int = 0, img_size: int = 224, patch: int = 16,
+             classes: int = 1000, depth: int | None = None) -> VitSpec:
+    """A ViT/DeiT-shaped integer model with seeded random weights: patch embedding (+ position embedding through
+    the residual branch of the linear layer), class token, `depth` encoder blocks, final LayerNorm, classifier.
+    The front end is calibrated by an fp64 shadow pass over the first two images; every block calibrates on its own
+    synthetic input (see make_block); the final LayerNorm and the classifier use fixed ranges (8 standard deviations
+    and 6 standard deviations of a unit-variance input)."""
+    m = VIT_MODELS[name]
+    D, H = m["D"], m["H"]
+    depth = m["depth"] if depth is None else depth
+    g = _rng(seed, 5)
+    gsz = img_size // patch
+    P, K = gsz * gsz, 3 * patch * patch
+    img_f = g.normal(0.0, 1.0, size=(B, 3, img_size, img_size))
+    image, S_img = quantize_sym(img_f, 8, np.int8)
+    del img_f
+    # ---- patch embedding + position embedding (fp64 shadow on two images)
+    Bc = min(B, 2)
+    rows = image[:Bc].reshape(Bc, 3, gsz, patch, gsz, patch).transpose(0, 2, 4, 1, 3, 5).reshape(Bc * P, K)
+    wf = g.normal(0.0, 0.02, size=(D, K))
+    bf = g.normal(0.0, 0.02, size=D)
+    wq, Sw = quantize_weight(wf, 8)
+    bq = np.round(bf / (S_img * Sw)).astype(np.int32)
+    pos_f = g.normal(0.0, 0.02, size=(P + 1, D))
+    cls_f = g.normal(0.0, 0.02, size=D)
+    pos, S_pos = quantize_sym(pos_f[1:], 8, np.int8)
+    tok = rows.astype(np.float64) @ (wq * Sw[:, None]).T * S_img + bq * (S_img * Sw) + np.tile(pos * S_pos, (Bc, 1))
+    S_tok = float(np.abs(tok).max()) / 127.0
+    embed = LinearSpec(wq, wq, bq, S_img * Sw / S_tok, 0, S_pos / S_tok, 0)
+    cls_row = np.clip(np.round((cls_f + pos_f[0]) / S_tok), -128, 127).astype(np.int8)
+    # ---- encoder blocks
+    shape = BlockShape("%s b%d" % (name, B), B, P + 1, D, H, D // H, 4 * D)
+    blocks = []
+    for i in range(depth):
+        spec = make_block(shape, seed=seed + 1 + i, calib_images=2)
+        spec.x = None
+        blocks.append(spec)
+    # ---- final LayerNorm and classifier
+    gamma = g.normal(1.0, 0.1, size=D).astype(np.float32)
+    beta = g.normal(0.0, 0.1, size=D).astype(np.float32)
+    S_ln = 8.0 * float(np.abs(gamma).max()) / 127.0
+    wf = g.normal(0.0, 0.02, size=(classes, D))
+    bf = g.normal(0.0, 0.02, size=classes)
+    wq, Sw = quantize_weight(wf, 8)
+    bq = np.round(bf / (S_ln * Sw)).astype(np.int32)
+    S_out = 6.0 * 0.02 * math.sqrt(D) / 127.0
+    head = LinearSpec(wq, wq, bq, S_ln * Sw / S_out)
+    return VitSpec(name, B, D, H, depth, img_size, patch, classes, image, embed, pos, cls_row, blocks,
+                   dict(gamma=gamma, beta=beta, out_scale=S_ln, out_zp=0), head)
