@@ -12,6 +12,7 @@ One step = one pass of the whole block over one batch of seeded synthetic input.
                Gelem/s and fraction of the measured HBM copy bandwidth;
   assignment   the Unified-Metric analysis (every candidate of every non-linear layer of the encoder scored and
                selected on the device) as evaluations/s, with the oracle's scores of the first block beside it;
+  models       whole DeiT-T/S/B forward latency at batch 8 (context beside the paper's latency table, other hardware);
   cpu_baseline the CPU oracle timed on the host cores on a bounded sample of the same workload, and the
                element-by-element comparison of the GPU output with it.
 `--impl reference` times the CPU oracle alone (rank 0 only).  Multi-GPU runs are independent replicas of the
@@ -378,6 +379,7 @@ def run_ours(args):
         nonlinear = bench_nonlinear(api, torch, dev, peaks, peak_kind)
     clocks.stop()
     assignment = bench_assignment(api, torch, dev) if rank == 0 else None
+    models = bench_models(api, torch, dev) if rank == 0 else None
 
     if rank != 0:
         if world > 1:
@@ -461,6 +463,7 @@ def run_ours(args):
         "stages": stages,
         "nonlinear": nonlinear,
         "assignment": assignment,
+        "models": models,
         "cpu_baseline": cpu,
     }))
     if world > 1:
@@ -524,6 +527,46 @@ def bench_nonlinear(api, torch, dev, peaks, peak_kind):
     gqd, bqd = torch.from_numpy(gq).to(dev), torch.from_numpy(bq).to(dev)
     record("iptq_layernorm", rows * dim, 2 * rows * dim, time_kernel(lambda: api.layernorm(xl, gqd, bqd, lc, out=yl)),
            "int8 [201728, 768] -> int8 (155 MB in)")
+    return out
+
+
+PAPER_LATENCY_MS = {"DeiT-T": 1.73, "DeiT-S": 3.46, "DeiT-B": 7.11}   # the paper's latency table: RTX 3090, TVM, batch 8
+
+
+def bench_models(api, torch, dev):
+    """Whole-model forward latency at batch 8 (the setting of the paper's latency table) for the three DeiT shapes
+    with seeded random weights: one CUDA-graph replay per forward pass, L2 flushed before each, CUDA events."""
+    from paper_2511_15369_b200 import vit
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    out = []
+    for name in ("DeiT-T", "DeiT-S", "DeiT-B"):
+        spec = synth.make_vit(name, 8, seed=0)
+        model = vit.VitModel(spec, TABLE, dev)
+        img = torch.from_numpy(spec.image).to(dev)
+        st = torch.cuda.Stream()
+        with torch.cuda.stream(st):
+            for _ in range(3):
+                model(img)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=st):
+                model(img)
+            ts = []
+            for _ in range(20):
+                flush.fill_(1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(st)
+                g.replay()
+                b.record(st)
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+        model.check()
+        ms = statistics.median(ts)
+        out.append({"model": name, "batch": 8, "ms": ms, "images_per_s": 8 / (ms * 1e-3),
+                    "tops": spec.gemm_ops() / (ms * 1e-3) / 1e12, "gop": spec.gemm_ops() / 1e9,
+                    "launches": model.launches_per_forward(),
+                    "paper_ms_rtx3090_tvm": PAPER_LATENCY_MS[name], "data": "synthetic image, random weights"})
+        del model, g, img
     return out
 
 
