@@ -69,26 +69,8 @@ def sub_batch(spec, images):
 def oracle_block(spec, table):
     """The CPU oracle's encoder block on `spec` (constants prepared by the oracle's own functions)."""
     import oracle
-    sm_v, gelu_v, ln1_v, ln2_v = table
-    sh = spec.shape
-    d = dict(B=sh.B, N=sh.N, D=sh.D, H=sh.H, dh=sh.dh, Dh=sh.Dh, w_bits=spec.w_bits,
-             sm_variant=sm_v, gelu_variant=gelu_v, ln1_variant=ln1_v, ln2_variant=ln2_v)
-    for name, ln, var in (("ln1", spec.ln1, ln1_v), ("ln2", spec.ln2, ln2_v)):
-        gq, bq, c = oracle.layernorm_prepare(ln["gamma"], ln["beta"], ln["out_scale"], ln["out_zp"], 8, var)
-        d[name + "_gamma"], d[name + "_beta"], d[name], d[name + "_ptf"] = gq, bq, c, ln.get("ptf")
-    for name, ls in (("qkv", spec.qkv), ("proj", spec.proj), ("fc1", spec.fc1), ("fc2", spec.fc2)):
-        rq = [oracle.requant_prepare(float(r)) for r in ls.ratio]
-        d["w_" + name], d["b_" + name] = ls.w_packed, ls.bias
-        d["m_" + name] = np.array([r.mult for r in rq], np.int32)
-        d["s_" + name] = np.array([r.shift for r in rq], np.int8)
-    d["sm"] = oracle.softmax_prepare(spec.softmax_scale, sh.N, 8, sm_v)
-    d["pv_rq"] = oracle.requant_prepare(spec.pv_ratio)
-    d["attn_bias"], d["mask_id"] = spec.attn_bias, spec.mask_id
-    d["res1_rq"] = oracle.requant_prepare(spec.proj.res_ratio / 65536, zp=spec.proj.res_zp)
-    d["res2_rq"] = oracle.requant_prepare(spec.fc2.res_ratio / 65536, zp=spec.fc2.res_zp)
-    gl = spec.gelu
-    d["gelu"] = oracle.gelu_prepare(gl["in_scale"], gl["in_bits"], gl["out_scale"], gl["out_zp"], 8, gelu_v)
-    d["proj_zp"], d["fc2_zp"] = spec.proj.out_zp, spec.fc2.out_zp
+    from oracle import compose
+    d = compose.block_params(spec, table)
     t0 = time.perf_counter()
     y = oracle.encoder_block(spec.x, d)
     return y, time.perf_counter() - t0

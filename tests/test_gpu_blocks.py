@@ -159,27 +159,8 @@ def test_attention_parity(api, orc, variant, B, H, N, dh, use_bias, use_mask):
 
 
 def _oracle_block(orc, spec, table):
-    sm_v, gelu_v, ln1_v, ln2_v = table
-    sh = spec.shape
-    d = dict(B=sh.B, N=sh.N, D=sh.D, H=sh.H, dh=sh.dh, Dh=sh.Dh, w_bits=spec.w_bits)
-    for name, lnspec, var in (("ln1", spec.ln1, ln1_v), ("ln2", spec.ln2, ln2_v)):
-        gq, bq, c = orc.layernorm_prepare(lnspec["gamma"], lnspec["beta"], lnspec["out_scale"], lnspec["out_zp"], 8, var)
-        d[name + "_gamma"], d[name + "_beta"], d[name] = gq, bq, c
-        d[name + "_ptf"] = lnspec.get("ptf")
-    for name, ls in (("qkv", spec.qkv), ("proj", spec.proj), ("fc1", spec.fc1), ("fc2", spec.fc2)):
-        rq = [orc.requant_prepare(float(r)) for r in ls.ratio]
-        d["w_" + name], d["b_" + name] = ls.w_packed, ls.bias
-        d["m_" + name] = np.array([r.mult for r in rq], np.int32)
-        d["s_" + name] = np.array([r.shift for r in rq], np.int8)
-    d["sm"] = orc.softmax_prepare(spec.softmax_scale, sh.N, 8, sm_v)
-    d["pv_rq"] = orc.requant_prepare(spec.pv_ratio)
-    d["attn_bias"], d["mask_id"] = spec.attn_bias, spec.mask_id
-    d["res1_rq"] = orc.requant_prepare(spec.proj.res_ratio / 65536, zp=spec.proj.res_zp)
-    d["res2_rq"] = orc.requant_prepare(spec.fc2.res_ratio / 65536, zp=spec.fc2.res_zp)
-    gl = spec.gelu
-    d["gelu"] = orc.gelu_prepare(gl["in_scale"], gl["in_bits"], gl["out_scale"], gl["out_zp"], 8, gelu_v)
-    d["proj_zp"], d["fc2_zp"] = spec.proj.out_zp, spec.fc2.out_zp
-    return orc.encoder_block(spec.x, d)
+    from oracle import compose
+    return orc.encoder_block(spec.x, compose.block_params(spec, table))
 
 
 @pytest.mark.parametrize("shape,w_bits,table", [
