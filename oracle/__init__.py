@@ -18,7 +18,8 @@ _SRC = os.path.join(_HERE, "iptq_oracle.c")
 _HDR = os.path.join(_HERE, "iptq_oracle.h")
 _LIB = os.path.join(_HERE, "liboracle_iptq.so")
 
-SM_BITEXP, SM_SHIFTMAX, SM_POLY = 0, 1, 2
+SM_BITEXP, SM_SHIFTMAX, SM_POLY, SM_LOG2 = 0, 1, 2, 3
+LOG2_ZERO = 255          # SM_LOG2 writes codes: probability 2^-code for 0..15, LOG2_ZERO for probability 0
 GELU_POLY4, GELU_POLY2, GELU_SHIFT = 0, 1, 2
 LN_SHIFT, LN_NEWTON, LN_PTF = 0, 1, 2
 

@@ -93,7 +93,9 @@ int oracle_softmax_prepare(double in_scale, int row_len, int out_bits, int varia
 {
     if (!out) return ORACLE_ERR_ARG;
     if (row_len < 1 || out_bits < 4 || out_bits > 8) return ORACLE_ERR_ARG;
-    if (variant != ORACLE_SM_BITEXP && variant != ORACLE_SM_SHIFTMAX && variant != ORACLE_SM_POLY) return ORACLE_ERR_ARG;
+    if (variant != ORACLE_SM_BITEXP && variant != ORACLE_SM_SHIFTMAX && variant != ORACLE_SM_POLY &&
+        variant != ORACLE_SM_LOG2) return ORACLE_ERR_ARG;
+    if (variant == ORACLE_SM_LOG2 && out_bits != 4) return ORACLE_ERR_ARG;   /* 4-bit log2 codes */
     if (!(in_scale > 0.0)) return ORACLE_ERR_RANGE;
     memset(out, 0, sizeof(*out));
     /* Eq. (14): the integer that stands for 1.0 is floor(1 / S_delta). */
@@ -108,7 +110,7 @@ int oracle_softmax_prepare(double in_scale, int row_len, int out_bits, int varia
     out->dcap = (int32_t)(34 * x0);
 
     int64_t unit;  /* value of the exponential at distance 0 */
-    if (variant == ORACLE_SM_POLY) {
+    if (variant == ORACLE_SM_POLY || variant == ORACLE_SM_LOG2) {
         /* reading: second-order exp polynomial of the cited polynomial method,
          * exp(p) ~ a (p + b)^2 + c on p in (-ln2, 0]; a is absorbed in the scale. */
         const double a = 0.3585, b = 1.353, cc = 0.344;
@@ -147,7 +149,7 @@ static int64_t phi_bitexp(int64_t u) { return fshr(u, 1) + fshr(u, 3) + fshr(u, 
 int64_t oracle_softmax_exp(int64_t d, const oracle_softmax_consts_t* c)
 {
     int64_t x0 = c->x0;
-    if (c->variant == ORACLE_SM_POLY) {
+    if (c->variant == ORACLE_SM_POLY || c->variant == ORACLE_SM_LOG2) {
         int64_t z = d / c->qln2;                       /* octave */
         int64_t p = -(d - z * c->qln2);                /* in (-qln2, 0] */
         int64_t poly = (p + c->qb) * (p + c->qb) + c->qc;
@@ -184,6 +186,21 @@ void oracle_softmax_row(const int64_t* s, const uint8_t* mask, int n, const orac
         if (d > c->dcap) d = c->dcap;
         e[j] = oracle_softmax_exp(d, c);
         sum += e[j];
+    }
+    if (c->variant == ORACLE_SM_LOG2) {
+        /* reading (the "logarithm" candidate of Sec. 3.2 is named, not defined): the probability is rounded to a
+         * power of two, p = 2^-code, code = round(log2(round(sum / e))) kept in 4 bits; smaller probabilities,
+         * and entries whose exponential is 0, are exactly 0 (code ORACLE_LOG2_ZERO).  Integer form of the
+         * rounded logarithm: the position of the leading one, plus one when the bit below it is set. */
+        for (int j = 0; j < n; j++) {
+            if (e[j] == 0) { p[j] = ORACLE_LOG2_ZERO; continue; }
+            int64_t r = (2 * sum + e[j]) / (2 * e[j]);             /* round(sum / e), halves up; >= 1 */
+            int fl = bitlen_u64((uint64_t)r) - 1;                  /* floor(log2 r) */
+            int code = fl + ((fl >= 1 && ((r >> (fl - 1)) & 1)) ? 1 : 0);
+            p[j] = code > 15 ? ORACLE_LOG2_ZERO : (uint8_t)code;
+        }
+        free(e);
+        return;
     }
     /* Eq. (15): IntDiv. */
     int64_t f = have ? (((int64_t)1 << c->M) / sum) : 0;
@@ -450,7 +467,13 @@ int oracle_attention_strided(const int8_t* q, const int8_t* k, const int8_t* v, 
             oracle_softmax_row(s, mask_id ? msk : NULL, N, sc, p);
             for (int d = 0; d < dh; d++) {
                 int64_t acc = 0;
-                for (int j = 0; j < N; j++) acc += (int64_t)p[j] * vp[j * tok_stride + d];
+                if (sc->variant == ORACLE_SM_LOG2) {
+                    /* shift-accumulate: p = 2^-code at scale 2^-15, i.e. the value shifted left by 15 - code */
+                    for (int j = 0; j < N; j++)
+                        if (p[j] != ORACLE_LOG2_ZERO) acc += (int64_t)vp[j * tok_stride + d] << (15 - p[j]);
+                } else {
+                    for (int j = 0; j < N; j++) acc += (int64_t)p[j] * vp[j * tok_stride + d];
+                }
                 out[(b * N + i) * (int64_t)(H * dh) + h * dh + d] = (int8_t)oracle_requant((int32_t)acc, out_rq);
             }
         }

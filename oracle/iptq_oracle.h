@@ -15,7 +15,7 @@
  * "reading:" beside the choice that was made.
  *
  * Parity status: every function below is pinned by CPU tests except
- *   - ORACLE_SM_POLY and ORACLE_GELU_SHIFT: the paper names these candidates
+ *   - ORACLE_SM_POLY, ORACLE_SM_LOG2 and ORACLE_GELU_SHIFT: the paper names these candidates
  *     (Sec. 3.2) but defines neither; pinned only against the float functions
  *     they approximate, with constants from the cited prior work
  *     ("parity unpinned" beyond that);
@@ -35,7 +35,10 @@ extern "C" {
 
 enum { ORACLE_OK = 0, ORACLE_ERR_RANGE = 1, ORACLE_ERR_ARG = 2 };
 
-enum { ORACLE_SM_BITEXP = 0, ORACLE_SM_SHIFTMAX = 1, ORACLE_SM_POLY = 2 };
+enum { ORACLE_SM_BITEXP = 0, ORACLE_SM_SHIFTMAX = 1, ORACLE_SM_POLY = 2, ORACLE_SM_LOG2 = 3 };
+/* ORACLE_SM_LOG2 writes codes instead of probabilities: p = 2^-code for code 0..15, ORACLE_LOG2_ZERO for p = 0;
+ * the attention then accumulates shifted values at scale 2^-15. */
+#define ORACLE_LOG2_ZERO 255
 enum { ORACLE_GELU_POLY4 = 0, ORACLE_GELU_POLY2 = 1, ORACLE_GELU_SHIFT = 2 };
 enum { ORACLE_LN_SHIFT = 0, ORACLE_LN_NEWTON = 1, ORACLE_LN_PTF = 2 };
 

@@ -105,13 +105,19 @@ def softmax_deq(probs: np.ndarray, out_bits: int) -> np.ndarray:
     return np.asarray(probs, dtype=np.float64) / float(1 << (out_bits - 1))
 
 
+def log2_deq(codes: np.ndarray) -> np.ndarray:
+    """Logarithm candidate: probability 2^-code for codes 0..15, 0 for the "zero" code 255."""
+    c = np.asarray(codes)
+    return np.where(c == 255, 0.0, np.exp2(-np.minimum(c, 15).astype(np.float64)))
+
+
 def affine_deq(y: np.ndarray, out_scale: float, out_zp: int) -> np.ndarray:
     return (np.asarray(y, dtype=np.float64) - float(out_zp)) * out_scale
 
 
 # ------------------------------------------------------------------ Eq. (20): operation counts (this library's reading)
 
-_SOFTMAX_PER_ELEM = {0: 21, 1: 17, 2: 15}     # SM_BITEXP, SM_SHIFTMAX, SM_POLY
+_SOFTMAX_PER_ELEM = {0: 21, 1: 17, 2: 15, 3: 22}     # SM_BITEXP, SM_SHIFTMAX, SM_POLY, SM_LOG2
 _GELU_PER_ELEM = {0: 20, 1: 19, 2: 33}        # GELU_POLY4, GELU_POLY2, GELU_SHIFT
 _LN_PER_ELEM = {0: 15, 1: 15, 2: 16}          # LN_SHIFT, LN_NEWTON, LN_PTF (one more shift per element)
 _LN_PER_ROW = {0: 34, 1: 22, 2: 22}           # variance 3, square root (10 fixed steps / about 6 Newton steps, 3 each), reciprocal 1
@@ -123,7 +129,8 @@ def op_count(kind: int, variant: int, rows: int, row_len: int) -> float:
     Softmax, per element: running max 1, distance 1, clamp 1, Eq. (7) 4, Eq. (8) 3 (divide, multiply, subtract),
     Phi + x0 6 (Bit-exp; 2 for Shiftmax), Eq. (9) 2, sum 1, Eq. (15) 2; one division per row.  Second-order
     polynomial exponential: max 1, distance 1, clamp 1, octave divide 1, remainder 2, polynomial 3, normalise 2,
-    octave shift 1, sum 1, Eq. (15) 2.
+    octave shift 1, sum 1, Eq. (15) 2.  Logarithm candidate: the same exponential and sum (13), round(sum / e) 4,
+    leading-one position 1, rounding bit 3, clamp 1, no division per row.
     GELU, per element: clamp 2, |x| 1, min 1, subtract 1, square 1, shift 1, second square 1 (fourth order only),
     C - (.) 1, sign 1, + C 1, shift 1, x * G 1, requantise 6 (multiply, round, shift, zero point, two clamps).
     Shift-based sigmoid form: 1.702 x by shifts 6, |.| and clamp 2, exponential 11, D + e 1, divide 1, select 1,
@@ -135,7 +142,7 @@ def op_count(kind: int, variant: int, rows: int, row_len: int) -> float:
     """
     n = float(rows) * float(row_len)
     if kind == SOFTMAX:
-        return _SOFTMAX_PER_ELEM[variant] * n + float(rows)
+        return _SOFTMAX_PER_ELEM[variant] * n + (0.0 if variant == 3 else float(rows))
     if kind == GELU:
         return _GELU_PER_ELEM[variant] * n
     if kind == LAYERNORM:
