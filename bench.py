@@ -587,7 +587,7 @@ def bench_assignment(api, torch, dev):
         layers, omega, n_eval = run()
         times.append(time.perf_counter() - t0)
     t = statistics.median(times)
-    names = {api.LAYER_SOFTMAX: ("bit", "shiftmax", "poly"), api.LAYER_GELU: ("poly4", "poly2", "shift"),
+    names = {api.LAYER_SOFTMAX: ("bit", "shiftmax", "poly", "log2"), api.LAYER_GELU: ("poly4", "poly2", "shift"),
              api.LAYER_LAYERNORM: ("shift", "newton", "ptf")}
     kinds = {api.LAYER_SOFTMAX: "softmax", api.LAYER_GELU: "gelu", api.LAYER_LAYERNORM: "layernorm"}
     chosen = {}
@@ -602,7 +602,8 @@ def bench_assignment(api, torch, dev):
         for c in l.candidates:
             v = c.variant
             if kind == "softmax":
-                q = om.softmax_deq(oracle.softmax(d["scores"], oracle.softmax_prepare(d["in_scale"], N, 8, v)), 8)
+                pq = oracle.softmax(d["scores"], oracle.softmax_prepare(d["in_scale"], N, 4 if v == 3 else 8, v))
+                q = om.log2_deq(pq) if v == 3 else om.softmax_deq(pq, 8)
                 x = om.softmax_float(d["scores"], d["in_scale"])
                 ops = om.op_count(om.SOFTMAX, v, d["scores"].shape[0], N)
             elif kind == "gelu":
@@ -621,7 +622,7 @@ def bench_assignment(api, torch, dev):
             agree += int(abs(term - c.term) <= 1e-9 * term and abs(pp - c.perturbation) <= 1e-9 * pp)
             terms.append(term)
     t_cpu = time.perf_counter() - t0
-    return {"workload": "DeiT-Small encoder, 49 non-linear layers, calibration batch 8 (synthetic), 3 candidates each",
+    return {"workload": "DeiT-Small encoder, 49 non-linear layers, calibration batch 8 (synthetic), 4 Softmax / 3 GELU / 3 LayerNorm candidates",
             "layers": len(layers), "evaluations": int(n_eval), "ms": 1e3 * t, "evaluations_per_s": n_eval / t,
             "omega": omega, "selected": chosen,
             "oracle_first_block": {"evaluations": compared, "agree_within_1e-9": agree, "seconds": t_cpu}}

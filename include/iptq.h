@@ -49,7 +49,8 @@ typedef enum {
 typedef enum {
     IPTQ_SM_BITEXP = 0,    /* Efficient Bit-Softmax, Eqs. (13)-(15) (the paper's own; default) */
     IPTQ_SM_SHIFTMAX = 1,  /* bit-shifting candidate, Eqs. (7)-(10) */
-    IPTQ_SM_POLY = 2       /* polynomial candidate (second-order integer exp) */
+    IPTQ_SM_POLY = 2,      /* polynomial candidate (second-order integer exp) */
+    IPTQ_SM_LOG2 = 3       /* logarithm candidate: probabilities rounded to powers of two, 4-bit codes */
 } iptq_softmax_variant;
 typedef enum {
     IPTQ_GELU_POLY4 = 0,   /* Data-aware Poly-GELU, Eqs. (3), (5) (the paper's own; default) */
@@ -92,7 +93,13 @@ int iptq_channel_requant_prepare(const double* ratios, int n, int32_t* mult, int
  * (Eq. (8)); e = ((Phi(-r) + x0) << nsh) >> q with Phi(u) = (u>>1)+(u>>3)+(u>>4)
  * (Eqs. (9), (13), (14)); p = (floor(2^M / sum e) * e) >> (M - (out_bits-1)) (Eq. (15)).
  * Output: uint8 probabilities at scale 2^-(out_bits-1), values in [0, 2^(out_bits-1)].
+ *
+ * IPTQ_SM_LOG2 (the "logarithm" candidate of Sec. 3.2, which the paper names without defining; out_bits must be
+ * 4): with the polynomial exponential e and its row sum, r = round(sum / e) and
+ * code = round(log2 r) = position of the leading one of r, plus one when the bit below it is set; the output byte
+ * is that code (probability 2^-code) for code <= 15 and IPTQ_LOG2_ZERO (probability 0) beyond or where e = 0.
  */
+#define IPTQ_LOG2_ZERO 255
 typedef struct {
     int32_t variant, out_bits, row_len;
     int32_t x0, nsh, M, dcap;
@@ -105,7 +112,8 @@ typedef struct {
 } iptq_softmax_consts;
 
 /* host.  in_scale: scale of the scores (1/sqrt(d_head) folded in); needs 8 <= floor(1/in_scale) < 2^24
- * and row_len * (x0 << nsh) < 2^31 (IPTQ_ERR_SCALE_RANGE); out_bits in [4, 8]; 1 <= row_len <= 1024. */
+ * and row_len * (x0 << nsh) < 2^31 (IPTQ_ERR_SCALE_RANGE); out_bits in [4, 8] (IPTQ_SM_LOG2: 4, else
+ * IPTQ_ERR_BITS); 1 <= row_len <= 1024. */
 int iptq_softmax_prepare(double in_scale, int row_len, int out_bits, iptq_softmax_variant variant,
                          iptq_softmax_consts* out /*host*/);
 /* The shift-based exponentials (IPTQ_SM_BITEXP, IPTQ_SM_SHIFTMAX) of Eq. (9) are 0 from some d = max - s on (a
@@ -320,7 +328,8 @@ int iptq_encoder_block_profiled(const int8_t* x, int8_t* y, const iptq_block_par
  * integer output, iptq_metric_*() evaluate X in fp64 on the de-quantised integer input and reduce
  *     sums[0] = sum X^2,   sums[1] = sum (X - Qd)^2
  * over the whole tensor with a fixed summation order (the same device and sizes give the same bits).
- *   Softmax:   X = softmax(in_scale * scores) per row;  Qd = probs * 2^-(out_bits-1)
+ *   Softmax:   X = softmax(in_scale * scores) per row;  Qd = probs * 2^-(out_bits-1), or, with out_bits =
+ *              IPTQ_PROBS_LOG2, 2^-code of the IPTQ_SM_LOG2 codes in probs (0 for IPTQ_LOG2_ZERO)
  *   GELU:      X = v/2 (1 + erf(v / sqrt 2)), v = in_scale * x;  Qd = (y - out_zp) * out_scale
  *   LayerNorm: X = (v - mean)/std * gamma + beta per row, v = x << ptf_shift[channel] (biased variance, no
  *              epsilon; a constant row gives beta);  Qd = (y - out_zp) * out_scale
@@ -329,6 +338,7 @@ int iptq_encoder_block_profiled(const int8_t* x, int8_t* y, const iptq_block_par
  * float [dim] (the float parameters handed to iptq_layernorm_prepare); ptf_shift nullable.  row_len <= 1024,
  * dim % 4 == 0 and dim <= 3072 as for the kernels measured.  Empty tensors give sums of 0. */
 #define IPTQ_METRIC_WORK_BYTES 32768
+#define IPTQ_PROBS_LOG2 0
 int iptq_metric_softmax(const int32_t* scores, const uint8_t* probs, int64_t rows, int row_len, double in_scale,
                         int out_bits, double* sums, void* work, iptq_stream_t stream);
 int iptq_metric_gelu(const int32_t* x, const int8_t* y, int64_t n, double in_scale, double out_scale, int out_zp,

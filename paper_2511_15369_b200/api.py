@@ -15,7 +15,9 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libiptq.so")
 
-SM_BITEXP, SM_SHIFTMAX, SM_POLY = 0, 1, 2
+SM_BITEXP, SM_SHIFTMAX, SM_POLY, SM_LOG2 = 0, 1, 2, 3
+LOG2_ZERO = 255          # SM_LOG2 output: code c <= 15 means probability 2^-c, LOG2_ZERO means 0
+PROBS_LOG2 = 0           # out_bits value that tells metric_softmax the bytes are SM_LOG2 codes
 GELU_POLY4, GELU_POLY2, GELU_SHIFT = 0, 1, 2
 LN_SHIFT, LN_NEWTON, LN_PTF = 0, 1, 2
 

@@ -16,7 +16,7 @@ import torch
 
 from . import api
 
-SOFTMAX_CANDIDATES = (api.SM_BITEXP, api.SM_SHIFTMAX, api.SM_POLY)
+SOFTMAX_CANDIDATES = (api.SM_BITEXP, api.SM_SHIFTMAX, api.SM_POLY, api.SM_LOG2)
 GELU_CANDIDATES = (api.GELU_POLY4, api.GELU_POLY2, api.GELU_SHIFT)
 LN_CANDIDATES = (api.LN_SHIFT, api.LN_NEWTON, api.LN_PTF)
 
@@ -72,14 +72,15 @@ class Analyzer:
         layer = Layer(name, api.LAYER_SOFTMAX)
         probs = torch.empty((rows, n), dtype=torch.uint8, device=scores.device)
         for v in variants:
+            bits = 4 if v == api.SM_LOG2 else out_bits         # the logarithm candidate writes 4-bit codes
             try:
-                c = api.softmax_prepare(in_scale, n, out_bits, v)
+                c = api.softmax_prepare(in_scale, n, bits, v)
             except api.IptqError:
                 continue                   # this candidate has no integer constants at this scale
             self._keep.append(api.softmax_table(c, scores.device))
             api.softmax(scores, c, out=probs)
             slot = self._slot()
-            api.metric_softmax(scores, probs, in_scale, out_bits, scratch=slot)
+            api.metric_softmax(scores, probs, in_scale, api.PROBS_LOG2 if v == api.SM_LOG2 else bits, scratch=slot)
             layer.candidates.append(Candidate(v, api.op_count(api.LAYER_SOFTMAX, v, rows, n), self.n_eval - 1))
         self.layers.append(layer)
         return layer

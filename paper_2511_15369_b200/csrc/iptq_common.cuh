@@ -137,7 +137,7 @@ struct ExpDev {
 template <int VARIANT>
 __device__ __forceinline__ unsigned exp_core_nd(int nd, const ExpDev& c)
 {
-    if (VARIANT == IPTQ_SM_POLY) {
+    if (VARIANT == IPTQ_SM_POLY || VARIANT == IPTQ_SM_LOG2) {
         const unsigned d = (unsigned)(-nd);
         unsigned z = __umulhi(d, c.div_mul) >> c.div_shift;          // octave: floor(d / qln2)
         int t = (int)(z * (unsigned)c.qln2) - (int)d + c.qb;           // p + qb, p in (-qln2, 0]
@@ -166,12 +166,24 @@ __device__ __forceinline__ unsigned exp_core(unsigned d, const ExpDev& c)
 // d >= 16 qz x0 / 23 + 15.  Returns 0 where no 16-bit table exists (polynomial variant, values of 2^16 and more).
 inline int exp_table_entries(const iptq_softmax_consts& sm)
 {
-    if (sm.variant == IPTQ_SM_POLY) return 0;
+    if (sm.variant == IPTQ_SM_POLY || sm.variant == IPTQ_SM_LOG2) return 0;
     int qz = 0;
     for (int64_t u = (int64_t)sm.x0 << sm.nsh; u; u >>= 1) ++qz;
     if (qz > 16) return 0;
     const int64_t n = (16 * (int64_t)qz * sm.x0) / 23 + 32;
     return n > (1 << 20) ? 0 : (int)n;
+}
+
+// Logarithm candidate: code = round(log2(round(sum / e))) for 0 < e <= sum < 2^31, IPTQ_LOG2_ZERO beyond 15 or for
+// e = 0.  round(sum / e) with halves up is (sum + (e >> 1)) / e: for odd e no multiple of e lies between
+// sum + (e - 1)/2 and sum + e/2.  The rounded logarithm is the position of the leading one, plus the bit below it.
+__device__ __forceinline__ unsigned log2_code(unsigned sum, unsigned e)
+{
+    if (e == 0) return IPTQ_LOG2_ZERO;
+    const unsigned r = (sum + (e >> 1)) / e;                 // >= 1
+    const int fl = 31 - __clz((int)r);
+    const unsigned code = (unsigned)fl + (fl >= 1 ? ((r >> (fl - 1)) & 1u) : 0u);
+    return code > 15u ? (unsigned)IPTQ_LOG2_ZERO : code;
 }
 
 // floor(2^M / sum) for 0 < sum < 2^31, M <= 40: the fp64 quotient cannot round across an integer

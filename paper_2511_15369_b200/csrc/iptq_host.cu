@@ -127,7 +127,9 @@ int iptq_softmax_prepare(double in_scale, int row_len, int out_bits, iptq_softma
     if (!out) return IPTQ_ERR_NULL;
     if (row_len < 1 || row_len > 1024) return IPTQ_ERR_SHAPE;
     if (out_bits < 4 || out_bits > 8) return IPTQ_ERR_BITS;
-    if (variant != IPTQ_SM_BITEXP && variant != IPTQ_SM_SHIFTMAX && variant != IPTQ_SM_POLY) return IPTQ_ERR_VARIANT;
+    if (variant != IPTQ_SM_BITEXP && variant != IPTQ_SM_SHIFTMAX && variant != IPTQ_SM_POLY &&
+        variant != IPTQ_SM_LOG2) return IPTQ_ERR_VARIANT;
+    if (variant == IPTQ_SM_LOG2 && out_bits != 4) return IPTQ_ERR_BITS;     // 4-bit codes
     if (!(in_scale > 0.0)) return IPTQ_ERR_SCALE_RANGE;
     std::memset(out, 0, sizeof(*out));
     const double one = std::floor(1.0 / in_scale);           // Eq. (14): the integer 1.0
@@ -137,7 +139,7 @@ int iptq_softmax_prepare(double in_scale, int row_len, int out_bits, iptq_softma
     out->x0 = (int32_t)x0;
     out->dcap = (int32_t)(34 * x0);
     int64_t unit;
-    if (variant == IPTQ_SM_POLY) {
+    if (variant == IPTQ_SM_POLY || variant == IPTQ_SM_LOG2) {
         const double a = 0.3585, b = 1.353, c = 0.344;       // exp(p) ~ a (p + b)^2 + c on (-ln 2, 0]
         const double l2 = std::floor(std::log(2.0) / in_scale);
         const double qb = std::floor(b / in_scale);

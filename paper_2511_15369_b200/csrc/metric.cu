@@ -70,7 +70,11 @@ metric_softmax_kernel(const int32_t* __restrict__ scores, const uint8_t* __restr
         den = warp_sum(den);
         for (int j = lane; j < n; j += 32) {
             const double X = exp((double)__ldg(sr + j) * in_scale - zmax) / den;
-            const double d = X - (double)__ldg(pr + j) * out_step;
+            const unsigned pb = __ldg(pr + j);
+            // out_step = 0: the byte is a logarithm-candidate code, 2^-code (255: zero) built from the exponent bits
+            const double Qd = out_step != 0.0 ? (double)pb * out_step
+                                              : (pb == IPTQ_LOG2_ZERO ? 0.0 : __longlong_as_double((long long)(1023 - (int)min(pb, 15u)) << 52));
+            const double d = X - Qd;
             ax2 += X * X;
             ae2 += d * d;
         }
@@ -165,12 +169,13 @@ int iptq_metric_softmax(const int32_t* scores, const uint8_t* probs, int64_t row
     int rc = metric_args_ok(sums, work);
     if (rc != IPTQ_OK) return rc;
     if (rows < 0 || row_len < 1 || row_len > 1024) return IPTQ_ERR_SHAPE;
-    if (out_bits < 4 || out_bits > 8) return IPTQ_ERR_BITS;
+    if (out_bits != IPTQ_PROBS_LOG2 && (out_bits < 4 || out_bits > 8)) return IPTQ_ERR_BITS;
     if (!(in_scale > 0.0)) return IPTQ_ERR_SCALE_RANGE;
     if (rows > 0 && (!scores || !probs)) return IPTQ_ERR_NULL;
     const int grid = metric_grid((rows + 7) / 8);
+    const double out_step = out_bits == IPTQ_PROBS_LOG2 ? 0.0 : 1.0 / (double)(1 << (out_bits - 1));
     launch_kernel(metric_softmax_kernel, grid, kMetricThreads, 0, stream, scores, probs, rows, row_len, in_scale,
-                  1.0 / (double)(1 << (out_bits - 1)), (double*)work);
+                  out_step, (double*)work);
     return metric_finish((double*)work, grid, sums, stream);
 }
 
@@ -234,12 +239,13 @@ double iptq_metric_term(double sqnr_db, double perturbation, double op_count, do
 // iterated to convergence) and the reciprocal (1).
 double iptq_op_count(int layer_kind, int variant, int64_t rows, int row_len)
 {
-    if (variant < 0 || variant > 2 || rows < 0 || row_len < 0) return -1.0;
+    if (variant < 0 || variant > (layer_kind == IPTQ_LAYER_SOFTMAX ? 3 : 2) || rows < 0 || row_len < 0) return -1.0;
     const double r = (double)rows, n = (double)rows * (double)row_len;
     switch (layer_kind) {
         case IPTQ_LAYER_SOFTMAX: {
-            static const double per_elem[3] = {21.0, 17.0, 15.0};
-            return per_elem[variant] * n + r;
+            // logarithm candidate: exponential and sum 13, round(sum / e) 4, leading one 1, rounding bit 3, clamp 1
+            static const double per_elem[4] = {21.0, 17.0, 15.0, 22.0};
+            return per_elem[variant] * n + (variant == IPTQ_SM_LOG2 ? 0.0 : r);
         }
         case IPTQ_LAYER_GELU: {
             static const double per_elem[3] = {20.0, 19.0, 33.0};

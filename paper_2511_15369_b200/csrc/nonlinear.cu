@@ -57,8 +57,16 @@ softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ pr
             sum += e;
         }
         sum = __reduce_add_sync(kFull, sum);
-        const unsigned f = intdiv_factor(sum, c.M) << c.f_shl;  // Eq. (15)
         uint8_t* pr = probs + row * n;
+        if (VARIANT == IPTQ_SM_LOG2) {
+#pragma unroll
+            for (int k = 0; k < NITER; ++k) {
+                const int j = lane + 32 * k;
+                if (j < n) __stcs(pr + j, (uint8_t)log2_code(sum, (unsigned)v[k]));
+            }
+            continue;
+        }
+        const unsigned f = intdiv_factor(sum, c.M) << c.f_shl;  // Eq. (15)
 #pragma unroll
         for (int k = 0; k < NITER; ++k) {
             const int j = lane + 32 * k;
@@ -152,7 +160,7 @@ template <int VARIANT, int NITER>
 static int launch_softmax2(const int32_t* s, uint8_t* p, int64_t rows, int n, const int32_t* bias, int64_t period,
                            const SoftmaxDev& c, cudaStream_t st)
 {
-    if constexpr (VARIANT != IPTQ_SM_POLY && NITER <= 8)
+    if constexpr (VARIANT != IPTQ_SM_POLY && VARIANT != IPTQ_SM_LOG2 && NITER <= 8)
     if (c.tab_n > 0 && ((c.tab_n + 8) & ~7) <= IPTQ_SOFTMAX_TABLE_MAX &&
         rows * n >= (c.tab_src ? kSmTabMinElemsCopy : kSmTabMinElemsBuild)) {
         // Tabulated exponential: worth the per-CTA table set-up once every warp has several rows.
@@ -547,6 +555,7 @@ int iptq_softmax(const int32_t* scores, uint8_t* probs, int64_t rows, int row_le
         case IPTQ_SM_BITEXP: return launch_softmax1<IPTQ_SM_BITEXP>(scores, probs, rows, row_len, bias, bias_period, c, stream);
         case IPTQ_SM_SHIFTMAX: return launch_softmax1<IPTQ_SM_SHIFTMAX>(scores, probs, rows, row_len, bias, bias_period, c, stream);
         case IPTQ_SM_POLY: return launch_softmax1<IPTQ_SM_POLY>(scores, probs, rows, row_len, bias, bias_period, c, stream);
+        case IPTQ_SM_LOG2: return launch_softmax1<IPTQ_SM_LOG2>(scores, probs, rows, row_len, bias, bias_period, c, stream);
         default: return IPTQ_ERR_VARIANT;
     }
 }

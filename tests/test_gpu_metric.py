@@ -56,6 +56,19 @@ def test_metric_softmax_parity(api, orc, metric, variant, rows, n):
     assert n == 1 or (want[1] > 0 and want[0] > want[1])
 
 
+@pytest.mark.parametrize("rows,n,scale", [(591, 197, synth.SOFTMAX_SCALE_ACC), (1000, 49, 1.0 / 700), (33, 1, 3e-4),
+                                          (300, 197, synth.SOFTMAX_SCALE_8BIT)])
+def test_metric_softmax_log2_candidate(api, orc, metric, rows, n, scale):
+    s = synth.quantize_scores(synth.softmax_logits(rows, n, seed=rows), scale)
+    codes = orc.softmax(s, orc.softmax_prepare(scale, n, 4, orc.SM_LOG2))
+    want = metric.error_sums(metric.softmax_float(s, scale), metric.log2_deq(codes))
+    sd = _cu(s)
+    cd = api.softmax(sd, api.softmax_prepare(scale, n, 4, api.SM_LOG2))
+    assert (cd.cpu().numpy() == codes).all()
+    got = api.metric_softmax(sd, cd, scale, api.PROBS_LOG2).cpu().numpy()
+    assert _close(got, want), (got, want)
+
+
 @pytest.mark.parametrize("out_bits", [8, 6, 4])
 def test_metric_softmax_out_bits_and_determinism(api, orc, metric, out_bits):
     S, rows, n = synth.SOFTMAX_SCALE_8BIT, 700, 197
@@ -137,9 +150,9 @@ def _oracle_analysis(orc, metric, layers, c_unit):
         if kind == "softmax":
             s, S = d["scores"], d["in_scale"]
             X = metric.softmax_float(s, S)
-            for v in (0, 1, 2):
-                p = orc.softmax(s, orc.softmax_prepare(S, s.shape[1], 8, v))
-                cands.append((v,) + metric.evaluate(X, metric.softmax_deq(p, 8),
+            for v in (0, 1, 2, 3):
+                p = orc.softmax(s, orc.softmax_prepare(S, s.shape[1], 4 if v == 3 else 8, v))
+                cands.append((v,) + metric.evaluate(X, metric.log2_deq(p) if v == 3 else metric.softmax_deq(p, 8),
                                                     metric.op_count(metric.SOFTMAX, v, s.shape[0], s.shape[1]), c_unit))
         elif kind == "gelu":
             x, S = d["x"], d["in_scale"]
@@ -167,7 +180,7 @@ def _oracle_analysis(orc, metric, layers, c_unit):
 
 @pytest.mark.parametrize("c_unit", [1.0e6, 1.0e9])
 def test_assignment_matches_oracle(api, orc, metric, c_unit):
-    """DeiT-Tiny-sized encoder, two blocks, one image: 9 layers, up to 27 evaluations."""
+    """DeiT-Tiny-sized encoder, two blocks, one image: 9 layers, up to 29 evaluations."""
     from paper_2511_15369_b200 import assign
     layers = list(synth.calibration_layers(192, 3, 197, 768, 2, 1, seed=4))
     an = assign.Analyzer(c_unit=c_unit)

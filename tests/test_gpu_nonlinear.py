@@ -112,6 +112,29 @@ def test_softmax_table_absent(api):
     assert rc == api.ERR_SHAPE and not c.table
 
 
+@pytest.mark.parametrize("rows,n", [(591, 197), (1000, 49), (33, 1), (17, 2), (9, 1000), (5000, 64)])
+@pytest.mark.parametrize("scale", [synth.SOFTMAX_SCALE_ACC, synth.SOFTMAX_SCALE_8BIT])
+def test_softmax_log2_parity(api, orc, rows, n, scale):
+    """Logarithm candidate: 4-bit power-of-two codes (255 = probability 0), with and without bias."""
+    s = synth.quantize_scores(synth.softmax_logits(rows, n, seed=rows + n), scale)
+    s[0] = 3                                                  # all-equal row
+    if n > 2:
+        s[1] = -(1 << 30) + 1
+        s[1, 1] = (1 << 30) - 1                               # everything but one entry vanishes
+    co = orc.softmax_prepare(scale, n, 4, orc.SM_LOG2)
+    ca = api.softmax_prepare(scale, n, 4, api.SM_LOG2)
+    want = orc.softmax(s, co)
+    got = api.softmax(_cu(s), ca).cpu().numpy()
+    assert (got == want).all()
+    assert ((got <= 15) | (got == api.LOG2_ZERO)).all()
+    bias = np.random.default_rng(1).integers(-2000, 2000, size=(4, n)).astype(np.int32)
+    got_b = api.softmax(_cu(s), ca, bias=_cu(bias)).cpu().numpy()
+    assert (got_b == orc.softmax(s, co, bias=bias, bias_period=4)).all()
+    with pytest.raises(api.IptqError) as e:
+        api.softmax_prepare(scale, n, 8, api.SM_LOG2)
+    assert e.value.status == api.ERR_BITS
+
+
 def test_softmax_edge_rows_and_bias(api, orc):
     n = 197
     rng = np.random.default_rng(3)

@@ -34,10 +34,10 @@ def test_metric_term_matches_oracle():
 
 def test_op_counts_and_selection_match_oracle():
     for kind in (0, 1, 2):
-        for v in (0, 1, 2):
+        for v in (0, 1, 2, 3) if kind == 0 else (0, 1, 2):
             for rows, n in ((1, 1), (197, 197), (9456, 197), (1576, 3072), (0, 64)):
                 assert api.op_count(kind, v, rows, n) == metric.op_count(kind, v, rows, n)
-    assert api.op_count(3, 0, 1, 1) < 0 and api.op_count(0, 3, 1, 1) < 0 and api.op_count(0, -1, 1, 1) < 0
+    assert api.op_count(3, 0, 1, 1) < 0 and api.op_count(0, 4, 1, 1) < 0 and api.op_count(1, 3, 1, 1) < 0 and api.op_count(0, -1, 1, 1) < 0
     rng = np.random.default_rng(2)
     for _ in range(50):
         t = list(rng.integers(0, 4, size=rng.integers(1, 6)) / 4.0)
