@@ -25,8 +25,10 @@ def block_params(spec, table) -> dict:
     for name, ls in (("qkv", spec.qkv), ("proj", spec.proj), ("fc1", spec.fc1), ("fc2", spec.fc2)):
         d["w_" + name], d["b_" + name] = ls.w_packed, ls.bias
         d["m_" + name], d["s_" + name] = _channel_requant(ls.ratio)
-    d["sm"] = oracle.softmax_prepare(spec.softmax_scale, sh.N, 8, sm_v)
-    d["pv_rq"] = oracle.requant_prepare(spec.pv_ratio)
+    # the logarithm candidate writes 4-bit codes and its P V product is at scale 2^-15 instead of 2^-7
+    log2 = sm_v == oracle.SM_LOG2
+    d["sm"] = oracle.softmax_prepare(spec.softmax_scale, sh.N, 4 if log2 else 8, sm_v)
+    d["pv_rq"] = oracle.requant_prepare(spec.pv_ratio / 256 if log2 else spec.pv_ratio)
     d["attn_bias"], d["mask_id"] = spec.attn_bias, spec.mask_id
     d["res1_rq"] = oracle.requant_prepare(spec.proj.res_ratio / 65536, zp=spec.proj.res_zp)
     d["res2_rq"] = oracle.requant_prepare(spec.fc2.res_ratio / 65536, zp=spec.fc2.res_zp)

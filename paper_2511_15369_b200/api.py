@@ -475,11 +475,13 @@ class EncoderBlock:
             setattr(p, "s_" + name, dev(s))
         p.attn_bias = dev(spec.attn_bias)
         p.mask_id = dev(spec.mask_id)
-        sc = softmax_prepare(spec.softmax_scale, sh.N, 8, sm_v)
+        # the logarithm candidate writes 4-bit codes and its P V product is at scale 2^-15 instead of 2^-7
+        log2 = sm_v == SM_LOG2
+        sc = softmax_prepare(spec.softmax_scale, sh.N, 4 if log2 else 8, sm_v)
         if softmax_table_on:
             self.keep.append(softmax_table(sc, device))
         p.sm = host(sc)
-        p.pv_rq = host(requant_prepare(spec.pv_ratio))
+        p.pv_rq = host(requant_prepare(spec.pv_ratio / 256 if log2 else spec.pv_ratio))
         p.proj_zp, p.fc2_zp = spec.proj.out_zp, spec.fc2.out_zp
         p.res1_rq = host(requant_prepare(spec.proj.res_ratio / 65536.0, zp=spec.proj.res_zp))
         p.res2_rq = host(requant_prepare(spec.fc2.res_ratio / 65536.0, zp=spec.fc2.res_zp))

@@ -34,6 +34,7 @@ struct AttnParams {
     int o_col;             // first TMEM column of O
     int q_bytes, k_bytes, v_bytes, stage_bytes;
     int p_off, p_bytes, xch_off, bar_off;
+    int p_plane;           // bytes of one P operand; the logarithm candidate keeps two per buffer (p_bytes = 2 p_plane)
     int stages;            // Q/K/V ring depth (3, or 2 when the exponential table needs the room)
     int lut_off, lut_n;    // exponential table: e(d) for d < lut_n, 0 beyond (lut_n = 0: no table)
     const uint16_t* lut_src;   // the same table in device memory (copied), or null (built by each CTA)
@@ -157,6 +158,11 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     // B = V [keys, DH]: MN-major (DH contiguous), DH-byte swizzle, 8-key groups 8*DH apart
                     const uint64_t db = umma_smem_desc(v_addr + ks * 32 * DH, 8 * DH, 8 * DH, DH);
                     umma_i8(tmem_o, da, db, idesc_o, ks != 0 ? 1u : 0u);
+                    if constexpr (VARIANT == IPTQ_SM_LOG2) {
+                        // low-order plane (probabilities 2^-8 .. 2^-15) into its own accumulator behind the first
+                        const uint64_t da2 = umma_smem_desc(p_addr + p.p_plane + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, 128);
+                        umma_i8(tmem_o + (uint32_t)DH, da2, db, idesc_o, ks != 0 ? 1u : 0u);
+                    }
                 }
                 umma_commit(&kv_empty[s_prev]);                // the stage may be refilled
                 umma_commit(o_full);
@@ -225,6 +231,14 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             if (mt * 128 + quad * 32 < p.N && part < OPARTS) {
                 uint32_t r[16];
                 tmem_ld16(trow + (uint32_t)(p.o_col + part * 16), r);
+                if constexpr (VARIANT == IPTQ_SM_LOG2) {
+                    // O = 2^8 * (high plane product) + (low plane product), at scale 2^-15
+                    uint32_t r2[16];
+                    tmem_ld16(trow + (uint32_t)(p.o_col + DH + part * 16), r2);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) r[j] = (uint32_t)(((int)r[j] << 8) + (int)r2[j]);
+                }
                 tmem_wait_ld();
                 int o[16];
 #pragma unroll
@@ -333,6 +347,34 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 xch_sum[part * 128 + rloc] = sum;
                 named_barrier(1 + quad, 128);
                 sum = (xch_sum[rloc] + xch_sum[128 + rloc]) + (xch_sum[256 + rloc] + xch_sum[384 + rloc]);
+                if constexpr (VARIANT == IPTQ_SM_LOG2) {
+                    // ---- logarithm candidate: p = 2^-code as the 16-bit value 2^(15 - code), split into a high and
+                    //      a low byte plane (exactly one of the two bytes is non-zero), both in the A-operand layout
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        if (i < nch) {
+                            uint32_t wh[4], wl[4];
+#pragma unroll
+                            for (int q4 = 0; q4 < 4; ++q4) {
+                                int hi[4], lo[4];
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) {
+                                    const unsigned code = log2_code(sum, v[i][q4 * 4 + t]);
+                                    const unsigned w16 = code <= 15u ? (0x8000u >> code) : 0u;
+                                    hi[t] = (int)(w16 >> 8);
+                                    lo[t] = (int)(w16 & 0xffu);
+                                }
+                                wh[q4] = pack4_sat_u8(hi[0], hi[1], hi[2], hi[3]);
+                                wl[q4] = pack4_sat_u8(lo[0], lo[1], lo[2], lo[3]);
+                            }
+                            const int c0 = (c_begin + i) * 16;
+                            const int chunk = (c0 & 127) >> 4;
+                            const uint32_t at = p_row + (uint32_t)((c0 >> 7) * 16384 + ((chunk ^ (rloc & 7)) << 4));
+                            st_shared_v4(at, wh[0], wh[1], wh[2], wh[3]);
+                            st_shared_v4(at + (uint32_t)p.p_plane, wl[0], wl[1], wl[2], wl[3]);
+                        }
+                    }
+                } else {
                 // ---- IntDiv (Eq. (15)) -> uint8 probabilities in the UMMA A-operand layout
                 const unsigned f = intdiv_factor(sum, p.M) << p.f_shl;
 #pragma unroll
@@ -355,6 +397,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                         st_shared_v4(p_row + (uint32_t)((c0 >> 7) * 16384 + ((chunk ^ (rloc & 7)) << 4)), w[0], w[1], w[2], w[3]);
                     }
                 }
+                }
             } else {
                 named_barrier_arrive(1 + quad, 128); named_barrier_arrive(1 + quad, 128);   // keeps the barrier generations aligned
             }
@@ -364,6 +407,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 const int c0 = p.npad_s;
                 const int chunk = (c0 & 127) >> 4;
                 st_shared_v4(p_row + (uint32_t)((c0 >> 7) * 16384 + ((chunk ^ (rloc & 7)) << 4)), 0u, 0u, 0u, 0u);
+                if constexpr (VARIANT == IPTQ_SM_LOG2)
+                    st_shared_v4(p_row + (uint32_t)(p.p_plane + (c0 >> 7) * 16384 + ((chunk ^ (rloc & 7)) << 4)), 0u, 0u, 0u, 0u);
             }
             fence_proxy_async_smem();            // generic-proxy stores -> visible to the tensor core's reads
             mbar_arrive(&p_ready[k & 1]);
@@ -445,6 +490,7 @@ static int launch_attn_v(int variant, const CUtensorMap& mq, const CUtensorMap& 
         case IPTQ_SM_BITEXP: return launch_attn<DH, IPTQ_SM_BITEXP>(mq, mk, mv, p, smem_bytes, st);
         case IPTQ_SM_SHIFTMAX: return launch_attn<DH, IPTQ_SM_SHIFTMAX>(mq, mk, mv, p, smem_bytes, st);
         case IPTQ_SM_POLY: return launch_attn<DH, IPTQ_SM_POLY>(mq, mk, mv, p, smem_bytes, st);
+        case IPTQ_SM_LOG2: return launch_attn<DH, IPTQ_SM_LOG2>(mq, mk, mv, p, smem_bytes, st);
         default: return IPTQ_ERR_VARIANT;
     }
 }
@@ -480,7 +526,8 @@ int attention_launch(const AttnArgs& a, cudaStream_t st)
     p.k_bytes = up1k(p.npad_s * a.dh);
     p.v_bytes = up1k(p.kpad * a.dh);
     p.stage_bytes = p.q_bytes + p.k_bytes + p.v_bytes;
-    p.p_bytes = ((p.kpad + 127) / 128) * 16384;
+    p.p_plane = ((p.kpad + 127) / 128) * 16384;
+    p.p_bytes = (a.sm->variant == IPTQ_SM_LOG2 ? 2 : 1) * p.p_plane;
     // Exponential table (shift-based variants with values below 2^16), where it fits beside 3 or 2 operand stages.
     p.lut_n = 0;
     p.stages = ATT_STAGES;
@@ -491,6 +538,8 @@ int attention_launch(const AttnArgs& a, cudaStream_t st)
         else if (fixed + 2 * p.stage_bytes + bytes <= 227 * 1024) { p.lut_n = (int)n; p.stages = 2; }
     }
     p.lut_src = (p.lut_n && a.sm->table && a.sm->table_n == p.lut_n) ? a.sm->table : nullptr;
+    // two operand planes per P buffer (logarithm candidate) leave room for a ring of two only
+    if (fixed + p.stages * p.stage_bytes > 226 * 1024) p.stages = 2;
     const int lut_bytes = p.lut_n ? (int)((2 * ((int64_t)p.lut_n + 1) + 255) & ~255) : 0;
     p.p_off = p.stages * p.stage_bytes;
     p.xch_off = p.p_off + 2 * p.p_bytes;
@@ -499,7 +548,7 @@ int attention_launch(const AttnArgs& a, cudaStream_t st)
     const int smem_bytes = p.bar_off + 256 + 1024;
     p.o_col = (p.npad_s + 31) & ~31;                     // O sits behind S in TMEM
     p.tmem_cols = 32;
-    while ((int)p.tmem_cols < p.o_col + a.dh) p.tmem_cols <<= 1;
+    while ((int)p.tmem_cols < p.o_col + (a.sm->variant == IPTQ_SM_LOG2 ? 2 : 1) * a.dh) p.tmem_cols <<= 1;
     p.bias = a.bias; p.mask_id = a.mask_id; p.out = a.out;
     p.ex = to_dev_exp(*a.sm);
     p.M = a.sm->M; p.f_shl = a.sm->f_shl; p.p_shr = a.sm->p_shr;

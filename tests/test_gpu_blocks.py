@@ -136,7 +136,7 @@ def test_mlp_parity(api, orc, variant, M, D, Dh):
     assert (got == want).all(), _mismatch(got, want)
 
 
-@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("variant", [0, 1, 2, 3])
 @pytest.mark.parametrize("B,H,N,dh,use_bias,use_mask", [
     (2, 3, 197, 64, False, False), (3, 2, 49, 32, True, False), (4, 3, 49, 32, True, True),
     (1, 1, 1, 64, False, False), (2, 2, 128, 64, False, False), (1, 2, 129, 32, False, False),
@@ -148,8 +148,10 @@ def test_attention_parity(api, orc, variant, B, H, N, dh, use_bias, use_mask):
     S = 3.0 / (1600.0 * np.sqrt(dh))
     bias = np.round(rng.normal(0, 1, size=(H, N, N)) / S).astype(np.int32) if use_bias else None
     mask_id = rng.integers(0, 3, size=(B, N)).astype(np.uint8) if use_mask else None
-    so, sa = orc.softmax_prepare(S, N, 8, variant), api.softmax_prepare(S, N, 8, variant)
-    ro, ra = orc.requant_prepare(0.011, zp=1), api.requant_prepare(0.011, zp=1)
+    bits = 4 if variant == 3 else 8                        # the logarithm candidate writes 4-bit codes ...
+    ratio = 0.011 / 256 if variant == 3 else 0.011         # ... and accumulates at scale 2^-15 instead of 2^-7
+    so, sa = orc.softmax_prepare(S, N, bits, variant), api.softmax_prepare(S, N, bits, variant)
+    ro, ra = orc.requant_prepare(ratio, zp=1), api.requant_prepare(ratio, zp=1)
     want = orc.attention_block(q, k, v, so, ro, bias, mask_id)
     ws = api.Workspace(api.attention_workspace_bytes(B, H, N, dh))
     got = api.attention_block(_cu(q), _cu(k), _cu(v), sa, ra, ws, _cu(bias), _cu(mask_id)).cpu().numpy()
@@ -169,6 +171,8 @@ def _oracle_block(orc, spec, table):
     (synth.BlockShape("DeiT-S b2 alt", 2, 197, 384, 6, 64, 1536), 8, (1, 1, 1, 1)),
     (synth.BlockShape("ViT-B b1 W4", 1, 197, 768, 12, 64, 3072), 4, (2, 2, 1, 0)),
     (synth.BlockShape("Swin-T 8 windows", 8, 49, 96, 3, 32, 384, True), 8, (0, 0, 0, 0)),
+    (synth.BlockShape("DeiT-S b2 log2", 2, 197, 384, 6, 64, 1536), 8, (3, 0, 0, 0)),
+    (synth.BlockShape("Swin-T 8 windows log2", 8, 49, 96, 3, 32, 384, True), 8, (3, 1, 1, 1)),
 ])
 def test_encoder_block_parity(api, orc, shape, w_bits, table):
     spec = synth.make_block(shape, seed=1, w_bits=w_bits, gelu_in_bits=14 if table[1] == 2 else 16)
