@@ -244,6 +244,9 @@ int iptq_linear_w4_static(const int8_t* x, const void* w_packed, const int32_t* 
  * bias: nullable dev int32 [H, N, N] at the score scale; mask_id: nullable dev uint8 [B, N]: the pair
  * (i, j) is masked (probability 0, excluded from max and sum) iff mask_id[b,i] != mask_id[b,j].
  * N <= 256, dh in {32, 64}; sm (host) prepared with row_len = N; out_rq: host.  ws: status block only.
+ * The real ratio of out_rq is 2^-(out_bits-1) * S_v / S_out.  With IPTQ_SM_LOG2 the probabilities are the powers
+ * of two 2^-code and the product is the shift-accumulate sum_j v_j << (15 - code_ij) (codes above 15: nothing),
+ * so out_rq's ratio is 2^-15 * S_v / S_out.
  */
 size_t iptq_attention_workspace_bytes(int64_t B, int H, int N, int dh);
 int iptq_attention_block(const int8_t* q, const int8_t* k, const int8_t* v, int8_t* out, int64_t B, int H,

@@ -16,7 +16,7 @@
  *
  * Parity status: every function below is pinned by CPU tests except
  *   - ORACLE_SM_POLY, ORACLE_SM_LOG2 and ORACLE_GELU_SHIFT: the paper names these candidates
- *     (Sec. 3.2) but defines neither; pinned only against the float functions
+ *     (Sec. 3.2) but defines none of them; pinned only against the float functions
  *     they approximate, with constants from the cited prior work
  *     ("parity unpinned" beyond that);
  *   - the three LayerNorm variants: named in Sec. 3.2, defined nowhere in the
