@@ -163,6 +163,15 @@ int iptq_gelu_table(const iptq_gelu_consts* consts, int8_t* table, iptq_stream_t
 /* host.  in_bits in [8, 16], out_bits in [4, 8]; floor(|b| / S') must be in [1, 2^15). */
 int iptq_gelu_prepare(double in_scale, int in_bits, double out_scale, int out_zp, int out_bits,
                       iptq_gelu_variant variant, iptq_gelu_consts* out /*host*/);
+/* Data-aware coefficients (Sec. 3.3, Eq. (4)): the paper re-computes (a, b) of Eq. (3) for the value range of the
+ * data, [min(T), max(T)], by least squares against erf.  iptq_gelu_fit does that on a uniform grid of `points`
+ * values over [lo, hi] (the paper gives the range, not the sample): *a, *b receive the coefficients (both
+ * negative), *rms (nullable) the root-mean-square residual.  Host only; 8 <= points <= 2^22, hi > lo.
+ * iptq_gelu_prepare_coeffs is iptq_gelu_prepare(IPTQ_GELU_POLY4) with these coefficients in place of the
+ * paper's constants (a, b < 0, else IPTQ_ERR_SCALE_RANGE); the kernels need nothing else. */
+int iptq_gelu_fit(double lo, double hi, int points, double* a /*host*/, double* b /*host*/, double* rms /*host*/);
+int iptq_gelu_prepare_coeffs(double in_scale, int in_bits, double out_scale, int out_zp, int out_bits, double a,
+                             double b, iptq_gelu_consts* out /*host*/);
 /* x: dev int32 [n] (clamped to in_bits inside); y: dev int8 [n]; consts: host. */
 int iptq_gelu(const int32_t* x, int8_t* y, int64_t n, const iptq_gelu_consts* consts, iptq_stream_t stream);
 

@@ -97,6 +97,8 @@ def lib():
         L.oracle_softmax_row.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.POINTER(SoftmaxConsts), C.c_void_p]
         L.oracle_gelu_prepare.argtypes = [C.c_double, C.c_int, C.c_double, C.c_int, C.c_int, C.c_int,
                                           C.POINTER(GeluConsts)]
+        L.oracle_gelu_prepare_coeffs.argtypes = [C.c_double, C.c_int, C.c_double, C.c_int, C.c_int, C.c_double,
+                                                 C.c_double, C.POINTER(GeluConsts)]
         L.oracle_gelu_core.restype = C.c_int64
         L.oracle_gelu_core.argtypes = [C.c_int64, C.POINTER(GeluConsts)]
         L.oracle_gelu_core_scale.restype = C.c_double
@@ -189,6 +191,14 @@ def gelu_prepare(in_scale, in_bits, out_scale, out_zp=0, out_bits=8, variant=GEL
     c = GeluConsts()
     _chk(lib().oracle_gelu_prepare(float(in_scale), in_bits, float(out_scale), out_zp, out_bits, variant,
                                    C.byref(c)), "gelu_prepare")
+    return c
+
+
+def gelu_prepare_coeffs(in_scale, in_bits, out_scale, out_zp, out_bits, a, b) -> GeluConsts:
+    """Quartic GELU with refitted erf coefficients (a, b) (Sec. 3.3, Eq. (4))."""
+    c = GeluConsts()
+    _chk(lib().oracle_gelu_prepare_coeffs(float(in_scale), in_bits, float(out_scale), out_zp, out_bits, float(a),
+                                          float(b), C.byref(c)), "gelu_prepare_coeffs")
     return c
 
 

@@ -227,8 +227,29 @@ int oracle_softmax(const int32_t* scores, uint8_t* probs, int64_t rows, int row_
 
 /* ---------- GELU (Sec. 3.3, Eqs. (1)-(5)) ------------------------------- */
 
+static int gelu_prepare_impl(double in_scale, int in_bits, double out_scale, int out_zp, int out_bits,
+                             int variant, double A, double Bf, oracle_gelu_consts_t* out);
+
 int oracle_gelu_prepare(double in_scale, int in_bits, double out_scale, int out_zp, int out_bits,
                         int variant, oracle_gelu_consts_t* out)
+{
+    /* Eq. (3): a = -0.019913, b = -2.698088 (quartic); the second-order
+     * erf polynomial of the cited prior work has a = -0.2888, b = -1.769. */
+    const double A = (variant == ORACLE_GELU_POLY4) ? 0.019913 : 0.2888;
+    const double Bf = (variant == ORACLE_GELU_POLY4) ? 2.698088 : 1.769;
+    return gelu_prepare_impl(in_scale, in_bits, out_scale, out_zp, out_bits, variant, A, Bf, out);
+}
+
+/* Quartic polynomial with coefficients refitted to the data range (Eq. (4)): a < 0, b < 0 as in Eq. (3). */
+int oracle_gelu_prepare_coeffs(double in_scale, int in_bits, double out_scale, int out_zp, int out_bits,
+                               double a, double b, oracle_gelu_consts_t* out)
+{
+    if (!(a < 0.0) || !(b < 0.0)) return ORACLE_ERR_RANGE;
+    return gelu_prepare_impl(in_scale, in_bits, out_scale, out_zp, out_bits, ORACLE_GELU_POLY4, -a, -b, out);
+}
+
+static int gelu_prepare_impl(double in_scale, int in_bits, double out_scale, int out_zp, int out_bits,
+                             int variant, double A, double Bf, oracle_gelu_consts_t* out)
 {
     if (!out) return ORACLE_ERR_ARG;
     if (in_bits < 8 || in_bits > 16 || out_bits < 4 || out_bits > 8) return ORACLE_ERR_ARG;
@@ -238,10 +259,6 @@ int oracle_gelu_prepare(double in_scale, int in_bits, double out_scale, int out_
     out->in_bits = in_bits;
     double Sy;
     if (variant == ORACLE_GELU_POLY4 || variant == ORACLE_GELU_POLY2) {
-        /* Eq. (3): a = -0.019913, b = -2.698088 (quartic); the second-order
-         * erf polynomial of the cited prior work has a = -0.2888, b = -1.769. */
-        const double A = (variant == ORACLE_GELU_POLY4) ? 0.019913 : 0.2888;
-        const double Bf = (variant == ORACLE_GELU_POLY4) ? 2.698088 : 1.769;
         double Sp = in_scale / sqrt(2.0);              /* scale of x / sqrt(2), Eq. (5) */
         double Bqd = floor(Bf / Sp);
         if (!(Bqd >= 1.0) || !(Bqd < 32768.0)) return ORACLE_ERR_RANGE;

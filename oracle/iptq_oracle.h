@@ -96,6 +96,9 @@ int oracle_softmax(const int32_t* scores, uint8_t* probs, int64_t rows, int row_
 /* ---- GELU ------------------------------------------------------------- */
 int oracle_gelu_prepare(double in_scale, int in_bits, double out_scale, int out_zp, int out_bits,
                         int variant, oracle_gelu_consts_t* out);
+/* The quartic variant with coefficients (a, b) of Eq. (3) refitted to the data range (Eq. (4)); a < 0, b < 0. */
+int oracle_gelu_prepare_coeffs(double in_scale, int in_bits, double out_scale, int out_zp, int out_bits,
+                               double a, double b, oracle_gelu_consts_t* out);
 /* Pre-requant integer y = x * (G >> gs) (or x * sigma_q) of one element. */
 int64_t oracle_gelu_core(int64_t x, const oracle_gelu_consts_t* c);
 /* Scale of the value oracle_gelu_core returns. */

@@ -101,6 +101,10 @@ def lib():
         L.iptq_gelu_prepare.argtypes = [C.c_double, C.c_int, C.c_double, C.c_int, C.c_int, C.c_int,
                                         C.POINTER(GeluConsts)]
         L.iptq_gelu.argtypes = [_vp, _vp, C.c_int64, C.POINTER(GeluConsts), _vp]
+        L.iptq_gelu_fit.argtypes = [C.c_double, C.c_double, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                    C.POINTER(C.c_double)]
+        L.iptq_gelu_prepare_coeffs.argtypes = [C.c_double, C.c_int, C.c_double, C.c_int, C.c_int, C.c_double,
+                                               C.c_double, C.POINTER(GeluConsts)]
         L.iptq_gelu_table.argtypes = [C.POINTER(GeluConsts), _vp, _vp]
         L.iptq_layernorm_prepare.argtypes = [C.c_int, _vp, _vp, C.c_double, C.c_int, C.c_int, C.c_int, _vp, _vp,
                                              C.POINTER(LnConsts)]
@@ -147,7 +151,7 @@ def lib():
 def exported_symbols():
     """Names declared in include/iptq.h (used by the CPU-side load test)."""
     return ["iptq_requant_prepare", "iptq_channel_requant_prepare", "iptq_softmax_prepare", "iptq_softmax", "iptq_softmax_table",
-            "iptq_gelu_prepare", "iptq_gelu", "iptq_gelu_table", "iptq_layernorm_prepare", "iptq_layernorm",
+            "iptq_gelu_prepare", "iptq_gelu", "iptq_gelu_table", "iptq_gelu_fit", "iptq_gelu_prepare_coeffs", "iptq_layernorm_prepare", "iptq_layernorm",
             "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_patchify", "iptq_attention_workspace_bytes", "iptq_attention_block",
             "iptq_mlp_workspace_bytes", "iptq_mlp_block", "iptq_encoder_block_workspace_bytes",
             "iptq_encoder_block", "iptq_encoder_block_profiled", "iptq_workspace_init", "iptq_check", "iptq_strerror", "iptq_launch_count",
@@ -273,6 +277,21 @@ def gelu(x, consts: GeluConsts, out=None):
 
 
 GELU_TABLE_SIZE = 65536
+
+
+def gelu_fit(lo, hi, points=4001):
+    """Data-aware coefficients of the quartic erf polynomial for inputs in [lo, hi] (Sec. 3.3, Eq. (4)).
+    Returns (a, b, rms residual)."""
+    a, b, r = C.c_double(), C.c_double(), C.c_double()
+    _chk(lib().iptq_gelu_fit(float(lo), float(hi), int(points), C.byref(a), C.byref(b), C.byref(r)), "iptq_gelu_fit")
+    return a.value, b.value, r.value
+
+
+def gelu_prepare_coeffs(in_scale, in_bits, out_scale, out_zp, out_bits, a, b) -> GeluConsts:
+    c = GeluConsts()
+    _chk(lib().iptq_gelu_prepare_coeffs(float(in_scale), in_bits, float(out_scale), out_zp, out_bits, float(a),
+                                        float(b), C.byref(c)), "iptq_gelu_prepare_coeffs")
+    return c
 
 
 def gelu_table(consts: GeluConsts, device="cuda"):

@@ -1,6 +1,7 @@
 // Host side of the iptq library: float scales -> integer constants, status helpers.
 #include <atomic>
 #include <cmath>
+#include <vector>
 #include <cstring>
 #include <mutex>
 
@@ -170,8 +171,83 @@ int iptq_softmax_prepare(double in_scale, int row_len, int out_bits, iptq_softma
     return IPTQ_OK;
 }
 
+static int gelu_prepare_with(double in_scale, int in_bits, double out_scale, int out_zp, int out_bits,
+                             iptq_gelu_variant variant, double A, double Bf, iptq_gelu_consts* out);
+
 int iptq_gelu_prepare(double in_scale, int in_bits, double out_scale, int out_zp, int out_bits,
                       iptq_gelu_variant variant, iptq_gelu_consts* out)
+{
+    const bool quartic = variant == IPTQ_GELU_POLY4;
+    // |a|, |b| of Eq. (3) / of the second-order erf polynomial
+    return gelu_prepare_with(in_scale, in_bits, out_scale, out_zp, out_bits, variant, quartic ? 0.019913 : 0.2888,
+                             quartic ? 2.698088 : 1.769, out);
+}
+
+int iptq_gelu_prepare_coeffs(double in_scale, int in_bits, double out_scale, int out_zp, int out_bits, double a,
+                             double b, iptq_gelu_consts* out)
+{
+    if (!(a < 0.0) || !(b < 0.0)) return IPTQ_ERR_SCALE_RANGE;
+    return gelu_prepare_with(in_scale, in_bits, out_scale, out_zp, out_bits, IPTQ_GELU_POLY4, -a, -b, out);
+}
+
+// Eq. (4): least squares of Eq. (3) against erf on a uniform grid over [lo, hi].  Both functions are odd, so the
+// grid is folded to u = |x|; for a fixed b the optimum a is the ratio of two sums, which leaves a search in b:
+// a scan over 400 values, then bisection on the sign of the slope between neighbours of the best cell.
+int iptq_gelu_fit(double lo, double hi, int points, double* a_out, double* b_out, double* rms_out)
+{
+    if (!a_out || !b_out) return IPTQ_ERR_NULL;
+    if (!(hi > lo) || points < 8 || points > (1 << 22)) return IPTQ_ERR_SHAPE;
+    std::vector<double> u, tgt;
+    u.reserve((size_t)points); tgt.reserve((size_t)points);
+    for (int i = 0; i < points; ++i) {
+        const double x = lo + (hi - lo) * (double)i / (double)(points - 1);
+        if (x == 0.0) continue;
+        u.push_back(std::fabs(x));
+        tgt.push_back(std::erf(std::fabs(x)));
+    }
+    if (u.size() < 4) return IPTQ_ERR_SHAPE;
+    auto a_of = [&](double b) {
+        long double num = 0.0L, den = 0.0L;
+        for (size_t i = 0; i < u.size(); ++i) {
+            const double c = std::min(u[i], -b) + b, t = c * c * c * c;
+            num += (long double)t * (tgt[i] - 1.0);
+            den += (long double)t * t;
+        }
+        return den > 0.0L ? (double)(num / den) : 0.0;
+    };
+    auto loss = [&](double b) {
+        const double a = a_of(b);
+        long double ss = 0.0L;
+        for (size_t i = 0; i < u.size(); ++i) {
+            const double c = std::min(u[i], -b) + b, t = c * c * c * c;
+            const double r = tgt[i] - (a * t + 1.0);
+            ss += (long double)r * r;
+        }
+        return (double)ss;
+    };
+    const double b_lo = -8.0, b_hi = -0.25;
+    const int cells = 400;
+    int best = 0;
+    double best_loss = loss(b_lo);
+    for (int k = 1; k <= cells; ++k) {
+        const double l = loss(b_lo + (b_hi - b_lo) * k / cells);
+        if (l < best_loss) { best_loss = l; best = k; }
+    }
+    double l = b_lo + (b_hi - b_lo) * std::max(best - 1, 0) / cells;
+    double r = b_lo + (b_hi - b_lo) * std::min(best + 1, cells) / cells;
+    for (int it = 0; it < 100 && r - l > 1e-13; ++it) {      // ternary search: the loss is unimodal inside the cell pair
+        const double m1 = l + (r - l) / 3.0, m2 = r - (r - l) / 3.0;
+        if (loss(m1) < loss(m2)) r = m2; else l = m1;
+    }
+    const double b = 0.5 * (l + r);
+    *a_out = a_of(b);
+    *b_out = b;
+    if (rms_out) *rms_out = std::sqrt(loss(b) / (double)u.size());
+    return IPTQ_OK;
+}
+
+static int gelu_prepare_with(double in_scale, int in_bits, double out_scale, int out_zp, int out_bits,
+                             iptq_gelu_variant variant, double A, double Bf, iptq_gelu_consts* out)
 {
     if (!out) return IPTQ_ERR_NULL;
     if (in_bits < 8 || in_bits > 16 || out_bits < 4 || out_bits > 8) return IPTQ_ERR_BITS;
@@ -181,8 +257,6 @@ int iptq_gelu_prepare(double in_scale, int in_bits, double out_scale, int out_zp
     double y_scale;
     if (variant == IPTQ_GELU_POLY4 || variant == IPTQ_GELU_POLY2) {
         const bool quartic = variant == IPTQ_GELU_POLY4;
-        const double A = quartic ? 0.019913 : 0.2888;         // |a| of Eq. (3) / of the second-order erf
-        const double Bf = quartic ? 2.698088 : 1.769;         // |b|
         const double sp = in_scale / std::sqrt(2.0);          // scale of x / sqrt(2)
         const double bq = std::floor(Bf / sp);
         if (!(bq >= 1.0 && bq < 32768.0)) return IPTQ_ERR_SCALE_RANGE;

@@ -185,6 +185,20 @@ def test_gelu_parity(api, orc, variant, n):
     assert (got == want).all()
 
 
+@pytest.mark.parametrize("bits,S,rng_", [(16, 1.3e-4, (-3.0, 3.0)), (14, 2.0 / 8191, (-1.4, 1.4)), (8, 8.0 / 127, (-5.0, 2.0))])
+def test_gelu_refitted_coefficients_exhaustive(api, orc, bits, S, rng_):
+    """Quartic GELU with coefficients refitted to a data range (Eq. (4)): every in_bits input and the clamp,
+    stand-alone kernel and tabulated form."""
+    a, b, _ = api.gelu_fit(rng_[0], rng_[1])
+    ca = api.gelu_prepare_coeffs(S, bits, 0.03, -7, 8, a, b)
+    co = orc.gelu_prepare_coeffs(S, bits, 0.03, -7, 8, a, b)
+    x = np.arange(-(1 << 17), 1 << 17, dtype=np.int32)
+    want = orc.gelu(x, co)
+    assert (api.gelu(_cu(x), ca).cpu().numpy() == want).all()
+    tab = api.gelu_table(ca).cpu().numpy()
+    assert (tab == want[(1 << 17) - 32768:(1 << 17) + 32768]).all()
+
+
 @pytest.mark.parametrize("variant", [0, 1, 2])
 @pytest.mark.parametrize("bits,S", [(8, 8.0 / 127), (12, 0.003), (16, 1.3e-4)])
 def test_gelu_exhaustive_inputs(api, orc, variant, bits, S):
