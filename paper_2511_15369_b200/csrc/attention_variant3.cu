@@ -1,0 +1,13 @@
+// Fused attention kernels of the IPTQ_SM_LOG2 Softmax variant (both head dimensions, every flag combination).
+#include "attention_kernel.cuh"
+
+namespace iptq {
+
+int attention_launch_variant3(int dh, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                              const AttnParams& p, int smem_bytes, cudaStream_t st)
+{
+    if (dh == 64) return launch_attn<64, IPTQ_SM_LOG2>(mq, mk, mv, p, smem_bytes, st);
+    return launch_attn<32, IPTQ_SM_LOG2>(mq, mk, mv, p, smem_bytes, st);
+}
+
+}  // namespace iptq
