@@ -12,6 +12,8 @@ One step = one pass of the whole block over one batch of seeded synthetic input.
                Gelem/s and fraction of the measured HBM copy bandwidth;
   assignment   the Unified-Metric analysis (every candidate of every non-linear layer of the encoder scored and
                selected on the device) as evaluations/s, with the oracle's scores of the first block beside it;
+  other_blocks the ViT-Base batch-128 and Swin-Tiny window blocks, timed like the headline block (context: the
+               headline metric stays the DeiT-Small block);
   models       whole DeiT-T/S/B forward latency at batch 8 (context beside the paper's latency table, other hardware);
   cpu_baseline the CPU oracle timed on the host cores on a bounded sample of the same workload, and the
                element-by-element comparison of the GPU output with it.
@@ -362,6 +364,7 @@ def run_ours(args):
     clocks.stop()
     assignment = bench_assignment(api, torch, dev) if rank == 0 else None
     models = bench_models(api, torch, dev) if rank == 0 else None
+    other_blocks = bench_other_blocks(api, torch, dev, peaks) if rank == 0 else None
 
     if rank != 0:
         if world > 1:
@@ -446,6 +449,7 @@ def run_ours(args):
         "nonlinear": nonlinear,
         "assignment": assignment,
         "models": models,
+        "other_blocks": other_blocks,
         "cpu_baseline": cpu,
     }))
     if world > 1:
@@ -509,6 +513,43 @@ def bench_nonlinear(api, torch, dev, peaks, peak_kind):
     gqd, bqd = torch.from_numpy(gq).to(dev), torch.from_numpy(bq).to(dev)
     record("iptq_layernorm", rows * dim, 2 * rows * dim, time_kernel(lambda: api.layernorm(xl, gqd, bqd, lc, out=yl)),
            "int8 [201728, 768] -> int8 (155 MB in)")
+    return out
+
+
+def bench_other_blocks(api, torch, dev, peaks):
+    """The other single-block configurations (ViT-Base batch 128, Swin-Tiny stage-1 windows), timed like the headline
+    one: CUDA-graph replay of one block step, L2 flushed before each, CUDA events, median of 20."""
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    out = []
+    for cfg in ("cfg2", "cfg3"):
+        shape = synth.CONFIGS[cfg]
+        spec = synth.make_block(shape, seed=0, calib_images=8 if shape.has_bias else 2)
+        blk = api.EncoderBlock(spec, TABLE, dev)
+        x = torch.from_numpy(spec.x).to(dev)
+        y = torch.empty_like(x)
+        st = torch.cuda.Stream()
+        with torch.cuda.stream(st):
+            for _ in range(3):
+                blk(x, y)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=st):
+                blk(x, y)
+            ts = []
+            for _ in range(20):
+                flush.fill_(1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(st)
+                g.replay()
+                b.record(st)
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+        blk.ws.check()
+        ms = statistics.median(ts)
+        tops = shape.gemm_ops() / (ms * 1e-3) / 1e12
+        out.append({"workload": "%s: %s" % (cfg, shape.name), "ms_per_step": ms, "tops": tops,
+                    "frac_int8_peak": tops / (peaks["bf16_tflops"] * INT8_OVER_BF16), "gop_per_step": shape.gemm_ops() / 1e9})
+        del blk, g, x, y, spec
     return out
 
 

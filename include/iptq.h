@@ -252,7 +252,9 @@ int iptq_linear_w4_static(const int8_t* x, const void* w_packed, const int32_t* 
  * q, k, v: dev int8 [B, H, N, dh] (zero point 0); out: dev int8 [B, N, H*dh];
  * bias: nullable dev int32 [H, N, N] at the score scale; mask_id: nullable dev uint8 [B, N]: the pair
  * (i, j) is masked (probability 0, excluded from max and sum) iff mask_id[b,i] != mask_id[b,j].
- * N <= 256, dh in {32, 64}; sm (host) prepared with row_len = N; out_rq: host.  ws: status block only.
+ * N <= 256, dh in {32, 64}; sm (host) prepared with row_len = N; out_rq: host.  ws: the status block, followed
+ * for N <= 64 by room for a transposed copy of the bias (iptq_attention_workspace_bytes() counts it; with a smaller
+ * workspace the call still works and reads the bias as it is, more slowly).
  * The real ratio of out_rq is 2^-(out_bits-1) * S_v / S_out.  With IPTQ_SM_LOG2 the probabilities are the powers
  * of two 2^-code and the product is the shift-accumulate sum_j v_j << (15 - code_ij) (codes above 15: nothing),
  * so out_rq's ratio is 2^-15 * S_v / S_out.

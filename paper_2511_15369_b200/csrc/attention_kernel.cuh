@@ -1,6 +1,7 @@
 #pragma once
 // Kernel and per-variant launcher of the fused integer attention (included by attention.cu and by the
 // attention_variant*.cu files, which instantiate one Softmax variant each so that they compile in parallel).
+// Problems of N <= 64 tokens take the kernel of attention_window.cuh instead.
 //
 // Fused integer attention: S = Q K^T (tcgen05 INT8 -> int32 in TMEM) -> (+bias, mask) -> integer Softmax of
 // Sec. 3.4 (Eqs. (6)-(15)) -> uint8 P written to shared memory in the tensor-core operand layout ->
@@ -38,14 +39,13 @@ struct AttnParams {
     int o_col;             // first TMEM column of O
     int q_bytes, k_bytes, v_bytes, stage_bytes;
     int p_off, p_bytes, xch_off, bar_off;
-    int pair;              // windows of N <= 64 tokens: an item is two (batch, head) problems, one per 64-row half of
-                           // the tile; each half reads only its own 64 key columns and P is zero off the diagonal
     int p_plane;           // bytes of one P operand; the logarithm candidate keeps two per buffer (p_bytes = 2 p_plane)
     int stages;            // Q/K/V ring depth (3, or 2 when the exponential table needs the room)
     int lut_off, lut_n;    // exponential table: e(d) for d < lut_n, 0 beyond (lut_n = 0: no table)
     const uint16_t* lut_src;   // the same table in device memory (copied), or null (built by each CTA)
     uint32_t tmem_cols;
     const int32_t* bias;   // [H, N, N] or null
+    const int4* bias_q;    // window kernel: the same bias as [H][ceil(N/4) column quads][64 rows] of 4 columns each, or null
     const uint8_t* mask_id;// [B, N] or null
     int8_t* out;           // [B, N, H*dh]
     ExpDev ex; int M, f_shl, p_shr;
@@ -64,10 +64,7 @@ __device__ __forceinline__ void decode_item(const AttnParams& p, int it, int& bh
 // USE_LUT: the integer exponential of Eqs. (7)-(14) depends only on d = max - s, is below 2^16 and vanishes for
 // d >= lut_n (a few times x0); each CTA tabulates it once in shared memory with the same arithmetic and the
 // Softmax step then costs one table read per score instead of some sixteen dependent integer instructions.
-// PAIR: problems of N <= 64 tokens (windows) are taken two per item, one per 64-row half of the tile: each half
-// reads its own 64 score columns only, the off-diagonal quarters of P stay zero, and the cross products the tensor
-// core computes on the way are never looked at.  Per-item overhead, which dominates such small problems, halves.
-template <int DH, int VARIANT, bool HAS_BIAS, bool HAS_MASK, bool PSHR, bool USE_LUT, bool PAIR>
+template <int DH, int VARIANT, bool HAS_BIAS, bool HAS_MASK, bool PSHR, bool USE_LUT>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, const AttnParams p)
@@ -128,29 +125,15 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     mbar_arrive(&kv_full[s]);                  // release: the consumers see the stop mark
                     break;
                 }
+                int bh, mt;
+                decode_item(p, it, bh, mt);
+                const int h = bh % p.H, b = bh / p.H;
                 item_of[s] = it;
                 uint8_t* st = smem + s * p.stage_bytes;
-                if (PAIR) {
-                    // two problems per item: 64-row boxes of q, k and v of each into the halves of the operand tiles
-                    const int n_here = 2 * it + 1 < p.B * p.H ? 2 : 1;
-                    mbar_expect_tx(&kv_full[s], (uint32_t)(n_here * 3 * 64 * DH));
-                    for (int w = 0; w < n_here; ++w) {
-                        const int bh = 2 * it + w;
-                        const int h = bh % p.H, b = bh / p.H;
-                        uint8_t* half = st + w * 64 * DH;
-                        tma_load_4d(half, &map_q, &kv_full[s], 0, 0, h, b);
-                        tma_load_4d(half + p.q_bytes, &map_k, &kv_full[s], 0, 0, h, b);
-                        tma_load_4d(half + p.q_bytes + p.k_bytes, &map_v, &kv_full[s], 0, 0, h, b);
-                    }
-                } else {
-                    int bh, mt;
-                    decode_item(p, it, bh, mt);
-                    const int h = bh % p.H, b = bh / p.H;
-                    mbar_expect_tx(&kv_full[s], (uint32_t)((128 + p.npad_s + p.kpad) * DH));   // bytes of the three full boxes
-                    tma_load_4d(st, &map_q, &kv_full[s], 0, mt * 128, h, b);
-                    tma_load_4d(st + p.q_bytes, &map_k, &kv_full[s], 0, 0, h, b);
-                    tma_load_4d(st + p.q_bytes + p.k_bytes, &map_v, &kv_full[s], 0, 0, h, b);
-                }
+                mbar_expect_tx(&kv_full[s], (uint32_t)((128 + p.npad_s + p.kpad) * DH));   // bytes of the three full boxes
+                tma_load_4d(st, &map_q, &kv_full[s], 0, mt * 128, h, b);
+                tma_load_4d(st + p.q_bytes, &map_k, &kv_full[s], 0, 0, h, b);
+                tma_load_4d(st + p.q_bytes + p.k_bytes, &map_v, &kv_full[s], 0, 0, h, b);
                 if (++s == p.stages) { s = 0; ph ^= 1u; }
             }
             // the last CTA to finish re-arms the counters for the next launch that uses this workspace
@@ -223,13 +206,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint32_t trow = tmem_base + ((uint32_t)(quad * 32) << 16);
         const uint32_t p_row0 = smem_u32(sP) + (uint32_t)((rloc >> 3) * 1024 + (rloc & 7) * 128);
         const int HD = p.H * DH;
-        // pair mode: rows 0..63 belong to the first problem and read S columns 0..63, rows 64..127 to the second
-        const int win = PAIR ? quad >> 1 : 0;
-        const int col_off = 64 * win;                          // S column of this row's key 0
-        const int chunks = (PAIR ? (p.N + 15) & ~15 : p.npad_s) >> 4;   // 16-column chunks of a row (<= 16)
+        const int chunks = p.npad_s >> 4;                      // 16-column chunks of a row (<= 16)
         const int cbase = chunks >> 2, crem = chunks & 3;
         const int nch = cbase + (part < crem ? 1 : 0);         // this thread's chunks (<= 4) ...
-        const int c_begin = 4 * win + part * cbase + min(part, crem);    // ... starting here
+        const int c_begin = part * cbase + min(part, crem);    // ... starting here
         const bool sat8 = p.orq.qmin == -128 && p.orq.qmax == 127;
         int s = 0; uint32_t ph = 0;
         uint16_t* lut = reinterpret_cast<uint16_t*>(smem + p.lut_off);
@@ -246,37 +226,15 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
             named_barrier(5, ATT_SOFTMAX_THREADS);              // the table is complete before anyone reads it
         }
-        if (PAIR) {
-            // the off-diagonal quarters of P (and key columns past the padded row length) are never written: zero once
-            int4* z = reinterpret_cast<int4*>(sP);
-            for (int i = (int)threadIdx.x - 64; i < 2 * p.p_bytes / 16; i += ATT_SOFTMAX_THREADS) z[i] = make_int4(0, 0, 0, 0);
-            fence_proxy_async_smem();
-            named_barrier(5, ATT_SOFTMAX_THREADS);
-        }
         grid_dep_wait();                                       // output rows are written only after this
 
         // requantises and stores this thread's share of the output tile of item (b, h, mt), count index k
-        // (PAIR: b is the item number, from which each half of the tile finds its own problem)
         auto epilogue = [&](int k, int b, int h, int mt) -> bool {
             if (!mbar_wait(o_full, (uint32_t)k & 1u, ctl, p.status, 16)) return false;
             tc_fence_after_sync();
-            int row;
-            bool warp_ok, row_ok;                              // some row of the warp is real; this one is
-            if (PAIR) {
-                const int bh = 2 * b + win;
-                const bool exists = bh < p.B * p.H;
-                row = rloc & 63;
-                warp_ok = exists && (quad & 1) * 32 < p.N;
-                row_ok = exists && row < p.N;
-                h = exists ? bh % p.H : 0;
-                b = exists ? bh / p.H : 0;
-            } else {
-                row = mt * 128 + rloc;
-                warp_ok = mt * 128 + quad * 32 < p.N;
-                row_ok = row < p.N;
-            }
+            const int row = mt * 128 + rloc;
             constexpr int OPARTS = DH / 16;                    // threads of a row that hold 16 output columns each
-            if (warp_ok && part < OPARTS) {
+            if (mt * 128 + quad * 32 < p.N && part < OPARTS) {
                 uint32_t r[16];
                 tmem_ld16(trow + (uint32_t)(p.o_col + part * 16), r);
                 if constexpr (VARIANT == IPTQ_SM_LOG2) {
@@ -294,7 +252,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     o[j] = requant_nosat((int)r[j], p.orq);
                     if (!sat8) o[j] = max(p.orq.qmin, min(p.orq.qmax, o[j]));
                 }
-                if (row_ok) {
+                if (row < p.N) {
                     int4 pk;
                     pk.x = (int)pack4_sat_s8(o[0], o[1], o[2], o[3]);
                     pk.y = (int)pack4_sat_s8(o[4], o[5], o[6], o[7]);
@@ -322,22 +280,12 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const int it = item_of[s];
             if (it < 0) break;
             if (++s == p.stages) { s = 0; ph ^= 1u; }
-            int bh, mt = 0, row;
-            bool valid, warp_rows;                             // warp_rows is warp-uniform: any valid row in this warp
-            if (PAIR) {
-                bh = 2 * it + win;
-                row = rloc & 63;
-                const bool exists = bh < p.B * p.H;
-                valid = exists && row < p.N;
-                warp_rows = exists && (quad & 1) * 32 < p.N;
-                if (!exists) bh = 0;
-            } else {
-                decode_item(p, it, bh, mt);
-                row = mt * 128 + rloc;
-                valid = row < p.N;
-                warp_rows = mt * 128 + quad * 32 < p.N;
-            }
+            int bh, mt;
+            decode_item(p, it, bh, mt);
             const int h = bh % p.H, b = bh / p.H;
+            const int row = mt * 128 + rloc;
+            const bool valid = row < p.N;
+            const bool warp_rows = mt * 128 + quad * 32 < p.N;            // warp-uniform: any valid row in this warp
             const int32_t* brow = HAS_BIAS ? p.bias + ((size_t)h * p.N + (valid ? row : 0)) * p.N : nullptr;
             const uint8_t* mrow = HAS_MASK ? p.mask_id + (size_t)b * p.N : nullptr;
             const unsigned my_id = HAS_MASK ? mrow[valid ? row : 0] : 0u;
@@ -364,7 +312,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     if (i < nch) {
-                        const int c0 = (c_begin + i) * 16 - col_off;          // first key of the chunk
+                        const int c0 = (c_begin + i) * 16;
                         if (HAS_BIAS || HAS_MASK || c0 + 16 > p.N) {          // warp-uniform
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
@@ -461,7 +409,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
             // key columns between npad_s and kpad (at most one 16-column chunk) meet zero rows of V, but the bytes
             // the tensor core reads there must be defined
-            if (part == 3 && p.kpad > p.npad_s && !PAIR) {
+            if (part == 3 && p.kpad > p.npad_s) {
                 const int c0 = p.npad_s;
                 const int chunk = (c0 & 127) >> 4;
                 st_shared_v4(p_row + (uint32_t)((c0 >> 7) * 16384 + ((chunk ^ (rloc & 7)) << 4)), 0u, 0u, 0u, 0u);
@@ -472,7 +420,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             mbar_arrive(&p_ready[k & 1]);
             // ---- output of the previous item: its P V product was issued right after that item's Softmax
             if (k > 0 && !epilogue(k - 1, pb, phd, pmt)) { ok = false; break; }
-            pb = PAIR ? it : b; phd = h; pmt = mt;
+            pb = b; phd = h; pmt = mt;
         }
         if (ok && k > 0) epilogue(k - 1, pb, phd, pmt);
     }
@@ -498,20 +446,16 @@ int launch_attn(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap&
     const int grid = std::min(p.items, sm_count());
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return IPTQ_ERR_CUDA;
-#define IPTQ_ATT_LAUNCH4(HB, HM, PS, LT, PR)                                                                      \
+#define IPTQ_ATT_LAUNCH3(HB, HM, PS, LT)                                                                          \
     do {                                                                                                          \
-        auto kern = attention_kernel<DH, VARIANT, HB, HM, PS, LT, PR>;                                            \
+        auto kern = attention_kernel<DH, VARIANT, HB, HM, PS, LT>;                                                \
         static int configured[64];          /* largest dynamic shared memory size set so far, per device */     \
         if (configured[dev] < smem_bytes) {                                                                       \
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) \
                 return IPTQ_ERR_CUDA;                                                                             \
             configured[dev] = smem_bytes;                                                                         \
         }                                                                                                         \
-        launch_kernel(kern, grid, ATT_THREADS, smem_bytes, st, mq, mk, mv, p);                                    \
-    } while (0)
-#define IPTQ_ATT_LAUNCH3(HB, HM, PS, LT)                                                                          \
-    do {                                                                                                          \
-        if (p.pair) IPTQ_ATT_LAUNCH4(HB, HM, PS, LT, true); else IPTQ_ATT_LAUNCH4(HB, HM, PS, LT, false);         \
+        launch_kernel(kern, grid, ATT_THREADS, smem_bytes, st, mq, mk, mv, p);                                               \
     } while (0)
 #define IPTQ_ATT_LAUNCH2(HB, HM, PS)                                                                              \
     do {                                                                                                          \
@@ -528,7 +472,6 @@ int launch_attn(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap&
 #undef IPTQ_ATT_LAUNCH
 #undef IPTQ_ATT_LAUNCH2
 #undef IPTQ_ATT_LAUNCH3
-#undef IPTQ_ATT_LAUNCH4
     note_launch();
     return last_launch_status();
 }

@@ -1,0 +1,13 @@
+// Window attention kernels (N <= 64) of the IPTQ_SM_SHIFTMAX Softmax variant (both head dimensions, every flag combination).
+#include "attention_window.cuh"
+
+namespace iptq {
+
+int window_launch_variant1(int dh, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                           const AttnParams& p, int smem_bytes, cudaStream_t st)
+{
+    if (dh == 64) return launch_window_attn<64, IPTQ_SM_SHIFTMAX>(mq, mk, mv, p, smem_bytes, st);
+    return launch_window_attn<32, IPTQ_SM_SHIFTMAX>(mq, mk, mv, p, smem_bytes, st);
+}
+
+}  // namespace iptq

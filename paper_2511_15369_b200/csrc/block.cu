@@ -28,13 +28,15 @@ struct AttnArgs {
     const int32_t* bias; const uint8_t* mask_id;
     const iptq_softmax_consts* sm; const iptq_requant* out_rq;
     StatusBlock* status;
+    int32_t* bias_t;       // 16-byte aligned scratch of attention_bias_t_bytes(H, N) for the window kernel's copy of the bias, or null
 };
 int attention_launch(const AttnArgs& a, cudaStream_t st);
+size_t attention_bias_t_bytes(int H, int N);
 
 static size_t a256(size_t v) { return (v + 255) & ~size_t(255); }
 
 struct BlockLayout {
-    size_t h1, qkv, att, x1, h2, hid, w_qkv, w_proj, w_fc1, w_fc2, total;
+    size_t h1, qkv, att, x1, h2, hid, w_qkv, w_proj, w_fc1, w_fc2, bias_t, total;
 };
 
 static BlockLayout block_layout(const iptq_block_params* p)
@@ -56,6 +58,8 @@ static BlockLayout block_layout(const iptq_block_params* p)
         l.w_fc1 = take(Dh * D);
         l.w_fc2 = take(D * Dh);
     }
+    l.bias_t = 0;
+    if (p->attn_bias && attention_bias_t_bytes(p->H, p->N)) l.bias_t = take(attention_bias_t_bytes(p->H, p->N));
     l.total = off;
     return l;
 }
@@ -134,7 +138,8 @@ static int encoder_block_run(const int8_t* x, int8_t* y, const iptq_block_params
     if ((rc = mark()) != IPTQ_OK) return rc;
     // a row of qkv is [q | k | v]; head h occupies columns h*dh .. of each third
     AttnArgs aa{qkv, qkv + D, qkv + 2 * D, (int64_t)3 * D, (int64_t)p->dh, (int64_t)p->N * 3 * D, att, p->B, p->H, p->N,
-                p->dh, p->attn_bias, p->mask_id, p->sm, p->pv_rq, status};
+                p->dh, p->attn_bias, p->mask_id, p->sm, p->pv_rq, status,
+                l.bias_t ? reinterpret_cast<int32_t*>(base + l.bias_t) : nullptr};
     if ((rc = attention_launch(aa, stream)) != IPTQ_OK) return rc;
     if ((rc = mark()) != IPTQ_OK) return rc;
     LinearArgs lp{att, wp, p->b_proj, p->m_proj, p->s_proj, p->proj_zp, x, p->res1_rq, nullptr, x1, T, D, D, status};

@@ -140,7 +140,10 @@ def test_mlp_parity(api, orc, variant, M, D, Dh):
 @pytest.mark.parametrize("B,H,N,dh,use_bias,use_mask", [
     (2, 3, 197, 64, False, False), (3, 2, 49, 32, True, False), (4, 3, 49, 32, True, True),
     (1, 1, 1, 64, False, False), (2, 2, 128, 64, False, False), (1, 2, 129, 32, False, False),
-    (1, 1, 256, 64, True, False), (2, 1, 80, 32, False, True), (5, 6, 197, 64, False, False)])
+    (1, 1, 256, 64, True, False), (2, 1, 80, 32, False, True), (5, 6, 197, 64, False, False),
+    # windows (N <= 64, two problems per item): odd problem counts, full and tiny windows, both head dimensions
+    (5, 1, 49, 64, True, True), (3, 3, 64, 32, False, False), (2, 3, 16, 32, True, False), (7, 1, 33, 64, False, True),
+    (2, 2, 1, 32, False, False), (40, 3, 49, 32, True, True), (1, 2, 64, 64, True, True)])
 def test_attention_parity(api, orc, variant, B, H, N, dh, use_bias, use_mask):
     rng = np.random.default_rng(B * 1000 + N + dh + variant)
     q, k, v = (np.clip(np.round(rng.normal(0, 40, size=(B, H, N, dh))), -128, 127).astype(np.int8) for _ in range(3))
