@@ -153,8 +153,8 @@ typedef struct {
 /* The integer GELU maps an in_bits-bit input (<= 16 bits) to 8 bits, so the whole function fits a 64 KB table:
  * table[x + 32768] = the value iptq_gelu() returns for x (x below/above the in_bits range is clamped first, as
  * in the kernel).  iptq_gelu_table() fills such a table with the same arithmetic; when consts->table points to it,
- * the FC1 epilogue of iptq_mlp_block() / iptq_encoder_block() keeps a copy in shared memory and replaces the
- * polynomial by one read per output.  The results are identical with and without the table.
+ * the FC1 epilogue of iptq_mlp_block() / iptq_encoder_block(), and iptq_gelu() on inputs of 2^20 elements and more,
+ * keep a copy in shared memory and replace the polynomial by one read per output.  The results are identical with and without the table.
  * table: dev int8 [IPTQ_GELU_TABLE_SIZE], 16-byte aligned, caller-owned; consts: host (its own `table` is ignored).
  * Work submitted to the stream after this call sees the complete table. */
 #define IPTQ_GELU_TABLE_SIZE 65536

@@ -252,6 +252,48 @@ gelu_kernel(const int32_t* __restrict__ x, int8_t* __restrict__ y, int64_t n, co
     if (t < n) y[t] = (int8_t)requant_full(gelu_core<VARIANT>(x[t], c), c.out);
 }
 
+// Tabulated form: with consts->table set (iptq_gelu_table) the whole function is a 64 KB table, copied once per CTA
+// into shared memory; an element then costs a clamp to 16 bits and one byte load.  Two CTAs of 1024 threads per SM.
+constexpr int kGeluTabThreads = 1024;
+
+__global__ void __launch_bounds__(kGeluTabThreads, 2)
+gelu_tab_kernel(const int32_t* __restrict__ x, int8_t* __restrict__ y, int64_t n, const int8_t* __restrict__ table)
+{
+    extern __shared__ __align__(16) int8_t gelu_tab[];
+    {
+        // written and fenced by iptq_gelu_table(): safe to read ahead of the dependency wait
+        const int4* src = reinterpret_cast<const int4*>(table);
+        int4* dst = reinterpret_cast<int4*>(gelu_tab);
+        for (int i = threadIdx.x; i < IPTQ_GELU_TABLE_SIZE / 16; i += kGeluTabThreads) dst[i] = __ldg(src + i);
+    }
+    __syncthreads();
+    const uint32_t mid = (uint32_t)__cvta_generic_to_shared(gelu_tab) + 32768u;      // address of table[0 + 32768]
+    grid_dep_launch();
+    grid_dep_wait();
+    auto look = [&](int v) -> int {
+        v = max(-32768, min(32767, v));
+        int r;
+        asm volatile("ld.shared.s8 %0, [%1];" : "=r"(r) : "r"(mid + (uint32_t)v));
+        return r;
+    };
+    auto four = [&](int4 a) -> unsigned { return pack4_sat_s8(look(a.x), look(a.y), look(a.z), look(a.w)); };
+    const int64_t nvec = n >> 2;
+    const int64_t stride = (int64_t)gridDim.x * kGeluTabThreads;
+    const int4* xv = reinterpret_cast<const int4*>(x);
+    unsigned* yv = reinterpret_cast<unsigned*>(y);
+    int64_t i = (int64_t)blockIdx.x * kGeluTabThreads + threadIdx.x;
+    for (; i + 3 * stride < nvec; i += 4 * stride) {
+        int4 a[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) a[u] = __ldcs(xv + i + u * stride);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) __stcs(yv + i + u * stride, four(a[u]));
+    }
+    for (; i < nvec; i += stride) yv[i] = four(__ldcs(xv + i));
+    const int64_t t = (nvec << 2) + (int64_t)blockIdx.x * kGeluTabThreads + threadIdx.x;
+    if (t < n) y[t] = (int8_t)look(x[t]);
+}
+
 // table[x + 32768] = integer GELU of x for every 16-bit x (the input clamp to in_bits is part of gelu_core)
 template <int VARIANT>
 __global__ void __launch_bounds__(256)
@@ -571,6 +613,16 @@ int iptq_gelu(const int32_t* x, int8_t* y, int64_t n, const iptq_gelu_consts* co
     int rc = check_requant(&consts->out);
     if (rc != IPTQ_OK) return rc;
     if (n == 0) return IPTQ_OK;
+    if (consts->table && n >= (1 << 20)) {
+        // tabulated: worth the 64 KB copy per CTA once every thread has a few vectors
+        if (!aligned16(consts->table)) return IPTQ_ERR_ALIGN;
+        const int64_t vecs = (n + 3) / 4;
+        const int grid = (int)std::min<int64_t>((vecs + kGeluTabThreads - 1) / kGeluTabThreads, (int64_t)sm_count() * 2);
+        cudaFuncSetAttribute(gelu_tab_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, IPTQ_GELU_TABLE_SIZE);
+        launch_kernel(gelu_tab_kernel, grid, kGeluTabThreads, IPTQ_GELU_TABLE_SIZE, stream, x, y, n, consts->table);
+        note_launch();
+        return last_launch_status();
+    }
     const GeluDev c = to_dev(*consts);
     const int threads = 256;
     const int64_t groups = (n + 3) / 4;

@@ -185,6 +185,21 @@ def test_gelu_parity(api, orc, variant, n):
     assert (got == want).all()
 
 
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("n", [(1 << 20) + 3, 3 * (1 << 20)])
+def test_gelu_tabulated_standalone(api, orc, variant, n):
+    """iptq_gelu with the table attached (inputs of 2^20 elements and more): values beyond 16 bits included."""
+    bits = 16 if variant != 2 else 12
+    xall, S = synth.quantize_sym(synth.gelu_values(1 << 16, seed=n + variant), bits)
+    x = np.tile(xall, (n + xall.size - 1) // xall.size)[:n].astype(np.int32)
+    x[:8] = [-(1 << 31), (1 << 31) - 1, -32769, 32768, -32768, 32767, 0, -1]
+    So, zp = synth.affine_out_quant(synth.gelu_ref(xall[:4096] * S))
+    want = orc.gelu(x, orc.gelu_prepare(S, bits, So, zp, 8, variant))
+    c = api.gelu_prepare(S, bits, So, zp, 8, variant)
+    keep = api.gelu_table(c)
+    assert (api.gelu(_cu(x), c).cpu().numpy() == want).all()
+
+
 @pytest.mark.parametrize("bits,S,rng_", [(16, 1.3e-4, (-3.0, 3.0)), (14, 2.0 / 8191, (-1.4, 1.4)), (8, 8.0 / 127, (-5.0, 2.0))])
 def test_gelu_refitted_coefficients_exhaustive(api, orc, bits, S, rng_):
     """Quartic GELU with coefficients refitted to a data range (Eq. (4)): every in_bits input and the clamp,
