@@ -30,7 +30,9 @@ template <int DH, int VARIANT> struct WinCfg {
     static_assert(G * GCOLS <= 512, "TMEM");
 };
 
-template <int DH, int VARIANT, bool HAS_BIAS, bool HAS_MASK, bool PSHR, bool USE_LUT>
+// FULL: 48 < N <= 64, i.e. every row has its four 16-column chunks (the Swin window of 49 tokens): the chunk loops
+// then carry no run-time conditions.
+template <int DH, int VARIANT, bool HAS_BIAS, bool HAS_MASK, bool PSHR, bool USE_LUT, bool FULL>
 __global__ void __launch_bounds__(WinCfg<DH, VARIANT>::THREADS, 1)
 window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                         const __grid_constant__ CUtensorMap map_v, const AttnParams p)
@@ -183,7 +185,7 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
         const uint32_t tO = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(g * W::GCOLS + 128);
         const uint32_t p_row = smem_u32(sP + g * W::P_BYTES) + (uint32_t)((rloc >> 3) * 1024 + (rloc & 7) * 128);
         const int HD = p.H * DH;
-        const int nch = ((p.N + 15) & ~15) >> 4;               // 16-column chunks of a row (1..4)
+        const int nch = FULL ? 4 : ((p.N + 15) & ~15) >> 4;    // 16-column chunks of a row (1..4)
         const bool sat8 = p.orq.qmin == -128 && p.orq.qmax == 127;
         const uint32_t lut_addr = smem_u32(lut);
         const int tid = (int)threadIdx.x - 64;                 // 0 .. 128 G - 1
@@ -246,6 +248,10 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
             tc_fence_before_sync();
             mbar_arrive(&s_empty[g]);                          // the MMA warp may overwrite S with the group's next item
             int mx = INT_MIN;
+            // most windows of a shifted layout lie inside one region: all labels equal, nothing to mask (the labels
+            // were requested before the wait for the scores and are first looked at here)
+            const unsigned id_0 = __shfl_sync(0xffffffffu, id_lo, 0);
+            const bool mixed = HAS_MASK && !__all_sync(0xffffffffu, (lane >= p.N || id_lo == id_0) && (lane + 32 >= p.N || id_hi == id_0));
             if (warp_rows) {
                 // ---- row maximum over the real, unmasked columns (Eq. (6)); padding and masked pairs become kPadScore
 #pragma unroll
@@ -266,16 +272,23 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
                                 v[i][4 * q4 + 2] += (uint32_t)q.z; v[i][4 * q4 + 3] += (uint32_t)q.w;
                             }
                         }
-                        if ((HAS_BIAS && !bq) || HAS_MASK || c0 + 16 > p.N) {          // warp-uniform
+                        // each case is straight-line code: the conditions are warp-uniform and tested once per chunk
+                        if (HAS_BIAS && !bq) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (c0 + j < p.N) v[i][j] += (uint32_t)__ldg(brow + c0 + j);
+                        }
+                        if (HAS_MASK && mixed) {
+                            // labels past column N are 0x100 and match no row, so this also pads the row end
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
-                                const int col = c0 + j;
-                                int sc = (int)v[i][j];
-                                bool use = col < p.N;
-                                if (HAS_BIAS && !bq && use) sc += __ldg(brow + col);
-                                if (HAS_MASK) use = use && __shfl_sync(0xffffffffu, col < 32 ? id_lo : id_hi, col & 31) == my_id;
-                                v[i][j] = (uint32_t)(use ? sc : kPadScore);
+                                const int col = c0 + j;                   // compile-time after unrolling: i and j are
+                                const unsigned id = __shfl_sync(0xffffffffu, col < 32 ? id_lo : id_hi, col & 31);
+                                v[i][j] = id == my_id ? v[i][j] : (uint32_t)kPadScore;
                             }
+                        } else if (c0 + 16 > p.N) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) v[i][j] = c0 + j < p.N ? v[i][j] : (uint32_t)kPadScore;
                         }
 #pragma unroll
                         for (int j = 0; j < 16; ++j) mx = max(mx, (int)v[i][j]);
@@ -412,9 +425,9 @@ int launch_window_attn(const CUtensorMap& mq, const CUtensorMap& mk, const CUten
     const int grid = std::min(p.items, sm_count());
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return IPTQ_ERR_CUDA;
-#define IPTQ_WIN_LAUNCH3(HB, HM, PS, LT)                                                                          \
+#define IPTQ_WIN_LAUNCH4(HB, HM, PS, LT, FL)                                                                      \
     do {                                                                                                          \
-        auto kern = window_attention_kernel<DH, VARIANT, HB, HM, PS, LT>;                                         \
+        auto kern = window_attention_kernel<DH, VARIANT, HB, HM, PS, LT, FL>;                                     \
         static int configured[64];          /* largest dynamic shared memory size set so far, per device */     \
         if (configured[dev] < smem_bytes) {                                                                       \
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) \
@@ -422,6 +435,10 @@ int launch_window_attn(const CUtensorMap& mq, const CUtensorMap& mk, const CUten
             configured[dev] = smem_bytes;                                                                         \
         }                                                                                                         \
         launch_kernel(kern, grid, W::THREADS, smem_bytes, st, mq, mk, mv, p);                                     \
+    } while (0)
+#define IPTQ_WIN_LAUNCH3(HB, HM, PS, LT)                                                                          \
+    do {                                                                                                          \
+        if (p.N > 48) IPTQ_WIN_LAUNCH4(HB, HM, PS, LT, true); else IPTQ_WIN_LAUNCH4(HB, HM, PS, LT, false);       \
     } while (0)
 #define IPTQ_WIN_LAUNCH2(HB, HM, PS)                                                                              \
     do {                                                                                                          \
@@ -438,6 +455,7 @@ int launch_window_attn(const CUtensorMap& mq, const CUtensorMap& mk, const CUten
 #undef IPTQ_WIN_LAUNCH
 #undef IPTQ_WIN_LAUNCH2
 #undef IPTQ_WIN_LAUNCH3
+#undef IPTQ_WIN_LAUNCH4
     note_launch();
     return last_launch_status();
 }
