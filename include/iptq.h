@@ -208,6 +208,11 @@ int iptq_layernorm(const int8_t* x, int8_t* y, int64_t rows, int dim, const int3
  * residual_rq: host; y: dev int8 [M, N].  K % 16 == 0, N % 16 == 0, K <= 4096.
  * ws: required (status block; plus N*K bytes of unpack scratch when w_bits = 4).
  */
+/* Packed int4 weights -> int8 [n_elems] (the format w_bits = 8 takes), for deployments that keep the W4 checkpoint
+ * packed on disk but unpack each weight once at load time instead of at every call: the same values, so the same
+ * results as w_bits = 4.  packed: dev [n_elems / 2] bytes; out: dev int8 [n_elems], both 16-byte aligned;
+ * n_elems even (IPTQ_ERR_SHAPE otherwise). */
+int iptq_unpack_int4(const void* packed, int8_t* out, int64_t n_elems, iptq_stream_t stream);
 size_t iptq_linear_workspace_bytes(int64_t M, int N, int K, int w_bits);
 int iptq_linear(const int8_t* x, const void* w, int w_bits, const int32_t* bias, const int32_t* mult,
                 const int8_t* shift, int32_t out_zp, const int8_t* residual, const iptq_requant* residual_rq,

@@ -115,6 +115,7 @@ def lib():
                                   C.c_int64, C.c_int, C.c_int, _vp, C.c_size_t, _vp]
         L.iptq_linear_w4_static.argtypes = [_vp, _vp, _vp, _vp, _vp, C.c_int32, _vp, C.POINTER(Requant), _vp,
                                             C.c_int64, C.c_int, C.c_int, _vp, _vp]
+        L.iptq_unpack_int4.argtypes = [_vp, _vp, C.c_int64, _vp]
         L.iptq_gather_rows.argtypes = [_vp, _vp, _vp, C.c_int64, C.c_int, C.c_int, _vp]
         L.iptq_patchify.argtypes = [_vp, _vp, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, _vp]
         L.iptq_attention_workspace_bytes.restype = C.c_size_t
@@ -152,7 +153,7 @@ def exported_symbols():
     """Names declared in include/iptq.h (used by the CPU-side load test)."""
     return ["iptq_requant_prepare", "iptq_channel_requant_prepare", "iptq_softmax_prepare", "iptq_softmax", "iptq_softmax_table",
             "iptq_gelu_prepare", "iptq_gelu", "iptq_gelu_table", "iptq_gelu_fit", "iptq_gelu_prepare_coeffs", "iptq_layernorm_prepare", "iptq_layernorm",
-            "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_patchify", "iptq_attention_workspace_bytes", "iptq_attention_block",
+            "iptq_unpack_int4", "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_patchify", "iptq_attention_workspace_bytes", "iptq_attention_block",
             "iptq_mlp_workspace_bytes", "iptq_mlp_block", "iptq_encoder_block_workspace_bytes",
             "iptq_encoder_block", "iptq_encoder_block_profiled", "iptq_workspace_init", "iptq_check", "iptq_strerror", "iptq_launch_count",
             "iptq_metric_softmax", "iptq_metric_gelu", "iptq_metric_layernorm", "iptq_softplus", "iptq_sqnr_db",
@@ -374,6 +375,14 @@ def layernorm(x, gamma_q, beta_q, consts: LnConsts, ptf_shift=None, out=None):
     return out
 
 
+def unpack_int4(w_packed):
+    """Packed int4 weights [N, K/2] -> int8 [N, K] on the device (what ``w_bits=8`` takes), once at load time."""
+    n, k2 = w_packed.shape
+    out = torch.empty((n, 2 * k2), dtype=torch.int8, device=w_packed.device)
+    _chk(lib().iptq_unpack_int4(_dp(w_packed), _dp(out), n * 2 * k2, _stream()), "iptq_unpack_int4")
+    return out
+
+
 def linear_workspace_bytes(M, N, K, w_bits=8):
     return int(lib().iptq_linear_workspace_bytes(M, N, K, w_bits))
 
@@ -460,12 +469,14 @@ class EncoderBlock:
     (or any object with the same fields) with the library's own ``*_prepare`` functions."""
 
     def __init__(self, spec, table=(SM_BITEXP, GELU_POLY4, LN_SHIFT, LN_SHIFT), device="cuda", gelu_table_on=True,
-                 softmax_table_on=True):
+                 softmax_table_on=True, unpack_w4_once=False):
         sh = spec.shape
         self.shape = sh
         self.keep = []          # host structs and device tensors referenced by raw pointers
         p = BlockParams()
-        p.B, p.N, p.D, p.H, p.dh, p.Dh, p.w_bits = sh.B, sh.N, sh.D, sh.H, sh.dh, sh.Dh, spec.w_bits
+        # W4 weights may be unpacked here, once, instead of by four kernels at every call (same values, same results)
+        w_bits = 8 if (spec.w_bits == 4 and unpack_w4_once) else spec.w_bits
+        p.B, p.N, p.D, p.H, p.dh, p.Dh, p.w_bits = sh.B, sh.N, sh.D, sh.H, sh.dh, sh.Dh, w_bits
         p.table = VariantTable(*table)
         sm_v, gelu_v, ln1_v, ln2_v = table
 
@@ -488,7 +499,12 @@ class EncoderBlock:
             setattr(p, name, host(c))
         for name, ls in (("qkv", spec.qkv), ("proj", spec.proj), ("fc1", spec.fc1), ("fc2", spec.fc2)):
             m, s = channel_requant_prepare(ls.ratio)
-            setattr(p, "w_" + name, dev(ls.w_packed))
+            if spec.w_bits == 4 and unpack_w4_once:
+                wt = unpack_int4(torch.from_numpy(np.ascontiguousarray(ls.w_packed)).to(device))
+                self.keep.append(wt)
+                setattr(p, "w_" + name, wt.data_ptr())
+            else:
+                setattr(p, "w_" + name, dev(ls.w_packed))
             setattr(p, "b_" + name, dev(ls.bias))
             setattr(p, "m_" + name, dev(m))
             setattr(p, "s_" + name, dev(s))

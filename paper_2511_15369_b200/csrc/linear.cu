@@ -651,4 +651,13 @@ int iptq_mlp_block(const int8_t* x, const void* w1, const int32_t* b1, const int
     return linear_launch(fc2, stream);
 }
 
+int iptq_unpack_int4(const void* packed, int8_t* out, int64_t n_elems, iptq_stream_t stream)
+{
+    if (n_elems < 0 || (n_elems & 1)) return IPTQ_ERR_SHAPE;
+    if (n_elems == 0) return IPTQ_OK;
+    if (!packed || !out) return IPTQ_ERR_NULL;
+    if (!aligned16(packed) || !aligned16(out)) return IPTQ_ERR_ALIGN;
+    return unpack_int4_launch(packed, out, n_elems, stream);
+}
+
 }  // extern "C"

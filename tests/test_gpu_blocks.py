@@ -190,3 +190,11 @@ def test_encoder_block_parity(api, orc, shape, w_bits, table):
     got2 = blk2(_cu(spec.x)).cpu().numpy()
     blk2.ws.check()
     assert (got2 == want).all(), _mismatch(got2, want)
+    if w_bits == 4:
+        # int4 weights unpacked once at load time instead of at every call
+        blk3 = api.EncoderBlock(spec, table, unpack_w4_once=True)
+        got3 = blk3(_cu(spec.x)).cpu().numpy()
+        blk3.ws.check()
+        assert (got3 == want).all(), _mismatch(got3, want)
+        wq = spec.qkv
+        assert (api.unpack_int4(_cu(wq.w_packed)).cpu().numpy() == wq.w).all()
