@@ -507,7 +507,7 @@ template <int NW>
 static int launch_ln(const int8_t* x, int8_t* y, int64_t rows, const int32_t* gq, const int32_t* bq,
                      const uint8_t* ptf_in, const LnDev& c, cudaStream_t st)
 {
-    constexpr int RW = NW <= 4 ? 4 : NW <= 8 ? 2 : 1;
+    constexpr int RW = NW == 1 ? 8 : NW <= 4 ? 4 : NW <= 8 ? 2 : 1;
     const int threads = 256;
     const int64_t want = ((rows + RW - 1) / RW + 7) / 8;
     const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 8);
