@@ -503,6 +503,113 @@ layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int6
     }
 }
 
+// Short rows (dim <= 128, dim % 16 == 0: the first Swin stage): four lanes share a row, so a warp step covers eight
+// rows.  Lane q of a row takes words q, q + 4, ... (WPL = dim / 16 words); row sums are two xor-shuffles over the
+// four lanes, and every lane then runs the scalar part (variance, square root, reciprocal) of its own row, so the
+// hundred dependent instructions of that part are shared by eight rows without any broadcast.
+template <int WPL, bool PTF, bool SAT8, bool ZPF>
+__global__ void __launch_bounds__(256)
+layernorm_short_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int64_t rows,
+                            const int32_t* __restrict__ gamma_q, const int32_t* __restrict__ beta_q,
+                            const uint8_t* __restrict__ ptf, const LnDev c)
+{
+    const int lane = threadIdx.x & 31;
+    const int q = lane & 3;                                   // position inside the row's four lanes
+    const int D = c.dim;                                      // = 16 * WPL
+    grid_dep_launch();
+    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t steps = (rows + 7) / 8;
+    int4 g[WPL], b[WPL];
+    unsigned sh[WPL];
+#pragma unroll
+    for (int k = 0; k < WPL; ++k) {
+        const int wi = q + 4 * k;
+        g[k] = __ldg(reinterpret_cast<const int4*>(gamma_q) + wi);
+        b[k] = __ldg(reinterpret_cast<const int4*>(beta_q) + wi);
+        sh[k] = PTF ? __ldg(reinterpret_cast<const unsigned*>(ptf) + wi) : 0u;
+    }
+    grid_dep_wait();                                          // gamma / beta above are static; the rows come from the previous kernel
+    const int om = c.out.mult, ornd = c.out.rnd, osh = c.out.shift, ozp = c.out.zp;
+    for (int64_t step = warp; step < steps; step += nwarps) {
+        const int64_t row = step * 8 + (lane >> 2);
+        const bool live = row < rows;
+        const int* xr = reinterpret_cast<const int*>(x + (live ? row : 0) * D);
+        int w[WPL];
+#pragma unroll
+        for (int k = 0; k < WPL; ++k) w[k] = live ? __ldcs(xr + q + 4 * k) : 0;
+        int s1 = 0;
+        unsigned s2 = 0;
+#pragma unroll
+        for (int k = 0; k < WPL; ++k) {
+            if (!PTF) {
+                s1 = __dp4a(w[k], 0x01010101, s1);
+                s2 = (unsigned)__dp4a(w[k], w[k], (int)s2);
+            } else {
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const int xv = ((int)(int8_t)(w[k] >> (8 * t))) << ((sh[k] >> (8 * t)) & 3);
+                    s1 += xv;
+                    s2 += (unsigned)(xv * xv);
+                }
+            }
+        }
+        s1 += __shfl_xor_sync(kFull, s1, 1); s2 += __shfl_xor_sync(kFull, s2, 1);
+        s1 += __shfl_xor_sync(kFull, s1, 2); s2 += __shfl_xor_sync(kFull, s2, 2);
+        const long long V = (long long)D * (long long)s2 - (long long)s1 * (long long)s1;            // D^2 var, exact
+        const unsigned long long rt = isqrt_variant((unsigned long long)V, c.variant);                // D * std
+        const long long F = rt ? (long long)floor_div_f64(1099511627776.0, (double)rt) : 0;          // floor(2^40 / rt)
+        const bool narrow = F < (1ll << 29);                  // then (u F) >> 30 = hi32(u * 4F)
+        const int F4 = (int)(F << 2);
+        int out[WPL];
+#pragma unroll
+        for (int k = 0; k < WPL; ++k) {
+            const unsigned wk = (unsigned)w[k];
+            auto elem = [&](int xv, int t, int gg, int bb) -> int {
+                if (PTF) xv <<= ((sh[k] >> (8 * t)) & 3);
+                const int u = D * xv - s1;                                   // D (x - mean)
+                const int nq = narrow ? __mulhi(u, F4) : (int)(((long long)u * F) >> 30);   // (x - mean) / std, Q10
+                int o = mad_hi(nq * gg + bb, om, ornd) >> osh;
+                if (!ZPF) o += ozp;
+                if (!SAT8) o = max(c.out.qmin, min(c.out.qmax, o));
+                return o;
+            };
+            const int o0 = elem(sext_byte<0>(wk), 0, g[k].x, b[k].x);
+            const int o1 = elem(sext_byte<1>(wk), 1, g[k].y, b[k].y);
+            const int o2 = elem(sext_byte<2>(wk), 2, g[k].z, b[k].z);
+            const int o3 = elem(sext_byte<3>(wk), 3, g[k].w, b[k].w);
+            out[k] = SAT8 ? (int)pack4_sat_s8(o0, o1, o2, o3) : (int)pack4_s8(o0, o1, o2, o3);
+        }
+        if (live) {
+            int* yr = reinterpret_cast<int*>(y + row * D);
+#pragma unroll
+            for (int k = 0; k < WPL; ++k) __stcs(yr + q + 4 * k, out[k]);
+        }
+    }
+}
+
+template <int WPL>
+static int launch_ln_short(const int8_t* x, int8_t* y, int64_t rows, const int32_t* gq, const int32_t* bq,
+                           const uint8_t* ptf_in, const LnDev& c, cudaStream_t st)
+{
+    const int threads = 256;
+    const int64_t want = ((rows + 7) / 8 + 7) / 8;
+    const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 8);
+    const bool sat8 = c.out.qmin == -128 && c.out.qmax == 127;
+    LnDev cc = c;
+    const long long rz = (long long)c.out.rnd + ((long long)c.out.zp << c.out.shift);
+    const bool zpf = rz > -(1ll << 30) && rz < (1ll << 30);
+    if (zpf) { cc.out.rnd = (int)rz; cc.out.zp = 0; }
+#define IPTQ_LNS_GO(P, S8, ZF) launch_kernel(layernorm_short_rows_kernel<WPL, P, S8, ZF>, grid, threads, 0, st, x, y, rows, gq, bq, ptf_in, cc)
+    if (c.variant == IPTQ_LN_PTF) { if (sat8) IPTQ_LNS_GO(true, true, false); else IPTQ_LNS_GO(true, false, false); }
+    else if (!sat8)               { IPTQ_LNS_GO(false, false, false); }
+    else if (zpf)                 { IPTQ_LNS_GO(false, true, true); }
+    else                          { IPTQ_LNS_GO(false, true, false); }
+#undef IPTQ_LNS_GO
+    note_launch();
+    return last_launch_status();
+}
+
 template <int NW>
 static int launch_ln(const int8_t* x, int8_t* y, int64_t rows, const int32_t* gq, const int32_t* bq,
                      const uint8_t* ptf_in, const LnDev& c, cudaStream_t st)
@@ -555,6 +662,17 @@ int layernorm_launch(const int8_t* x, int8_t* y, int64_t rows, int dim, const in
     if (rows == 0) return IPTQ_OK;
     LnDev c;
     c.variant = consts->variant; c.dim = dim; c.out = to_dev(consts->out);
+    if ((dim & 15) == 0 && dim <= 128 && rows >= 64) {
+        switch (dim / 16) {                                   // words per lane with four lanes per row
+            case 1: return launch_ln_short<1>(x, y, rows, gq, bq, ptf, c, st);
+            case 2: return launch_ln_short<2>(x, y, rows, gq, bq, ptf, c, st);
+            case 3: return launch_ln_short<3>(x, y, rows, gq, bq, ptf, c, st);
+            case 4: return launch_ln_short<4>(x, y, rows, gq, bq, ptf, c, st);
+            case 6: return launch_ln_short<6>(x, y, rows, gq, bq, ptf, c, st);
+            case 8: return launch_ln_short<8>(x, y, rows, gq, bq, ptf, c, st);
+            default: break;                                   // other widths take the general kernel
+        }
+    }
     const int nw = (dim / 4 + 31) / 32;
     switch (nw) {
         case 1: return launch_ln<1>(x, y, rows, gq, bq, ptf, c, st);

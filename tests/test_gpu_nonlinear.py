@@ -243,15 +243,17 @@ def test_layernorm_parity(api, orc, variant, rows, dim):
     assert (got == want).all()
 
 
-def test_layernorm_degenerate_rows(api, orc):
-    dim = 192
+@pytest.mark.parametrize("dim,rows", [(192, 40), (96, 75), (128, 64), (16, 100), (48, 333)])
+def test_layernorm_degenerate_rows(api, orc, dim, rows):
+    """Constant rows, extreme variances, a ragged last step -- for the general kernel (dim 192) and for the
+    four-lanes-per-row kernel of short rows (dim <= 128, at least 64 rows)."""
     rng = np.random.default_rng(5)
-    x = rng.integers(-128, 128, size=(40, dim)).astype(np.int8)
+    x = rng.integers(-128, 128, size=(rows, dim)).astype(np.int8)
     x[0] = 0
     x[1] = 127                                  # zero variance
     x[2] = -128
     x[3] = 0
-    x[3, 17] = 1                                # smallest non-zero variance
+    x[3, dim // 2] = 1                          # smallest non-zero variance
     x[4, ::2] = 127
     x[4, 1::2] = -128                           # largest variance
     # rows whose D^2 var + 1 is a perfect square make the fixed-step square root stop one above
@@ -259,8 +261,10 @@ def test_layernorm_degenerate_rows(api, orc):
     x[5, :3] = [1, 1, 1]
     gamma = rng.normal(1, 0.1, dim).astype(np.float32)
     beta = rng.normal(0, 0.1, dim).astype(np.float32)
-    for variant in (0, 1):
-        gq, bq, co = orc.layernorm_prepare(gamma, beta, 0.02, 3, 8, variant)
-        _, _, ca = api.layernorm_prepare(gamma, beta, 0.02, 3, 8, variant)
-        got = api.layernorm(_cu(x), _cu(gq), _cu(bq), ca).cpu().numpy()
-        assert (got == orc.layernorm(x, gq, bq, co)).all()
+    for variant in (0, 1, 2):
+        for out_bits, zp in ((8, 3), (6, -2)):
+            ptf = synth.ptf_shifts(x) if variant == 2 else None
+            gq, bq, co = orc.layernorm_prepare(gamma, beta, 0.02 * (1 << (8 - out_bits)), zp, out_bits, variant)
+            _, _, ca = api.layernorm_prepare(gamma, beta, 0.02 * (1 << (8 - out_bits)), zp, out_bits, variant)
+            got = api.layernorm(_cu(x), _cu(gq), _cu(bq), ca, None if ptf is None else _cu(ptf)).cpu().numpy()
+            assert (got == orc.layernorm(x, gq, bq, co, ptf)).all()
