@@ -217,6 +217,12 @@ size_t iptq_linear_workspace_bytes(int64_t M, int N, int K, int w_bits);
 int iptq_linear(const int8_t* x, const void* w, int w_bits, const int32_t* bias, const int32_t* mult,
                 const int8_t* shift, int32_t out_zp, const int8_t* residual, const iptq_requant* residual_rq,
                 int8_t* y, int64_t M, int N, int K, void* ws, size_t ws_bytes, iptq_stream_t stream);
+/* The same layer with activations out_bits wide (4..8; the W6A6 setting of Sec. 4 uses 6): y is clamped to
+ * [-2^(out_bits-1), 2^(out_bits-1) - 1] instead of the int8 range, still stored as int8.  iptq_linear() is out_bits = 8. */
+int iptq_linear_bits(const int8_t* x, const void* w, int w_bits, const int32_t* bias, const int32_t* mult,
+                     const int8_t* shift, int32_t out_zp, const int8_t* residual, const iptq_requant* residual_rq,
+                     int8_t* y, int64_t M, int N, int K, int out_bits, void* ws, size_t ws_bytes,
+                     iptq_stream_t stream);
 
 /* ------------------------------------------------------------------ 4-bit-weight GEMM without any allocation
  * (No counterpart in the paper: this is a packaging variant of iptq_linear(w_bits = 4) for callers that
@@ -317,6 +323,8 @@ typedef struct {
     const void* w_fc1; const int32_t *b_fc1, *m_fc1; const int8_t* s_fc1; const iptq_gelu_consts* gelu;
     const void* w_fc2; const int32_t *b_fc2, *m_fc2; const int8_t* s_fc2; int32_t fc2_zp;
     const iptq_requant* res2_rq;
+    int32_t act_bits;              /* width of the QKV / proj / FC2 outputs: 0 or 8 = int8; 6 with 6-bit LayerNorm, Softmax,
+                                      attention and GELU constants is the W6A6 setting of the detection results (Sec. 4) */
 } iptq_block_params;
 
 size_t iptq_encoder_block_workspace_bytes(const iptq_block_params* p /*host*/);

@@ -62,6 +62,7 @@ class BlockParams(C.Structure):
         ("w_fc2", C.c_void_p), ("b_fc2", C.c_void_p), ("m_fc2", C.c_void_p), ("s_fc2", C.c_void_p),
         ("fc2_zp", C.c_int32),
         ("res2_rq", C.c_void_p),
+        ("act_bits", C.c_int32),
     ]
 
 
@@ -112,6 +113,8 @@ def lib():
                                        C.c_void_p, C.POINTER(LnConsts)]
         L.oracle_linear.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int]
+        L.oracle_linear_bits.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int]
         L.oracle_attention_block.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int,
                                              C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.POINTER(SoftmaxConsts),
                                              C.POINTER(Requant)]
@@ -243,12 +246,12 @@ def layernorm(x: np.ndarray, gq: np.ndarray, bq: np.ndarray, c: LnConsts, ptf_sh
 
 
 # ---------------------------------------------------------------- GEMM carriers and blocks
-def linear(x, w, bias, mult, shift, out_zp=0, residual=None, residual_rq=None, w_bits=8):
+def linear(x, w, bias, mult, shift, out_zp=0, residual=None, residual_rq=None, w_bits=8, out_bits=8):
     M, K = x.shape
     N = w.shape[0]
     y = np.empty((M, N), dtype=np.int8)
-    _chk(lib().oracle_linear(_p(x), _p(w), w_bits, _p(bias), _p(mult), _p(shift), out_zp, _p(residual),
-                             _ref(residual_rq), _p(y), M, N, K), "linear")
+    _chk(lib().oracle_linear_bits(_p(x), _p(w), w_bits, _p(bias), _p(mult), _p(shift), out_zp, _p(residual),
+                                  _ref(residual_rq), _p(y), M, N, K, out_bits), "linear")
     return y
 
 

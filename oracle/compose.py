@@ -17,23 +17,25 @@ def block_params(spec, table) -> dict:
     """Field dictionary of ``oracle.encoder_block`` for a block spec and a (softmax, gelu, ln1, ln2) variant table."""
     sm_v, gelu_v, ln1_v, ln2_v = table
     sh = spec.shape
-    d = dict(B=sh.B, N=sh.N, D=sh.D, H=sh.H, dh=sh.dh, Dh=sh.Dh, w_bits=spec.w_bits,
+    ab = getattr(spec, "a_bits", 8)                # activation width: 8, or 6 for the W6A6 setting
+    d = dict(B=sh.B, N=sh.N, D=sh.D, H=sh.H, dh=sh.dh, Dh=sh.Dh, w_bits=4 if spec.w_bits == 4 else 8, act_bits=ab,
              sm_variant=sm_v, gelu_variant=gelu_v, ln1_variant=ln1_v, ln2_variant=ln2_v)
     for name, ln, var in (("ln1", spec.ln1, ln1_v), ("ln2", spec.ln2, ln2_v)):
-        gq, bq, c = oracle.layernorm_prepare(ln["gamma"], ln["beta"], ln["out_scale"], ln["out_zp"], 8, var)
+        gq, bq, c = oracle.layernorm_prepare(ln["gamma"], ln["beta"], ln["out_scale"], ln["out_zp"], ab, var)
         d[name + "_gamma"], d[name + "_beta"], d[name], d[name + "_ptf"] = gq, bq, c, ln.get("ptf")
     for name, ls in (("qkv", spec.qkv), ("proj", spec.proj), ("fc1", spec.fc1), ("fc2", spec.fc2)):
         d["w_" + name], d["b_" + name] = ls.w_packed, ls.bias
         d["m_" + name], d["s_" + name] = _channel_requant(ls.ratio)
     # the logarithm candidate writes 4-bit codes and its P V product is at scale 2^-15 instead of 2^-7
     log2 = sm_v == oracle.SM_LOG2
-    d["sm"] = oracle.softmax_prepare(spec.softmax_scale, sh.N, 4 if log2 else 8, sm_v)
-    d["pv_rq"] = oracle.requant_prepare(spec.pv_ratio / 256 if log2 else spec.pv_ratio)
+    qa = 1 << (ab - 1)
+    d["sm"] = oracle.softmax_prepare(spec.softmax_scale, sh.N, 4 if log2 else ab, sm_v)
+    d["pv_rq"] = oracle.requant_prepare(spec.pv_ratio * qa / 32768 if log2 else spec.pv_ratio, 0, -qa, qa - 1)
     d["attn_bias"], d["mask_id"] = spec.attn_bias, spec.mask_id
     d["res1_rq"] = oracle.requant_prepare(spec.proj.res_ratio / 65536, zp=spec.proj.res_zp)
     d["res2_rq"] = oracle.requant_prepare(spec.fc2.res_ratio / 65536, zp=spec.fc2.res_zp)
     gl = spec.gelu
-    d["gelu"] = oracle.gelu_prepare(gl["in_scale"], gl["in_bits"], gl["out_scale"], gl["out_zp"], 8, gelu_v)
+    d["gelu"] = oracle.gelu_prepare(gl["in_scale"], gl["in_bits"], gl["out_scale"], gl["out_zp"], ab, gelu_v)
     d["proj_zp"], d["fc2_zp"] = spec.proj.out_zp, spec.fc2.out_zp
     return d
 

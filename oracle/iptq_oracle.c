@@ -437,7 +437,18 @@ int oracle_linear(const int8_t* x, const void* w, int w_bits, const int32_t* bia
                   const int8_t* shift, int32_t out_zp, const int8_t* residual, const oracle_requant_t* residual_rq,
                   int8_t* y, int64_t M, int N, int K)
 {
+    return oracle_linear_bits(x, w, w_bits, bias, mult, shift, out_zp, residual, residual_rq, y, M, N, K, 8);
+}
+
+/* The same layer with out_bits-wide activations (W6A6 setting): the output is clamped to
+ * [-2^(out_bits-1), 2^(out_bits-1) - 1] instead of the int8 range. */
+int oracle_linear_bits(const int8_t* x, const void* w, int w_bits, const int32_t* bias, const int32_t* mult,
+                       const int8_t* shift, int32_t out_zp, const int8_t* residual,
+                       const oracle_requant_t* residual_rq, int8_t* y, int64_t M, int N, int K, int out_bits)
+{
     if (!x || !w || !mult || !shift || !y) return ORACLE_ERR_ARG;
+    if (out_bits < 4 || out_bits > 8) return ORACLE_ERR_ARG;
+    const int64_t qmin = -((int64_t)1 << (out_bits - 1)), qmax = ((int64_t)1 << (out_bits - 1)) - 1;
     if (w_bits != 8 && w_bits != 4) return ORACLE_ERR_ARG;
     if (residual && !residual_rq) return ORACLE_ERR_ARG;
 #pragma omp parallel for schedule(static)
@@ -451,7 +462,7 @@ int oracle_linear(const int8_t* x, const void* w, int w_bits, const int32_t* bia
                 int64_t rr = ((int64_t)residual[m * N + n] - residual_rq->zp) << 16;
                 v += requant_noclamp(rr, residual_rq->mult, residual_rq->shift);
             }
-            y[m * N + n] = (int8_t)clamp64(v + out_zp, -128, 127);
+            y[m * N + n] = (int8_t)clamp64(v + out_zp, qmin, qmax);
         }
     }
     return ORACLE_OK;
@@ -513,6 +524,16 @@ int oracle_mlp_block(const int8_t* x, const void* w1, const int32_t* b1, const i
                      const int8_t* s2, int32_t out_zp, const int8_t* residual, const oracle_requant_t* residual_rq,
                      int8_t* y, int64_t M, int D, int Dh, int w_bits)
 {
+    return oracle_mlp_block_bits(x, w1, b1, m1, s1, gc, w2, b2, m2, s2, out_zp, residual, residual_rq, y, M, D, Dh,
+                                 w_bits, 8);
+}
+
+int oracle_mlp_block_bits(const int8_t* x, const void* w1, const int32_t* b1, const int32_t* m1, const int8_t* s1,
+                          const oracle_gelu_consts_t* gc, const void* w2, const int32_t* b2, const int32_t* m2,
+                          const int8_t* s2, int32_t out_zp, const int8_t* residual,
+                          const oracle_requant_t* residual_rq, int8_t* y, int64_t M, int D, int Dh, int w_bits,
+                          int out_bits)
+{
     if (!x || !w1 || !m1 || !s1 || !gc || !y) return ORACLE_ERR_ARG;
     if (w_bits != 8 && w_bits != 4) return ORACLE_ERR_ARG;
     int8_t* h = w2 ? (int8_t*)malloc((size_t)M * (size_t)Dh) : y;
@@ -529,7 +550,7 @@ int oracle_mlp_block(const int8_t* x, const void* w1, const int32_t* b1, const i
         }
     }
     if (!w2) return ORACLE_OK;
-    int rc = oracle_linear(h, w2, w_bits, b2, m2, s2, out_zp, residual, residual_rq, y, M, D, Dh);
+    int rc = oracle_linear_bits(h, w2, w_bits, b2, m2, s2, out_zp, residual, residual_rq, y, M, D, Dh, out_bits);
     free(h);
     return rc;
 }
@@ -540,22 +561,23 @@ int oracle_encoder_block(const int8_t* x, int8_t* y, const oracle_block_params_t
     int64_t T = p->B * p->N;
     int D = p->D;
     int rc;
+    const int ab = p->act_bits ? p->act_bits : 8;      /* activation width of the three linear outputs */
     int8_t* h1 = (int8_t*)malloc((size_t)T * D);
     int8_t* qkv = (int8_t*)malloc((size_t)T * 3 * D);
     int8_t* att = (int8_t*)malloc((size_t)T * D);
     int8_t* x1 = (int8_t*)malloc((size_t)T * D);
     int8_t* h2 = (int8_t*)malloc((size_t)T * D);
     rc = oracle_layernorm(x, h1, T, D, p->ln1_gamma, p->ln1_beta, p->ln1_ptf, p->ln1);
-    if (!rc) rc = oracle_linear(h1, p->w_qkv, p->w_bits, p->b_qkv, p->m_qkv, p->s_qkv, 0, NULL, NULL, qkv, T, 3 * D, D);
+    if (!rc) rc = oracle_linear_bits(h1, p->w_qkv, p->w_bits, p->b_qkv, p->m_qkv, p->s_qkv, 0, NULL, NULL, qkv, T, 3 * D, D, ab);
     /* qkv row = [q | k | v], head h at columns h*dh */
     if (!rc) rc = oracle_attention_strided(qkv, qkv + D, qkv + 2 * D, att, p->B, p->H, p->N, p->dh,
                                            3 * (int64_t)D, p->dh, (int64_t)p->N * 3 * D,
                                            p->attn_bias, p->mask_id, p->sm, p->pv_rq);
-    if (!rc) rc = oracle_linear(att, p->w_proj, p->w_bits, p->b_proj, p->m_proj, p->s_proj, p->proj_zp,
-                                x, p->res1_rq, x1, T, D, D);
+    if (!rc) rc = oracle_linear_bits(att, p->w_proj, p->w_bits, p->b_proj, p->m_proj, p->s_proj, p->proj_zp,
+                                     x, p->res1_rq, x1, T, D, D, ab);
     if (!rc) rc = oracle_layernorm(x1, h2, T, D, p->ln2_gamma, p->ln2_beta, p->ln2_ptf, p->ln2);
-    if (!rc) rc = oracle_mlp_block(h2, p->w_fc1, p->b_fc1, p->m_fc1, p->s_fc1, p->gelu, p->w_fc2, p->b_fc2,
-                                   p->m_fc2, p->s_fc2, p->fc2_zp, x1, p->res2_rq, y, T, D, p->Dh, p->w_bits);
+    if (!rc) rc = oracle_mlp_block_bits(h2, p->w_fc1, p->b_fc1, p->m_fc1, p->s_fc1, p->gelu, p->w_fc2, p->b_fc2,
+                                        p->m_fc2, p->s_fc2, p->fc2_zp, x1, p->res2_rq, y, T, D, p->Dh, p->w_bits, ab);
     free(h1); free(qkv); free(att); free(x1); free(h2);
     return rc;
 }

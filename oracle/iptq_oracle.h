@@ -116,6 +116,9 @@ int oracle_layernorm(const int8_t* x, int8_t* y, int64_t rows, int dim, const in
 int oracle_linear(const int8_t* x, const void* w, int w_bits, const int32_t* bias, const int32_t* mult,
                   const int8_t* shift, int32_t out_zp, const int8_t* residual, const oracle_requant_t* residual_rq,
                   int8_t* y, int64_t M, int N, int K);
+int oracle_linear_bits(const int8_t* x, const void* w, int w_bits, const int32_t* bias, const int32_t* mult,
+                       const int8_t* shift, int32_t out_zp, const int8_t* residual,
+                       const oracle_requant_t* residual_rq, int8_t* y, int64_t M, int N, int K, int out_bits);
 int oracle_attention_block(const int8_t* q, const int8_t* k, const int8_t* v, int8_t* out, int64_t B, int H, int N,
                            int dh, const int32_t* bias, const uint8_t* mask_id, const oracle_softmax_consts_t* sc,
                            const oracle_requant_t* out_rq);
@@ -128,6 +131,12 @@ int oracle_mlp_block(const int8_t* x, const void* w1, const int32_t* b1, const i
                      const oracle_gelu_consts_t* gc, const void* w2, const int32_t* b2, const int32_t* m2,
                      const int8_t* s2, int32_t out_zp, const int8_t* residual, const oracle_requant_t* residual_rq,
                      int8_t* y, int64_t M, int D, int Dh, int w_bits);
+
+int oracle_mlp_block_bits(const int8_t* x, const void* w1, const int32_t* b1, const int32_t* m1, const int8_t* s1,
+                          const oracle_gelu_consts_t* gc, const void* w2, const int32_t* b2, const int32_t* m2,
+                          const int8_t* s2, int32_t out_zp, const int8_t* residual,
+                          const oracle_requant_t* residual_rq, int8_t* y, int64_t M, int D, int Dh, int w_bits,
+                          int out_bits);
 
 /* Parameters of one encoder block (all host pointers). */
 typedef struct {
@@ -143,6 +152,7 @@ typedef struct {
     const void* w_fc1; const int32_t *b_fc1, *m_fc1; const int8_t* s_fc1; const oracle_gelu_consts_t* gelu;
     const void* w_fc2; const int32_t *b_fc2, *m_fc2; const int8_t* s_fc2; int32_t fc2_zp;
     const oracle_requant_t* res2_rq;
+    int32_t act_bits;      /* width of the QKV / proj / FC2 outputs: 0 or 8 = int8, 6 = the W6A6 setting */
 } oracle_block_params_t;
 /* x [B*N, D] -> y [B*N, D]; scratch is allocated inside (host malloc). */
 int oracle_encoder_block(const int8_t* x, int8_t* y, const oracle_block_params_t* p);

@@ -68,6 +68,7 @@ class BlockParams(C.Structure):
         ("w_fc2", C.c_void_p), ("b_fc2", C.c_void_p), ("m_fc2", C.c_void_p), ("s_fc2", C.c_void_p),
         ("fc2_zp", C.c_int32),
         ("res2_rq", C.c_void_p),
+        ("act_bits", C.c_int32),
     ]
 
 
@@ -113,6 +114,8 @@ def lib():
         L.iptq_linear_workspace_bytes.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
         L.iptq_linear.argtypes = [_vp, _vp, C.c_int, _vp, _vp, _vp, C.c_int32, _vp, C.POINTER(Requant), _vp,
                                   C.c_int64, C.c_int, C.c_int, _vp, C.c_size_t, _vp]
+        L.iptq_linear_bits.argtypes = [_vp, _vp, C.c_int, _vp, _vp, _vp, C.c_int32, _vp, C.POINTER(Requant), _vp,
+                                       C.c_int64, C.c_int, C.c_int, C.c_int, _vp, C.c_size_t, _vp]
         L.iptq_linear_w4_static.argtypes = [_vp, _vp, _vp, _vp, _vp, C.c_int32, _vp, C.POINTER(Requant), _vp,
                                             C.c_int64, C.c_int, C.c_int, _vp, _vp]
         L.iptq_unpack_int4.argtypes = [_vp, _vp, C.c_int64, _vp]
@@ -153,7 +156,7 @@ def exported_symbols():
     """Names declared in include/iptq.h (used by the CPU-side load test)."""
     return ["iptq_requant_prepare", "iptq_channel_requant_prepare", "iptq_softmax_prepare", "iptq_softmax", "iptq_softmax_table",
             "iptq_gelu_prepare", "iptq_gelu", "iptq_gelu_table", "iptq_gelu_fit", "iptq_gelu_prepare_coeffs", "iptq_layernorm_prepare", "iptq_layernorm",
-            "iptq_unpack_int4", "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_patchify", "iptq_attention_workspace_bytes", "iptq_attention_block",
+            "iptq_unpack_int4", "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_bits", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_patchify", "iptq_attention_workspace_bytes", "iptq_attention_block",
             "iptq_mlp_workspace_bytes", "iptq_mlp_block", "iptq_encoder_block_workspace_bytes",
             "iptq_encoder_block", "iptq_encoder_block_profiled", "iptq_workspace_init", "iptq_check", "iptq_strerror", "iptq_launch_count",
             "iptq_metric_softmax", "iptq_metric_gelu", "iptq_metric_layernorm", "iptq_softplus", "iptq_sqnr_db",
@@ -387,13 +390,15 @@ def linear_workspace_bytes(M, N, K, w_bits=8):
     return int(lib().iptq_linear_workspace_bytes(M, N, K, w_bits))
 
 
-def linear(x, w, bias, mult, shift, ws: Workspace, out_zp=0, residual=None, residual_rq=None, w_bits=8, out=None):
+def linear(x, w, bias, mult, shift, ws: Workspace, out_zp=0, residual=None, residual_rq=None, w_bits=8, out=None,
+           out_bits=8):
     M, K = x.shape
     N = w.shape[0]
     if out is None:
         out = torch.empty((M, N), dtype=torch.int8, device=x.device)
-    _chk(lib().iptq_linear(_dp(x), _dp(w), w_bits, _dp(bias), _dp(mult), _dp(shift), out_zp, _dp(residual),
-                           _ref(residual_rq), _dp(out), M, N, K, ws.ptr, ws.nbytes, _stream()), "iptq_linear")
+    _chk(lib().iptq_linear_bits(_dp(x), _dp(w), w_bits, _dp(bias), _dp(mult), _dp(shift), out_zp, _dp(residual),
+                                _ref(residual_rq), _dp(out), M, N, K, out_bits, ws.ptr, ws.nbytes, _stream()),
+         "iptq_linear")
     return out
 
 
@@ -475,9 +480,11 @@ class EncoderBlock:
         self.keep = []          # host structs and device tensors referenced by raw pointers
         p = BlockParams()
         # W4 weights may be unpacked here, once, instead of by four kernels at every call (same values, same results)
-        w_bits = 8 if (spec.w_bits == 4 and unpack_w4_once) else spec.w_bits
+        w_bits = 8 if (spec.w_bits == 4 and unpack_w4_once) or spec.w_bits == 6 else spec.w_bits   # 6-bit weights are int8 values
+        ab = getattr(spec, "a_bits", 8)                # activation width: 8, or 6 for the W6A6 setting
         p.B, p.N, p.D, p.H, p.dh, p.Dh, p.w_bits = sh.B, sh.N, sh.D, sh.H, sh.dh, sh.Dh, w_bits
         p.table = VariantTable(*table)
+        p.act_bits = ab
         sm_v, gelu_v, ln1_v, ln2_v = table
 
         def dev(a):
@@ -492,7 +499,7 @@ class EncoderBlock:
             return C.addressof(s)
 
         for name, lnspec, var in (("ln1", spec.ln1, ln1_v), ("ln2", spec.ln2, ln2_v)):
-            gq, bq, c = layernorm_prepare(lnspec["gamma"], lnspec["beta"], lnspec["out_scale"], lnspec["out_zp"], 8, var)
+            gq, bq, c = layernorm_prepare(lnspec["gamma"], lnspec["beta"], lnspec["out_scale"], lnspec["out_zp"], ab, var)
             setattr(p, name + "_gamma", dev(gq))
             setattr(p, name + "_beta", dev(bq))
             setattr(p, name + "_ptf", dev(lnspec.get("ptf")))
@@ -512,16 +519,17 @@ class EncoderBlock:
         p.mask_id = dev(spec.mask_id)
         # the logarithm candidate writes 4-bit codes and its P V product is at scale 2^-15 instead of 2^-7
         log2 = sm_v == SM_LOG2
-        sc = softmax_prepare(spec.softmax_scale, sh.N, 4 if log2 else 8, sm_v)
+        sc = softmax_prepare(spec.softmax_scale, sh.N, 4 if log2 else ab, sm_v)
         if softmax_table_on:
             self.keep.append(softmax_table(sc, device))
         p.sm = host(sc)
-        p.pv_rq = host(requant_prepare(spec.pv_ratio / 256 if log2 else spec.pv_ratio))
+        qa = 1 << (ab - 1)
+        p.pv_rq = host(requant_prepare(spec.pv_ratio * qa / 32768 if log2 else spec.pv_ratio, 0, -qa, qa - 1))
         p.proj_zp, p.fc2_zp = spec.proj.out_zp, spec.fc2.out_zp
         p.res1_rq = host(requant_prepare(spec.proj.res_ratio / 65536.0, zp=spec.proj.res_zp))
         p.res2_rq = host(requant_prepare(spec.fc2.res_ratio / 65536.0, zp=spec.fc2.res_zp))
         gl = spec.gelu
-        gc = gelu_prepare(gl["in_scale"], gl["in_bits"], gl["out_scale"], gl["out_zp"], 8, gelu_v)
+        gc = gelu_prepare(gl["in_scale"], gl["in_bits"], gl["out_scale"], gl["out_zp"], ab, gelu_v)
         if gelu_table_on:
             self.keep.append(gelu_table(gc, device))
         p.gelu = host(gc)

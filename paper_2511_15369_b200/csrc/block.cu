@@ -15,6 +15,7 @@ struct LinearArgs {
     int8_t* y;
     int64_t M; int N, K;
     StatusBlock* status;
+    int out_bits = 8;                                          // width of the output activations (plain and residual epilogues)
 };
 int linear_launch(const LinearArgs& a, cudaStream_t st);
 int unpack_int4_launch(const void* packed, int8_t* out, int64_t n_elems, cudaStream_t st);
@@ -133,7 +134,9 @@ static int encoder_block_run(const int8_t* x, int8_t* y, const iptq_block_params
 
     if ((rc = layernorm_launch(x, h1, T, D, p->ln1_gamma, p->ln1_beta, p->ln1_ptf, p->ln1, stream)) != IPTQ_OK) return rc;
     if ((rc = mark()) != IPTQ_OK) return rc;
-    LinearArgs lq{h1, wq, p->b_qkv, p->m_qkv, p->s_qkv, 0, nullptr, nullptr, nullptr, qkv, T, 3 * D, D, status};
+    const int ab = p->act_bits ? p->act_bits : 8;            // width of the QKV / proj / FC2 outputs
+    if (ab < 4 || ab > 8) return IPTQ_ERR_BITS;
+    LinearArgs lq{h1, wq, p->b_qkv, p->m_qkv, p->s_qkv, 0, nullptr, nullptr, nullptr, qkv, T, 3 * D, D, status, ab};
     if ((rc = linear_launch(lq, stream)) != IPTQ_OK) return rc;
     if ((rc = mark()) != IPTQ_OK) return rc;
     // a row of qkv is [q | k | v]; head h occupies columns h*dh .. of each third
@@ -142,7 +145,7 @@ static int encoder_block_run(const int8_t* x, int8_t* y, const iptq_block_params
                 l.bias_t ? reinterpret_cast<int32_t*>(base + l.bias_t) : nullptr};
     if ((rc = attention_launch(aa, stream)) != IPTQ_OK) return rc;
     if ((rc = mark()) != IPTQ_OK) return rc;
-    LinearArgs lp{att, wp, p->b_proj, p->m_proj, p->s_proj, p->proj_zp, x, p->res1_rq, nullptr, x1, T, D, D, status};
+    LinearArgs lp{att, wp, p->b_proj, p->m_proj, p->s_proj, p->proj_zp, x, p->res1_rq, nullptr, x1, T, D, D, status, ab};
     if ((rc = linear_launch(lp, stream)) != IPTQ_OK) return rc;
     if ((rc = mark()) != IPTQ_OK) return rc;
     if ((rc = layernorm_launch(x1, h2, T, D, p->ln2_gamma, p->ln2_beta, p->ln2_ptf, p->ln2, stream)) != IPTQ_OK) return rc;
@@ -150,7 +153,7 @@ static int encoder_block_run(const int8_t* x, int8_t* y, const iptq_block_params
     LinearArgs l1{h2, w1, p->b_fc1, p->m_fc1, p->s_fc1, 0, nullptr, nullptr, p->gelu, hid, T, Dh, D, status};
     if ((rc = linear_launch(l1, stream)) != IPTQ_OK) return rc;
     if ((rc = mark()) != IPTQ_OK) return rc;
-    LinearArgs l2{hid, w2, p->b_fc2, p->m_fc2, p->s_fc2, p->fc2_zp, x1, p->res2_rq, nullptr, y, T, D, Dh, status};
+    LinearArgs l2{hid, w2, p->b_fc2, p->m_fc2, p->s_fc2, p->fc2_zp, x1, p->res2_rq, nullptr, y, T, D, Dh, status, ab};
     if ((rc = linear_launch(l2, stream)) != IPTQ_OK) return rc;
     return mark();
 }

@@ -86,6 +86,7 @@ struct GemmParams {
     int num_m_tiles, num_n_tiles;
     const int32_t* bias; const int32_t* mult; const int8_t* shift;
     int out_zp;
+    int qmin, qmax;                                   // output range of the plain / residual epilogues when it is not int8
     int res_mult, res_rnd, res_shift, res_off;        // residual branch: ((res << 16) - res_off) through R
     GeluDev gelu;
     const int8_t* gelu_tab;                           // device table of the integer GELU, or null
@@ -340,6 +341,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     } else {
                         v += p.out_zp;
                     }
+                    if (EPI != EPI_GELU && !SAT8) v = max(p.qmin, min(p.qmax, v));   // activations narrower than 8 bits
                     o[j] = v;
                 }
                 st_shared_v4(out_blk + swz32(lane, ch), pack4_sat_s8(o[0], o[1], o[2], o[3]),
@@ -412,6 +414,7 @@ struct LinearArgs {
     int8_t* y;
     int64_t M; int N, K;
     StatusBlock* status;
+    int out_bits = 8;                                          // width of the output activations (plain and residual epilogues)
 };
 
 template <int BN, int EPI, int GV, bool SAT8, bool GTAB = false>
@@ -453,6 +456,7 @@ int linear_launch(const LinearArgs& a, cudaStream_t st)
         if (a.gelu->variant < 0 || a.gelu->variant > 2) return IPTQ_ERR_VARIANT;
         int rc = check_requant(&a.gelu->out); if (rc != IPTQ_OK) return rc;
     }
+    if (a.out_bits < 4 || a.out_bits > 8) return IPTQ_ERR_BITS;
     if (!a.status) return IPTQ_ERR_WORKSPACE;
     if (a.M == 0) return IPTQ_OK;
     // 128-wide tiles use the tensor core fully and re-read the activations less often, but rebuild the rounding
@@ -469,6 +473,7 @@ static int linear_launch_bn(const LinearArgs& a, cudaStream_t st)
     p.num_m_tiles = (int)((a.M + BM - 1) / BM);
     p.num_n_tiles = (a.N + BN - 1) / BN;
     p.bias = a.bias; p.mult = a.mult; p.shift = a.shift; p.out_zp = a.out_zp;
+    p.qmin = -(1 << (a.out_bits - 1)); p.qmax = (1 << (a.out_bits - 1)) - 1;
     p.res_mult = p.res_rnd = p.res_shift = p.res_off = 0;
     if (a.residual) {
         p.res_mult = a.residual_rq->mult; p.res_shift = a.residual_rq->shift;
@@ -516,6 +521,10 @@ static int linear_launch_bn(const LinearArgs& a, cudaStream_t st)
         }
 #undef IPTQ_GEMM_GELU
     }
+    if (a.out_bits != 8) {
+        if (a.residual) return launch_gemm<BN, EPI_RESIDUAL, 0, false>(ma, mb, my, mr, p, st);
+        return launch_gemm<BN, EPI_REQUANT, 0, false>(ma, mb, my, mr, p, st);
+    }
     if (a.residual) return launch_gemm<BN, EPI_RESIDUAL, 0, true>(ma, mb, my, mr, p, st);
     return launch_gemm<BN, EPI_REQUANT, 0, true>(ma, mb, my, mr, p, st);
 }
@@ -562,7 +571,17 @@ int iptq_linear(const int8_t* x, const void* w, int w_bits, const int32_t* bias,
                 const int8_t* shift, int32_t out_zp, const int8_t* residual, const iptq_requant* residual_rq,
                 int8_t* y, int64_t M, int N, int K, void* ws, size_t ws_bytes, iptq_stream_t stream)
 {
+    return iptq_linear_bits(x, w, w_bits, bias, mult, shift, out_zp, residual, residual_rq, y, M, N, K, 8, ws, ws_bytes,
+                            stream);
+}
+
+int iptq_linear_bits(const int8_t* x, const void* w, int w_bits, const int32_t* bias, const int32_t* mult,
+                     const int8_t* shift, int32_t out_zp, const int8_t* residual, const iptq_requant* residual_rq,
+                     int8_t* y, int64_t M, int N, int K, int out_bits, void* ws, size_t ws_bytes,
+                     iptq_stream_t stream)
+{
     if (w_bits != 8 && w_bits != 4) return IPTQ_ERR_BITS;
+    if (out_bits < 4 || out_bits > 8) return IPTQ_ERR_BITS;
     if (!ws) return IPTQ_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(ws) & 255u) return IPTQ_ERR_ALIGN;
     if (N < 1 || K < 1) return IPTQ_ERR_SHAPE;
@@ -577,7 +596,7 @@ int iptq_linear(const int8_t* x, const void* w, int w_bits, const int32_t* bias,
         w8 = scratch;
     }
     LinearArgs a{x, w8, bias, mult, shift, out_zp, residual, residual_rq, nullptr, y, M, N, K,
-                 static_cast<StatusBlock*>(ws)};
+                 static_cast<StatusBlock*>(ws), out_bits};
     return linear_launch(a, stream);
 }
 

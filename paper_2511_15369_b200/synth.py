@@ -223,21 +223,25 @@ class BlockSpec:
     fc1: LinearSpec | None = None                  # ratio = S_x*S_w[n] / S_gelu_in
     fc2: LinearSpec | None = None
     softmax_scale: float = 0.0                     # scale of the int32 scores (1/sqrt(dh) folded in)
-    pv_ratio: float = 0.0                          # 2^-7 * S_v / S_attn
+    pv_ratio: float = 0.0                          # 2^-(a_bits-1) * S_v / S_attn
     gelu: dict = field(default_factory=dict)       # in_scale, in_bits, out_scale, out_zp
     attn_bias: np.ndarray | None = None            # int32 [H, N, N] at the score scale
     mask_id: np.ndarray | None = None              # uint8 [B, N]
+    a_bits: int = 8                                # activation width (8, or 6 for W6A6)
 
 
 def make_block(shape: BlockShape, seed: int = 0, w_bits: int = 8, gelu_in_bits: int = 16,
-               calib_images: int = 2, mask_id: np.ndarray | None = None) -> BlockSpec:
+               calib_images: int = 2, mask_id: np.ndarray | None = None, a_bits: int = 8) -> BlockSpec:
     """Draw one encoder block (weights, input) and calibrate every intermediate scale
-    with an fp64 shadow forward over the first ``calib_images`` attention problems."""
+    with an fp64 shadow forward over the first ``calib_images`` attention problems.
+    ``w_bits`` 8 / 6 / 4 and ``a_bits`` 8 / 6 give the W8A8, W6A6 and W4A8 settings (6-bit values are stored as
+    int8, 4-bit weights are packed)."""
+    qa = float((1 << (a_bits - 1)) - 1)             # largest activation code
     g = _rng(seed, 3)
     T, D, H, dh, Dh, N = shape.T, shape.D, shape.H, shape.dh, shape.Dh, shape.N
     # block input: the LayerNorm-input distribution
     xin, g1, b1, _ = ln_values(T, D, seed)
-    x, Sx = quantize_sym(xin, 8, np.int8)
+    x, Sx = quantize_sym(xin, a_bits, np.int8)
     del xin
     Tc = min(T, calib_images * N)
     Bc = Tc // N
@@ -252,12 +256,13 @@ def make_block(shape: BlockShape, seed: int = 0, w_bits: int = 8, gelu_in_bits: 
         wp = pack_int4(wq) if w_bits_ == 4 else wq
         return wq, Sw, bq, wp
 
-    spec = BlockSpec(shape=shape, w_bits=w_bits, x=x)
+    spec = BlockSpec(shape=shape, w_bits=w_bits, x=x, a_bits=a_bits)
     # ---- LN1
     h1 = layernorm_ref(xc, g1, b1)
-    S_h1 = float(np.abs(h1).max()) / 127.0
-    spec.ln1 = dict(gamma=g1, beta=b1, out_scale=S_h1, out_zp=0)
-    h1 = np.clip(np.round(h1 / S_h1), -128, 127) * S_h1
+    S_h1 = float(np.abs(h1).max()) / qa
+    # the block's activations carry one scale per tensor, so the power-of-two factors LN_PTF takes are all 2^0
+    spec.ln1 = dict(gamma=g1, beta=b1, out_scale=S_h1, out_zp=0, ptf=np.zeros(shape.D, np.uint8))
+    h1 = np.clip(np.round(h1 / S_h1), -qa - 1, qa) * S_h1
     # ---- QKV; a gain on the q/k rows puts the logits on config 0's N(0, 3^2) spread
     wf, bf = draw_w(3 * D, D)
     q0 = h1 @ wf[:D].T + bf[:D]
@@ -268,9 +273,9 @@ def make_block(shape: BlockShape, seed: int = 0, w_bits: int = 8, gelu_in_bits: 
     bf[:2 * D] *= gain
     wq, Sw, bq, wp = qlin(wf, bf, S_h1, w_bits)
     qkv = h1 @ (wq * Sw[:, None]).T + bq * (S_h1 * Sw)
-    S_qkv = float(np.abs(qkv).max()) / 127.0
+    S_qkv = float(np.abs(qkv).max()) / qa
     spec.qkv = LinearSpec(wq, wp, bq, S_h1 * Sw / S_qkv)
-    qkv = np.clip(np.round(qkv / S_qkv), -128, 127) * S_qkv
+    qkv = np.clip(np.round(qkv / S_qkv), -qa - 1, qa) * S_qkv
     # ---- attention
     spec.softmax_scale = S_qkv * S_qkv / math.sqrt(dh)
     qh = qkv[:, :D].reshape(Bc, N, H, dh)
@@ -287,23 +292,24 @@ def make_block(shape: BlockShape, seed: int = 0, w_bits: int = 8, gelu_in_bits: 
         lg = np.where(mm[:, None], -1e9, lg)
     P = softmax_ref(lg)
     att = np.einsum("bhnm,bmhd->bnhd", P, vh).reshape(Tc, D)
-    S_att = float(np.abs(att).max()) / 127.0
-    spec.pv_ratio = (2.0 ** -7) * S_qkv / S_att
-    att = np.clip(np.round(att / S_att), -128, 127) * S_att
+    # floor on the scale: the dyadic requantiser takes ratios below 1/4
+    S_att = max(float(np.abs(att).max()) / qa, 4.2 * (2.0 ** -(a_bits - 1)) * S_qkv)
+    spec.pv_ratio = (2.0 ** -(a_bits - 1)) * S_qkv / S_att
+    att = np.clip(np.round(att / S_att), -qa - 1, qa) * S_att
     # ---- proj + residual
     wf, bf = draw_w(D, D)
     wq, Sw, bq, wp = qlin(wf, bf, S_att, w_bits)
     x1 = att @ (wq * Sw[:, None]).T + bq * (S_att * Sw) + xc
-    S_x1 = float(np.abs(x1).max()) / 127.0
+    S_x1 = float(np.abs(x1).max()) / qa
     spec.proj = LinearSpec(wq, wp, bq, S_att * Sw / S_x1, 0, Sx / S_x1, 0)
-    x1 = np.clip(np.round(x1 / S_x1), -128, 127) * S_x1
+    x1 = np.clip(np.round(x1 / S_x1), -qa - 1, qa) * S_x1
     # ---- LN2
     g2 = g.normal(1.0, 0.1, size=D).astype(np.float32)
     b2 = g.normal(0.0, 0.1, size=D).astype(np.float32)
     h2 = layernorm_ref(x1, g2, b2)
-    S_h2 = float(np.abs(h2).max()) / 127.0
-    spec.ln2 = dict(gamma=g2, beta=b2, out_scale=S_h2, out_zp=0)
-    h2 = np.clip(np.round(h2 / S_h2), -128, 127) * S_h2
+    S_h2 = float(np.abs(h2).max()) / qa
+    spec.ln2 = dict(gamma=g2, beta=b2, out_scale=S_h2, out_zp=0, ptf=np.zeros(shape.D, np.uint8))
+    h2 = np.clip(np.round(h2 / S_h2), -qa - 1, qa) * S_h2
     # ---- FC1 + GELU; a gain puts the GELU input on config 0's N(-0.3, 1.2^2) spread
     wf, bf = draw_w(Dh, D)
     a0 = h2 @ wf.T + bf
@@ -321,16 +327,16 @@ def make_block(shape: BlockShape, seed: int = 0, w_bits: int = 8, gelu_in_bits: 
         gelu_in_bits -= 1
     spec.fc1 = LinearSpec(wq, wp, bq, S_h2 * Sw / S_gin)
     hid = gelu_ref(a)
-    S_hid, zp_hid = affine_out_quant(hid, 8)
+    S_hid, zp_hid = affine_out_quant(hid, a_bits)
     spec.gelu = dict(in_scale=S_gin, in_bits=gelu_in_bits, out_scale=S_hid, out_zp=zp_hid)
-    hid_q = np.clip(np.round(hid / S_hid) + zp_hid, -128, 127)
+    hid_q = np.clip(np.round(hid / S_hid) + zp_hid, -qa - 1, qa)
     hid = (hid_q - zp_hid) * S_hid
     # ---- FC2 + residual; the hidden zero point is folded into the bias
     wf, bf = draw_w(D, Dh)
     wq, Sw, bq, wp = qlin(wf, bf, S_hid, w_bits)
     bq = (bq.astype(np.int64) - zp_hid * wq.astype(np.int64).sum(axis=1)).astype(np.int32)
     yf = hid_q @ (wq * Sw[:, None]).T * S_hid + bq * (S_hid * Sw) + x1
-    S_y = float(np.abs(yf).max()) / 127.0
+    S_y = float(np.abs(yf).max()) / qa
     spec.fc2 = LinearSpec(wq, wp, bq, S_hid * Sw / S_y, 0, S_x1 / S_y, 0)
     return spec
 

@@ -67,6 +67,31 @@ def test_linear_parity(api, orc, M, N, K):
     assert (got == want).all(), _mismatch(got, want)
 
 
+@pytest.mark.parametrize("out_bits", [6, 4])
+def test_linear_narrow_outputs(api, orc, out_bits):
+    """Outputs clamped to a signed range narrower than 8 bits (W6A6 activations), plain and residual epilogue."""
+    M, N, K = 333, 384, 192
+    rng = np.random.default_rng(out_bits)
+    x, w, bias, ratios = _linear_case(rng, M, N, K)
+    ma, sa = api.channel_requant_prepare(ratios)
+    ws = api.Workspace(api.linear_workspace_bytes(M, N, K))
+    want = orc.linear(x, w, bias, ma, sa, out_zp=1, out_bits=out_bits)
+    got = api.linear(_cu(x), _cu(w), _cu(bias), _cu(ma), _cu(sa), ws, out_zp=1, out_bits=out_bits).cpu().numpy()
+    ws.check()
+    q = 1 << (out_bits - 1)
+    assert want.min() == -q and want.max() == q - 1
+    assert (got == want).all(), _mismatch(got, want)
+    res = rng.integers(-q, q, size=(M, N)).astype(np.int8)
+    rro, rra = orc.requant_prepare(0.9 / 65536, zp=-1), api.requant_prepare(0.9 / 65536, zp=-1)
+    want = orc.linear(x, w, None, ma, sa, out_zp=-2, residual=res, residual_rq=rro, out_bits=out_bits)
+    got = api.linear(_cu(x), _cu(w), None, _cu(ma), _cu(sa), ws, out_zp=-2, residual=_cu(res), residual_rq=rra,
+                     out_bits=out_bits).cpu().numpy()
+    ws.check()
+    assert (got == want).all(), _mismatch(got, want)
+    with pytest.raises(api.IptqError):
+        api.linear(_cu(x), _cu(w), None, _cu(ma), _cu(sa), ws, out_bits=9)
+
+
 def test_linear_w4(api, orc):
     rng = np.random.default_rng(44)
     M, N, K = 200, 256, 384
@@ -175,10 +200,29 @@ def _oracle_block(orc, spec, table):
     (synth.BlockShape("ViT-B b1 W4", 1, 197, 768, 12, 64, 3072), 4, (2, 2, 1, 0)),
     (synth.BlockShape("Swin-T 8 windows", 8, 49, 96, 3, 32, 384, True), 8, (0, 0, 0, 0)),
     (synth.BlockShape("DeiT-S b2 log2", 2, 197, 384, 6, 64, 1536), 8, (3, 0, 0, 0)),
+    (synth.BlockShape("DeiT-T b2 ptf", 2, 197, 192, 3, 64, 768), 8, (1, 0, 2, 2)),
     (synth.BlockShape("Swin-T 8 windows log2", 8, 49, 96, 3, 32, 384, True), 8, (3, 1, 1, 1)),
 ])
 def test_encoder_block_parity(api, orc, shape, w_bits, table):
-    spec = synth.make_block(shape, seed=1, w_bits=w_bits, gelu_in_bits=14 if table[1] == 2 else 16)
+    _block_parity(api, orc, synth.make_block(shape, seed=1, w_bits=w_bits, gelu_in_bits=14 if table[1] == 2 else 16),
+                  w_bits, table)
+
+
+@pytest.mark.parametrize("shape,table", [
+    (synth.BlockShape("DeiT-S b2 W6A6", 2, 197, 384, 6, 64, 1536), (0, 0, 0, 0)),
+    (synth.BlockShape("DeiT-T b3 W6A6 alt", 3, 197, 192, 3, 64, 768), (1, 1, 1, 2)),
+    (synth.BlockShape("Swin-T 8 windows W6A6", 8, 49, 96, 3, 32, 384, True), (2, 0, 0, 0)),
+    (synth.BlockShape("DeiT-S b1 W6A6 log2", 1, 197, 384, 6, 64, 1536), (3, 0, 0, 0)),
+])
+def test_encoder_block_w6a6_parity(api, orc, shape, table):
+    """6-bit weights and activations (Table 1, W6A6): every operator of the block emits signed 6-bit codes."""
+    spec = synth.make_block(shape, seed=2, w_bits=6, a_bits=6)
+    _block_parity(api, orc, spec, 6, table)
+    y = api.EncoderBlock(spec, table)(_cu(spec.x)).cpu().numpy()
+    assert y.min() >= -32 and y.max() <= 31
+
+
+def _block_parity(api, orc, spec, w_bits, table):
     want = _oracle_block(orc, spec, table)
     blk = api.EncoderBlock(spec, table)
     got = blk(_cu(spec.x)).cpu().numpy()

@@ -409,6 +409,11 @@ def test_linear_against_int64_matmul(orc, w_bits):
     assert (y == want).all()
     y0 = orc.linear(x, wp, None, mult, shift, w_bits=w_bits)
     assert (y0 == np.clip(_np_requant_vec(acc - bias, mult, shift), -128, 127)).all()
+    # narrower activations (the W6A6 setting): the same sum, clamped to the out_bits range
+    for bits in (6, 4):
+        yb = orc.linear(x, wp, bias, mult, shift, out_zp=5, residual=res, residual_rq=rrq, w_bits=w_bits, out_bits=bits)
+        assert (yb == np.clip(main + rterm + 5, -(1 << (bits - 1)), (1 << (bits - 1)) - 1)).all()
+        assert yb.min() == -(1 << (bits - 1)) and yb.max() == (1 << (bits - 1)) - 1
 
 
 def test_attention_against_composition(orc):
@@ -476,6 +481,35 @@ def test_encoder_block_is_the_chain_of_its_parts(orc, w_bits):
     assert (y == want).all()
     # and the whole integer block tracks the fp64 computation it quantises (loose: W4 is coarse)
     assert np.abs(hid.astype(int)).max() > 20 and len(np.unique(y)) > 20
+
+
+def test_encoder_block_w6a6_is_the_chain_of_its_parts(orc):
+    """6-bit weights and activations (the W6A6 column of Table 1): every tensor between two operators stays in
+    the signed 6-bit range (residual stream included), and the block is the chain of the stand-alone operators
+    run at that width."""
+    from oracle import compose
+    shape = synth.BlockShape("tiny", 2, 21, 32, 2, 16, 64, True)
+    spec = synth.make_block(shape, seed=5, w_bits=6, a_bits=6)
+    for lin in (spec.qkv, spec.proj, spec.fc1, spec.fc2):
+        assert np.abs(lin.w.astype(int)).max() <= 31
+    assert np.abs(spec.x.astype(int)).max() <= 32
+    d = compose.block_params(spec, (0, 0, 0, 0))
+    y = orc.encoder_block(spec.x, d)
+    T, D = shape.T, shape.D
+    h1 = orc.layernorm(spec.x, d["ln1_gamma"], d["ln1_beta"], d["ln1"])
+    qkv = orc.linear(h1, d["w_qkv"], d["b_qkv"], d["m_qkv"], d["s_qkv"], out_bits=6)
+    to_heads = lambda a: np.ascontiguousarray(a.reshape(shape.B, shape.N, shape.H, shape.dh).transpose(0, 2, 1, 3))
+    att = orc.attention_block(to_heads(qkv[:, :D]), to_heads(qkv[:, D:2 * D]), to_heads(qkv[:, 2 * D:]),
+                              d["sm"], d["pv_rq"], d["attn_bias"], None).reshape(T, D)
+    x1 = orc.linear(att, d["w_proj"], d["b_proj"], d["m_proj"], d["s_proj"], d["proj_zp"], spec.x, d["res1_rq"],
+                    out_bits=6)
+    h2 = orc.layernorm(x1, d["ln2_gamma"], d["ln2_beta"], d["ln2"])
+    hid = orc.mlp_block(h2, d["w_fc1"], d["b_fc1"], d["m_fc1"], d["s_fc1"], d["gelu"])
+    want = orc.linear(hid, d["w_fc2"], d["b_fc2"], d["m_fc2"], d["s_fc2"], d["fc2_zp"], x1, d["res2_rq"], out_bits=6)
+    for t in (h1, qkv, att, x1, h2, hid, want):
+        assert t.min() >= -32 and t.max() <= 31
+    assert (y == want).all()
+    assert len(np.unique(y)) > 20 and len(np.unique(hid)) > 10
 
 
 def test_mlp_block_fc1_epilogue(orc):
