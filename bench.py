@@ -12,8 +12,8 @@ One step = one pass of the whole block over one batch of seeded synthetic input.
                Gelem/s and fraction of the measured HBM copy bandwidth;
   assignment   the Unified-Metric analysis (every candidate of every non-linear layer of the encoder scored and
                selected on the device) as evaluations/s, with the oracle's scores of the first block beside it;
-  other_blocks the ViT-Base batch-128 and Swin-Tiny window blocks, timed like the headline block (context: the
-               headline metric stays the DeiT-Small block);
+  other_blocks the ViT-Base batch-128 block (8- and 4-bit weights), the Swin-Tiny window block and the 6-bit DeiT-Small
+               block, timed like the headline block (context: the headline metric stays the W8A8 DeiT-Small block);
   models       whole DeiT-T/S/B forward latency at batch 8 (context beside the paper's latency table, other hardware);
   cpu_baseline the CPU oracle timed on the host cores on a bounded sample of the same workload, and the
                element-by-element comparison of the GPU output with it.
@@ -518,14 +518,17 @@ def bench_nonlinear(api, torch, dev, peaks, peak_kind):
 
 
 def bench_other_blocks(api, torch, dev, peaks):
-    """The other single-block configurations (ViT-Base batch 128, Swin-Tiny stage-1 windows), timed like the headline
-    one: CUDA-graph replay of one block step, L2 flushed before each, CUDA events, median of 20."""
+    """The other single-block configurations (ViT-Base batch 128 with 8- and 4-bit weights, Swin-Tiny stage-1 windows,
+    the headline block at 6 bits), timed like the headline one: CUDA-graph replay of one block step, L2 flushed before each, CUDA events, median of 20."""
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
     out = []
-    for cfg in ("cfg2", "cfg3"):
+    cases = [("cfg2", "W8A8", {}, {}), ("cfg2", "W4A8, weights unpacked at every call", {"w_bits": 4}, {}),
+             ("cfg2", "W4A8, weights unpacked once at load time", {"w_bits": 4}, {"unpack_w4_once": True}),
+             ("cfg3", "W8A8", {}, {}), ("cfg1", "W6A6", {"w_bits": 6, "a_bits": 6}, {})]
+    for cfg, label, spec_kw, blk_kw in cases:
         shape = synth.CONFIGS[cfg]
-        spec = synth.make_block(shape, seed=0, calib_images=8 if shape.has_bias else 2)
-        blk = api.EncoderBlock(spec, TABLE, dev)
+        spec = synth.make_block(shape, seed=0, calib_images=8 if shape.has_bias else 2, **spec_kw)
+        blk = api.EncoderBlock(spec, TABLE, dev, **blk_kw)
         x = torch.from_numpy(spec.x).to(dev)
         y = torch.empty_like(x)
         st = torch.cuda.Stream()
@@ -548,7 +551,7 @@ def bench_other_blocks(api, torch, dev, peaks):
         blk.ws.check()
         ms = statistics.median(ts)
         tops = shape.gemm_ops() / (ms * 1e-3) / 1e12
-        out.append({"workload": "%s: %s" % (cfg, shape.name), "ms_per_step": ms, "tops": tops,
+        out.append({"workload": "%s: %s, %s" % (cfg, shape.name, label), "ms_per_step": ms, "tops": tops,
                     "frac_int8_peak": tops / (peaks["bf16_tflops"] * INT8_OVER_BF16), "gop_per_step": shape.gemm_ops() / 1e9})
         del blk, g, x, y, spec
     return out
