@@ -70,10 +70,11 @@ constexpr uint32_t TMEM_COLS = 512;
 // replicated over the 128 lanes so that a thread reads them with the same instruction as its accumulators):
 //   BN =  96: mult, rounding constant, shift           (5 x 96 = 480 columns)
 //   BN = 128: mult, shift - 1; the rounding constant 2^(shift-1) is rebuilt with one shift  (4 x 128 = 512 columns)
-// GTAB: the FC1 epilogue reads the integer GELU from a 64 KB table in shared memory (one ring stage fewer).
+// GTAB: the FC1 epilogue reads the integer GELU from a 64 KB table in shared memory, which leaves room for a shorter ring.
+// The ring takes what shared memory is left: deeper rings changed nothing at K = 384 and gave 3 % at K = 768 / 3072.
 template <int BN, bool GTAB = false>
 struct GemmCfg {
-    static constexpr int STAGES = (BN == 96 ? 5 : 4) - (GTAB ? 1 : 0);
+    static constexpr int STAGES = GTAB ? (BN == 96 ? 4 : 3) : (BN == 96 ? 7 : 5);
     static constexpr int EPI_PARTS = BN / COLS;          // epilogue warps per TMEM lane quadrant
     static constexpr int EPI_WARPS = 4 * EPI_PARTS;
     static constexpr int THREADS = 32 * (2 + EPI_WARPS);
