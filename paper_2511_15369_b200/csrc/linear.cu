@@ -85,6 +85,7 @@ struct GemmCfg {
 struct GemmParams {
     int M, N, K;
     int num_m_tiles, num_n_tiles;
+    int stages;                                       // ring stages in use
     const int32_t* bias; const int32_t* mult; const int8_t* shift;
     int out_zp;
     int qmin, qmax;                                   // output range of the plain / residual epilogues when it is not int8
@@ -101,16 +102,16 @@ struct GemmSmem {
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_BYTES = BN * BK;
     static constexpr int WARP_TILE = 32 * COLS;                                   // bytes of one warp's output block
-    static constexpr int OFF_A = 0;
-    static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
-    static constexpr int OFF_OUT = OFF_B + STAGES * B_BYTES;                     // [EPI_WARPS][32 rows][COLS] int8
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;                        // one ring stage: A tile, then B tile
+    static constexpr int OFF_OUT = 0;                                             // [EPI_WARPS][32 rows][COLS] int8
     static constexpr int OFF_RES = OFF_OUT + EPI_WARPS * WARP_TILE;              // same shape, residual tiles
     static constexpr int OFF_BIAS = OFF_RES + EPI_WARPS * WARP_TILE;             // [EPI_WARPS][COLS] int32
     static constexpr int OFF_TAB = OFF_BIAS + EPI_WARPS * COLS * 4;              // GELU table (GTAB only)
     static constexpr int OFF_BAR = OFF_TAB + (GTAB ? IPTQ_GELU_TABLE_SIZE : 0);
     static constexpr int NUM_BARS = 2 * STAGES + 4 + EPI_WARPS;
-    static constexpr int OFF_END = OFF_BAR + NUM_BARS * 8 + 16;
-    static constexpr int TOTAL = OFF_END + 1024;                                 // slack for 1024-byte alignment
+    static constexpr int OFF_RING = (OFF_BAR + NUM_BARS * 8 + 16 + 1023) & ~1023; // the ring comes last: its length is a launch parameter
+    static constexpr int total(int stages) { return OFF_RING + stages * STAGE_BYTES + 1024; }   // slack for 1024-byte alignment
+    static constexpr int TOTAL = total(STAGES);
 };
 
 // Byte offset of 16-byte chunk `chunk` (0/1) of row `row` inside a [32][32]-byte block written/read by TMA with
@@ -133,8 +134,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     constexpr uint32_t TM_MULT = G::TM_MULT, TM_RND = G::TM_RND, TM_SHIFT = G::TM_SHIFT;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* sA = smem + L::OFF_A;
-    uint8_t* sB = smem + L::OFF_B;
+    uint8_t* sA = smem + L::OFF_RING;
+    uint8_t* sB = sA + L::A_BYTES;
+    const int stages = p.stages;                     // ring stages in use (<= STAGES)
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
     uint64_t* empty_bar = full_bar + STAGES;
     uint64_t* acc_full = empty_bar + STAGES;      // [2]
@@ -181,9 +183,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(&empty_bar[s], ph ^ 1u, ctl, p.status, 1)) { ok = false; break; }
                     mbar_expect_tx(&full_bar[s], L::A_BYTES + L::B_BYTES);
-                    tma_load_2d(sA + s * L::A_BYTES, &map_a, &full_bar[s], kb * BK, mt * BM);
-                    tma_load_2d(sB + s * L::B_BYTES, &map_b, &full_bar[s], kb * BK, n0);
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                    tma_load_2d(sA + s * L::STAGE_BYTES, &map_a, &full_bar[s], kb * BK, mt * BM);
+                    tma_load_2d(sB + s * L::STAGE_BYTES, &map_b, &full_bar[s], kb * BK, n0);
+                    if (++s == stages) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
             }
@@ -204,8 +206,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(&full_bar[s], ph, ctl, p.status, 3)) { ok = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t a_addr = smem_u32(sA + s * L::A_BYTES);
-                    const uint32_t b_addr = smem_u32(sB + s * L::B_BYTES);
+                    const uint32_t a_addr = smem_u32(sA + s * L::STAGE_BYTES);
+                    const uint32_t b_addr = smem_u32(sB + s * L::STAGE_BYTES);
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k) {
                         // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart; a k-step is 32 bytes
@@ -214,7 +216,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         umma_i8(tacc, da, db, idesc, 1u);
                     }
                     umma_commit(&empty_bar[s]);               // frees the stage once these MMAs have read it
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                    if (++s == stages) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
                 umma_commit(&acc_full[ab]);                   // accumulator complete
@@ -435,7 +437,12 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUten
     // every CTA serves one column tile; the SMs are split evenly among the column tiles
     const int per_n = std::max(1, std::min(sm_count() / p.num_n_tiles, p.num_m_tiles));
     const int grid = p.num_n_tiles * per_n;
-    launch_kernel(kern, grid, GemmCfg<BN>::THREADS, L::TOTAL, st, ma, mb, my, mr, p);
+    // a ring much longer than one tile's K loop buys nothing, and a smaller footprint lets the next kernel's CTAs
+    // become resident earlier
+    GemmParams q = p;
+    const int kblocks = (p.K + BK - 1) / BK;
+    q.stages = std::max(2, std::min(L::STAGES, kblocks + 1));
+    launch_kernel(kern, grid, GemmCfg<BN>::THREADS, L::total(q.stages), st, ma, mb, my, mr, q);
     note_launch();
     return last_launch_status();
 }
