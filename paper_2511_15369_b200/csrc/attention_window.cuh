@@ -90,7 +90,7 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
             int s = 0; uint32_t ph = 0;
             int stops = 0;                                     // stop marks written so far (every group needs one)
             for (;;) {
-                if (!mbar_wait<true>(&kv_empty[s], ph ^ 1u, ctl, p.status, 21)) break;
+                if (!mbar_wait(&kv_empty[s], ph ^ 1u, ctl, p.status, 21)) break;
                 const int it = stops ? p.items : atomicAdd(&p.status->work_next, 1);
                 if (it >= p.items) {
                     item_of[s] = -1;
@@ -127,8 +127,8 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
             const uint32_t idesc_o = umma_idesc_i8(128, DH, false, true, false, true);     // u8 P (K-major) x s8 V (MN-major)
             auto issue_pv = [&](int j) -> bool {                // item count index j: its P is (about to be) ready
                 const int g = j % G, n = j / G, sj = j % ST;
-                if (!mbar_wait<true>(&p_ready[g], (uint32_t)n & 1u, ctl, p.status, 24)) return false;
-                if (!mbar_wait<true>(&o_empty[g], ((uint32_t)n & 1u) ^ 1u, ctl, p.status, 22)) return false;   // previous O of the group has been read
+                if (!mbar_wait(&p_ready[g], (uint32_t)n & 1u, ctl, p.status, 24)) return false;
+                if (!mbar_wait(&o_empty[g], ((uint32_t)n & 1u) ^ 1u, ctl, p.status, 22)) return false;   // previous O of the group has been read
                 tc_fence_after_sync();
                 const uint32_t tmem_o = tmem_base + (uint32_t)(g * W::GCOLS + 128);
                 const uint32_t p_addr = smem_u32(sP + g * W::P_BYTES);
@@ -151,12 +151,12 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
             for (int k = 0;; ++k) {
                 if (k < k_stop) {
                     const int sk = k % ST;
-                    if (!mbar_wait<true>(&kv_full[sk], (uint32_t)(k / ST) & 1u, ctl, p.status, 23)) break;
+                    if (!mbar_wait(&kv_full[sk], (uint32_t)(k / ST) & 1u, ctl, p.status, 23)) break;
                     if (item_of[sk] < 0) {
                         k_stop = k;
                     } else {
                         const int g = k % G, n = k / G;
-                        if (!mbar_wait<true>(&s_empty[g], ((uint32_t)n & 1u) ^ 1u, ctl, p.status, 28)) break;   // the group holds its previous S in registers
+                        if (!mbar_wait(&s_empty[g], ((uint32_t)n & 1u) ^ 1u, ctl, p.status, 28)) break;   // the group holds its previous S in registers
                         tc_fence_after_sync();
                         const uint32_t q_addr = smem_u32(smem + sk * W::STAGE_BYTES);
                         const uint32_t k_addr = q_addr + 128 * DH;
@@ -211,7 +211,7 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
 
         for (int k = g, n = 0;; k += G, ++n) {
             const int sk = k % ST;
-            if (!mbar_wait<true>(&kv_full[sk], (uint32_t)(k / ST) & 1u, ctl, p.status, 27)) break;   // acquire: the item number is visible
+            if (!mbar_wait(&kv_full[sk], (uint32_t)(k / ST) & 1u, ctl, p.status, 27)) break;   // acquire: the item number is visible
             const int it = item_of[sk];
             if (it < 0) break;
             int bh = 2 * it + win;
@@ -238,7 +238,7 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
             const unsigned id_lo = HAS_MASK && lane < p.N ? mrow[lane] : 0x100u;
             const unsigned id_hi = HAS_MASK && lane + 32 < p.N ? mrow[lane + 32] : 0x100u;
 
-            if (!mbar_wait<true>(&s_full[g], (uint32_t)n & 1u, ctl, p.status, 25)) break;
+            if (!mbar_wait(&s_full[g], (uint32_t)n & 1u, ctl, p.status, 25)) break;
             tc_fence_after_sync();
             uint32_t v[4][16];
 #pragma unroll
@@ -350,7 +350,7 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
             fence_proxy_async_smem();            // generic-proxy stores -> visible to the tensor core's reads
             mbar_arrive(&p_ready[g]);
             // ---- output of this item: the other groups' items fill the time the P V product takes
-            if (!mbar_wait<true>(&o_full[g], (uint32_t)n & 1u, ctl, p.status, 26)) break;
+            if (!mbar_wait(&o_full[g], (uint32_t)n & 1u, ctl, p.status, 26)) break;
             tc_fence_after_sync();
             if (warp_rows) {
                 int8_t* orow = p.out + ((size_t)b * p.N + row) * HD + h * DH;

@@ -38,28 +38,17 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// One try.  SUSPEND: the thread may be suspended by the hardware for up to `kSuspendNs`, so a waiting warp costs a
-// handful of issue slots per wait instead of spinning beside the working warps, but it wakes later than a spinning
-// one (measured: the GEMM and the general attention kernel lose 2-4 % to that; the window attention kernel, whose
-// row threads share the issue slots with the waiting warps, gains about 1 %).
-constexpr uint32_t kSuspendNs = 20000;
-template <bool SUSPEND>
+// One try.  The plain form returns within the hardware's own short limit; the form with a suspend-time hint costs
+// fewer issue slots while waiting but wakes the warp late (measured: 2-4 % on every tensor-core kernel), so it is
+// not used.
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
 {
     uint32_t ok;
-    if constexpr (SUSPEND) {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-            "selp.b32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendNs) : "memory");
-    } else {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.b32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    }
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
 
@@ -68,20 +57,15 @@ struct CtaControl {
     volatile int abort;
 };
 
-// tries before a wait gives up (seconds in total either way): a suspended try may block for up to kSuspendNs, a
-// plain one returns within the hardware's own short limit
-constexpr uint32_t kWaitSpinsSuspend = 1u << 18;
-constexpr uint32_t kWaitSpinsPlain = 1u << 24;
+constexpr uint32_t kWaitSpins = 1u << 24;      // tries before a wait gives up: tenths of a second at the very least
 
 // Bounded wait.  Returns false when the wait ran out or another role already aborted; the first
 // waiter to give up records (where, blockIdx) in the status block.
-template <bool SUSPEND = false>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, CtaControl* ctl, StatusBlock* status,
                                           int where)
 {
-    constexpr uint32_t spins = SUSPEND ? kWaitSpinsSuspend : kWaitSpinsPlain;
-    for (uint32_t spin = 0; spin < spins; ++spin) {
-        if (mbar_try_wait<SUSPEND>(bar, parity)) return true;
+    for (uint32_t spin = 0; spin < kWaitSpins; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
         if ((spin & 15u) == 15u && ctl->abort) return false;
     }
     ctl->abort = 1;
