@@ -311,26 +311,28 @@ def run_ours(args):
 
     # ---- end to end from pinned host buffers: every step copies its input host -> device, runs the block and copies
     #      the result device -> host.  A whole step (copy in, the block's launches, copy out) is one CUDA graph; steps
-    #      are independent, so two buffer sets (each with its own block workspace) alternate on two streams and the
-    #      copies of one step overlap the block of its neighbour.
+    #      are independent, so four buffer sets (each with its own block workspace) take turns on four streams and the
+    #      copies of one step overlap the block and the copies of its neighbours.
+    E2E_SETS = 4                                        # a step is a chain of three phases: four sets keep all of them busy
     xh = torch.from_numpy(spec.x).pin_memory()
-    yh = [torch.empty_like(xh).pin_memory() for _ in range(2)]
-    xd = [torch.empty_like(x) for _ in range(2)]
-    yd = [torch.empty_like(x) for _ in range(2)]
-    blks = [blk, api.EncoderBlock(spec, TABLE, device=dev)]
+    yh = [torch.empty_like(xh).pin_memory() for _ in range(E2E_SETS)]
+    xd = [torch.empty_like(x) for _ in range(E2E_SETS)]
+    yd = [torch.empty_like(x) for _ in range(E2E_SETS)]
+    blks = [blk] + [api.EncoderBlock(spec, TABLE, device=dev) for _ in range(E2E_SETS - 1)]
 
     def e2e_step(i):
         xd[i].copy_(xh, non_blocking=True)
         blks[i](xd[i], yd[i])
         yh[i].copy_(yd[i], non_blocking=True)
 
-    graphs = [capture(lambda i=i: e2e_step(i)) for i in range(2)]
-    s_e2e = [torch.cuda.Stream(device=dev) for _ in range(2)]
+    graphs = [capture(lambda i=i: e2e_step(i)) for i in range(E2E_SETS)]
+    s_e2e = [torch.cuda.Stream(device=dev) for _ in range(E2E_SETS)]
 
     def e2e_steps(n):
         for k in range(n):
-            with torch.cuda.stream(s_e2e[k & 1]):
-                graphs[k & 1].replay()                     # replays on one stream run in order: buffer set reuse is safe
+            i = k % E2E_SETS
+            with torch.cuda.stream(s_e2e[i]):
+                graphs[i].replay()                         # replays on one stream run in order: buffer set reuse is safe
         for st_ in s_e2e:
             torch.cuda.current_stream().wait_stream(st_)
 
@@ -347,7 +349,7 @@ def run_ours(args):
     windows.append((t0, time.perf_counter()))
     total_e2e = max_over_ranks(e0.elapsed_time(e1))
     e2e_value = job_tops(ops, K, world, total_e2e)
-    got_full = yh[(K - 1) & 1].numpy().copy()
+    got_full = yh[(K - 1) % E2E_SETS].numpy().copy()
     for b_ in blks:
         b_.ws.check()
 
@@ -436,7 +438,7 @@ def run_ours(args):
                    "cache": "L2 flushed (256 MiB write) before every timed step, outside the event pairs",
                    "launch": "each step is one CUDA-graph replay of the launches iptq_encoder_block() enqueues"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(xh.numel()), "d2h_bytes_per_step": int(yh[0].numel()),
-                "ms_per_step": total_e2e / K, "pipelining": "one CUDA graph per step (copy in, block, copy out); two buffer sets alternate on two streams"},
+                "ms_per_step": total_e2e / K, "pipelining": "one CUDA graph per step (copy in, block, copy out); four buffer sets take turns on four streams"},
         "gpu_launches": int(launches),
         "clocks": clock_summary,
         "roofline": roofline,
