@@ -353,6 +353,23 @@ def run_ours(args):
     for b_ in blks:
         b_.ws.check()
 
+    # the host link as this machine gives it (one direction at a time, 64 MiB pinned copies): the floor of an end-to-end step
+    def link_gbs(dst, src):
+        ts = []
+        for _ in range(4):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            dst.copy_(src, non_blocking=True)
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return src.numel() / (min(ts) * 1e-3) / 1e9
+    hbuf = torch.empty(64 << 20, dtype=torch.uint8).pin_memory()
+    dbuf = torch.empty(64 << 20, dtype=torch.uint8, device=dev)
+    link = {"h2d_gbs": link_gbs(dbuf, hbuf), "d2h_gbs": link_gbs(hbuf, dbuf)}
+    link["floor_ms_per_step"] = 1e3 * max(xh.numel() / (link["h2d_gbs"] * 1e9), yh[0].numel() / (link["d2h_gbs"] * 1e9))
+    del hbuf, dbuf
+
     # ---- stand-alone non-linear kernels on tensors larger than L2
     peaks, peak_kind = measured_peaks()
     nonlinear = []
@@ -438,7 +455,7 @@ def run_ours(args):
                    "cache": "L2 flushed (256 MiB write) before every timed step, outside the event pairs",
                    "launch": "each step is one CUDA-graph replay of the launches iptq_encoder_block() enqueues"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(xh.numel()), "d2h_bytes_per_step": int(yh[0].numel()),
-                "ms_per_step": total_e2e / K, "pipelining": "one CUDA graph per step (copy in, block, copy out); four buffer sets take turns on four streams"},
+                "ms_per_step": total_e2e / K, "host_link": link, "pipelining": "one CUDA graph per step (copy in, block, copy out); four buffer sets take turns on four streams"},
         "gpu_launches": int(launches),
         "clocks": clock_summary,
         "roofline": roofline,
