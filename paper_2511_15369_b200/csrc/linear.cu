@@ -468,8 +468,10 @@ int linear_launch(const LinearArgs& a, cudaStream_t st)
     if (!a.status) return IPTQ_ERR_WORKSPACE;
     if (a.M == 0) return IPTQ_OK;
     // 128-wide tiles use the tensor core fully and re-read the activations less often, but rebuild the rounding
-    // constant per output (two more instructions); measured, they win only for the plain epilogue at small K
-    const bool wide = a.N % 128 == 0 && (a.N % 96 != 0 || (!a.gelu && !a.residual && a.K <= 768));
+    // constant per output (two more instructions); measured, they win for the plain epilogue and for the tabulated
+    // GELU epilogue at small K (ViT-Base FC1: 24 column tiles on 144 CTAs instead of 32 on 128), not for the
+    // polynomial GELU or the residual epilogue
+    const bool wide = a.N % 128 == 0 && (a.N % 96 != 0 || ((!a.gelu || a.gelu->table) && !a.residual && a.K <= 768));
     return wide ? linear_launch_bn<128>(a, st) : linear_launch_bn<96>(a, st);
 }
 
