@@ -57,16 +57,31 @@ struct CtaControl {
     volatile int abort;
 };
 
-constexpr uint32_t kWaitSpins = 1u << 24;      // tries before a wait gives up: tenths of a second at the very least
+// A wait gives up after kWaitNs of wall time (read from the global timer every 1024 tries), far above any legitimate
+// wait, which is bounded by the previous kernel's run time; kWaitSpins bounds it as well should the timer stand still.
+constexpr uint64_t kWaitNs = 2000000000ull;
+constexpr uint32_t kWaitSpins = 1u << 28;
+__device__ __forceinline__ uint64_t global_timer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 
 // Bounded wait.  Returns false when the wait ran out or another role already aborted; the first
 // waiter to give up records (where, blockIdx) in the status block.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, CtaControl* ctl, StatusBlock* status,
                                           int where)
 {
+    uint64_t t0 = 0;
     for (uint32_t spin = 0; spin < kWaitSpins; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((spin & 15u) == 15u && ctl->abort) return false;
+        if ((spin & 1023u) == 1023u) {
+            const uint64_t t = global_timer_ns();
+            if (t0 == 0) t0 = t;
+            else if (t - t0 > kWaitNs) break;
+        }
     }
     ctl->abort = 1;
     if (status && atomicExch(&status->timeout_flag, 1) == 0) {
