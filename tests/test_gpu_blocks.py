@@ -119,7 +119,8 @@ def test_linear_errors(api):
 
 
 @pytest.mark.parametrize("variant", [0, 1, 2])
-@pytest.mark.parametrize("M,D,Dh", [(197, 192, 768), (333, 384, 1536), (64, 96, 384)])
+# hidden widths 768 / 1536 / 384 take 128-wide column tiles with the tabulated GELU, 288 the 96-wide ones
+@pytest.mark.parametrize("M,D,Dh", [(197, 192, 768), (333, 384, 1536), (64, 96, 384), (130, 96, 288)])
 def test_mlp_parity(api, orc, variant, M, D, Dh):
     rng = np.random.default_rng(M + variant)
     x = rng.integers(-128, 128, size=(M, D)).astype(np.int8)
