@@ -216,7 +216,7 @@ def test_encoder_block_parity(api, orc, shape, w_bits, table):
     (synth.BlockShape("DeiT-S b1 W6A6 log2", 1, 197, 384, 6, 64, 1536), (3, 0, 0, 0)),
 ])
 def test_encoder_block_w6a6_parity(api, orc, shape, table):
-    """6-bit weights and activations (Table 1, W6A6): every operator of the block emits signed 6-bit codes."""
+    """6-bit weights and activations (the W6A6 column of the object-detection results, Table 8): every operator of the block emits signed 6-bit codes."""
     spec = synth.make_block(shape, seed=2, w_bits=6, a_bits=6)
     _block_parity(api, orc, spec, 6, table)
     y = api.EncoderBlock(spec, table)(_cu(spec.x)).cpu().numpy()

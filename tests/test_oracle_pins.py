@@ -484,7 +484,7 @@ def test_encoder_block_is_the_chain_of_its_parts(orc, w_bits):
 
 
 def test_encoder_block_w6a6_is_the_chain_of_its_parts(orc):
-    """6-bit weights and activations (the W6A6 column of Table 1): every tensor between two operators stays in
+    """6-bit weights and activations (the W6A6 column of the object-detection results, Table 8): every tensor between two operators stays in
     the signed 6-bit range (residual stream included), and the block is the chain of the stand-alone operators
     run at that width."""
     from oracle import compose
