@@ -19,6 +19,8 @@ struct LinearArgs {
 };
 int linear_launch(const LinearArgs& a, cudaStream_t st);
 int unpack_int4_launch(const void* packed, int8_t* out, int64_t n_elems, cudaStream_t st);
+int unpack_int4_multi_launch(const void* const* packed, int8_t* const* out, const int64_t* n_elems, int count,
+                             cudaStream_t st);
 int layernorm_launch(const int8_t* x, int8_t* y, int64_t rows, int dim, const int32_t* gq, const int32_t* bq,
                      const uint8_t* ptf, const iptq_ln_consts* consts, cudaStream_t st);
 struct AttnArgs {
@@ -125,11 +127,16 @@ static int encoder_block_run(const int8_t* x, int8_t* y, const iptq_block_params
         struct { const void* src; size_t off; int64_t n; const int8_t** dst; } u[4] = {
             {p->w_qkv, l.w_qkv, (int64_t)3 * D * D, &wq}, {p->w_proj, l.w_proj, (int64_t)D * D, &wp},
             {p->w_fc1, l.w_fc1, (int64_t)Dh * D, &w1}, {p->w_fc2, l.w_fc2, (int64_t)D * Dh, &w2}};
-        for (auto& e : u) {
-            int8_t* dst = reinterpret_cast<int8_t*>(base + e.off);
-            if ((rc = unpack_int4_launch(e.src, dst, e.n, stream)) != IPTQ_OK) return rc;
-            *e.dst = dst;
+        const void* srcs[4];
+        int8_t* dsts[4];
+        int64_t ns[4];
+        for (int i = 0; i < 4; ++i) {
+            srcs[i] = u[i].src;
+            dsts[i] = reinterpret_cast<int8_t*>(base + u[i].off);
+            ns[i] = u[i].n;
+            *u[i].dst = dsts[i];
         }
+        if ((rc = unpack_int4_multi_launch(srcs, dsts, ns, 4, stream)) != IPTQ_OK) return rc;   // one launch for the four matrices
     }
 
     if ((rc = layernorm_launch(x, h1, T, D, p->ln1_gamma, p->ln1_beta, p->ln1_ptf, p->ln1, stream)) != IPTQ_OK) return rc;

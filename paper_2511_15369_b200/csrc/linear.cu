@@ -407,6 +407,71 @@ int unpack_int4_launch(const void* packed, int8_t* out, int64_t n_elems, cudaStr
     return last_launch_status();
 }
 
+// Up to four weight matrices in one launch (the head of a W4 encoder block): 16 packed bytes -> 32 int8 per step.
+// The low nibbles L and high nibbles H of a word are sign-extended byte-wise ((v ^ 8) - 8, with bit 7 set during the
+// subtraction so that no borrow crosses a byte) and interleaved back into element order.
+struct UnpackSegs {
+    const uint4* src[4];
+    uint4* dst[4];
+    int64_t nvec[4];           // 16-byte input vectors per segment
+};
+
+__device__ __forceinline__ unsigned sext_nibbles(unsigned v)
+{
+    return (((v ^ 0x08080808u) | 0x80808080u) - 0x08080808u) ^ 0x80808080u;
+}
+
+__global__ void __launch_bounds__(256) unpack_int4_multi_kernel(const UnpackSegs s)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    grid_dep_launch();
+    grid_dep_wait();                                // the scratch may still be read by the previous kernel
+#pragma unroll 1
+    for (int seg = 0; seg < 4; ++seg) {
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < s.nvec[seg]; i += stride) {
+            const uint4 pk = __ldg(s.src[seg] + i);
+            const unsigned w[4] = {pk.x, pk.y, pk.z, pk.w};
+            unsigned o[8];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const unsigned lo = sext_nibbles(w[k] & 0x0f0f0f0fu), hi = sext_nibbles((w[k] >> 4) & 0x0f0f0f0fu);
+                o[2 * k] = __byte_perm(lo, hi, 0x5140);        // elements 0..3 of the word: l0 h0 l1 h1
+                o[2 * k + 1] = __byte_perm(lo, hi, 0x7362);    // elements 4..7: l2 h2 l3 h3
+            }
+            s.dst[seg][2 * i] = make_uint4(o[0], o[1], o[2], o[3]);
+            s.dst[seg][2 * i + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+        }
+    }
+}
+
+// count <= 4 matrices; falls back to one launch per matrix when a pointer or a size does not allow 16-byte vectors
+int unpack_int4_multi_launch(const void* const* packed, int8_t* const* out, const int64_t* n_elems, int count,
+                             cudaStream_t st)
+{
+    bool vec = count >= 1 && count <= 4;
+    for (int i = 0; vec && i < count; ++i)
+        vec = aligned16(packed[i]) && aligned16(out[i]) && n_elems[i] % 32 == 0;
+    if (!vec) {
+        for (int i = 0; i < count; ++i) {
+            int rc = unpack_int4_launch(packed[i], out[i], n_elems[i], st);
+            if (rc != IPTQ_OK) return rc;
+        }
+        return IPTQ_OK;
+    }
+    UnpackSegs s{};
+    int64_t total = 0;
+    for (int i = 0; i < count; ++i) {
+        s.src[i] = static_cast<const uint4*>(packed[i]);
+        s.dst[i] = reinterpret_cast<uint4*>(out[i]);
+        s.nvec[i] = n_elems[i] / 32;
+        total = std::max(total, s.nvec[i]);
+    }
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((total + 255) / 256, (int64_t)sm_count() * 8));
+    launch_kernel(unpack_int4_multi_kernel, grid, 256, 0, st, s);
+    note_launch();
+    return last_launch_status();
+}
+
 // ---------------------------------------------------------------- launcher
 struct LinearArgs {
     const int8_t* x; const int8_t* w;                          // w already int8 [N, K]
