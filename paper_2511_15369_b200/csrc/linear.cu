@@ -398,7 +398,7 @@ __global__ void unpack_int4_kernel(const uint8_t* __restrict__ packed, int8_t* _
     }
 }
 
-int unpack_int4_launch(const void* packed, int8_t* out, int64_t n_elems, cudaStream_t st)
+static int unpack_int4_bytes_launch(const void* packed, int8_t* out, int64_t n_elems, cudaStream_t st)
 {
     const int64_t nbytes = n_elems / 2;
     const int grid = (int)std::min<int64_t>((nbytes + 255) / 256, (int64_t)sm_count() * 8);
@@ -453,7 +453,7 @@ int unpack_int4_multi_launch(const void* const* packed, int8_t* const* out, cons
         vec = aligned16(packed[i]) && aligned16(out[i]) && n_elems[i] % 32 == 0;
     if (!vec) {
         for (int i = 0; i < count; ++i) {
-            int rc = unpack_int4_launch(packed[i], out[i], n_elems[i], st);
+            int rc = unpack_int4_bytes_launch(packed[i], out[i], n_elems[i], st);
             if (rc != IPTQ_OK) return rc;
         }
         return IPTQ_OK;
@@ -470,6 +470,12 @@ int unpack_int4_multi_launch(const void* const* packed, int8_t* const* out, cons
     launch_kernel(unpack_int4_multi_kernel, grid, 256, 0, st, s);
     note_launch();
     return last_launch_status();
+}
+
+// one matrix: the vector kernel when pointers and size allow it, the byte-wise one otherwise
+int unpack_int4_launch(const void* packed, int8_t* out, int64_t n_elems, cudaStream_t st)
+{
+    return unpack_int4_multi_launch(&packed, &out, &n_elems, 1, st);
 }
 
 // ---------------------------------------------------------------- launcher

@@ -106,6 +106,17 @@ def test_linear_w4(api, orc):
     assert (want == orc.linear(x, w, bias, ma, sa)).all()
 
 
+@pytest.mark.parametrize("n,k", [(1, 34), (3, 30), (16, 64), (40, 48), (96, 1536)])
+def test_unpack_int4(api, n, k):
+    """Every nibble value in every position; sizes that take the 16-byte vector kernel and sizes that fall back to the
+    byte-wise one (the expected values are the definition: low nibble first, two's complement)."""
+    rng = np.random.default_rng(n * k)
+    q = rng.integers(-8, 8, size=(n, k)).astype(np.int8)
+    q.reshape(-1)[:16] = np.arange(-8, 8)
+    got = api.unpack_int4(_cu(synth.pack_int4(q))).cpu().numpy()
+    assert (got == q).all()
+
+
 def test_linear_errors(api):
     import torch
     ws = api.Workspace(256)
