@@ -732,16 +732,15 @@ int iptq_mlp_block(const int8_t* x, const void* w1, const int32_t* b1, const int
     const int8_t* w1_8 = static_cast<const int8_t*>(w1);
     const int8_t* w2_8 = static_cast<const int8_t*>(w2);
     if (w_bits == 4) {
-        int8_t* u1 = reinterpret_cast<int8_t*>(base + off);
-        int rc = unpack_int4_launch(w1, u1, (int64_t)D * Dh, stream);
+        // both matrices in one launch
+        const void* srcs[2] = {w1, w2};
+        int8_t* dsts[2] = {reinterpret_cast<int8_t*>(base + off),
+                           reinterpret_cast<int8_t*>(base + off + align256((size_t)D * (size_t)Dh))};
+        const int64_t ns[2] = {(int64_t)D * Dh, (int64_t)D * Dh};
+        int rc = unpack_int4_multi_launch(srcs, dsts, ns, w2 ? 2 : 1, stream);
         if (rc != IPTQ_OK) return rc;
-        w1_8 = u1;
-        if (w2) {
-            int8_t* u2 = reinterpret_cast<int8_t*>(base + off + align256((size_t)D * (size_t)Dh));
-            rc = unpack_int4_launch(w2, u2, (int64_t)D * Dh, stream);
-            if (rc != IPTQ_OK) return rc;
-            w2_8 = u2;
-        }
+        w1_8 = dsts[0];
+        if (w2) w2_8 = dsts[1];
     }
     // FC1 with the GELU epilogue; without FC2 the activations go straight to y
     LinearArgs fc1{x, w1_8, b1, m1, s1, 0, nullptr, nullptr, gelu, w2 ? hidden : y, M, Dh, D, status};

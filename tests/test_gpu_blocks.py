@@ -106,6 +106,35 @@ def test_linear_w4(api, orc):
     assert (want == orc.linear(x, w, bias, ma, sa)).all()
 
 
+def test_mlp_w4(api, orc):
+    """FC1 + GELU + FC2 with packed 4-bit weights (both matrices unpacked by one launch), with and without FC2."""
+    rng = np.random.default_rng(45)
+    M, D, Dh = 150, 96, 384
+    x = rng.integers(-128, 128, size=(M, D)).astype(np.int8)
+    w1 = rng.integers(-8, 8, size=(Dh, D)).astype(np.int8)
+    w2 = rng.integers(-8, 8, size=(D, Dh)).astype(np.int8)
+    b1 = rng.integers(-500, 500, size=Dh).astype(np.int32)
+    b2 = rng.integers(-500, 500, size=D).astype(np.int32)
+    m1, s1 = api.channel_requant_prepare((2047 / (4 * 74.0 * 4.6 * np.sqrt(D))) * 2.0 ** rng.uniform(-0.3, 0.3, size=Dh))
+    m2, s2 = api.channel_requant_prepare(2.0 ** rng.uniform(-9, -7, size=D))
+    go, ga = orc.gelu_prepare(4.0 / 2047, 12, 0.03, -100, 8, 0), api.gelu_prepare(4.0 / 2047, 12, 0.03, -100, 8, 0)
+    p1, p2 = synth.pack_int4(w1), synth.pack_int4(w2)
+    res = rng.integers(-128, 128, size=(M, D)).astype(np.int8)
+    rro, rra = orc.requant_prepare(0.5 / 65536), api.requant_prepare(0.5 / 65536)
+    ws = api.Workspace(api.mlp_workspace_bytes(M, D, Dh, 4))
+    want_h = orc.mlp_block(x, p1, b1, m1, s1, go, w_bits=4)
+    got_h = api.mlp_block(_cu(x), _cu(p1), _cu(b1), _cu(m1), _cu(s1), ga, ws, w_bits=4).cpu().numpy()
+    ws.check()
+    assert len(np.unique(want_h)) > 30
+    assert (got_h == want_h).all(), _mismatch(got_h, want_h)
+    want = orc.mlp_block(x, p1, b1, m1, s1, go, p2, b2, m2, s2, 1, res, rro, w_bits=4)
+    got = api.mlp_block(_cu(x), _cu(p1), _cu(b1), _cu(m1), _cu(s1), ga, ws, _cu(p2), _cu(b2), _cu(m2), _cu(s2), 1,
+                        _cu(res), rra, w_bits=4).cpu().numpy()
+    ws.check()
+    assert (got == want).all(), _mismatch(got, want)
+    assert (want == orc.mlp_block(x, w1, b1, m1, s1, go, w2, b2, m2, s2, 1, res, rro)).all()
+
+
 @pytest.mark.parametrize("n,k", [(1, 34), (3, 30), (16, 64), (40, 48), (96, 1536)])
 def test_unpack_int4(api, n, k):
     """Every nibble value in every position; sizes that take the 16-byte vector kernel and sizes that fall back to the
