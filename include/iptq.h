@@ -116,20 +116,23 @@ typedef struct {
  * IPTQ_ERR_BITS); 1 <= row_len <= 1024. */
 int iptq_softmax_prepare(double in_scale, int row_len, int out_bits, iptq_softmax_variant variant,
                          iptq_softmax_consts* out /*host*/);
-/* The shift-based exponentials (IPTQ_SM_BITEXP, IPTQ_SM_SHIFTMAX) of Eq. (9) are 0 from some d = max - s on (a
- * few x0) and, where x0 << nsh < 2^16, fit 16 bits, so the whole function is a short table.  iptq_softmax() and
- * the attention kernel build that table per CTA in shared memory; iptq_softmax_table() writes it once to device
- * memory with the same arithmetic -- e(0) .. e(n - 1), then zeros up to the next multiple of 8 entries -- and
- * stores the pointer and n in consts, after which the kernels copy it instead.  Results are identical either way.
- * *consts: host, updated (table = NULL, table_n = 0 and nothing written where this variant or scale has no such
+/* The integer exponential of every variant (Eq. (9) for IPTQ_SM_BITEXP / IPTQ_SM_SHIFTMAX, the second-order
+ * polynomial behind IPTQ_SM_POLY / IPTQ_SM_LOG2) is a function of d = max - s alone, is 0 from some d on (a few
+ * x0) and, where its largest value is below 2^16, fits 16 bits, so the whole function is a short table.
+ * iptq_softmax() and the attention kernels build that table per CTA in shared memory; iptq_softmax_table() writes
+ * it once to device memory with the same arithmetic -- e(0) .. e(n - 1), then zeros up to the next multiple of 8
+ * entries -- and stores the pointer and n in consts, after which the kernels copy it instead.  Results are
+ * identical either way.
+ * *consts: host, updated (table = NULL, table_n = 0 and nothing written where this scale has no such
  * table).  table: dev uint16 [capacity], 16-byte aligned, caller-owned, must outlive every use of consts;
  * IPTQ_ERR_SHAPE when capacity is too small (IPTQ_SOFTMAX_TABLE_MAX entries always suffice: larger tables are
  * not used by the kernels and count as "no table").  Work submitted to the stream after this call sees the
  * complete table. */
 #define IPTQ_SOFTMAX_TABLE_MAX 51200
 int iptq_softmax_table(iptq_softmax_consts* consts, uint16_t* table, int32_t capacity, iptq_stream_t stream);
-/* scores: dev int32 [rows, row_len], |score| < 2^30.  probs: dev uint8 [rows, row_len].
- * bias: nullable dev int32 [bias_period, row_len] at the score scale; row i adds bias row (i % bias_period).
+/* scores: dev int32 [rows, row_len], |score| < 2^30 (with a bias: |score + bias| < 2^30).  probs: dev uint8
+ * [rows, row_len].  bias: nullable dev int32 [bias_period, row_len] at the score scale; row i adds bias row
+ * (i % bias_period).
  * consts: host.  No workspace. */
 int iptq_softmax(const int32_t* scores, uint8_t* probs, int64_t rows, int row_len, const int32_t* bias,
                  int64_t bias_period, const iptq_softmax_consts* consts, iptq_stream_t stream);
@@ -263,18 +266,24 @@ int iptq_linear_w4_static(const int8_t* x, const void* w_packed, const int32_t* 
  * q, k, v: dev int8 [B, H, N, dh] (zero point 0); out: dev int8 [B, N, H*dh];
  * bias: nullable dev int32 [H, N, N] at the score scale; mask_id: nullable dev uint8 [B, N]: the pair
  * (i, j) is masked (probability 0, excluded from max and sum) iff mask_id[b,i] != mask_id[b,j].
- * N <= 256, dh in {32, 64}; sm (host) prepared with row_len = N; out_rq: host.  ws: the status block, followed
- * for N <= 64 by room for a transposed copy of the bias (iptq_attention_workspace_bytes() counts it; with a smaller
- * workspace the call still works and reads the bias as it is, more slowly).
+ * N <= 256, dh in {32, 64}; sm (host) prepared with row_len = N; out_rq: host.  ws: the status block.
  * The real ratio of out_rq is 2^-(out_bits-1) * S_v / S_out.  With IPTQ_SM_LOG2 the probabilities are the powers
  * of two 2^-code and the product is the shift-accumulate sum_j v_j << (15 - code_ij) (codes above 15: nothing),
  * so out_rq's ratio is 2^-15 * S_v / S_out.
+ *
+ * The relative-position bias of a window model is a weight.  For N <= 64 the kernel gives one thread a whole score
+ * row, and reads the bias fastest from a copy laid out as [H][ceil(N/4)][64 rows] x 4 int32 columns (zeros past
+ * column N).  iptq_attention_bias_prepare() writes that copy once, at load time, into caller-owned device memory of
+ * iptq_attention_bias_bytes(H, N) bytes (16-byte aligned; 0 bytes and nothing to do for N > 64); pass it as
+ * bias_t together with bias.  With bias_t == NULL the row-major bias is read as it is (same results, slower).
  */
 size_t iptq_attention_workspace_bytes(int64_t B, int H, int N, int dh);
+size_t iptq_attention_bias_bytes(int H, int N);
+int iptq_attention_bias_prepare(const int32_t* bias, int32_t* bias_t, int H, int N, iptq_stream_t stream);
 int iptq_attention_block(const int8_t* q, const int8_t* k, const int8_t* v, int8_t* out, int64_t B, int H,
-                         int N, int dh, const int32_t* bias, const uint8_t* mask_id,
-                         const iptq_softmax_consts* sm, const iptq_requant* out_rq, void* ws, size_t ws_bytes,
-                         iptq_stream_t stream);
+                         int N, int dh, const int32_t* bias, const int32_t* bias_t /*nullable*/,
+                         const uint8_t* mask_id, const iptq_softmax_consts* sm, const iptq_requant* out_rq,
+                         void* ws, size_t ws_bytes, iptq_stream_t stream);
 
 /* ------------------------------------------------------------------ fused MLP
  * FC1 (INT8 GEMM) with the integer GELU of Sec. 3.3 applied in the int32 epilogue:
@@ -325,6 +334,7 @@ typedef struct {
     const iptq_requant* res2_rq;
     int32_t act_bits;              /* width of the QKV / proj / FC2 outputs: 0 or 8 = int8; 6 with 6-bit LayerNorm, Softmax,
                                       attention and GELU constants is the W6A6 setting of the detection results (Sec. 4) */
+    const int32_t* attn_bias_t;    /* nullable: attn_bias as laid out by iptq_attention_bias_prepare() (N <= 64) */
 } iptq_block_params;
 
 size_t iptq_encoder_block_workspace_bytes(const iptq_block_params* p /*host*/);
@@ -377,8 +387,9 @@ int iptq_metric_layernorm(const int8_t* x, const int8_t* y, int64_t rows, int di
 /* Host part.  iptq_sqnr_db returns +inf for sum_err2 == 0.  iptq_metric_term: op_count is divided by c_unit before
  * N() (the paper gives no unit; raw counts of 1e7 and more would leave N(C) as the only term that matters).
  * iptq_op_count: integer operations of one layer on [rows, row_len] (GELU: rows * row_len elements) counted from
- * this library's integer definitions, one per add / subtract / multiply / shift / compare / divide; returns a
- * negative value for an unknown kind or variant.  iptq_metric_select: index of the largest term, the first of
+ * this library's integer definitions, one per binary add / subtract / multiply / divide / shift / mask and per
+ * comparison (sign flips, copies and prepared constants are free; a value that is the same for a whole row counts
+ * once per row); returns a negative value for an unknown kind or variant.  iptq_metric_select: index of the largest term, the first of
  * equals; -1 for n < 1. */
 typedef enum { IPTQ_LAYER_SOFTMAX = 0, IPTQ_LAYER_GELU = 1, IPTQ_LAYER_LAYERNORM = 2 } iptq_layer_kind;
 double iptq_softplus(double v);

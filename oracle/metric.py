@@ -117,10 +117,15 @@ def affine_deq(y: np.ndarray, out_scale: float, out_zp: int) -> np.ndarray:
 
 # ------------------------------------------------------------------ Eq. (20): operation counts (this library's reading)
 
-_SOFTMAX_PER_ELEM = {0: 21, 1: 17, 2: 15, 3: 22}     # SM_BITEXP, SM_SHIFTMAX, SM_POLY, SM_LOG2
-_GELU_PER_ELEM = {0: 20, 1: 19, 2: 33}        # GELU_POLY4, GELU_POLY2, GELU_SHIFT
-_LN_PER_ELEM = {0: 15, 1: 15, 2: 16}          # LN_SHIFT, LN_NEWTON, LN_PTF (one more shift per element)
-_LN_PER_ROW = {0: 34, 1: 22, 2: 22}           # variance 3, square root (10 fixed steps / about 6 Newton steps, 3 each), reciprocal 1
+# Counted mechanically: one per binary add / subtract / multiply / divide / shift / mask and per comparison (min, max,
+# |.|, sign and leading-one position are one each); sign flips, copies, constants prepared before inference and
+# values that do not change inside a row (counted once per row) are not per-element operations.
+_SOFTMAX_PER_ELEM = {0: 21, 1: 17, 2: 15, 3: 25}     # SM_BITEXP, SM_SHIFTMAX, SM_POLY, SM_LOG2
+_SOFTMAX_PER_ROW = {0: 1, 1: 1, 2: 1, 3: 1}          # the division of Eq. (15); logarithm candidate: twice the row sum
+_GELU_PER_ELEM = {0: 21, 1: 20, 2: 34}               # GELU_POLY4, GELU_POLY2, GELU_SHIFT
+_LN_PER_ELEM = {0: 16, 1: 16, 2: 17}                 # LN_SHIFT, LN_NEWTON, LN_PTF (one more shift per element)
+LN_NEWTON_NOMINAL_STEPS = 5                          # most steps the iterated square root takes on LayerNorm rows of the workload
+_LN_PER_ROW = {0: 38, 1: 28, 2: 28}                  # variance 3, start value 4, steps (10 x 3 / 5 x 4), reciprocal 1
 
 
 def op_count(kind: int, variant: int, rows: int, row_len: int) -> float:
@@ -129,20 +134,20 @@ def op_count(kind: int, variant: int, rows: int, row_len: int) -> float:
     Softmax, per element: running max 1, distance 1, clamp 1, Eq. (7) 4, Eq. (8) 3 (divide, multiply, subtract),
     Phi + x0 6 (Bit-exp; 2 for Shiftmax), Eq. (9) 2, sum 1, Eq. (15) 2; one division per row.  Second-order
     polynomial exponential: max 1, distance 1, clamp 1, octave divide 1, remainder 2, polynomial 3, normalise 2,
-    octave shift 1, sum 1, Eq. (15) 2.  Logarithm candidate: the same exponential and sum (13), round(sum / e) 4,
-    leading-one position 1, rounding bit 3, clamp 1, no division per row.
+    octave shift 1, sum 1, Eq. (15) 2.  Logarithm candidate: the same exponential and sum (13), zero test 1,
+    round(sum / e) 3 (twice the sum once per row), leading-one position 2, rounding bit 5, range test 1.
     GELU, per element: clamp 2, |x| 1, min 1, subtract 1, square 1, shift 1, second square 1 (fourth order only),
-    C - (.) 1, sign 1, + C 1, shift 1, x * G 1, requantise 6 (multiply, round, shift, zero point, two clamps).
-    Shift-based sigmoid form: 1.702 x by shifts 6, |.| and clamp 2, exponential 11, D + e 1, divide 1, select 1,
-    multiply 1, shift 1, x * sigma 1, clamp 2, requantise 6.
+    C - (.) 1, sign 1, times E 1, + C 1, shift 1, x * G 1, requantise 7 (multiply, high word, round, shift, zero
+    point, two clamps).  Shift-based sigmoid form: clamp 2, 1.702 x by shifts 6, |.| and clamp 2, exponential 11,
+    D + e 1, divide 1, select 1, multiply 1, shift 1, x * sigma 1, requantise 7.
     LayerNorm, per element: sum 1, square-and-add 2, D x - sum 2, times reciprocal and shift 2, gamma/beta 2,
-    requantise 6 (the power-of-two-factor variant shifts the input first: 1 more); per row: variance 3, square
-    root steps of 3 operations (divide, add, shift) -- 10 in the fixed-step variant, about 6 when iterated to
-    convergence -- and one reciprocal.
+    requantise 7 (the power-of-two-factor variant shifts the input first: 1 more); per row: variance 3, start
+    value of the square root 4, steps of the recurrence (divide, add, shift: 10 in the fixed-step variant; with
+    the comparison that ends the iteration, 5 steps when iterated to convergence) and one reciprocal.
     """
     n = float(rows) * float(row_len)
     if kind == SOFTMAX:
-        return _SOFTMAX_PER_ELEM[variant] * n + (0.0 if variant == 3 else float(rows))
+        return _SOFTMAX_PER_ELEM[variant] * n + _SOFTMAX_PER_ROW[variant] * float(rows)
     if kind == GELU:
         return _GELU_PER_ELEM[variant] * n
     if kind == LAYERNORM:

@@ -69,6 +69,7 @@ class BlockParams(C.Structure):
         ("fc2_zp", C.c_int32),
         ("res2_rq", C.c_void_p),
         ("act_bits", C.c_int32),
+        ("attn_bias_t", C.c_void_p),
     ]
 
 
@@ -123,7 +124,10 @@ def lib():
         L.iptq_patchify.argtypes = [_vp, _vp, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, _vp]
         L.iptq_attention_workspace_bytes.restype = C.c_size_t
         L.iptq_attention_workspace_bytes.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
-        L.iptq_attention_block.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, C.c_int, C.c_int, C.c_int, _vp, _vp,
+        L.iptq_attention_bias_bytes.restype = C.c_size_t
+        L.iptq_attention_bias_bytes.argtypes = [C.c_int, C.c_int]
+        L.iptq_attention_bias_prepare.argtypes = [_vp, _vp, C.c_int, C.c_int, _vp]
+        L.iptq_attention_block.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, C.c_int, C.c_int, C.c_int, _vp, _vp, _vp,
                                            C.POINTER(SoftmaxConsts), C.POINTER(Requant), _vp, C.c_size_t, _vp]
         L.iptq_mlp_workspace_bytes.restype = C.c_size_t
         L.iptq_mlp_workspace_bytes.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
@@ -156,7 +160,7 @@ def exported_symbols():
     """Names declared in include/iptq.h (used by the CPU-side load test)."""
     return ["iptq_requant_prepare", "iptq_channel_requant_prepare", "iptq_softmax_prepare", "iptq_softmax", "iptq_softmax_table",
             "iptq_gelu_prepare", "iptq_gelu", "iptq_gelu_table", "iptq_gelu_fit", "iptq_gelu_prepare_coeffs", "iptq_layernorm_prepare", "iptq_layernorm",
-            "iptq_unpack_int4", "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_bits", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_patchify", "iptq_attention_workspace_bytes", "iptq_attention_block",
+            "iptq_unpack_int4", "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_bits", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_patchify", "iptq_attention_workspace_bytes", "iptq_attention_bias_bytes", "iptq_attention_bias_prepare", "iptq_attention_block",
             "iptq_mlp_workspace_bytes", "iptq_mlp_block", "iptq_encoder_block_workspace_bytes",
             "iptq_encoder_block", "iptq_encoder_block_profiled", "iptq_workspace_init", "iptq_check", "iptq_strerror", "iptq_launch_count",
             "iptq_metric_softmax", "iptq_metric_gelu", "iptq_metric_layernorm", "iptq_softplus", "iptq_sqnr_db",
@@ -443,12 +447,25 @@ def attention_workspace_bytes(B, H, N, dh):
     return int(lib().iptq_attention_workspace_bytes(B, H, N, dh))
 
 
-def attention_block(q, k, v, sm: SoftmaxConsts, out_rq: Requant, ws: Workspace, bias=None, mask_id=None, out=None):
+def attention_bias_prepare(bias):
+    """The relative-position bias [H, N, N] (N <= 64) in the layout the window kernel reads fastest, written once at
+    load time; returns the device tensor to pass as ``bias_t`` (None for N > 64, where there is no such layout)."""
+    H, N, _ = bias.shape
+    nbytes = int(lib().iptq_attention_bias_bytes(H, N))
+    if nbytes == 0:
+        return None
+    t = torch.empty(nbytes // 4, dtype=torch.int32, device=bias.device)
+    _chk(lib().iptq_attention_bias_prepare(_dp(bias), _dp(t), H, N, _stream()), "iptq_attention_bias_prepare")
+    return t
+
+
+def attention_block(q, k, v, sm: SoftmaxConsts, out_rq: Requant, ws: Workspace, bias=None, mask_id=None, out=None,
+                    bias_t=None):
     B, H, N, dh = q.shape
     if out is None:
         out = torch.empty((B, N, H * dh), dtype=torch.int8, device=q.device)
-    _chk(lib().iptq_attention_block(_dp(q), _dp(k), _dp(v), _dp(out), B, H, N, dh, _dp(bias), _dp(mask_id),
-                                    C.byref(sm), C.byref(out_rq), ws.ptr, ws.nbytes, _stream()),
+    _chk(lib().iptq_attention_block(_dp(q), _dp(k), _dp(v), _dp(out), B, H, N, dh, _dp(bias), _dp(bias_t),
+                                    _dp(mask_id), C.byref(sm), C.byref(out_rq), ws.ptr, ws.nbytes, _stream()),
          "iptq_attention_block")
     return out
 
@@ -516,6 +533,11 @@ class EncoderBlock:
             setattr(p, "m_" + name, dev(m))
             setattr(p, "s_" + name, dev(s))
         p.attn_bias = dev(spec.attn_bias)
+        if spec.attn_bias is not None:
+            bt = attention_bias_prepare(self.keep[-1])      # a weight: laid out once, here
+            if bt is not None:
+                self.keep.append(bt)
+                p.attn_bias_t = bt.data_ptr()
         p.mask_id = dev(spec.mask_id)
         # the logarithm candidate writes 4-bit codes and its P V product is at scale 2^-15 instead of 2^-7
         log2 = sm_v == SM_LOG2

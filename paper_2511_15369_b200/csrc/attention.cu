@@ -1,6 +1,7 @@
 // Host side of the fused integer attention: argument checks, tile geometry, tensor maps, dispatch to the
 // per-variant kernel files.
 #include "attention_window.cuh"
+#include "iptq_internal.cuh"
 
 namespace iptq {
 
@@ -21,21 +22,8 @@ int window_launch_variant2(int dh, const CUtensorMap& mq, const CUtensorMap& mk,
 int window_launch_variant3(int dh, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                            const AttnParams& p, int smem_bytes, cudaStream_t st);
 
-// ---------------------------------------------------------------- launcher (strided q/k/v so that the encoder
-// block can read heads straight out of the fused QKV activation)
-struct AttnArgs {
-    const int8_t *q, *k, *v;
-    int64_t tok_stride, head_stride, batch_stride;     // in bytes (= elements)
-    int8_t* out;
-    int64_t B; int H, N, dh;
-    const int32_t* bias; const uint8_t* mask_id;
-    const iptq_softmax_consts* sm; const iptq_requant* out_rq;
-    StatusBlock* status;
-    int32_t* bias_t;       // 16-byte aligned scratch of attention_bias_t_bytes(H, N) for the window kernel's copy of the bias, or null
-};
-
 // Bytes of the re-laid-out bias the window kernel (N <= 64) reads: [H][ceil(N/4) column quads][64 rows] x 4 int32.
-size_t attention_bias_t_bytes(int H, int N) { return N <= 64 ? (size_t)H * (size_t)((N + 3) / 4) * 64 * 16 : 0; }
+static size_t attention_bias_t_bytes(int H, int N) { return N <= 64 ? (size_t)H * (size_t)((N + 3) / 4) * 64 * 16 : 0; }
 
 // out[h][c4][r] = bias[h][r][4 c4 .. 4 c4 + 3] (0 past column N): one 16-byte load gives a thread four columns of
 // its row, and the 32 rows of a warp are 512 contiguous bytes.
@@ -43,7 +31,7 @@ __global__ void __launch_bounds__(256)
 bias_relayout_kernel(const int32_t* __restrict__ bias, int4* __restrict__ out, int H, int N)
 {
     grid_dep_launch();
-    grid_dep_wait();                                   // an earlier attention launch may still be reading `out`
+    grid_dep_wait();
     const int C4 = (N + 3) / 4;
     const int total = H * C4 * N;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
@@ -74,7 +62,8 @@ static int launch_attn_v(bool window, int dh, int variant, const CUtensorMap& mq
     }
 }
 
-int attention_launch(const AttnArgs& a, cudaStream_t st)
+// Host-side argument checks alone: nothing is enqueued.
+static int attention_check(const AttnArgs& a)
 {
     if (!a.sm || !a.out_rq) return IPTQ_ERR_NULL;
     if (a.B < 0 || a.B > (1 << 24) || a.H < 1 || a.H > 1024 || a.N < 1 || a.N > 256) return IPTQ_ERR_SHAPE;
@@ -88,10 +77,17 @@ int attention_launch(const AttnArgs& a, cudaStream_t st)
     if (a.B == 0) return IPTQ_OK;
     if (!a.q || !a.k || !a.v || !a.out) return IPTQ_ERR_NULL;
     if (!aligned16(a.q) || !aligned16(a.k) || !aligned16(a.v) || !aligned16(a.out) ||
-        (a.bias && (reinterpret_cast<uintptr_t>(a.bias) & 3u)) || (a.tok_stride & 15) || (a.head_stride & 15) ||
-        (a.batch_stride & 15))
+        (a.bias && (reinterpret_cast<uintptr_t>(a.bias) & 3u)) || (a.bias_t && !aligned16(a.bias_t)) ||
+        (a.tok_stride & 15) || (a.head_stride & 15) || (a.batch_stride & 15))
         return IPTQ_ERR_ALIGN;
     if (a.B * a.H * ((a.N + 127) / 128) > (int64_t)1 << 30) return IPTQ_ERR_SHAPE;
+    return IPTQ_OK;
+}
+
+int attention_launch(const AttnArgs& a, cudaStream_t st)
+{
+    int rc = attention_check(a);
+    if (rc != IPTQ_OK || a.B == 0) return rc;
 
     AttnParams p;
     p.B = (int)a.B; p.H = a.H; p.N = a.N; p.dh = a.dh;
@@ -156,14 +152,7 @@ int attention_launch(const AttnArgs& a, cudaStream_t st)
     }
     p.lut_src = (p.lut_n && a.sm->table && a.sm->table_n == p.lut_n) ? a.sm->table : nullptr;
     p.bias = a.bias; p.mask_id = a.mask_id; p.out = a.out;
-    p.bias_q = nullptr;
-    if (window && a.bias && a.bias_t) {
-        const int total = a.H * ((a.N + 3) / 4) * a.N;
-        launch_kernel(bias_relayout_kernel, std::min((total + 255) / 256, 4 * sm_count()), 256, 0, st, a.bias,
-                      reinterpret_cast<int4*>(a.bias_t), a.H, a.N);
-        note_launch();
-        p.bias_q = reinterpret_cast<const int4*>(a.bias_t);
-    }
+    p.bias_q = (window && a.bias && a.bias_t) ? reinterpret_cast<const int4*>(a.bias_t) : nullptr;
     p.ex = to_dev_exp(*a.sm);
     p.M = a.sm->M; p.f_shl = a.sm->f_shl; p.p_shr = a.sm->p_shr;
     p.orq = to_dev(*a.out_rq);
@@ -188,22 +177,30 @@ using namespace iptq;
 
 extern "C" {
 
-size_t iptq_attention_workspace_bytes(int64_t, int H, int N, int)
+size_t iptq_attention_workspace_bytes(int64_t, int, int, int) { return kStatusBytes; }
+
+size_t iptq_attention_bias_bytes(int H, int N) { return (H < 1 || N < 1) ? 0 : attention_bias_t_bytes(H, N); }
+
+int iptq_attention_bias_prepare(const int32_t* bias, int32_t* bias_t, int H, int N, iptq_stream_t stream)
 {
-    return kStatusBytes + ((attention_bias_t_bytes(H, N) + 255) & ~size_t(255));
+    if (H < 1 || H > 1024 || N < 1 || N > 256) return IPTQ_ERR_SHAPE;
+    if (attention_bias_t_bytes(H, N) == 0) return IPTQ_OK;          // N > 64: the row-major bias is what the kernel reads
+    if (!bias || !bias_t) return IPTQ_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(bias) & 3u) || !aligned16(bias_t)) return IPTQ_ERR_ALIGN;
+    const int total = H * ((N + 3) / 4) * N;
+    launch_kernel(bias_relayout_kernel, std::min((total + 255) / 256, 4 * sm_count()), 256, 0, stream, bias,
+                  reinterpret_cast<int4*>(bias_t), H, N);
+    note_launch();
+    return last_launch_status();
 }
 
 int iptq_attention_block(const int8_t* q, const int8_t* k, const int8_t* v, int8_t* out, int64_t B, int H,
-                         int N, int dh, const int32_t* bias, const uint8_t* mask_id,
+                         int N, int dh, const int32_t* bias, const int32_t* bias_t, const uint8_t* mask_id,
                          const iptq_softmax_consts* sm, const iptq_requant* out_rq, void* ws, size_t ws_bytes,
                          iptq_stream_t stream)
 {
     if (!ws || ws_bytes < kStatusBytes) return IPTQ_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(ws) & 255u) return IPTQ_ERR_ALIGN;
-    // the transposed-bias scratch sits behind the status block when the workspace has room for it
-    int32_t* bias_t = nullptr;
-    if (bias && N >= 1 && N <= 64 && H >= 1 && ws_bytes >= kStatusBytes + attention_bias_t_bytes(H, N))
-        bias_t = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + kStatusBytes);
     AttnArgs a{q, k, v, (int64_t)dh, (int64_t)N * dh, (int64_t)H * N * dh, out, B, H, N, dh, bias, mask_id, sm, out_rq,
                static_cast<StatusBlock*>(ws), bias_t};
     return attention_launch(a, stream);

@@ -28,7 +28,6 @@ namespace iptq {
 constexpr int ATT_THREADS = 576;
 constexpr int ATT_SOFTMAX_THREADS = 512;
 constexpr int ATT_STAGES = 3;              // upper bound of the Q/K/V ring depth
-constexpr int kPadScore = -(1 << 30);     // a score this low has exponential 0 for every row maximum below 2^30
 
 struct AttnParams {
     int B, H, N, dh;
@@ -307,7 +306,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             mbar_arrive(s_empty);                              // the MMA warp may overwrite S with the next item's scores
             if (warp_rows) {
                 // ---- row maximum over the real, unmasked columns (Eq. (6)); padding and masked pairs become
-                //      kPadScore, a bias is added in place, so that the next step needs no case analysis
+                //      kNoScore, a bias is added in place, so that the next step needs no case analysis
                 int mx = INT_MIN;
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
@@ -321,7 +320,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                                 bool use = col < p.N;
                                 if (HAS_BIAS && use) sc += __ldg(brow + col);
                                 if (HAS_MASK && use) use = (mrow[col] == my_id);
-                                v[i][j] = (uint32_t)(use ? sc : kPadScore);
+                                v[i][j] = (uint32_t)(use ? sc : kNoScore);
                             }
                         }
 #pragma unroll
@@ -340,10 +339,10 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                         for (int j = 0; j < 16; ++j) {
                             unsigned e;
                             if (USE_LUT) {
-                                const unsigned d = min((unsigned)(mx - (int)v[i][j]), (unsigned)p.lut_n);
+                                const unsigned d = min((unsigned)mx - v[i][j], (unsigned)p.lut_n);
                                 asm volatile("ld.shared.u16 %0, [%1];" : "=r"(e) : "r"(lut_addr + 2u * d));
                             } else {
-                                e = exp_core_nd<VARIANT>((int)v[i][j] - mx, p.ex);
+                                e = exp_core_nd<VARIANT>(exp_distance(mx, (int)v[i][j]), p.ex);
                             }
                             sum += e;
                             v[i][j] = e;

@@ -253,7 +253,7 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
             const unsigned id_0 = __shfl_sync(0xffffffffu, id_lo, 0);
             const bool mixed = HAS_MASK && !__all_sync(0xffffffffu, (lane >= p.N || id_lo == id_0) && (lane + 32 >= p.N || id_hi == id_0));
             if (warp_rows) {
-                // ---- row maximum over the real, unmasked columns (Eq. (6)); padding and masked pairs become kPadScore
+                // ---- row maximum over the real, unmasked columns (Eq. (6)); padding and masked pairs become kNoScore
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     if (i < nch) {
@@ -284,11 +284,11 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
                             for (int j = 0; j < 16; ++j) {
                                 const int col = c0 + j;                   // compile-time after unrolling: i and j are
                                 const unsigned id = __shfl_sync(0xffffffffu, col < 32 ? id_lo : id_hi, col & 31);
-                                v[i][j] = id == my_id ? v[i][j] : (uint32_t)kPadScore;
+                                v[i][j] = id == my_id ? v[i][j] : (uint32_t)kNoScore;
                             }
                         } else if (c0 + 16 > p.N) {
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) v[i][j] = c0 + j < p.N ? v[i][j] : (uint32_t)kPadScore;
+                            for (int j = 0; j < 16; ++j) v[i][j] = c0 + j < p.N ? v[i][j] : (uint32_t)kNoScore;
                         }
 #pragma unroll
                         for (int j = 0; j < 16; ++j) mx = max(mx, (int)v[i][j]);
@@ -303,10 +303,10 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
                         for (int j = 0; j < 16; ++j) {
                             unsigned e;
                             if (USE_LUT) {
-                                const unsigned d = min((unsigned)(mx - (int)v[i][j]), (unsigned)p.lut_n);
+                                const unsigned d = min((unsigned)mx - v[i][j], (unsigned)p.lut_n);
                                 asm volatile("ld.shared.u16 %0, [%1];" : "=r"(e) : "r"(lut_addr + 2u * d));
                             } else {
-                                e = exp_core_nd<VARIANT>((int)v[i][j] - mx, p.ex);
+                                e = exp_core_nd<VARIANT>(exp_distance(mx, (int)v[i][j]), p.ex);
                             }
                             sum += e;
                             v[i][j] = e;

@@ -2,44 +2,14 @@
 // LN1 -> QKV GEMM -> fused attention (reads heads straight out of the QKV activation) -> proj GEMM
 // (+ residual) -> LN2 -> FC1 GEMM with GELU epilogue -> FC2 GEMM (+ residual).  Each layer runs the
 // approximation variant its constants name (the per-layer table of Sec. 3.2).
-#include "tc_common.cuh"
+#include "iptq_internal.cuh"
 
 namespace iptq {
-
-struct LinearArgs {
-    const int8_t* x; const int8_t* w;
-    const int32_t* bias; const int32_t* mult; const int8_t* shift;
-    int32_t out_zp;
-    const int8_t* residual; const iptq_requant* residual_rq;
-    const iptq_gelu_consts* gelu;
-    int8_t* y;
-    int64_t M; int N, K;
-    StatusBlock* status;
-    int out_bits = 8;                                          // width of the output activations (plain and residual epilogues)
-};
-int linear_launch(const LinearArgs& a, cudaStream_t st);
-int unpack_int4_launch(const void* packed, int8_t* out, int64_t n_elems, cudaStream_t st);
-int unpack_int4_multi_launch(const void* const* packed, int8_t* const* out, const int64_t* n_elems, int count,
-                             cudaStream_t st);
-int layernorm_launch(const int8_t* x, int8_t* y, int64_t rows, int dim, const int32_t* gq, const int32_t* bq,
-                     const uint8_t* ptf, const iptq_ln_consts* consts, cudaStream_t st);
-struct AttnArgs {
-    const int8_t *q, *k, *v;
-    int64_t tok_stride, head_stride, batch_stride;
-    int8_t* out;
-    int64_t B; int H, N, dh;
-    const int32_t* bias; const uint8_t* mask_id;
-    const iptq_softmax_consts* sm; const iptq_requant* out_rq;
-    StatusBlock* status;
-    int32_t* bias_t;       // 16-byte aligned scratch of attention_bias_t_bytes(H, N) for the window kernel's copy of the bias, or null
-};
-int attention_launch(const AttnArgs& a, cudaStream_t st);
-size_t attention_bias_t_bytes(int H, int N);
 
 static size_t a256(size_t v) { return (v + 255) & ~size_t(255); }
 
 struct BlockLayout {
-    size_t h1, qkv, att, x1, h2, hid, w_qkv, w_proj, w_fc1, w_fc2, bias_t, total;
+    size_t h1, qkv, att, x1, h2, hid, w_qkv, w_proj, w_fc1, w_fc2, total;
 };
 
 static BlockLayout block_layout(const iptq_block_params* p)
@@ -61,8 +31,6 @@ static BlockLayout block_layout(const iptq_block_params* p)
         l.w_fc1 = take(Dh * D);
         l.w_fc2 = take(D * Dh);
     }
-    l.bias_t = 0;
-    if (p->attn_bias && attention_bias_t_bytes(p->H, p->N)) l.bias_t = take(attention_bias_t_bytes(p->H, p->N));
     l.total = off;
     return l;
 }
@@ -148,8 +116,7 @@ static int encoder_block_run(const int8_t* x, int8_t* y, const iptq_block_params
     if ((rc = mark()) != IPTQ_OK) return rc;
     // a row of qkv is [q | k | v]; head h occupies columns h*dh .. of each third
     AttnArgs aa{qkv, qkv + D, qkv + 2 * D, (int64_t)3 * D, (int64_t)p->dh, (int64_t)p->N * 3 * D, att, p->B, p->H, p->N,
-                p->dh, p->attn_bias, p->mask_id, p->sm, p->pv_rq, status,
-                l.bias_t ? reinterpret_cast<int32_t*>(base + l.bias_t) : nullptr};
+                p->dh, p->attn_bias, p->mask_id, p->sm, p->pv_rq, status, p->attn_bias_t};
     if ((rc = attention_launch(aa, stream)) != IPTQ_OK) return rc;
     if ((rc = mark()) != IPTQ_OK) return rc;
     LinearArgs lp{att, wp, p->b_proj, p->m_proj, p->s_proj, p->proj_zp, x, p->res1_rq, nullptr, x1, T, D, D, status, ab};

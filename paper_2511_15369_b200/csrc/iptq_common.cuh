@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <limits.h>
 #include <stdint.h>
 
 #include "iptq.h"
@@ -161,12 +162,32 @@ __device__ __forceinline__ unsigned exp_core(unsigned d, const ExpDev& c)
     return exp_core_nd<VARIANT>(-(int)d, c);
 }
 
-// Length of the exponential table for the shift-based variants: e(d) = 0 once the octave count q of Eq. (8)
-// reaches qz, the bit length of the largest value x0 << nsh; -Q_p >= 23 (d >> 4) puts that at
-// d >= 16 qz x0 / 23 + 15.  Returns 0 where no 16-bit table exists (polynomial variant, values of 2^16 and more).
+// Scores that take no part in a row (columns past the row end, masked pairs) carry this value.  The distance to the
+// row maximum is formed in unsigned arithmetic, mx - kNoScore >= 2^30 for every admissible maximum (|score| < 2^30),
+// and clamped (exp_distance below, or at the table length), so that such a column gets the exponential 0 whatever
+// the row holds -- also when every real score of the row is close to -2^30.
+constexpr int kNoScore = INT_MIN;
+// -(max - s) for the evaluated exponential: exact for real scores (the distance is below 2^31), -(2^31 - 1) for
+// kNoScore, where every variant of exp_core_nd returns 0.
+__host__ __device__ __forceinline__ int exp_distance(int mx, int s)
+{
+    const unsigned d = (unsigned)mx - (unsigned)s;
+    return -(int)(d < 0x7fffffffu ? d : 0x7fffffffu);
+}
+
+// Length of the exponential table: e(d) = 0 for every d >= the value returned; 0 where no 16-bit table exists.
+// Shift-based variants: e vanishes once the octave count q of Eq. (8) reaches qz, the bit length of the largest
+// value x0 << nsh; -Q_p >= 23 (d >> 4) puts that at d >= 16 qz x0 / 23 + 15.  Polynomial exponential (also behind
+// the logarithm candidate): the value at p = 0 is normalised to 14 bits and is the largest, so e vanishes from
+// octave 14 on, d >= 14 qln2.
 inline int exp_table_entries(const iptq_softmax_consts& sm)
 {
-    if (sm.variant == IPTQ_SM_POLY || sm.variant == IPTQ_SM_LOG2) return 0;
+    if (sm.variant == IPTQ_SM_POLY || sm.variant == IPTQ_SM_LOG2) {
+        const int64_t top = (((int64_t)sm.qb * sm.qb + sm.qc) << sm.norm_l) >> sm.norm_r;
+        if (top >= (1 << 14) || sm.qln2 < 1) return 0;
+        const int64_t n = 14 * (int64_t)sm.qln2 + 8;
+        return n > (1 << 20) ? 0 : (int)n;
+    }
     int qz = 0;
     for (int64_t u = (int64_t)sm.x0 << sm.nsh; u; u >>= 1) ++qz;
     if (qz > 16) return 0;

@@ -14,6 +14,7 @@
 #include <mutex>
 
 #include "tc_common.cuh"
+#include "iptq_internal.cuh"
 
 namespace iptq {
 
@@ -479,18 +480,6 @@ int unpack_int4_launch(const void* packed, int8_t* out, int64_t n_elems, cudaStr
 }
 
 // ---------------------------------------------------------------- launcher
-struct LinearArgs {
-    const int8_t* x; const int8_t* w;                          // w already int8 [N, K]
-    const int32_t* bias; const int32_t* mult; const int8_t* shift;
-    int32_t out_zp;
-    const int8_t* residual; const iptq_requant* residual_rq;
-    const iptq_gelu_consts* gelu;                              // non-null: FC1 + GELU epilogue
-    int8_t* y;
-    int64_t M; int N, K;
-    StatusBlock* status;
-    int out_bits = 8;                                          // width of the output activations (plain and residual epilogues)
-};
-
 template <int BN, int EPI, int GV, bool SAT8, bool GTAB = false>
 static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& my, const CUtensorMap& mr,
                        const GemmParams& p, cudaStream_t st)
@@ -521,7 +510,7 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUten
 template <int BN>
 static int linear_launch_bn(const LinearArgs& a, cudaStream_t st);
 
-int linear_launch(const LinearArgs& a, cudaStream_t st)
+int linear_check(const LinearArgs& a)
 {
     if (!a.x || !a.w || !a.mult || !a.shift || !a.y) return IPTQ_ERR_NULL;
     if (a.M < 0 || a.M > (int64_t)1 << 30 || a.N < 16 || a.K < 16 || a.K > 4096 || (a.N & 15) || (a.K & 15))
@@ -534,9 +523,17 @@ int linear_launch(const LinearArgs& a, cudaStream_t st)
         if (a.gelu->in_bits < 8 || a.gelu->in_bits > 16) return IPTQ_ERR_BITS;
         if (a.gelu->variant < 0 || a.gelu->variant > 2) return IPTQ_ERR_VARIANT;
         int rc = check_requant(&a.gelu->out); if (rc != IPTQ_OK) return rc;
+        if (a.gelu->table && !aligned16(a.gelu->table)) return IPTQ_ERR_ALIGN;
     }
     if (a.out_bits < 4 || a.out_bits > 8) return IPTQ_ERR_BITS;
     if (!a.status) return IPTQ_ERR_WORKSPACE;
+    return IPTQ_OK;
+}
+
+int linear_launch(const LinearArgs& a, cudaStream_t st)
+{
+    const int rc0 = linear_check(a);
+    if (rc0 != IPTQ_OK) return rc0;
     if (a.M == 0) return IPTQ_OK;
     // 128-wide tiles use the tensor core fully and re-read the activations less often, but rebuild the rounding
     // constant per output (two more instructions); measured, they win for the plain epilogue and for the tabulated
@@ -668,16 +665,15 @@ int iptq_linear_bits(const int8_t* x, const void* w, int w_bits, const int32_t* 
     if (N < 1 || K < 1) return IPTQ_ERR_SHAPE;
     if (ws_bytes < iptq_linear_workspace_bytes(M, N, K, w_bits)) return IPTQ_ERR_WORKSPACE;
     if (!w) return IPTQ_ERR_NULL;
-    const int8_t* w8 = static_cast<const int8_t*>(w);
-    if (w_bits == 4) {
-        if (K & 1) return IPTQ_ERR_SHAPE;
-        int8_t* scratch = static_cast<int8_t*>(ws) + kStatusBytes;
-        int rc = unpack_int4_launch(w, scratch, (int64_t)N * K, stream);
-        if (rc != IPTQ_OK) return rc;
-        w8 = scratch;
-    }
+    // every argument is checked before the first launch (the unpack kernel included)
+    const int8_t* w8 = w_bits == 4 ? static_cast<const int8_t*>(ws) + kStatusBytes : static_cast<const int8_t*>(w);
     LinearArgs a{x, w8, bias, mult, shift, out_zp, residual, residual_rq, nullptr, y, M, N, K,
                  static_cast<StatusBlock*>(ws), out_bits};
+    int rc = linear_check(a);
+    if (rc != IPTQ_OK) return rc;
+    if (w_bits == 4) {
+        if (M > 0 && (rc = unpack_int4_launch(w, const_cast<int8_t*>(w8), (int64_t)N * K, stream)) != IPTQ_OK) return rc;
+    }
     return linear_launch(a, stream);
 }
 
@@ -693,15 +689,14 @@ int iptq_linear_w4_static(const int8_t* x, const void* w_packed, const int32_t* 
     uint8_t* base = nullptr;
     int rc = static_scratch_ptr(&base);            // first call on this device: looks the array's address up
     if (rc != IPTQ_OK) return rc;
-    StatusBlock* st = static_cast<StatusBlock*>(status);
-    if (!st) {
-        // the built-in status block keeps the previous call's contents: it must start at zero
-        st = reinterpret_cast<StatusBlock*>(base);
-        if (cudaMemsetAsync(st, 0, kStatusBytes, stream) != cudaSuccess) return IPTQ_ERR_CUDA;
-    }
+    StatusBlock* st = status ? static_cast<StatusBlock*>(status) : reinterpret_cast<StatusBlock*>(base);
     int8_t* w8 = reinterpret_cast<int8_t*>(base + kStatusBytes);
-    if ((rc = unpack_int4_launch(w_packed, w8, (int64_t)N * K, stream)) != IPTQ_OK) return rc;
     LinearArgs a{x, w8, bias, mult, shift, out_zp, residual, residual_rq, nullptr, y, M, N, K, st};
+    if ((rc = linear_check(a)) != IPTQ_OK) return rc;          // nothing is enqueued for a call that is rejected
+    if (M == 0) return IPTQ_OK;
+    // the built-in status block keeps the previous call's contents: it must start at zero
+    if (!status && cudaMemsetAsync(st, 0, kStatusBytes, stream) != cudaSuccess) return IPTQ_ERR_CUDA;
+    if ((rc = unpack_int4_launch(w_packed, w8, (int64_t)N * K, stream)) != IPTQ_OK) return rc;
     return linear_launch(a, stream);
 }
 
@@ -731,22 +726,26 @@ int iptq_mlp_block(const int8_t* x, const void* w1, const int32_t* b1, const int
     size_t off = kStatusBytes + align256((size_t)M * (size_t)Dh);
     const int8_t* w1_8 = static_cast<const int8_t*>(w1);
     const int8_t* w2_8 = static_cast<const int8_t*>(w2);
+    int8_t* dsts[2] = {reinterpret_cast<int8_t*>(base + off),
+                       reinterpret_cast<int8_t*>(base + off + align256((size_t)D * (size_t)Dh))};
     if (w_bits == 4) {
-        // both matrices in one launch
-        const void* srcs[2] = {w1, w2};
-        int8_t* dsts[2] = {reinterpret_cast<int8_t*>(base + off),
-                           reinterpret_cast<int8_t*>(base + off + align256((size_t)D * (size_t)Dh))};
-        const int64_t ns[2] = {(int64_t)D * Dh, (int64_t)D * Dh};
-        int rc = unpack_int4_multi_launch(srcs, dsts, ns, w2 ? 2 : 1, stream);
-        if (rc != IPTQ_OK) return rc;
         w1_8 = dsts[0];
         if (w2) w2_8 = dsts[1];
     }
     // FC1 with the GELU epilogue; without FC2 the activations go straight to y
     LinearArgs fc1{x, w1_8, b1, m1, s1, 0, nullptr, nullptr, gelu, w2 ? hidden : y, M, Dh, D, status};
-    int rc = linear_launch(fc1, stream);
-    if (rc != IPTQ_OK || !w2) return rc;
     LinearArgs fc2{hidden, w2_8, b2, m2, s2, out_zp, residual, residual_rq, nullptr, y, M, D, Dh, status};
+    // every argument of both layers is checked before the first launch (the unpack kernel included)
+    int rc = linear_check(fc1);
+    if (rc == IPTQ_OK && w2) rc = linear_check(fc2);
+    if (rc != IPTQ_OK) return rc;
+    if (w_bits == 4) {
+        const void* srcs[2] = {w1, w2};
+        const int64_t ns[2] = {(int64_t)D * Dh, (int64_t)D * Dh};
+        if (M > 0 && (rc = unpack_int4_multi_launch(srcs, dsts, ns, w2 ? 2 : 1, stream)) != IPTQ_OK) return rc;   // both matrices in one launch
+    }
+    rc = linear_launch(fc1, stream);
+    if (rc != IPTQ_OK || !w2) return rc;
     return linear_launch(fc2, stream);
 }
 

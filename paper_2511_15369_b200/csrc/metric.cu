@@ -229,31 +229,34 @@ double iptq_metric_term(double sqnr_db, double perturbation, double op_count, do
     return 3.0 / (inv_nq + iptq_softplus(perturbation) + iptq_softplus(op_count / c_unit));
 }
 
-// Operations per element / per row of the integer definitions in this library (one per add, subtract, multiply,
-// shift, compare, divide).  Softmax: max, distance, clamp (3), Eq. (7) (4), Eq. (8) (3), Phi and + x0 (6; Shiftmax
-// 2), Eq. (9) (2), sum (1), Eq. (15) (2), one division per row; the polynomial exponential has 15.  GELU: clamp
-// (2), |x|, min, subtract (3), two squares and a shift (3; second order 2), C - (.), sign, + C (3), shift and
-// x * G (2), requantisation (6, also the LayerNorm's); the shift-based sigmoid form has 33.  LayerNorm: sums (3),
-// D x - sum (2), reciprocal multiply and shift (2), gamma and beta (2), requantisation (6), one more shift with
-// power-of-two factors; per row the variance (3), 3 operations per square-root step (10 fixed steps, about 6 when
-// iterated to convergence) and the reciprocal (1).
+// Operations per element / per row of the integer definitions in this library: one per binary add, subtract,
+// multiply, divide, shift or mask and per comparison (min, max, |.|, sign and leading-one position count as one);
+// sign flips, copies, constants prepared before inference and values that are the same for a whole row are not
+// per-element operations.  Softmax: max, distance, clamp (3), Eq. (7) (4), Eq. (8) (3), Phi and + x0 (6; Shiftmax
+// 2), Eq. (9) (2), sum (1), Eq. (15) (2), one division per row; the polynomial exponential has 15, the logarithm
+// candidate 13 for exponential and sum plus 12 for the rounded ratio and its rounded logarithm.  GELU: clamp (2),
+// |x|, min, subtract (3), two squares and a shift (3; second order 2), C - (.), sign, times, + C (4), shift and
+// x * G (2), requantisation (7: multiply, high word, round, shift, zero point, two clamps; also the LayerNorm's);
+// the shift-based sigmoid form has 34.  LayerNorm: sums (3), D x - sum (2), reciprocal multiply and shift (2),
+// gamma and beta (2), requantisation (7), one more shift with power-of-two factors; per row the variance (3), the
+// start value of the square root (4), its steps (10 fixed steps of 3 operations; 5 steps of 4 when iterated to
+// convergence, the most the rows of the workloads need) and the reciprocal (1).
 double iptq_op_count(int layer_kind, int variant, int64_t rows, int row_len)
 {
     if (variant < 0 || variant > (layer_kind == IPTQ_LAYER_SOFTMAX ? 3 : 2) || rows < 0 || row_len < 0) return -1.0;
     const double r = (double)rows, n = (double)rows * (double)row_len;
     switch (layer_kind) {
         case IPTQ_LAYER_SOFTMAX: {
-            // logarithm candidate: exponential and sum 13, round(sum / e) 4, leading one 1, rounding bit 3, clamp 1
-            static const double per_elem[4] = {21.0, 17.0, 15.0, 22.0};
-            return per_elem[variant] * n + (variant == IPTQ_SM_LOG2 ? 0.0 : r);
+            static const double per_elem[4] = {21.0, 17.0, 15.0, 25.0};
+            return per_elem[variant] * n + r;
         }
         case IPTQ_LAYER_GELU: {
-            static const double per_elem[3] = {20.0, 19.0, 33.0};
+            static const double per_elem[3] = {21.0, 20.0, 34.0};
             return per_elem[variant] * n;
         }
         case IPTQ_LAYER_LAYERNORM: {
-            static const double per_elem[3] = {15.0, 15.0, 16.0};
-            static const double per_row[3] = {34.0, 22.0, 22.0};
+            static const double per_elem[3] = {16.0, 16.0, 17.0};
+            static const double per_row[3] = {38.0, 28.0, 28.0};
             return per_elem[variant] * n + per_row[variant] * r;
         }
         default: return -1.0;

@@ -19,9 +19,6 @@ struct SoftmaxDev {
     const uint16_t* tab_src;   // the table in device memory, or null: each CTA builds it
 };
 
-// Lanes past the row end carry a score so low that the clamp at -dcap applies and the exponential is 0.
-constexpr int kPadScore = -(1 << 30);
-
 template <int VARIANT, int NITER, bool HAS_BIAS, bool PSHR>
 __global__ void __launch_bounds__(256)
 softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ probs, int64_t rows, int n,
@@ -40,7 +37,7 @@ softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ pr
 #pragma unroll
         for (int k = 0; k < NITER; ++k) {
             const int j = lane + 32 * k;
-            int s = kPadScore;
+            int s = kNoScore;                                  // lanes past the row end
             if (j < n) {
                 s = __ldcs(sr + j);
                 if (HAS_BIAS) s += __ldg(br + j);
@@ -52,7 +49,7 @@ softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ pr
         unsigned sum = 0;
 #pragma unroll
         for (int k = 0; k < NITER; ++k) {
-            const unsigned e = exp_core_nd<VARIANT>(v[k] - mx, c.ex);
+            const unsigned e = exp_core_nd<VARIANT>(exp_distance(mx, v[k]), c.ex);
             v[k] = (int)e;
             sum += e;
         }
@@ -77,8 +74,9 @@ softmax_rows_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict__ pr
     }
 }
 
-// Tabulated form for the shift-based variants: the exponential of Eq. (9) is 0 beyond a few multiples of x0 and
-// below 2^16, so each CTA keeps it as a table in shared memory (copied from the one iptq_softmax_table() wrote, or
+// Tabulated form: the integer exponential (Eq. (9), or the second-order polynomial of the other two candidates)
+// depends on max - s alone, is 0 beyond a few multiples of x0 and below 2^16, so each CTA keeps it as a table in
+// shared memory (copied from the one iptq_softmax_table() wrote, or
 // built here with the same arithmetic) and a score costs one 16-bit shared-memory load instead of the evaluation.
 // Two CTAs of 1024 threads per SM: 32 registers per thread, 64 warps to cover the load latency.
 constexpr int kSmTabThreads = 1024;
@@ -117,7 +115,7 @@ softmax_rows_tab_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict_
         const int32_t* br = HAS_BIAS ? bias + (row % bias_period) * n + lane : nullptr;
 #pragma unroll
         for (int k = 0; k < NITER; ++k) {
-            int s = kPadScore;
+            int s = kNoScore;                                  // lanes past the row end
             if (k < NITER - 1 || tail_ok) {
                 s = __ldcs(sr + 32 * k);
                 if (HAS_BIAS) s += __ldg(br + 32 * k);
@@ -140,8 +138,14 @@ softmax_rows_tab_kernel(const int32_t* __restrict__ scores, uint8_t* __restrict_
             sum += e;
         }
         sum = __reduce_add_sync(kFull, sum);
-        const unsigned f = intdiv_factor(sum, c.M) << c.f_shl;  // Eq. (15)
         uint8_t* pr = probs + row * n + lane;
+        if constexpr (VARIANT == IPTQ_SM_LOG2) {
+#pragma unroll
+            for (int k = 0; k < NITER; ++k)
+                if (k < NITER - 1 || tail_ok) __stcs(pr + 32 * k, (uint8_t)log2_code(sum, (unsigned)v[k]));
+            return;
+        }
+        const unsigned f = intdiv_factor(sum, c.M) << c.f_shl;  // Eq. (15)
 #pragma unroll
         for (int k = 0; k < NITER; ++k) {
             unsigned pv = __umulhi(f, (unsigned)v[k]);
@@ -160,7 +164,7 @@ template <int VARIANT, int NITER>
 static int launch_softmax2(const int32_t* s, uint8_t* p, int64_t rows, int n, const int32_t* bias, int64_t period,
                            const SoftmaxDev& c, cudaStream_t st)
 {
-    if constexpr (VARIANT != IPTQ_SM_POLY && VARIANT != IPTQ_SM_LOG2 && NITER <= 8)
+    if constexpr (NITER <= 8)
     if (c.tab_n > 0 && ((c.tab_n + 8) & ~7) <= IPTQ_SOFTMAX_TABLE_MAX &&
         rows * n >= (c.tab_src ? kSmTabMinElemsCopy : kSmTabMinElemsBuild)) {
         // Tabulated exponential: worth the per-CTA table set-up once every warp has several rows.
@@ -795,8 +799,9 @@ int iptq_softmax_table(iptq_softmax_consts* consts, uint16_t* table, int32_t cap
     if (capacity < n_pad) return IPTQ_ERR_SHAPE;
     const ExpDev ex = to_dev_exp(*consts);
     const int threads = 256, grid = (n_pad + threads - 1) / threads;
-    if (consts->variant == IPTQ_SM_BITEXP) launch_kernel(softmax_table_kernel<IPTQ_SM_BITEXP>, grid, threads, 0, stream, table, n, n_pad, ex);
-    else                                   launch_kernel(softmax_table_kernel<IPTQ_SM_SHIFTMAX>, grid, threads, 0, stream, table, n, n_pad, ex);
+    if (consts->variant == IPTQ_SM_BITEXP)        launch_kernel(softmax_table_kernel<IPTQ_SM_BITEXP>, grid, threads, 0, stream, table, n, n_pad, ex);
+    else if (consts->variant == IPTQ_SM_SHIFTMAX) launch_kernel(softmax_table_kernel<IPTQ_SM_SHIFTMAX>, grid, threads, 0, stream, table, n, n_pad, ex);
+    else                                          launch_kernel(softmax_table_kernel<IPTQ_SM_POLY>, grid, threads, 0, stream, table, n, n_pad, ex);   // also behind the logarithm candidate
     stream_fence_kernel<<<1, 32, 0, stream>>>();
     note_launch();
     const int rc = last_launch_status();

@@ -111,7 +111,7 @@ def test_argument_errors_are_reported_before_any_launch(api):
     assert e.value.status == api.ERR_VARIANT
     assert L.iptq_linear(None, None, 5, None, None, None, 0, None, None, None, 8, 16, 16, None, 0, None) == api.ERR_BITS
     assert L.iptq_linear(None, None, 8, None, None, None, 0, None, None, None, 8, 16, 16, None, 0, None) == api.ERR_WORKSPACE
-    assert L.iptq_attention_block(None, None, None, None, 1, 1, 49, 32, None, None, None, None, None, 0, None) \
+    assert L.iptq_attention_block(None, None, None, None, 1, 1, 49, 32, None, None, None, None, None, None, 0, None) \
         == api.ERR_WORKSPACE
     assert api.lib().iptq_strerror(api.ERR_TIMEOUT).decode() != ""
     assert api.linear_workspace_bytes(100, 256, 384, 4) >= 256 + 256 * 384
