@@ -4,12 +4,9 @@
 //   - FC1: requantise to the GELU input scale, integer GELU (Sec. 3.3, Eqs. (3), (5)), requantise to int8.
 // No int32 intermediate is written to HBM.
 //
-// One persistent CTA per SM, 14 warps: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM),
-// warps 2..13 = epilogue (three warps per TMEM lane quadrant, each taking a third of the tile's columns).
-// The accumulator is double-buffered in TMEM so that the epilogue of tile i overlaps the mainloop of tile i+1.
-// Per-column requantisation constants live in TMEM beside the accumulators (shared-memory reads of them would
-// cost one load per output and saturate the load/store pipe); the bias is written into each accumulator before
-// the MMAs start, which then always accumulate.
+// One persistent CTA per SM, 18 warps: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM), warps 2..17 =
+// epilogue.  The accumulator is double-buffered in TMEM so that the epilogue of tile i overlaps the mainloop of
+// tile i+1.
 #include <algorithm>
 #include <mutex>
 
@@ -60,87 +57,61 @@ int make_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint6
 }
 
 // ---------------------------------------------------------------- kernel
-enum { EPI_REQUANT = 0, EPI_RESIDUAL = 1, EPI_GELU = 2 };
+// The product is computed transposed, D^T[channel, token] = W X^T: the weight tile is the A operand (128 output
+// channels = the 128 TMEM lanes), the activation tile the B operand (TN tokens = TMEM columns).  A thread of the
+// epilogue then owns ONE output channel, so the per-channel requantisation constants (bias, multiplier, shift,
+// rounding constant) are four registers instead of per-column vectors, and nothing but the accumulator is read
+// from TMEM.  The outputs of a warp (32 channels x TN/4 tokens) go through a shared-memory block in the row-major
+// [token][channel] order of y and leave with one TMA store, which also clips at M and N.
+enum { EPI_REQUANT = 0, EPI_RESIDUAL = 1, EPI_GELU = 2, EPI_GELU_TAB = 3 };
 
-constexpr int BM = 128;          // rows per tile = TMEM lanes
-constexpr int BK = 128;          // bytes of K per stage = one 128-byte swizzle row = 4 MMA k-steps
-constexpr int COLS = 32;         // columns per epilogue warp: bytes per output row, one 32-byte swizzle row
+constexpr int BK = 128;                  // bytes of K per ring stage = one 128-byte swizzle row = 4 MMA k-steps
+constexpr int CT = 128;                  // output channels per tile = TMEM lanes
+constexpr int W_BYTES = CT * BK;         // weight tile of one stage
+constexpr int MAX_STAGES = 8;
+constexpr int EPI_WARPS = 16;            // 4 TMEM lane quadrants x 4 token quarters
+constexpr int GEMM_THREADS = 32 * (2 + EPI_WARPS);
+constexpr int ACC_COLS = 256;            // TMEM columns between the two accumulators
 constexpr uint32_t TMEM_COLS = 512;
-
-// Tile width BN is 96 or 128.  TMEM holds two accumulators plus per-column constant rows (one row = BN words,
-// replicated over the 128 lanes so that a thread reads them with the same instruction as its accumulators):
-//   BN =  96: mult, rounding constant, shift           (5 x 96 = 480 columns)
-//   BN = 128: mult, shift - 1; the rounding constant 2^(shift-1) is rebuilt with one shift  (4 x 128 = 512 columns)
-// GTAB: the FC1 epilogue reads the integer GELU from a 64 KB table in shared memory, which leaves room for a shorter ring.
-// The ring takes what shared memory is left: deeper rings changed nothing at K = 384 and gave 3 % at K = 768 / 3072.
-template <int BN, bool GTAB = false>
-struct GemmCfg {
-    static constexpr int STAGES = GTAB ? (BN == 96 ? 4 : 3) : (BN == 96 ? 7 : 5);
-    static constexpr int EPI_PARTS = BN / COLS;          // epilogue warps per TMEM lane quadrant
-    static constexpr int EPI_WARPS = 4 * EPI_PARTS;
-    static constexpr int THREADS = 32 * (2 + EPI_WARPS);
-    static constexpr uint32_t TM_MULT = 2 * BN, TM_RND = 3 * BN, TM_SHIFT = BN == 96 ? 4 * BN : 3 * BN;
-    static constexpr bool HAS_RND = BN == 96;
-};
+constexpr int SMEM_LIMIT = 227 * 1024;
 
 struct GemmParams {
-    int M, N, K;
-    int num_m_tiles, num_n_tiles;
-    int stages;                                       // ring stages in use
+    int M, N, K;                                      // tokens, output channels, reduction length
+    int TN;                                           // tokens per tile: 64, 128, 192 or 256
+    int n_ct, n_tt;                                   // channel tiles, token tiles
+    int stages, stage_bytes;                          // TMA ring
+    int off_res, off_tab, off_bar, off_ring;          // shared-memory layout (the output blocks start at 0)
     const int32_t* bias; const int32_t* mult; const int8_t* shift;
     int out_zp;
-    int qmin, qmax;                                   // output range of the plain / residual epilogues when it is not int8
+    int qmin, qmax;                                   // output range
     int res_mult, res_rnd, res_shift, res_off;        // residual branch: ((res << 16) - res_off) through R
     GeluDev gelu;
-    const int8_t* gelu_tab;                           // device table of the integer GELU, or null
+    const int8_t* gelu_tab;                           // device table of the integer GELU (EPI_GELU_TAB)
     StatusBlock* status;
 };
 
-template <int BN, bool GTAB = false>
-struct GemmSmem {
-    static constexpr int STAGES = GemmCfg<BN, GTAB>::STAGES;
-    static constexpr int EPI_WARPS = GemmCfg<BN, GTAB>::EPI_WARPS;
-    static constexpr int A_BYTES = BM * BK;
-    static constexpr int B_BYTES = BN * BK;
-    static constexpr int WARP_TILE = 32 * COLS;                                   // bytes of one warp's output block
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;                        // one ring stage: A tile, then B tile
-    static constexpr int OFF_OUT = 0;                                             // [EPI_WARPS][32 rows][COLS] int8
-    static constexpr int OFF_RES = OFF_OUT + EPI_WARPS * WARP_TILE;              // same shape, residual tiles
-    static constexpr int OFF_BIAS = OFF_RES + EPI_WARPS * WARP_TILE;             // [EPI_WARPS][COLS] int32
-    static constexpr int OFF_TAB = OFF_BIAS + EPI_WARPS * COLS * 4;              // GELU table (GTAB only)
-    static constexpr int OFF_BAR = OFF_TAB + (GTAB ? IPTQ_GELU_TABLE_SIZE : 0);
-    static constexpr int NUM_BARS = 2 * STAGES + 4 + EPI_WARPS;
-    static constexpr int OFF_RING = (OFF_BAR + NUM_BARS * 8 + 16 + 1023) & ~1023; // the ring comes last: its length is a launch parameter
-    static constexpr int total(int stages) { return OFF_RING + stages * STAGE_BYTES + 1024; }   // slack for 1024-byte alignment
-    static constexpr int TOTAL = total(STAGES);
-};
+// The i-th tile of this CTA: tiles are numbered with the channel tile fastest, so that CTAs running side by side
+// share an activation tile in L2.
+__device__ __forceinline__ bool gemm_tile(const GemmParams& p, int i, int& tt, int& ct)
+{
+    const int t = (int)blockIdx.x + i * (int)gridDim.x;
+    tt = t / p.n_ct;
+    ct = t - tt * p.n_ct;
+    return tt < p.n_tt;
+}
 
-// Byte offset of 16-byte chunk `chunk` (0/1) of row `row` inside a [32][32]-byte block written/read by TMA with
-// the 32-byte swizzle (chunk bit XOR bit 7 of the address); also keeps a warp's per-row 16-byte accesses
-// conflict-free.
-__device__ __forceinline__ uint32_t swz32(int row, int chunk) { return (uint32_t)(row * 32 + ((chunk ^ ((row >> 2) & 1)) << 4)); }
-
-// One CTA works on ONE column tile (blockIdx.x % num_n_tiles) and walks down its row tiles, so the per-column
-// constants are set up once per CTA: mult / rounding / shift in TMEM, the bias in shared memory, from where the
-// epilogue writes it back into each accumulator it has just drained (the MMAs then always accumulate).
-template <int BN, int EPI, int GELU_VARIANT, bool SAT8, bool GTAB>
-__global__ void __launch_bounds__(GemmCfg<BN>::THREADS, 1)
-gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+template <int EPI, int GELU_VARIANT>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_res,
                const GemmParams p)
 {
-    using L = GemmSmem<BN, GTAB>;
-    using G = GemmCfg<BN, GTAB>;
-    constexpr int STAGES = G::STAGES, EPI_WARPS = G::EPI_WARPS;
-    constexpr uint32_t TM_MULT = G::TM_MULT, TM_RND = G::TM_RND, TM_SHIFT = G::TM_SHIFT;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* sA = smem + L::OFF_RING;
-    uint8_t* sB = sA + L::A_BYTES;
-    const int stages = p.stages;                     // ring stages in use (<= STAGES)
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
-    uint64_t* empty_bar = full_bar + STAGES;
-    uint64_t* acc_full = empty_bar + STAGES;      // [2]
+    uint8_t* ring = smem + p.off_ring;
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + p.off_bar);
+    uint64_t* empty_bar = full_bar + MAX_STAGES;
+    uint64_t* acc_full = empty_bar + MAX_STAGES;  // [2]
     uint64_t* acc_empty = acc_full + 2;           // [2]
     uint64_t* res_bar = acc_empty + 2;            // [EPI_WARPS]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(res_bar + EPI_WARPS);
@@ -149,18 +120,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int kblocks = (p.K + BK - 1) / BK;
-    const int n0 = (int)(blockIdx.x % (unsigned)p.num_n_tiles) * BN;
-    const int mt0 = (int)(blockIdx.x / (unsigned)p.num_n_tiles);
-    const int mt_step = (int)(gridDim.x / (unsigned)p.num_n_tiles);
+    const int stages = p.stages;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EPI_WARPS); }
         for (int w = 0; w < EPI_WARPS; ++w) mbar_init(&res_bar[w], 1);
         ctl->abort = 0;
         fence_barrier_init();
-        prefetch_tensormap(&map_a);
-        prefetch_tensormap(&map_b);
+        prefetch_tensormap(&map_w);
+        prefetch_tensormap(&map_x);
         prefetch_tensormap(&map_y);
         if (EPI == EPI_RESIDUAL) prefetch_tensormap(&map_res);
     }
@@ -177,15 +146,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (elect_one()) {
-            grid_dep_wait();                                   // the activations come from the previous kernel
+            grid_dep_wait();                                   // the activations (and unpacked weights) come from earlier kernels
             int s = 0; uint32_t ph = 0;
-            for (int mt = mt0; mt < p.num_m_tiles; mt += mt_step) {
+            int tt, ct;
+            for (int i = 0; gemm_tile(p, i, tt, ct); ++i) {
                 bool ok = true;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(&empty_bar[s], ph ^ 1u, ctl, p.status, 1)) { ok = false; break; }
-                    mbar_expect_tx(&full_bar[s], L::A_BYTES + L::B_BYTES);
-                    tma_load_2d(sA + s * L::STAGE_BYTES, &map_a, &full_bar[s], kb * BK, mt * BM);
-                    tma_load_2d(sB + s * L::STAGE_BYTES, &map_b, &full_bar[s], kb * BK, n0);
+                    uint8_t* st = ring + s * p.stage_bytes;
+                    mbar_expect_tx(&full_bar[s], (uint32_t)p.stage_bytes);
+                    tma_load_2d(st, &map_w, &full_bar[s], kb * BK, ct * CT);
+                    tma_load_2d(st + W_BYTES, &map_x, &full_bar[s], kb * BK, tt * p.TN);
                     if (++s == stages) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
@@ -194,27 +165,27 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (elect_one()) {
-            constexpr uint32_t idesc = umma_idesc_i8(BM, BN, true, true, false, false);
+            const uint32_t idesc = umma_idesc_i8(CT, p.TN, true, true, false, false);
             int s = 0; uint32_t ph = 0;
-            int it = 0;
-            for (int mt = mt0; mt < p.num_m_tiles; mt += mt_step, ++it) {
+            int tt, ct;
+            for (int it = 0; gemm_tile(p, it, tt, ct); ++it) {
                 const int ab = it & 1;
-                // the accumulator holds the bias, written by the epilogue warps (first at start-up, then after each drain)
-                if (!mbar_wait(&acc_empty[ab], (uint32_t)(it >> 1) & 1u, ctl, p.status, 2)) break;
+                // the epilogue warps have pulled this accumulator's previous contents into registers
+                if (!mbar_wait(&acc_empty[ab], ((uint32_t)(it >> 1) & 1u) ^ 1u, ctl, p.status, 2)) break;
                 tc_fence_after_sync();
-                const uint32_t tacc = tmem_base + (uint32_t)(ab * BN);
+                const uint32_t tacc = tmem_base + (uint32_t)(ab * ACC_COLS);
                 bool ok = true;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(&full_bar[s], ph, ctl, p.status, 3)) { ok = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t a_addr = smem_u32(sA + s * L::STAGE_BYTES);
-                    const uint32_t b_addr = smem_u32(sB + s * L::STAGE_BYTES);
+                    const uint32_t w_addr = smem_u32(ring + s * p.stage_bytes);
+                    const uint32_t x_addr = w_addr + W_BYTES;
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k) {
                         // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart; a k-step is 32 bytes
-                        const uint64_t da = umma_smem_desc(a_addr + k * 32, 16, 1024, 128);
-                        const uint64_t db = umma_smem_desc(b_addr + k * 32, 16, 1024, 128);
-                        umma_i8(tacc, da, db, idesc, 1u);
+                        const uint64_t da = umma_smem_desc(w_addr + k * 32, 16, 1024, 128);
+                        const uint64_t db = umma_smem_desc(x_addr + k * 32, 16, 1024, 128);
+                        umma_i8(tacc, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
                     }
                     umma_commit(&empty_bar[s]);               // frees the stage once these MMAs have read it
                     if (++s == stages) { s = 0; ph ^= 1u; }
@@ -225,145 +196,133 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else {
         // ------------------------------------------------------------ epilogue warps
-        // Warp (quad, part) owns TMEM lanes 32*quad.. (the only ones it may touch) and columns part*COLS.. of
-        // every tile: it turns them into a [32 rows][COLS] int8 block in shared memory and stores that block
-        // with one TMA copy; nothing in the epilogue synchronises across warps.
+        // Warp (quad, part) owns TMEM lanes 32*quad.. (the only ones it may touch) = 32 output channels, and the
+        // token columns part * TN/4 .. of every tile; lane = channel.  Nothing here synchronises across warps.
         const int ew = warp - 2;
         const int quad = warp & 3;
         const int part = ew >> 2;
-        int* sbias = reinterpret_cast<int*>(smem + L::OFF_BIAS) + ew * COLS;
-        const uint32_t bias_addr = smem_u32(sbias);
-        const uint32_t out_blk = smem_u32(smem + L::OFF_OUT + ew * L::WARP_TILE);
-        uint8_t* res_ptr = smem + L::OFF_RES + ew * L::WARP_TILE;
-        const uint32_t res_blk = smem_u32(res_ptr);
-        const int col0 = n0 + part * COLS;
-        const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(part * COLS);
+        const int tpp = p.TN >> 2;                             // tokens per part: 16, 32, 48 or 64
+        const int nchunks = tpp >> 4;                          // 16-token chunks: 1..4
+        uint8_t* out_blk = smem + ew * (tpp * 32);            // [tpp tokens][32 channels] int8
+        const uint32_t out_lane = smem_u32(out_blk) + (uint32_t)lane;
+        uint8_t* res_blk = smem + p.off_res + ew * (tpp * 32);
+        const uint32_t res_lane = smem_u32(res_blk) + (uint32_t)lane;
         uint32_t res_ph = 0;
-        {
-            // ---- once per CTA: this warp's per-column constants (lane = column)
-            const int n = col0 + lane;
-            int cb = 0, cm = 1 << 30, cr = 1, cs = 1;
-            if (n < p.N) {
-                cs = (int)__ldg(p.shift + n);
-                cb = p.bias ? __ldg(p.bias + n) : 0;
-                cm = __ldg(p.mult + n);
-                cr = 1 << (cs - 1);
-            }
-            if (!G::HAS_RND) cs -= 1;                         // the shift row holds shift - 1
-            sbias[lane] = cb;
-            __syncwarp();
-            uint32_t v[16];
-#pragma unroll
-            for (int ch = 0; ch < COLS / 16; ++ch) {
-#pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] = (uint32_t)__shfl_sync(0xffffffffu, cm, ch * 16 + j);
-                tmem_st16(tlane + TM_MULT + ch * 16, v);
-                if (G::HAS_RND) {
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] = (uint32_t)__shfl_sync(0xffffffffu, cr, ch * 16 + j);
-                    tmem_st16(tlane + TM_RND + ch * 16, v);
-                }
-#pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] = (uint32_t)__shfl_sync(0xffffffffu, cs, ch * 16 + j);
-                tmem_st16(tlane + TM_SHIFT + ch * 16, v);
-#pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] = (uint32_t)__shfl_sync(0xffffffffu, cb, ch * 16 + j);
-                tmem_st16(tlane + ch * 16, v);                // both accumulators start from the bias
-                tmem_st16(tlane + BN + ch * 16, v);
-            }
-            tmem_wait_st();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) { mbar_arrive(&acc_empty[0]); mbar_arrive(&acc_empty[1]); }
-        }
-        const uint32_t tab_mid = smem_u32(smem + L::OFF_TAB) + 32768u;      // address of table[0 + 32768]
-        if (GTAB) {
+        const uint32_t tab_mid = smem_u32(smem + p.off_tab) + 32768u;      // address of table[0 + 32768]
+        if (EPI == EPI_GELU_TAB) {
             // the GELU table is static data: copy it while the previous kernel may still be running
             const int4* src = reinterpret_cast<const int4*>(p.gelu_tab);
-            int4* dst = reinterpret_cast<int4*>(smem + L::OFF_TAB);
+            int4* dst = reinterpret_cast<int4*>(smem + p.off_tab);
             for (int i = ew * 32 + lane; i < IPTQ_GELU_TABLE_SIZE / 16; i += EPI_WARPS * 32) dst[i] = __ldg(src + i);
             named_barrier(1, EPI_WARPS * 32);
         }
         grid_dep_wait();                                       // residual reads and output writes come after this
-        int it = 0;
-        for (int mt = mt0; mt < p.num_m_tiles; mt += mt_step, ++it) {
+        // Nothing in a tile's epilogue waits for something that was started in the same tile: the channel constants
+        // and the residual block of tile i + 1 are requested during tile i.
+        auto load_consts = [&](int ct_, int& cm_, int& cs_, int& cb_) {
+            const int c = ct_ * CT + quad * 32 + lane;
+            cm_ = 1 << 30; cs_ = 1; cb_ = 0;
+            if (c < p.N) {
+                cm_ = __ldg(p.mult + c);
+                cs_ = (int)__ldg(p.shift + c);
+                cb_ = p.bias ? __ldg(p.bias + c) : 0;
+            }
+        };
+        auto request_residual = [&](int tt_, int ct_) {
+            const int c0_ = ct_ * CT + quad * 32, tok0_ = tt_ * p.TN + part * tpp;
+            if (c0_ < p.N && tok0_ < p.M && lane == 0) {
+                mbar_expect_tx(&res_bar[ew], (uint32_t)(tpp * 32));
+                tma_load_2d(res_blk, &map_res, &res_bar[ew], c0_, tok0_);
+            }
+        };
+        int tt, ct;
+        bool have = gemm_tile(p, 0, tt, ct);
+        int cm, cs, cb;
+        if (have) {
+            load_consts(ct, cm, cs, cb);
+            if (EPI == EPI_RESIDUAL) request_residual(tt, ct);
+        }
+        for (int it = 0; have; ++it) {
+            int ntt, nct, ncm, ncs, ncb;
+            const bool nhave = gemm_tile(p, it + 1, ntt, nct);
+            if (nhave) load_consts(nct, ncm, ncs, ncb);        // in flight during this tile
             const int ab = it & 1;
             const uint32_t abph = (uint32_t)(it >> 1) & 1u;
-            const int row0 = mt * BM + quad * 32;
-            const bool active = row0 < p.M && col0 < p.N;     // warp-uniform
-            // the previous tile's store must have read the staging block before it is rewritten
-            if (lane == 0) bulk_wait_read_all();
-            __syncwarp();
-            if (EPI == EPI_RESIDUAL && active && lane == 0) {
-                mbar_expect_tx(&res_bar[ew], L::WARP_TILE);
-                tma_load_2d(res_ptr, &map_res, &res_bar[ew], col0, row0);
-            }
+            const int c0 = ct * CT + quad * 32;               // first channel of this warp
+            const int tok0 = tt * p.TN + part * tpp;          // first token of this warp
+            const bool active = c0 < p.N && tok0 < p.M;       // warp-uniform
+            const int crnd = 1 << (cs - 1);
             if (!mbar_wait(&acc_full[ab], abph, ctl, p.status, 4)) break;
             tc_fence_after_sync();
+            // the previous tile's store has read the output block (it was issued a whole K loop ago)
+            if (lane == 0) bulk_wait_read_all();
+            __syncwarp();
             if (EPI == EPI_RESIDUAL && active) {
                 if (!mbar_wait(&res_bar[ew], res_ph, ctl, p.status, 5)) break;
                 res_ph ^= 1u;
             }
-            const uint32_t tacc = tlane + (uint32_t)(ab * BN);
+            const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * ACC_COLS + part * tpp);
+            uint32_t acc[2][16];
+            tmem_ld16(tacc, acc[0]);
 #pragma unroll
-            for (int ch = 0; ch < COLS / 16; ++ch) {
-                uint32_t acc[16], cm[16], cr[G::HAS_RND ? 16 : 1], cs[16];
-                tmem_ld16(tacc + ch * 16, acc);
-                tmem_ld16(tlane + TM_MULT + ch * 16, cm);
-                if constexpr (G::HAS_RND) tmem_ld16(tlane + TM_RND + ch * 16, cr);
-                tmem_ld16(tlane + TM_SHIFT + ch * 16, cs);
-                uint32_t bv[16];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const uint4 t = ld_shared_v4(bias_addr + ch * 64 + q * 16);
-                    bv[4 * q] = t.x; bv[4 * q + 1] = t.y; bv[4 * q + 2] = t.z; bv[4 * q + 3] = t.w;
-                }
-                tmem_wait_ld();
-                tmem_st16(tacc + ch * 16, bv);                // re-arm this accumulator with the bias
-                if (!active) continue;
-                uint4 resv = make_uint4(0, 0, 0, 0);
-                if (EPI == EPI_RESIDUAL) resv = ld_shared_v4(res_blk + swz32(lane, ch));
-                const uint32_t resw[4] = {resv.x, resv.y, resv.z, resv.w};
-                int o[16];
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    int v;
-                    if constexpr (G::HAS_RND) v = requant_core((int)acc[j], (int)cm[j], (int)cr[j], (int)cs[j]);
-                    else v = (mad_hi((int)acc[j], (int)cm[j], 1 << cs[j]) >> cs[j]) >> 1;   // cs = shift - 1
-                    if (EPI == EPI_GELU && GTAB) {
-                        v = max(-32768, min(32767, v));
-                        asm volatile("ld.shared.s8 %0, [%1];" : "=r"(v) : "r"(tab_mid + (uint32_t)v));
-                    } else if (EPI == EPI_GELU) {
-                        v = gelu_core<GELU_VARIANT>(v, p.gelu);
-                        v = requant_nosat(v, p.gelu.out);
-                        if (!SAT8) v = max(p.gelu.out.qmin, min(p.gelu.out.qmax, v));
-                    } else if (EPI == EPI_RESIDUAL) {
-                        // byte j of the residual word, sign-extended, widened by 2^16 and requantised
-                        const int rb = (j & 3) == 0 ? sext_byte<0>(resw[j >> 2]) : (j & 3) == 1 ? sext_byte<1>(resw[j >> 2])
-                                     : (j & 3) == 2 ? sext_byte<2>(resw[j >> 2]) : sext_byte<3>(resw[j >> 2]);
-                        v += requant_core(rb * 65536 - p.res_off, p.res_mult, p.res_rnd, p.res_shift) + p.out_zp;
+            for (int ch = 0; ch < 4; ++ch) {
+                if (ch < nchunks) {                            // warp-uniform
+                    tmem_wait_ld();                            // chunk ch is in registers
+                    if (ch + 1 < nchunks) {
+                        tmem_ld16(tacc + (uint32_t)((ch + 1) * 16), acc[(ch + 1) & 1]);   // in flight during the arithmetic
                     } else {
-                        v += p.out_zp;
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&acc_empty[ab]);   // the MMA warp may refill this accumulator
                     }
-                    if (EPI != EPI_GELU && !SAT8) v = max(p.qmin, min(p.qmax, v));   // activations narrower than 8 bits
-                    o[j] = v;
+                    if (active) {
+                        // Three passes over the chunk, so that the shared-memory reads (volatile, hence kept in
+                        // program order with the stores) are issued back to back instead of one per stored byte.
+                        int v[16], r[16];
+                        if (EPI == EPI_RESIDUAL) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                asm volatile("ld.shared.s8 %0, [%1];" : "=r"(r[j]) : "r"(res_lane + (uint32_t)((ch * 16 + j) * 32)));
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            v[j] = requant_core((int)acc[ch & 1][j] + cb, cm, crnd, cs);
+                            if (EPI == EPI_GELU_TAB) {
+                                v[j] = max(-32768, min(32767, v[j]));
+                            } else if (EPI == EPI_GELU) {
+                                v[j] = requant_nosat(gelu_core<GELU_VARIANT>(v[j], p.gelu), p.gelu.out);
+                                v[j] = max(p.gelu.out.qmin, min(p.gelu.out.qmax, v[j]));
+                            } else if (EPI == EPI_RESIDUAL) {
+                                v[j] += requant_core(r[j] * 65536 - p.res_off, p.res_mult, p.res_rnd, p.res_shift) + p.out_zp;
+                                v[j] = max(p.qmin, min(p.qmax, v[j]));
+                            } else {
+                                v[j] = max(p.qmin, min(p.qmax, v[j] + p.out_zp));
+                            }
+                        }
+                        if (EPI == EPI_GELU_TAB) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                asm volatile("ld.shared.s8 %0, [%1];" : "=r"(v[j]) : "r"(tab_mid + (uint32_t)v[j]));
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            asm volatile("st.shared.u8 [%0], %1;" ::"r"(out_lane + (uint32_t)((ch * 16 + j) * 32)), "r"(v[j]) : "memory");
+                    }
                 }
-                st_shared_v4(out_blk + swz32(lane, ch), pack4_sat_s8(o[0], o[1], o[2], o[3]),
-                             pack4_sat_s8(o[4], o[5], o[6], o[7]), pack4_sat_s8(o[8], o[9], o[10], o[11]),
-                             pack4_sat_s8(o[12], o[13], o[14], o[15]));
             }
-            tmem_wait_st();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[ab]);       // the MMA warp may refill this accumulator
             if (active) {
-                fence_proxy_async_smem();                     // this lane's st.shared -> visible to the TMA engine
+                fence_proxy_async_smem();                     // this lane's shared-memory stores -> visible to the TMA engine
                 __syncwarp();
                 if (lane == 0) {
-                    tma_store_2d(&map_y, smem + L::OFF_OUT + ew * L::WARP_TILE, col0, row0);   // clipped at M and N
+                    tma_store_2d(&map_y, out_blk, c0, tok0);  // clipped at N and M
                     bulk_commit();
                 }
             }
+            if (EPI == EPI_RESIDUAL && nhave) {
+                __syncwarp();                                  // every lane has read its residual bytes of this tile
+                request_residual(ntt, nct);
+            }
+            have = nhave; tt = ntt; ct = nct; cm = ncm; cs = ncs; cb = ncb;
         }
         if (lane == 0) bulk_wait_all();                       // stores complete before shared memory goes away
     }
@@ -480,35 +439,23 @@ int unpack_int4_launch(const void* packed, int8_t* out, int64_t n_elems, cudaStr
 }
 
 // ---------------------------------------------------------------- launcher
-template <int BN, int EPI, int GV, bool SAT8, bool GTAB = false>
-static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& my, const CUtensorMap& mr,
-                       const GemmParams& p, cudaStream_t st)
+template <int EPI, int GV>
+static int launch_gemm(const CUtensorMap& mw, const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& mr,
+                       const GemmParams& p, int grid, int smem_bytes, cudaStream_t st)
 {
-    using L = GemmSmem<BN, GTAB>;
-    auto kern = gemm_i8_kernel<BN, EPI, GV, SAT8, GTAB>;
+    auto kern = gemm_i8_kernel<EPI, GV>;
     static bool configured[64];               // one attribute call per instantiation and device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return IPTQ_ERR_CUDA;
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) != cudaSuccess)
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT) != cudaSuccess)
             return IPTQ_ERR_CUDA;
         configured[dev] = true;
     }
-    // every CTA serves one column tile; the SMs are split evenly among the column tiles
-    const int per_n = std::max(1, std::min(sm_count() / p.num_n_tiles, p.num_m_tiles));
-    const int grid = p.num_n_tiles * per_n;
-    // a ring much longer than one tile's K loop buys nothing, and a smaller footprint lets the next kernel's CTAs
-    // become resident earlier
-    GemmParams q = p;
-    const int kblocks = (p.K + BK - 1) / BK;
-    q.stages = std::max(2, std::min(L::STAGES, kblocks + 1));
-    launch_kernel(kern, grid, GemmCfg<BN>::THREADS, L::total(q.stages), st, ma, mb, my, mr, q);
+    launch_kernel(kern, grid, GEMM_THREADS, smem_bytes, st, mw, mx, my, mr, p);
     note_launch();
     return last_launch_status();
 }
-
-template <int BN>
-static int linear_launch_bn(const LinearArgs& a, cudaStream_t st);
 
 int linear_check(const LinearArgs& a)
 {
@@ -530,26 +477,37 @@ int linear_check(const LinearArgs& a)
     return IPTQ_OK;
 }
 
+// Shared-memory layout for a tile width: output blocks, residual blocks, GELU table, barriers, then as many ring
+// stages as fit.  Returns the number of stages (0: does not fit).
+static int gemm_layout(GemmParams& p, int TN, bool residual, bool table, int kblocks, int* smem_bytes)
+{
+    const int blocks = EPI_WARPS * (TN / 4) * 32;             // = 128 TN bytes
+    p.TN = TN;
+    p.off_res = blocks;
+    p.off_tab = p.off_res + (residual ? blocks : 0);
+    p.off_bar = p.off_tab + (table ? IPTQ_GELU_TABLE_SIZE : 0);
+    p.off_ring = (p.off_bar + (2 * MAX_STAGES + 4 + EPI_WARPS) * 8 + 16 + 1023) & ~1023;
+    p.stage_bytes = W_BYTES + TN * BK;
+    const int room = SMEM_LIMIT - 1024 - p.off_ring;          // 1024: slack for the alignment of the dynamic base
+    if (room < 0) return 0;
+    int stages = std::min(MAX_STAGES, room / p.stage_bytes);
+    // a ring much longer than one tile's K loop buys nothing, and a smaller footprint lets the next kernel's CTAs
+    // become resident earlier
+    stages = std::min(stages, std::max(2, kblocks + 1));
+    p.stages = stages;
+    *smem_bytes = p.off_ring + stages * p.stage_bytes + 1024;
+    return stages;
+}
+
 int linear_launch(const LinearArgs& a, cudaStream_t st)
 {
     const int rc0 = linear_check(a);
     if (rc0 != IPTQ_OK) return rc0;
     if (a.M == 0) return IPTQ_OK;
-    // 128-wide tiles use the tensor core fully and re-read the activations less often, but rebuild the rounding
-    // constant per output (two more instructions); measured, they win for the plain epilogue and for the tabulated
-    // GELU epilogue at small K (ViT-Base FC1: 24 column tiles on 144 CTAs instead of 32 on 128), not for the
-    // polynomial GELU or the residual epilogue
-    const bool wide = a.N % 128 == 0 && (a.N % 96 != 0 || ((!a.gelu || a.gelu->table) && !a.residual && a.K <= 768));
-    return wide ? linear_launch_bn<128>(a, st) : linear_launch_bn<96>(a, st);
-}
 
-template <int BN>
-static int linear_launch_bn(const LinearArgs& a, cudaStream_t st)
-{
     GemmParams p;
     p.M = (int)a.M; p.N = a.N; p.K = a.K;
-    p.num_m_tiles = (int)((a.M + BM - 1) / BM);
-    p.num_n_tiles = (a.N + BN - 1) / BN;
+    p.n_ct = (a.N + CT - 1) / CT;
     p.bias = a.bias; p.mult = a.mult; p.shift = a.shift; p.out_zp = a.out_zp;
     p.qmin = -(1 << (a.out_bits - 1)); p.qmax = (1 << (a.out_bits - 1)) - 1;
     p.res_mult = p.res_rnd = p.res_shift = p.res_off = 0;
@@ -560,51 +518,64 @@ static int linear_launch_bn(const LinearArgs& a, cudaStream_t st)
     p.status = a.status;
     if (a.gelu) p.gelu = to_dev(*a.gelu);
     else { iptq_gelu_consts z{}; z.in_bits = 8; z.out.shift = 1; p.gelu = to_dev(z); }
+    const bool table = a.gelu && a.gelu->table;
+    p.gelu_tab = table ? a.gelu->table : nullptr;
 
-    CUtensorMap ma, mb, my, mr;
-    int rc;
-    {
-        const uint64_t dims[2] = {(uint64_t)a.K, (uint64_t)a.M};
-        const uint64_t str[1] = {(uint64_t)a.K};
-        const uint32_t box[2] = {BK, BM};
-        if ((rc = make_tensor_map_u8(&ma, a.x, 2, dims, str, box, 128)) != IPTQ_OK) return rc;
+    // Tile width: the widest that fits beside a ring of at least three stages and is not mostly padding.  What
+    // bounds a tile is shared-memory bandwidth (128 bytes per clock): every operand byte is written once by the
+    // copy engine and read once by the tensor core, (16 KB + 128 TN) bytes per 128-byte block of K each way, so a
+    // wide tile, which amortises the weight tile, beat every narrower one that was measured, even where it leaves
+    // the last round of tiles half empty.
+    const int kblocks = (a.K + BK - 1) / BK;
+    const int sms = sm_count();
+    int best_tn = 0, smem_bytes = 0;
+    for (int TN : {256, 192, 128, 64}) {
+        GemmParams q = p;
+        int sb;
+        if (TN > 64 && a.M <= TN - 64) continue;              // a narrower tile covers all tokens
+        if (gemm_layout(q, TN, a.residual != nullptr, table, kblocks, &sb) < std::min(3, kblocks + 1)) continue;
+        best_tn = TN;
+        break;
     }
+    if (best_tn == 0) return IPTQ_ERR_SHAPE;
+    gemm_layout(p, best_tn, a.residual != nullptr, table, kblocks, &smem_bytes);
+    const int64_t n_tt = (a.M + p.TN - 1) / p.TN;
+    if ((int64_t)p.n_ct * n_tt > (int64_t)1 << 30) return IPTQ_ERR_SHAPE;
+    p.n_tt = (int)n_tt;
+    const int grid = (int)std::min<int64_t>((int64_t)p.n_ct * n_tt, sms);
+
+    CUtensorMap mw, mx, my, mr;
+    int rc;
     {
         const uint64_t dims[2] = {(uint64_t)a.K, (uint64_t)a.N};
         const uint64_t str[1] = {(uint64_t)a.K};
-        const uint32_t box[2] = {BK, BN};
-        if ((rc = make_tensor_map_u8(&mb, a.w, 2, dims, str, box, 128)) != IPTQ_OK) return rc;
+        const uint32_t box[2] = {BK, CT};
+        if ((rc = make_tensor_map_u8(&mw, a.w, 2, dims, str, box, 128)) != IPTQ_OK) return rc;
     }
     {
-        // output and residual: one [32 rows][COLS] block per epilogue warp, clipped at M and N by the copy engine
+        const uint64_t dims[2] = {(uint64_t)a.K, (uint64_t)a.M};
+        const uint64_t str[1] = {(uint64_t)a.K};
+        const uint32_t box[2] = {BK, (uint32_t)p.TN};
+        if ((rc = make_tensor_map_u8(&mx, a.x, 2, dims, str, box, 128)) != IPTQ_OK) return rc;
+    }
+    {
+        // output and residual: one [TN / 4 tokens][32 channels] block per epilogue warp, clipped at M and N by the copy engine
         const uint64_t dims[2] = {(uint64_t)a.N, (uint64_t)a.M};
         const uint64_t str[1] = {(uint64_t)a.N};
-        const uint32_t box[2] = {COLS, 32};
-        if ((rc = make_tensor_map_u8(&my, a.y, 2, dims, str, box, 32)) != IPTQ_OK) return rc;
-        if ((rc = make_tensor_map_u8(&mr, a.residual ? a.residual : a.y, 2, dims, str, box, 32)) != IPTQ_OK) return rc;
+        const uint32_t box[2] = {32, (uint32_t)(p.TN / 4)};
+        if ((rc = make_tensor_map_u8(&my, a.y, 2, dims, str, box, 0)) != IPTQ_OK) return rc;
+        if ((rc = make_tensor_map_u8(&mr, a.residual ? a.residual : a.y, 2, dims, str, box, 0)) != IPTQ_OK) return rc;
     }
-    p.gelu_tab = a.gelu ? a.gelu->table : nullptr;
-    if (a.gelu && a.gelu->table) {
-        if (!aligned16(a.gelu->table)) return IPTQ_ERR_ALIGN;
-        return launch_gemm<BN, EPI_GELU, 0, true, true>(ma, mb, my, mr, p, st);    // the variant is in the table
-    }
+    if (table) return launch_gemm<EPI_GELU_TAB, 0>(mw, mx, my, mr, p, grid, smem_bytes, st);   // the variant is in the table
     if (a.gelu) {
-        const bool sat8 = a.gelu->out.qmin == -128 && a.gelu->out.qmax == 127;
-#define IPTQ_GEMM_GELU(V) (sat8 ? launch_gemm<BN, EPI_GELU, V, true>(ma, mb, my, mr, p, st) \
-                                : launch_gemm<BN, EPI_GELU, V, false>(ma, mb, my, mr, p, st))
         switch (a.gelu->variant) {
-            case IPTQ_GELU_POLY4: return IPTQ_GEMM_GELU(IPTQ_GELU_POLY4);
-            case IPTQ_GELU_POLY2: return IPTQ_GEMM_GELU(IPTQ_GELU_POLY2);
-            default: return IPTQ_GEMM_GELU(IPTQ_GELU_SHIFT);
+            case IPTQ_GELU_POLY4: return launch_gemm<EPI_GELU, IPTQ_GELU_POLY4>(mw, mx, my, mr, p, grid, smem_bytes, st);
+            case IPTQ_GELU_POLY2: return launch_gemm<EPI_GELU, IPTQ_GELU_POLY2>(mw, mx, my, mr, p, grid, smem_bytes, st);
+            default: return launch_gemm<EPI_GELU, IPTQ_GELU_SHIFT>(mw, mx, my, mr, p, grid, smem_bytes, st);
         }
-#undef IPTQ_GEMM_GELU
     }
-    if (a.out_bits != 8) {
-        if (a.residual) return launch_gemm<BN, EPI_RESIDUAL, 0, false>(ma, mb, my, mr, p, st);
-        return launch_gemm<BN, EPI_REQUANT, 0, false>(ma, mb, my, mr, p, st);
-    }
-    if (a.residual) return launch_gemm<BN, EPI_RESIDUAL, 0, true>(ma, mb, my, mr, p, st);
-    return launch_gemm<BN, EPI_REQUANT, 0, true>(ma, mb, my, mr, p, st);
+    if (a.residual) return launch_gemm<EPI_RESIDUAL, 0>(mw, mx, my, mr, p, grid, smem_bytes, st);
+    return launch_gemm<EPI_REQUANT, 0>(mw, mx, my, mr, p, grid, smem_bytes, st);
 }
 
 static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }

@@ -74,10 +74,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, CtaCon
                                           int where)
 {
     uint64_t t0 = 0;
-    for (uint32_t spin = 0; spin < kWaitSpins; ++spin) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 15u) == 15u && ctl->abort) return false;
-        if ((spin & 1023u) == 1023u) {
+    // 16 tries in a row cost nothing but the tries; the abort flag and the clock are looked at between such runs
+    for (uint32_t run = 0; run < kWaitSpins / 16; ++run) {
+#pragma unroll 1
+        for (int i = 0; i < 16; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (ctl->abort) return false;
+        if ((run & 63u) == 63u) {
             const uint64_t t = global_timer_ns();
             if (t0 == 0) t0 = t;
             else if (t - t0 > kWaitNs) break;
@@ -92,7 +95,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, CtaCon
     return false;
 }
 
-// ---------------------------------------------------------------- TMA (no multicast anywhere)
+// ---------------------------------------------------------------- TMA tile copies, one CTA per copy
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");

@@ -227,6 +227,39 @@ def test_attention_parity(api, orc, variant, B, H, N, dh, use_bias, use_mask):
     ws.check()
     assert len(np.unique(want)) > 10 or N == 1
     assert (got == want).all(), _mismatch(got, want)
+    if use_bias and N <= 64:
+        # the same call with the bias laid out once at load time (what an encoder block of a window model does)
+        bias_d = _cu(bias)
+        bias_t = api.attention_bias_prepare(bias_d)
+        assert bias_t is not None
+        got = api.attention_block(_cu(q), _cu(k), _cu(v), sa, ra, ws, bias_d, _cu(mask_id), bias_t=bias_t).cpu().numpy()
+        ws.check()
+        assert (got == want).all(), _mismatch(got, want)
+
+
+@pytest.mark.parametrize("variant", [0, 2, 3])
+@pytest.mark.parametrize("B,H,N,dh,use_mask,table", [(2, 2, 197, 64, False, True), (3, 1, 49, 32, True, True),
+                                                      (2, 2, 80, 32, True, False), (1, 3, 130, 64, True, True)])
+def test_attention_scores_at_the_bottom_of_the_range(api, orc, variant, B, H, N, dh, use_mask, table):
+    """Biased scores close to -2^30 in every row (the lowest the contract admits): padding columns and masked pairs
+    must still contribute exactly nothing, with the exponential from the table and evaluated."""
+    rng = np.random.default_rng(N + variant)
+    q, k, v = (np.clip(np.round(rng.normal(0, 40, size=(B, H, N, dh))), -128, 127).astype(np.int8) for _ in range(3))
+    S = 3.0 / (1600.0 * np.sqrt(dh))
+    # |q.k| <= 128 * 128 * 64 = 2^20: the bias puts every score within 2^21 + 2^16 of -2^30
+    bias = (-(1 << 30) + (1 << 21) + rng.integers(0, 1 << 16, size=(H, N, N))).astype(np.int32)
+    mask_id = rng.integers(0, 3, size=(B, N)).astype(np.uint8) if use_mask else None
+    bits = 4 if variant == 3 else 8
+    ratio = 0.011 / 256 if variant == 3 else 0.011
+    so, sa = orc.softmax_prepare(S, N, bits, variant), api.softmax_prepare(S, N, bits, variant)
+    keep = api.softmax_table(sa) if table else None
+    ro, ra = orc.requant_prepare(ratio, zp=1), api.requant_prepare(ratio, zp=1)
+    want = orc.attention_block(q, k, v, so, ro, bias, mask_id)
+    ws = api.Workspace(api.attention_workspace_bytes(B, H, N, dh))
+    got = api.attention_block(_cu(q), _cu(k), _cu(v), sa, ra, ws, _cu(bias), _cu(mask_id)).cpu().numpy()
+    ws.check()
+    assert (got == want).all(), _mismatch(got, want)
+    del keep
 
 
 def _oracle_block(orc, spec, table):

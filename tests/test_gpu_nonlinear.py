@@ -53,7 +53,7 @@ def test_softmax_parity(api, orc, variant, rows, n, scale):
     assert (got == want).all()
 
 
-@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("variant", [0, 1, 2, 3])
 @pytest.mark.parametrize("scale", [synth.SOFTMAX_SCALE_ACC, synth.SOFTMAX_SCALE_8BIT])
 @pytest.mark.parametrize("rows,n,use_table", [(6001, 197, True), (86017, 197, False), (86017, 197, True),
                                               (40003, 49, True), (9000, 208, True)])
@@ -65,11 +65,14 @@ def test_softmax_tabulated_parity(api, orc, variant, scale, rows, n, use_table):
     s0[7] = -(1 << 30) + 1
     s0[7, n // 2] = (1 << 30) - 1                  # largest admissible distance to the row maximum
     s0[8] = 12345                                  # all-equal row
+    s0[9] = -(1 << 30) + 3001                      # every entry at the bottom of the admissible range (bias included)
+    s0[10] = -(1 << 30) + 3001 + np.arange(n) * 7
     reps = (rows + base - 1) // base
     s = np.ascontiguousarray(np.tile(s0, (reps, 1))[:rows])
     bias = np.random.default_rng(5).integers(-3000, 3000, size=(3, n)).astype(np.int32)
-    co = orc.softmax_prepare(scale, n, 8, variant)
-    ca = api.softmax_prepare(scale, n, 8, variant)
+    bits = 4 if variant == 3 else 8
+    co = orc.softmax_prepare(scale, n, bits, variant)
+    ca = api.softmax_prepare(scale, n, bits, variant)
     keep = api.softmax_table(ca) if use_table else None
     assert (keep is not None) == use_table and bool(ca.table) == use_table
     want0 = orc.softmax(s0, co)
@@ -82,27 +85,28 @@ def test_softmax_tabulated_parity(api, orc, variant, scale, rows, n, use_table):
     assert (got_b[sub] == want_b).all()
 
 
-@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("variant", [0, 1, 2, 3])
 @pytest.mark.parametrize("scale,n", [(synth.SOFTMAX_SCALE_ACC, 197), (synth.SOFTMAX_SCALE_8BIT, 197), (1.0 / 700, 49)])
 def test_softmax_table_contents(api, orc, variant, scale, n):
     """The device table holds the oracle's exponential for every tabulated distance, and the oracle's
     exponential is 0 at every distance the table leaves out (up to the clamp of Eq. (6))."""
-    co = orc.softmax_prepare(scale, n, 8, variant)
-    ca = api.softmax_prepare(scale, n, 8, variant)
+    bits = 4 if variant == 3 else 8
+    co = orc.softmax_prepare(scale, n, bits, variant)
+    ca = api.softmax_prepare(scale, n, bits, variant)
     t = api.softmax_table(ca)
     assert t is not None and 0 < ca.table_n < api.SOFTMAX_TABLE_MAX
     tab = t.cpu().numpy().view(np.uint16)
     want = np.array([orc.softmax_exp(d, co) for d in range(ca.table_n)])
     assert (tab[:ca.table_n] == want).all()
     assert tab[ca.table_n] == 0
-    assert tab[0] == co.x0 << co.nsh
+    assert tab[0] == (co.x0 << co.nsh if variant < 2 else orc.softmax_exp(0, co))
     for d in list(range(ca.table_n, min(co.dcap, ca.table_n + 5000))) + list(range(ca.table_n, co.dcap + 1, 97)) + [co.dcap]:
         assert orc.softmax_exp(d, co) == 0, d
 
 
 def test_softmax_table_absent(api):
     import torch
-    c = api.softmax_prepare(synth.SOFTMAX_SCALE_ACC, 197, 8, 2)       # polynomial exponential: no table
+    c = api.softmax_prepare(1.0 / 8000.5, 49, 8, 2)                   # polynomial exponential, table too long
     assert api.softmax_table(c) is None and not c.table and c.table_n == 0
     c = api.softmax_prepare(1.0 / ((1 << 20) - 2.5), 49)               # x0 too large for a shared-memory table
     assert api.softmax_table(c) is None and not c.table
@@ -133,6 +137,33 @@ def test_softmax_log2_parity(api, orc, rows, n, scale):
     with pytest.raises(api.IptqError) as e:
         api.softmax_prepare(scale, n, 8, api.SM_LOG2)
     assert e.value.status == api.ERR_BITS
+
+
+@pytest.mark.parametrize("n", [197, 49, 1000, 1])
+@pytest.mark.parametrize("variant", [0, 1, 2, 3])
+def test_softmax_rows_at_the_bottom_of_the_range(api, orc, variant, n):
+    """Rows whose every entry sits at -2^30 + 1 (the lowest admissible score), with and without a bias: lanes past
+    the row end must contribute nothing although the row maximum is as low as a score can be.  Small inputs take
+    the evaluated kernel, large ones the tabulated kernel (table built per CTA and copied from device memory)."""
+    lo = -(1 << 30) + 1
+    bits = 4 if variant == 3 else 8
+    for scale in (synth.SOFTMAX_SCALE_ACC, synth.SOFTMAX_SCALE_8BIT):
+        co = orc.softmax_prepare(scale, n, bits, variant)
+        ca = api.softmax_prepare(scale, n, bits, variant)
+        block = np.full((64, n), lo, dtype=np.int32)
+        block[1::2] += np.random.default_rng(n).integers(0, 5000, size=(32, n)).astype(np.int32)
+        bias = np.random.default_rng(2).integers(0, 4000, size=(4, n)).astype(np.int32)
+        want, want_b = orc.softmax(block, co), orc.softmax(block, co, bias=bias, bias_period=4)
+        assert (api.softmax(_cu(block), ca).cpu().numpy() == want).all()
+        assert (api.softmax(_cu(block), ca, bias=_cu(bias)).cpu().numpy() == want_b).all()
+        if n <= 256:
+            reps = ((17 << 20) // (64 * n)) + 1                     # past the size where every CTA builds the table
+            big = _cu(np.tile(block, (reps, 1)))
+            assert (api.softmax(big, ca).cpu().numpy() == np.tile(want, (reps, 1))).all()
+            keep = api.softmax_table(ca)
+            assert (api.softmax(big, ca).cpu().numpy() == np.tile(want, (reps, 1))).all()
+            assert (api.softmax(big, ca, bias=_cu(bias)).cpu().numpy() == np.tile(want_b, (reps, 1))).all()
+            del keep
 
 
 def test_softmax_edge_rows_and_bias(api, orc):
