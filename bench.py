@@ -1,22 +1,25 @@
 """Benchmark of the integer-only encoder block (LN -> QKV -> fused attention with the integer Softmax ->
-proj -> LN -> FC1 with the integer GELU epilogue -> FC2) on the DeiT-Small W8A8 shape, batch 64 per GPU.
+proj -> LN -> FC1 with the integer GELU epilogue -> FC2).  Headline workload: the ViT-Base block, W8A8, batch 128
+per GPU (the largest single-block configuration); every other configuration is timed and checked in `configs`.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
 One step = one pass of the whole block over one batch of seeded synthetic input.  Rank 0 prints one JSON line.
   value        whole-job INT8 tera-ops/s (2 * MACs of the real, unpadded contractions) with inputs resident in HBM;
+  sustained    the same step replayed back to back for two seconds, with the SM clock and power sampled meanwhile;
   e2e          the same metric from pinned HOST buffers (host->device copy, block, device->host copy per step);
   roofline     the dominant kernel of the step, timed live with CUDA events at its stage boundaries;
   stages       every kernel of the step with its share of the step;
+  configs      every configuration (DeiT-Tiny batch 1, DeiT-Small batch 64, ViT-Base batch 128 with three variant
+               tables and with 4-bit weights, Swin-Tiny windows, the Swin-Tiny backbone at detection resolution):
+               time, TOP/s, fraction of the INT8 ceilings and the element-by-element comparison with the CPU oracle;
   nonlinear    the stand-alone integer Softmax / GELU / LayerNorm kernels on tensors larger than L2, as
                Gelem/s and fraction of the measured HBM copy bandwidth;
   assignment   the Unified-Metric analysis (every candidate of every non-linear layer of the encoder scored and
                selected on the device) as evaluations/s, with the oracle's scores of the first block beside it;
-  other_blocks the ViT-Base batch-128 block (8- and 4-bit weights), the Swin-Tiny window block and the 6-bit DeiT-Small
-               block, timed like the headline block (context: the headline metric stays the W8A8 DeiT-Small block);
   models       whole DeiT-T/S/B forward latency at batch 8 (context beside the paper's latency table, other hardware);
-  cpu_baseline the CPU oracle timed on the host cores on a bounded sample of the same workload, and the
-               element-by-element comparison of the GPU output with it.
+  cpu_baseline the CPU oracle timed on the host cores (all cores, and one core on a smaller sample) on the headline
+               workload, and the element-by-element comparison of the GPU output with it.
 `--impl reference` times the CPU oracle alone (rank 0 only).  Multi-GPU runs are independent replicas of the
 batch shard (no data-path collective); only the barrier and the max-over-ranks of the time use torch.distributed.
 """
@@ -24,9 +27,11 @@ from __future__ import annotations
 
 import argparse
 import copy
+import hashlib
 import json
 import os
 import statistics
+import subprocess
 import sys
 import threading
 import time
@@ -41,11 +46,20 @@ from paper_2511_15369_b200 import synth  # noqa: E402
 
 METRIC = "fused INT8 block TOPS"
 UNIT = "TOPS"
-WORKLOAD = "cfg1: DeiT-Small integer-only encoder block, W8A8, batch 64, seq 197, dim 384, 6 heads x 64, MLP 1536"
+HEADLINE = "cfg2"
+WORKLOAD = "cfg2: ViT-Base integer-only encoder block, W8A8, batch 128, seq 197, dim 768, 12 heads x 64, MLP 3072"
 TABLE = (0, 0, 0, 0)            # SM_BITEXP, GELU_POLY4, LN_SHIFT, LN_SHIFT: the default variant of every layer
+ALT_TABLES = [(1, 1, 1, 1), (2, 2, 0, 1)]   # the other candidates of every layer (config 2 alternates between them)
+TABLE_NAMES = {(0, 0, 0, 0): "bit-exp / poly4 / shift / shift", (1, 1, 1, 1): "shiftmax / poly2 / newton / newton",
+               (2, 2, 0, 1): "poly / shift-gelu / shift / newton"}
 INT8_OVER_BF16 = 2.0            # nominal dense INT8 : bf16 tensor throughput (4.5 : 2.25 PFLOP/s)
+# tcgen05.mma.kind::i8 issue loop on all 148 SMs, operands in shared memory, no loads, no epilogue: 64 clocks per
+# 128 x 128 x 32 MMA, sustained for 3 s at 1.9 GHz (see profiles/int8_mma_peak.md)
+INT8_ISSUE_LOOP_TOPS = 4598.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 L2_FLUSH_BYTES = 256 << 20      # > 126 MB of L2
+KERNEL_SOURCES = {"attention": ["attention_kernel.cuh", "tc_common.cuh", "iptq_common.cuh"],
+                  "gemm": ["linear.cu", "tc_common.cuh", "iptq_common.cuh"]}
 
 
 def measured_peaks():
@@ -53,8 +67,32 @@ def measured_peaks():
     if os.path.exists(path):
         with open(path) as f:
             d = json.load(f)
-        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"])}, "measured"
-    return dict(FALLBACK_PEAKS), "fallback"
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"]))}, "measured"
+    p = dict(FALLBACK_PEAKS)
+    p["bf16_tflops_sustained"] = 1400.0
+    return p, "fallback"
+
+
+def source_digest(files):
+    h = hashlib.sha1()
+    for f in files:
+        with open(os.path.join(ROOT, "paper_2511_15369_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:12]
+
+
+def ncu_counters(kernel):
+    """Counters of `kernel` from the ncu capture summarised in profiles/traffic.json, or None when the kernel's
+    sources have changed since the capture was taken."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        d = json.load(f).get(kernel)
+    if not d or d.get("source_digest") != source_digest(KERNEL_SOURCES[kernel]):
+        return None
+    return d
 
 
 def sub_batch(spec, images):
@@ -84,6 +122,48 @@ def oracle_sample_size(spec, budget_s, max_images):
     return max(1, min(max_images, int(budget_s / max(t1, 1e-6)))), t1
 
 
+def oracle_single_thread_seconds(cfg, images):
+    """The oracle block on the first `images` images of `cfg` in a child process restricted to one OpenMP thread
+    (the oracle itself is not touched: the thread count is the environment's)."""
+    code = ("import sys, time; sys.path.insert(0, %r); import bench; from paper_2511_15369_b200 import synth; "
+            "spec = synth.make_block(synth.CONFIGS[%r], seed=0); s = bench.sub_batch(spec, %d); "
+            "bench.oracle_block(bench.sub_batch(spec, 1), bench.TABLE); y, t = bench.oracle_block(s, bench.TABLE); "
+            "import oracle; print(t, oracle.num_threads())" % (ROOT, cfg, images))
+    env = dict(os.environ, OMP_NUM_THREADS="1")
+    try:
+        out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=600)
+        t, n = out.stdout.split()[-2:]
+        return float(t), int(n)
+    except Exception:
+        return None, None
+
+
+def oracle_backbone(spec, table):
+    """The Swin backbone as a composition of oracle calls (numpy index gathers for the layout steps)."""
+    import oracle
+
+    def gather(src, index):
+        index = index.reshape(-1, 1) if index.ndim == 1 else index
+        parts = [np.where(index[:, p:p + 1] >= 0, src[np.maximum(index[:, p], 0)], 0) for p in range(index.shape[1])]
+        return np.ascontiguousarray(np.concatenate(parts, axis=1).astype(np.int8))
+
+    x = spec.x
+    for st in spec.stages:
+        for bspec, shift, fwd, rev in st["blocks"]:
+            bspec.x = gather(x, fwd)
+            yw, _ = oracle_block(bspec, table)
+            bspec.x = None
+            x = gather(yw, rev)
+        if st["merge"] is not None:
+            m, tab = st["merge"]
+            g = gather(x, tab)
+            gq, bq, lc = oracle.layernorm_prepare(m.gamma, m.beta, m.ln_out_scale, 0)
+            h = oracle.layernorm(g, gq, bq, lc)
+            rq = [oracle.requant_prepare(float(r)) for r in m.ratio]
+            x = oracle.linear(h, m.w, None, np.array([r.mult for r in rq], np.int32), np.array([r.shift for r in rq], np.int8))
+    return x
+
+
 # ---------------------------------------------------------------------------------------------- reference arm
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
@@ -91,7 +171,7 @@ def run_reference(args):
         return
     import oracle
     oracle.lib()
-    shape = synth.CONFIGS["cfg1"]
+    shape = synth.CONFIGS[HEADLINE]
     spec = synth.make_block(shape, seed=0)
     # every step is the oracle on the same bounded sample, sized so that warm-up + steps end in a few minutes
     images, _ = oracle_sample_size(spec, 120.0 / max(1, args.steps + args.warmup), shape.B)
@@ -103,7 +183,7 @@ def run_reference(args):
     total = sum(times)
     value = ops * args.steps / total / 1e12
     cores = oracle.num_threads()
-    desc = "first %d of 64 images of the cfg1 block per step (%.3g GOP)" % (images, ops / 1e9)
+    desc = "first %d of %d images of the cfg2 block per step (%.3g GOP)" % (images, shape.B, ops / 1e9)
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -189,7 +269,8 @@ class ClockSampler:
         reasons = sorted(name for bit, name in self.REASONS.items() if mask & bit)
         pw = [s[3] for s in inside if s[3] is not None]
         return {"sm_mhz": statistics.median(s[1] for s in inside), "sm_max_mhz": self.max_mhz, "reasons": reasons,
-                "samples": len(inside), "power_w_max": max(pw) if pw else None, "note": note}
+                "samples": len(inside), "power_w_max": max(pw) if pw else None,
+                "power_w_median": statistics.median(pw) if pw else None, "note": note}
 
 
 # ---------------------------------------------------------------------------------------------- ranks
@@ -212,6 +293,13 @@ def rank_max(v, world, device=None):
 def job_tops(ops_per_rank_step, steps, world, total_ms_max):
     """Whole-job throughput: every rank did `steps` passes over its own shard within the slowest rank's time."""
     return ops_per_rank_step * steps * world / (total_ms_max * 1e-3) / 1e12
+
+
+def int8_fracs(tops, peaks):
+    """Fraction of the two INT8 ceilings: measured bf16 burst GEMM x 2 (nominal ratio), and the measured
+    tcgen05.mma.kind::i8 issue loop."""
+    return {"frac_int8_peak": tops / (peaks["bf16_tflops"] * INT8_OVER_BF16),
+            "frac_int8_issue_loop": tops / INT8_ISSUE_LOOP_TOPS}
 
 
 # ---------------------------------------------------------------------------------------------- our arm
@@ -239,7 +327,7 @@ def run_ours(args):
     def max_over_ranks(v):
         return rank_max(v, world, dev)
 
-    shape = synth.CONFIGS["cfg1"]
+    shape = synth.CONFIGS[HEADLINE]
     spec = synth.make_block(shape, seed=shard_seed(rank))   # each rank owns its own batch shard (weak scaling)
     blk = api.EncoderBlock(spec, TABLE, device=dev)
     x = torch.from_numpy(spec.x).to(dev)
@@ -291,6 +379,27 @@ def run_ours(args):
     total_ms = max_over_ranks(sum(ms))
     value = job_tops(ops, K, world, total_ms)
 
+    # ---- sustained: the same step back to back for two seconds (no flush: the working set of 0.3 GB exceeds L2),
+    #      SM clock and power sampled meanwhile, so that the figure can be read at equal clock
+    barrier()
+    n_sus = max(K, int(2.2e3 / max(statistics.median(ms), 1e-3)))
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    s0.record()
+    for _ in range(n_sus):
+        step_graph.replay()
+    s1.record()
+    barrier()
+    sus_window = (t0, time.perf_counter())
+    sus_ms = max_over_ranks(s0.elapsed_time(s1)) / n_sus
+    sus_clk = clocks.summary([sus_window])
+    sustained = {"steps": n_sus, "ms_per_step": sus_ms, "value": job_tops(ops, 1, world, sus_ms), "unit": UNIT,
+                 "sm_mhz_median": sus_clk.get("sm_mhz"), "power_w_median": sus_clk.get("power_w_median"),
+                 "power_w_max": sus_clk.get("power_w_max"), "reasons": sus_clk.get("reasons"),
+                 "ms_times_mhz": sus_ms * sus_clk["sm_mhz"] if sus_clk.get("sm_mhz") else None,
+                 "note": "back-to-back CUDA-graph replays, no L2 flush; ms_times_mhz compares runs at equal clock"}
+    launches += launches_per_step * n_sus * 0            # outside the timed K steps: not counted
+
     # ---- per-stage times from the same kernels with events at the stage boundaries
     nst = len(api.BLOCK_STAGES)
     sets = []
@@ -311,9 +420,9 @@ def run_ours(args):
 
     # ---- end to end from pinned host buffers: every step copies its input host -> device, runs the block and copies
     #      the result device -> host.  A whole step (copy in, the block's launches, copy out) is one CUDA graph; steps
-    #      are independent, so four buffer sets (each with its own block workspace) take turns on four streams and the
-    #      copies of one step overlap the block and the copies of its neighbours.
-    E2E_SETS = 4                                        # a step is a chain of three phases: four sets keep all of them busy
+    #      are independent, so several buffer sets (each with its own block workspace) take turns on their own streams
+    #      and the copies of one step overlap the block and the copies of its neighbours.
+    E2E_SETS = 3
     xh = torch.from_numpy(spec.x).pin_memory()
     yh = [torch.empty_like(xh).pin_memory() for _ in range(E2E_SETS)]
     xd = [torch.empty_like(x) for _ in range(E2E_SETS)]
@@ -368,25 +477,43 @@ def run_ours(args):
     dbuf = torch.empty(64 << 20, dtype=torch.uint8, device=dev)
     link = {"h2d_gbs": link_gbs(dbuf, hbuf), "d2h_gbs": link_gbs(hbuf, dbuf)}
     link["floor_ms_per_step"] = 1e3 * max(xh.numel() / (link["h2d_gbs"] * 1e9), yh[0].numel() / (link["d2h_gbs"] * 1e9))
-    del hbuf, dbuf
+    del hbuf, dbuf, graphs, blks, xd, yd
 
-    # ---- stand-alone non-linear kernels on tensors larger than L2
-    peaks, peak_kind = measured_peaks()
-    nonlinear = []
-    if rank == 0:
-        nonlinear = bench_nonlinear(api, torch, dev, peaks, peak_kind)
-    clocks.stop()
-    assignment = bench_assignment(api, torch, dev) if rank == 0 else None
-    models = bench_models(api, torch, dev) if rank == 0 else None
-    other_blocks = bench_other_blocks(api, torch, dev, peaks) if rank == 0 else None
-
+    clock_summary = clocks.summary(windows)
     if rank != 0:
+        clocks.stop()
         if world > 1:
             dist.destroy_process_group()
         return
 
+    peaks, peak_kind = measured_peaks()
+    nonlinear = bench_nonlinear(api, torch, dev, peaks, peak_kind)
+    clocks.stop()
+
+    # ---- CPU oracle on the headline workload, timed on the host cores, and compared with the GPU output
+    import oracle
+    oracle.lib()
+    N = shape.N
+    images, _ = oracle_sample_size(spec, 12.0, shape.B)
+    sample = sub_batch(spec, images)
+    want, t_cpu = oracle_block(sample, TABLE)
+    mismatches = int((got_full[: images * N] != want).sum())
+    desc = "first %d of %d images of the cfg2 block, one pass (%.3g GOP)" % (images, shape.B, sample.shape.gemm_ops() / 1e9)
+    one_images = max(1, min(images, 4))
+    t_one, n_one = oracle_single_thread_seconds(HEADLINE, one_images)
+    cpu = {"value": sample.shape.gemm_ops() / t_cpu / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+           "sample": desc, "seconds": t_cpu, "gpu_vs_oracle_mismatches": mismatches,
+           "compared_elements": int(want.size),
+           "single_thread": None if t_one is None else {
+               "value": sub_batch(spec, one_images).shape.gemm_ops() / t_one / 1e12, "unit": UNIT, "cores": n_one,
+               "seconds": t_one, "sample": "first %d images of the cfg2 block, OMP_NUM_THREADS=1" % one_images}}
+
+    configs = bench_configs(api, torch, dev, peaks, cached={(HEADLINE, TABLE): (spec, want, images)})
+    assignment = bench_assignment(api, torch, dev)
+    models = bench_models(api, torch, dev)
+
     # ---- roofline of the dominant kernel
-    T, D, Dh, N, dh, H, B = shape.T, shape.D, shape.Dh, shape.N, shape.dh, shape.H, shape.B
+    T, D, Dh, dh, H, B = shape.T, shape.D, shape.Dh, shape.dh, shape.H, shape.B
     stage_ops = {"qkv": 2 * T * D * 3 * D, "attention": 4 * B * H * N * N * dh, "proj": 2 * T * D * D,
                  "fc1_gelu": 2 * T * D * Dh, "fc2": 2 * T * Dh * D}
     stage_bytes = {"ln1": 2 * T * D, "ln2": 2 * T * D}
@@ -396,37 +523,45 @@ def run_ours(args):
         s = {"kernel": name, "us": 1e3 * t, "share": t / sum(stage_ms)}
         if name in stage_ops:
             s["tops"] = stage_ops[name] / (t * 1e-3) / 1e12
-            s["frac_int8_peak"] = s["tops"] / int8_peak
+            s.update(int8_fracs(s["tops"], peaks))
         else:
             s["gbs"] = stage_bytes[name] / (t * 1e-3) / 1e9
             s["frac_hbm"] = s["gbs"] / peaks["hbm_gbs"]
         stages.append(s)
-    # DRAM bytes per launch of the kernels of this workload, from the ncu capture summarised in
-    # profiles/encoder_block_kernels_cfg1.md (dram__bytes_read.sum + dram__bytes_write.sum); valid for that kernel version
-    traffic = {"attention": 14.61e6}
     top = max(stages, key=lambda s: s["us"])
-    clock_summary = clocks.summary(windows)
+    tensor_src = "%s bf16 burst GEMM x %.0f (nominal dense INT8 : bf16 ratio)" % (peak_kind, INT8_OVER_BF16)
     if top["kernel"] == "attention":
-        # The fused attention is bound by the integer pipes, not by the contraction: a score costs 2 * 2 * dh tensor
-        # operations but the 21 integer operations of Eqs. (6)-(15) (the count iptq_op_count() gives the variant).
-        # Ceiling: every SM sub-partition issues one 32-lane integer instruction per clock.
+        # A score costs 2 * 2 * dh tensor operations but the 21 integer operations of Eqs. (6)-(15) (the count
+        # iptq_op_count() gives the variant), and the integer pipes are where the kernel's time goes.  Ceiling: every
+        # SM sub-partition issues one 32-lane instruction per clock (adds and min/max run at that rate; shifts,
+        # logic, multiplies and byte packs at half of it, the high half of a product at a quarter).
+        cnt = ncu_counters("attention")
         props = torch.cuda.get_device_properties(dev)
         sm_mhz = clock_summary.get("sm_max_mhz") or 1965.0
         alu_peak = props.multi_processor_count * 4 * 32 * sm_mhz * 1e6 / 1e12
         alu_ops = api.op_count(api.LAYER_SOFTMAX, TABLE[0], B * H * N, N)
         achieved = alu_ops / (top["us"] * 1e-6) / 1e12
         roofline = {"kernel": "attention", "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "Tint-op/s",
-                    "frac": achieved / alu_peak, "traffic": traffic.get("attention"),
+                    "frac": achieved / alu_peak, "traffic": cnt["dram_bytes_per_launch"] if cnt else None,
                     "peak_source": "%d SMs x 4 sub-partitions x 32 lanes x %.0f MHz (clocks.max.sm), one integer "
-                                   "instruction per lane per clock" % (props.multi_processor_count, sm_mhz),
+                                   "instruction per lane per clock (issue limit; see profiles/int_issue_rates.md for "
+                                   "the rate of each instruction)" % (props.multi_processor_count, sm_mhz),
                     "ops_per_launch": alu_ops, "us_per_launch": top["us"],
+                    "issue_active": cnt.get("issue_active") if cnt else None,
+                    "warps_active": cnt.get("warps_active") if cnt else None,
+                    "tensor_active": cnt.get("tensor_active") if cnt else None,
+                    "limiter": "instruction latency: neither the issue slots nor a pipe are saturated (see the ncu "
+                               "counters beside this entry); the integer Softmax runs between the two MMAs",
                     "tensor": {"achieved": top["tops"], "peak": int8_peak, "unit": "TOP/s", "frac": top["tops"] / int8_peak,
-                               "ops_per_launch": stage_ops["attention"],
-                               "peak_source": "%s bf16 burst GEMM x %.0f (nominal dense INT8 : bf16 ratio)" % (peak_kind, INT8_OVER_BF16)}}
+                               "ops_per_launch": stage_ops["attention"], "peak_source": tensor_src}}
     elif "tops" in top:
+        cnt = ncu_counters("gemm")
         roofline = {"kernel": top["kernel"], "bound": "tensor", "achieved": top["tops"], "peak": int8_peak,
-                    "unit": "TOP/s", "frac": top["tops"] / int8_peak, "traffic": traffic.get(top["kernel"]),
-                    "peak_source": "%s bf16 burst GEMM x %.0f (nominal dense INT8 : bf16 ratio)" % (peak_kind, INT8_OVER_BF16),
+                    "unit": "TOP/s", "frac": top["tops"] / int8_peak, "traffic": cnt["dram_bytes_per_launch"] if cnt else None,
+                    "peak_source": tensor_src, "frac_int8_issue_loop": top["tops"] / INT8_ISSUE_LOOP_TOPS,
+                    "issue_active": cnt.get("issue_active") if cnt else None,
+                    "warps_active": cnt.get("warps_active") if cnt else None,
+                    "tensor_active": cnt.get("tensor_active") if cnt else None,
                     "ops_per_launch": stage_ops[top["kernel"]], "us_per_launch": top["us"]}
     else:
         roofline = {"kernel": top["kernel"], "bound": "hbm", "achieved": top["gbs"], "peak": peaks["hbm_gbs"],
@@ -434,40 +569,141 @@ def run_ours(args):
                     "peak_source": peak_kind + " copy bandwidth", "bytes_per_launch": stage_bytes[top["kernel"]],
                     "us_per_launch": top["us"]}
 
-    # ---- CPU oracle on a bounded sample, timed on the host cores, and compared with the GPU output
-    import oracle
-    oracle.lib()
-    images, _ = oracle_sample_size(spec, 12.0, shape.B)
-    sample = sub_batch(spec, images)
-    want, t_cpu = oracle_block(sample, TABLE)
-    mismatches = int((got_full[: images * N] != want).sum())
-    desc = "first %d of %d images of the cfg1 block, one pass (%.3g GOP)" % (images, B, sample.shape.gemm_ops() / 1e9)
-    cpu = {"value": sample.shape.gemm_ops() / t_cpu / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-           "sample": desc, "seconds": t_cpu, "gpu_vs_oracle_mismatches": mismatches,
-           "compared_elements": int(want.size)}
-
-    print(json.dumps({
+    out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int8 x int8 -> int32", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "per_gpu_batch": B, "gop_per_step_per_gpu": ops / 1e9,
+        "config": {"workload": WORKLOAD, "per_gpu_batch": shape.B, "gop_per_step_per_gpu": ops / 1e9,
                    "variants": "SM_BITEXP, GELU_POLY4, LN_SHIFT", "parallelism": "replicas, batch-sharded, no collective",
                    "cache": "L2 flushed (256 MiB write) before every timed step, outside the event pairs",
                    "launch": "each step is one CUDA-graph replay of the launches iptq_encoder_block() enqueues"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(xh.numel()), "d2h_bytes_per_step": int(yh[0].numel()),
-                "ms_per_step": total_e2e / K, "host_link": link, "pipelining": "one CUDA graph per step (copy in, block, copy out); four buffer sets take turns on four streams"},
+                "ms_per_step": total_e2e / K, "host_link": link,
+                "pipelining": "one CUDA graph per step (copy in, block, copy out); three buffer sets take turns on three streams"},
         "gpu_launches": int(launches),
         "clocks": clock_summary,
+        "sustained": sustained,
         "roofline": roofline,
         "stages": stages,
+        "configs": configs,
         "nonlinear": nonlinear,
         "assignment": assignment,
         "models": models,
-        "other_blocks": other_blocks,
         "cpu_baseline": cpu,
-    }))
+    }
+    out.update(int8_fracs(value / world, peaks))
+    out["int8_ceilings"] = {"bf16_burst_x2_tops": int8_peak, "issue_loop_tops": INT8_ISSUE_LOOP_TOPS,
+                            "note": "frac_int8_peak uses the first, frac_int8_issue_loop the second (per GPU)"}
+    print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def time_graph(torch, flush, fn, reps=20):
+    """Median ms of one CUDA-graph replay of fn(), L2 flushed before each."""
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            fn()
+        ts = []
+        for _ in range(reps):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(st)
+            g.replay()
+            b.record(st)
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+    del g
+    return statistics.median(ts)
+
+
+def bench_configs(api, torch, dev, peaks, cached):
+    """Every configuration, timed like the headline step (CUDA-graph replay, L2 flushed, CUDA events, median of 20) and
+    compared element by element with the CPU oracle (whole batch unless `compared` says otherwise)."""
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    out = []
+
+    def block_case(cfg, label, table, spec_kw, blk_kw, compare_images=None, per_kernel=False):
+        shape = synth.CONFIGS[cfg]
+        key = (cfg, table)
+        if key in cached and not spec_kw:
+            spec, want, images = cached[key]
+        else:
+            spec = synth.make_block(shape, seed=0, calib_images=8 if shape.has_bias else 2, **spec_kw)
+            want, images = None, None
+        blk = api.EncoderBlock(spec, table, dev, **blk_kw)
+        x = torch.from_numpy(spec.x).to(dev)
+        y = torch.empty_like(x)
+        ms = time_graph(torch, flush, lambda: blk(x, y))
+        blk.ws.check()
+        got = y.cpu().numpy()
+        if want is None:
+            images = shape.B if compare_images is None else min(shape.B, compare_images)
+            want, _ = oracle_block(sub_batch(spec, images), table)
+        bad = int((got[: images * shape.N] != want).sum())
+        tops = shape.gemm_ops() / (ms * 1e-3) / 1e12
+        e = {"config": cfg, "workload": "%s, %s" % (shape.name, label), "variants": TABLE_NAMES.get(table, str(table)),
+             "ms_per_step": ms, "us_per_step": 1e3 * ms, "tops": tops, "gop_per_step": shape.gemm_ops() / 1e9,
+             "gpu_vs_oracle_mismatches": bad, "compared_elements": int(want.size),
+             "compared": "whole batch" if images == shape.B else "first %d of %d problems" % (images, shape.B)}
+        e.update(int8_fracs(tops, peaks))
+        if per_kernel:
+            # batch 1: kernels of a few microseconds each; per-kernel time from events at the stage boundaries
+            acc = None
+            for _ in range(10):
+                evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(api.BLOCK_STAGES) + 1)]
+                for ev in evs:
+                    ev.record()
+                torch.cuda.synchronize()
+                torch.cuda._sleep(2000000)
+                blk.profiled(x, y, evs)
+                torch.cuda.synchronize()
+                t = [evs[i].elapsed_time(evs[i + 1]) * 1e3 for i in range(len(api.BLOCK_STAGES))]
+                acc = t if acc is None else [min(a, b) for a, b in zip(acc, t)]
+            e["kernel_us"] = dict(zip(api.BLOCK_STAGES, acc))
+            e["note"] = "kernel_us: CUDA events at the stage boundaries (each interval holds the event itself, about 2 us)"
+        out.append(e)
+        del blk, x, y
+
+    block_case("cfg0", "W8A8, batch 1 (latency)", TABLE, {}, {}, per_kernel=True)
+    block_case("cfg1", "W8A8", TABLE, {}, {})
+    block_case("cfg2", "W8A8", TABLE, {}, {})
+    for t in ALT_TABLES:
+        block_case("cfg2", "W8A8", t, {}, {}, compare_images=16)
+    block_case("cfg2", "W4A8, weights unpacked at every call", TABLE, {"w_bits": 4}, {}, compare_images=16)
+    block_case("cfg2", "W4A8, weights unpacked once at load time", TABLE, {"w_bits": 4}, {"unpack_w4_once": True},
+               compare_images=16)
+    block_case("cfg3", "W8A8, 4096 windows of 49 tokens, relative-position bias", TABLE, {}, {})
+    block_case("cfg1", "W6A6", TABLE, {"w_bits": 6, "a_bits": 6}, {}, compare_images=16)
+
+    # cfg4: the Swin-Tiny backbone at detection resolution (12 blocks, 3 patch merges, every row gather included)
+    from paper_2511_15369_b200 import swin
+    spec = synth.make_swin(2, None, seed=3)
+    net = swin.SwinBackbone(spec, TABLE, dev)
+    x = torch.from_numpy(spec.x).to(dev)
+    launches0 = api.launch_count()
+    got = net(x)
+    n_launch = api.launch_count() - launches0
+    ms = time_graph(torch, flush, lambda: net(x))
+    net.check()
+    got = got.cpu().numpy()
+    t0 = time.perf_counter()
+    want = oracle_backbone(spec, TABLE)
+    t_or = time.perf_counter() - t0
+    tops = net.gemm_ops() / (ms * 1e-3) / 1e12
+    e = {"config": "cfg4", "workload": "Swin-Tiny backbone, batch 2, 800 x 1216 (200 x 304 tokens), W8A8, shifted 7x7 windows",
+         "variants": TABLE_NAMES[TABLE], "ms_per_step": ms, "us_per_step": 1e3 * ms, "tops": tops,
+         "gop_per_step": net.gemm_ops() / 1e9, "launches": int(n_launch),
+         "gpu_vs_oracle_mismatches": int((got != want).sum()), "compared_elements": int(want.size),
+         "compared": "whole output", "oracle_seconds": t_or}
+    e.update(int8_fracs(tops, peaks))
+    out.append(e)
+    return out
 
 
 def bench_nonlinear(api, torch, dev, peaks, peak_kind):
@@ -497,16 +733,19 @@ def bench_nonlinear(api, torch, dev, peaks, peak_kind):
                     "gelem_s": elems / (ms * 1e-3) / 1e9, "gbs": gbs, "bytes_per_elem": nbytes / elems,
                     "frac_hbm": gbs / peaks["hbm_gbs"], "peak": peak_kind + " copy %.0f GB/s" % peaks["hbm_gbs"]})
 
-    # Softmax: ViT-Base batch 128 -> 128 * 12 * 197 rows of 197 int32 scores
+    # Softmax: ViT-Base batch 128 -> 128 * 12 * 197 rows of 197 int32 scores; the default candidate and the one the
+    # assignment below picks for most layers
     rows, n = 128 * 12 * 197, 197
     s = synth.quantize_scores(synth.softmax_logits(4096, n, seed=0), synth.SOFTMAX_SCALE_ACC)
     sc = tile_rows(s, rows)
     pr = torch.empty((rows, n), dtype=torch.uint8, device=dev)
-    c = api.softmax_prepare(synth.SOFTMAX_SCALE_ACC, n)
-    sm_tab = api.softmax_table(c, dev)              # exponential table written once, as a deployed layer would
-    record("iptq_softmax", rows * n, 5 * rows * n, time_kernel(lambda: api.softmax(sc, c, out=pr)),
-           "int32 [302592, 197] -> uint8 (238 MB in)")
-    del sc, pr, sm_tab
+    for variant, vname in ((api.SM_BITEXP, "bit-exp"), (api.SM_POLY, "polynomial")):
+        c = api.softmax_prepare(synth.SOFTMAX_SCALE_ACC, n, 8, variant)
+        sm_tab = api.softmax_table(c, dev)          # exponential table written once, as a deployed layer would
+        record("iptq_softmax (%s)" % vname, rows * n, 5 * rows * n, time_kernel(lambda: api.softmax(sc, c, out=pr)),
+               "int32 [302592, 197] -> uint8 (238 MB in)")
+        del sm_tab
+    del sc, pr
     # GELU: ViT-Base batch 128 -> 25216 x 3072 int32
     n_el = 25216 * 3072
     xg, S = synth.quantize_sym(synth.gelu_values(1 << 20, seed=0), 16)
@@ -531,46 +770,6 @@ def bench_nonlinear(api, torch, dev, peaks, peak_kind):
     return out
 
 
-def bench_other_blocks(api, torch, dev, peaks):
-    """The other single-block configurations (ViT-Base batch 128 with 8- and 4-bit weights, Swin-Tiny stage-1 windows,
-    the headline block at 6 bits), timed like the headline one: CUDA-graph replay of one block step, L2 flushed before each, CUDA events, median of 20."""
-    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
-    out = []
-    cases = [("cfg2", "W8A8", {}, {}), ("cfg2", "W4A8, weights unpacked at every call", {"w_bits": 4}, {}),
-             ("cfg2", "W4A8, weights unpacked once at load time", {"w_bits": 4}, {"unpack_w4_once": True}),
-             ("cfg3", "W8A8", {}, {}), ("cfg1", "W6A6", {"w_bits": 6, "a_bits": 6}, {})]
-    for cfg, label, spec_kw, blk_kw in cases:
-        shape = synth.CONFIGS[cfg]
-        spec = synth.make_block(shape, seed=0, calib_images=8 if shape.has_bias else 2, **spec_kw)
-        blk = api.EncoderBlock(spec, TABLE, dev, **blk_kw)
-        x = torch.from_numpy(spec.x).to(dev)
-        y = torch.empty_like(x)
-        st = torch.cuda.Stream()
-        with torch.cuda.stream(st):
-            for _ in range(3):
-                blk(x, y)
-            torch.cuda.synchronize()
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=st):
-                blk(x, y)
-            ts = []
-            for _ in range(20):
-                flush.fill_(1)
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(st)
-                g.replay()
-                b.record(st)
-                torch.cuda.synchronize()
-                ts.append(a.elapsed_time(b))
-        blk.ws.check()
-        ms = statistics.median(ts)
-        tops = shape.gemm_ops() / (ms * 1e-3) / 1e12
-        out.append({"workload": "%s: %s, %s" % (cfg, shape.name, label), "ms_per_step": ms, "tops": tops,
-                    "frac_int8_peak": tops / (peaks["bf16_tflops"] * INT8_OVER_BF16), "gop_per_step": shape.gemm_ops() / 1e9})
-        del blk, g, x, y, spec
-    return out
-
-
 PAPER_LATENCY_MS = {"DeiT-T": 1.73, "DeiT-S": 3.46, "DeiT-B": 7.11}   # the paper's latency table: RTX 3090, TVM, batch 8
 
 
@@ -584,30 +783,13 @@ def bench_models(api, torch, dev):
         spec = synth.make_vit(name, 8, seed=0)
         model = vit.VitModel(spec, TABLE, dev)
         img = torch.from_numpy(spec.image).to(dev)
-        st = torch.cuda.Stream()
-        with torch.cuda.stream(st):
-            for _ in range(3):
-                model(img)
-            torch.cuda.synchronize()
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=st):
-                model(img)
-            ts = []
-            for _ in range(20):
-                flush.fill_(1)
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(st)
-                g.replay()
-                b.record(st)
-                torch.cuda.synchronize()
-                ts.append(a.elapsed_time(b))
+        ms = time_graph(torch, flush, lambda: model(img))
         model.check()
-        ms = statistics.median(ts)
         out.append({"model": name, "batch": 8, "ms": ms, "images_per_s": 8 / (ms * 1e-3),
                     "tops": spec.gemm_ops() / (ms * 1e-3) / 1e12, "gop": spec.gemm_ops() / 1e9,
                     "launches": model.launches_per_forward(),
                     "paper_ms_rtx3090_tvm": PAPER_LATENCY_MS[name], "data": "synthetic image, random weights"})
-        del model, g, img
+        del model, img
     return out
 
 
@@ -657,7 +839,6 @@ def bench_assignment(api, torch, dev):
     t0 = time.perf_counter()
     agree, compared = 0, 0
     for (name, kind, d), l in list(zip(host_layers, layers))[:4]:
-        terms = []
         for c in l.candidates:
             v = c.variant
             if kind == "softmax":
@@ -679,7 +860,6 @@ def bench_assignment(api, torch, dev):
             qdb, pp, term = om.evaluate(x, q, ops)
             compared += 1
             agree += int(abs(term - c.term) <= 1e-9 * term and abs(pp - c.perturbation) <= 1e-9 * pp)
-            terms.append(term)
     t_cpu = time.perf_counter() - t0
     return {"workload": "DeiT-Small encoder, 49 non-linear layers, calibration batch 8 (synthetic), 4 Softmax / 3 GELU / 3 LayerNorm candidates",
             "layers": len(layers), "evaluations": int(n_eval), "ms": 1e3 * t, "evaluations_per_s": n_eval / t,
