@@ -404,6 +404,17 @@ int iptq_metric_select(const double* terms /*host*/, int n);
  * abandoned a bounded wait, IPTQ_ERR_CUDA if the stream reports an error, else IPTQ_OK. */
 int iptq_workspace_init(void* ws, size_t ws_bytes, iptq_stream_t stream);
 int iptq_check(iptq_stream_t stream, const void* ws);
+/* Every wait inside the tensor-core kernels (on a copy, on the tensor core, on another warp) is bounded: after the
+ * limit it records itself in the status block -- flag, id of the wait, block index, at int32 offsets 0, 1, 2 -- makes
+ * its CTA drain and return, and iptq_check() reports IPTQ_ERR_TIMEOUT.  The limit is 2 s unless the workspace
+ * carries its own: iptq_workspace_set_wait_limit() stores one in the status block (microseconds; 0 = default;
+ * enqueued on the stream; iptq_workspace_init() clears it again).  The host pointer is read during the call.
+ * iptq_selftest_wait_timeout() (no counterpart in the paper: a diagnostic) launches one warp that waits on a
+ * barrier nothing arrives at, so that the give-up path can be observed on a healthy device: afterwards iptq_check()
+ * returns IPTQ_ERR_TIMEOUT with wait id 99 and block 0, the kernel has returned, and the workspace is usable
+ * again after iptq_workspace_init(). */
+int iptq_workspace_set_wait_limit(void* ws, size_t ws_bytes, int32_t microseconds, iptq_stream_t stream);
+int iptq_selftest_wait_timeout(void* ws, size_t ws_bytes, iptq_stream_t stream);
 const char* iptq_strerror(int status);
 /* Number of kernels the library has launched so far in this process (for launch accounting). */
 int64_t iptq_launch_count(void);

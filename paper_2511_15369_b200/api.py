@@ -141,6 +141,8 @@ def lib():
                                                   C.POINTER(C.c_void_p), C.c_int]
         L.iptq_workspace_init.argtypes = [_vp, C.c_size_t, _vp]
         L.iptq_check.argtypes = [_vp, _vp]
+        L.iptq_workspace_set_wait_limit.argtypes = [_vp, C.c_size_t, C.c_int32, _vp]
+        L.iptq_selftest_wait_timeout.argtypes = [_vp, C.c_size_t, _vp]
         L.iptq_metric_softmax.argtypes = [_vp, _vp, C.c_int64, C.c_int, C.c_double, C.c_int, _vp, _vp, _vp]
         L.iptq_metric_gelu.argtypes = [_vp, _vp, C.c_int64, C.c_double, C.c_double, C.c_int, _vp, _vp, _vp]
         L.iptq_metric_layernorm.argtypes = [_vp, _vp, C.c_int64, C.c_int, _vp, _vp, _vp, C.c_double, C.c_int, _vp,
@@ -162,7 +164,7 @@ def exported_symbols():
             "iptq_gelu_prepare", "iptq_gelu", "iptq_gelu_table", "iptq_gelu_fit", "iptq_gelu_prepare_coeffs", "iptq_layernorm_prepare", "iptq_layernorm",
             "iptq_unpack_int4", "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_bits", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_patchify", "iptq_attention_workspace_bytes", "iptq_attention_bias_bytes", "iptq_attention_bias_prepare", "iptq_attention_block",
             "iptq_mlp_workspace_bytes", "iptq_mlp_block", "iptq_encoder_block_workspace_bytes",
-            "iptq_encoder_block", "iptq_encoder_block_profiled", "iptq_workspace_init", "iptq_check", "iptq_strerror", "iptq_launch_count",
+            "iptq_encoder_block", "iptq_encoder_block_profiled", "iptq_workspace_init", "iptq_check", "iptq_workspace_set_wait_limit", "iptq_selftest_wait_timeout", "iptq_strerror", "iptq_launch_count",
             "iptq_metric_softmax", "iptq_metric_gelu", "iptq_metric_layernorm", "iptq_softplus", "iptq_sqnr_db",
             "iptq_metric_term", "iptq_op_count", "iptq_metric_select"]
 
@@ -248,6 +250,20 @@ class Workspace:
 
     def check(self):
         _chk(lib().iptq_check(_stream(), self.ptr), "iptq_check")
+
+    def reset(self):
+        """Clears the status block (after a reported time-out the workspace is usable again)."""
+        _chk(lib().iptq_workspace_init(self.ptr, self.nbytes, _stream()), "iptq_workspace_init")
+
+    def set_wait_limit(self, microseconds: int):
+        _chk(lib().iptq_workspace_set_wait_limit(self.ptr, self.nbytes, int(microseconds), _stream()),
+             "iptq_workspace_set_wait_limit")
+
+    def status_words(self):
+        """The first int32 fields of the status block: (flag, wait id, block, work_next, work_done, wait limit)."""
+        torch.cuda.synchronize()
+        off = self.ptr - self.buf.data_ptr()
+        return self.buf[off:off + 24].cpu().view(torch.int32).tolist()
 
 
 # ------------------------------------------------------------------ device entry points

@@ -24,7 +24,8 @@ struct StatusBlock {
     int32_t block;            // blockIdx.x of the CTA that gave up
     int32_t work_next;        // next work item of a kernel that hands out items dynamically (0 between launches)
     int32_t work_done;        // CTAs of that kernel that have finished (0 between launches)
-    int32_t pad[59];
+    int32_t wait_limit_us;    // limit of a bounded device-side wait in microseconds; 0 = the default (2 s)
+    int32_t pad[58];
 };
 static_assert(sizeof(StatusBlock) == 256, "status block is 256 bytes");
 constexpr size_t kStatusBytes = 256;

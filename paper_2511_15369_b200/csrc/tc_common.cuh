@@ -59,6 +59,7 @@ struct CtaControl {
 
 // A wait gives up after kWaitNs of wall time (read from the global timer every 1024 tries), far above any legitimate
 // wait, which is bounded by the previous kernel's run time; kWaitSpins bounds it as well should the timer stand still.
+// A workspace may carry its own limit in the status block (iptq_workspace_set_wait_limit).
 constexpr uint64_t kWaitNs = 2000000000ull;
 constexpr uint32_t kWaitSpins = 1u << 28;
 __device__ __forceinline__ uint64_t global_timer_ns()
@@ -83,7 +84,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, CtaCon
         if ((run & 63u) == 63u) {
             const uint64_t t = global_timer_ns();
             if (t0 == 0) t0 = t;
-            else if (t - t0 > kWaitNs) break;
+            else {
+                const int32_t us = status ? *reinterpret_cast<volatile int32_t*>(&status->wait_limit_us) : 0;
+                if (t - t0 > (us > 0 ? (uint64_t)us * 1000ull : kWaitNs)) break;
+            }
         }
     }
     ctl->abort = 1;

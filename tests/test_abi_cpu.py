@@ -113,6 +113,15 @@ def test_argument_errors_are_reported_before_any_launch(api):
     assert L.iptq_linear(None, None, 8, None, None, None, 0, None, None, None, 8, 16, 16, None, 0, None) == api.ERR_WORKSPACE
     assert L.iptq_attention_block(None, None, None, None, 1, 1, 49, 32, None, None, None, None, None, None, 0, None) \
         == api.ERR_WORKSPACE
+    # a rejected call with packed 4-bit weights has launched nothing, the unpack kernel included
+    n0 = L.iptq_launch_count()
+    fake = 4096                                               # a non-NULL, 256-byte aligned stand-in: never dereferenced
+    assert L.iptq_linear(None, fake, 4, None, fake, fake, 0, None, None, fake, 8, 16, 16, fake, 1 << 20, None) == api.ERR_NULL
+    assert L.iptq_linear(fake, fake, 4, None, fake, fake, 0, None, None, fake, 8, 24, 16, fake, 1 << 20, None) == api.ERR_SHAPE
+    g2 = api.gelu_prepare(1.3e-4, 16, 0.03, 0)
+    assert L.iptq_mlp_block(fake, fake, None, fake, fake, C.byref(g2), fake, None, None, fake, 0, None, None, fake,
+                            8, 16, 64, 4, fake, 1 << 20, None) == api.ERR_NULL    # FC2's multiplier is missing
+    assert L.iptq_launch_count() == n0
     assert api.lib().iptq_strerror(api.ERR_TIMEOUT).decode() != ""
     assert api.linear_workspace_bytes(100, 256, 384, 4) >= 256 + 256 * 384
     assert api.mlp_workspace_bytes(100, 384, 1536) >= 256 + 100 * 1536

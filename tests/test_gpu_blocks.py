@@ -316,3 +316,26 @@ def _block_parity(api, orc, spec, w_bits, table):
         assert (got3 == want).all(), _mismatch(got3, want)
         wq = spec.qkv
         assert (api.unpack_int4(_cu(wq.w_packed)).cpu().numpy() == wq.w).all()
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_workspace_recovers(api, orc):
+    """A wait nothing ever satisfies (the self-test kernel waits on a barrier without arrivals) gives up after the
+    workspace's limit, records itself, and the kernel returns: iptq_check reports the time-out, and the same
+    workspace runs an ordinary layer bit-exactly after it has been re-initialised."""
+    rng = np.random.default_rng(77)
+    M, N, K = 300, 256, 128
+    x, w, bias, ratios = _linear_case(rng, M, N, K)
+    ma, sa = api.channel_requant_prepare(ratios)
+    ws = api.Workspace(api.linear_workspace_bytes(M, N, K))
+    ws.set_wait_limit(1000)                                     # 1 ms instead of 2 s
+    assert api.lib().iptq_selftest_wait_timeout(ws.ptr, ws.nbytes, None) == api.OK
+    with pytest.raises(api.IptqError) as e:
+        ws.check()
+    assert e.value.status == api.ERR_TIMEOUT
+    flag, where, block, work_next, work_done, limit = ws.status_words()
+    assert flag == 1 and where == 99 and block == 0 and work_next == 0 and work_done == 0 and limit == 1000
+    ws.reset()
+    assert ws.status_words()[:3] == [0, 0, 0]
+    got = api.linear(_cu(x), _cu(w), _cu(bias), _cu(ma), _cu(sa), ws, out_zp=3).cpu().numpy()
+    ws.check()
+    assert (got == orc.linear(x, w, bias, ma, sa, out_zp=3)).all()

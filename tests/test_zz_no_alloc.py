@@ -3,9 +3,11 @@
 Some users of the library run where device memory must not be allocated (a serving loop that may never hit
 cudaMalloc, a plug-in given a fixed set of buffers), so they cannot supply the workspace the regular entry point
 unpacks the weights into.  The static variant keeps that scratch in a device array owned by the library and
-shared by every call.  Because the array keeps whatever the previous call left in it, the check is made on two
-calls in a row with different weights and shapes (the second one smaller, so stale bytes of the first remain
-behind it), each compared bit for bit with the regular entry point.  This file sorts last on purpose.
+shared by every call.  Because the array keeps whatever the previous call left in it, the check is made on
+calls in a row with different weights and shapes (later ones smaller, so stale bytes of the first remain
+behind them; the last one with packed weights at an odd address, which takes the byte-wise unpack), each
+compared bit for bit with the regular entry point, and the free device memory the driver reports has to be the
+same before and after each call.  This file sorts last on purpose.
 """
 import numpy as np
 import pytest
@@ -39,16 +41,27 @@ def test_static_scratch_variant_matches_the_workspace_variant_twice_in_a_row(api
     rng = np.random.default_rng(2024)
     cu = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
     rq = api.requant_prepare(0.7 / 65536, zp=3)
-    for M, N, K in [(300, 768, 3072), (197, 96, 32)]:          # second call: smaller weights, stale bytes behind them
+    for M, N, K, odd in [(300, 768, 3072, False), (197, 96, 32, False), (50, 48, 32, True)]:   # later calls: smaller weights, stale bytes behind them
         x, wp, bias, ratios, res = _case(rng, M, N, K)
         m, s = api.channel_requant_prepare(ratios)
-        args = (cu(x), cu(wp), cu(bias), cu(m), cu(s))
+        wp_d = cu(wp)
+        if odd:                                                  # the same bytes, one byte further on: no 16-byte vectors
+            buf = torch.empty(wp.size + 16, dtype=torch.uint8, device="cuda")
+            buf[1:1 + wp.size] = wp_d.reshape(-1)
+            wp_d = buf[1:1 + wp.size].view(N, K // 2)
+            assert wp_d.data_ptr() % 2 == 1
+        args = (cu(x), wp_d, cu(bias), cu(m), cu(s))
         ws = api.Workspace(api.linear_workspace_bytes(M, N, K, 4))
         want = api.linear(*args, ws, out_zp=-5, residual=cu(res), residual_rq=rq, w_bits=4)
         ws.check()
         out = torch.empty((M, N), dtype=torch.int8, device="cuda")
-        got = api.linear_w4_static(*args, out_zp=-5, residual=cu(res), residual_rq=rq, out=out)
+        res_d = cu(res)
+        api.linear_w4_static(*args, out_zp=-5, residual=res_d, residual_rq=rq, out=out)   # includes a first call's address look-up
         torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]              # cudaMemGetInfo: what the driver has left
+        got = api.linear_w4_static(*args, out_zp=-5, residual=res_d, residual_rq=rq, out=out)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the amount of free device memory"
         assert len(torch.unique(want)) > 20
         assert torch.equal(got, want), "%d of %d differ" % (int((got != want).sum()), want.numel())
         # with a caller-owned status block the outcome can be queried through iptq_check
