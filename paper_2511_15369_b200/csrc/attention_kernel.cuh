@@ -90,11 +90,11 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
         mbar_init(s_full, 1);
-        mbar_init(s_empty, ATT_SOFTMAX_THREADS);
-        mbar_init(&p_ready[0], ATT_SOFTMAX_THREADS);
-        mbar_init(&p_ready[1], ATT_SOFTMAX_THREADS);
+        mbar_init(s_empty, ATT_SOFTMAX_THREADS / 32);       // one arrival per Softmax warp (512 arrivals on one
+        mbar_init(&p_ready[0], ATT_SOFTMAX_THREADS / 32);  // barrier word serialise and cost more than the Softmax itself)
+        mbar_init(&p_ready[1], ATT_SOFTMAX_THREADS / 32);
         mbar_init(o_full, 1);
-        mbar_init(o_empty, ATT_SOFTMAX_THREADS);
+        mbar_init(o_empty, ATT_SOFTMAX_THREADS / 32);
         ctl->abort = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_q);
@@ -261,7 +261,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 }
             }
             tc_fence_before_sync();
-            mbar_arrive(o_empty);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(o_empty);
             return true;
         };
 
@@ -303,11 +304,12 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 if (warp_rows && i < nch) tmem_ld16(trow + (uint32_t)((c_begin + i) * 16), v[i]);
             tmem_wait_ld();
             tc_fence_before_sync();
-            mbar_arrive(s_empty);                              // the MMA warp may overwrite S with the next item's scores
+            __syncwarp();
+            if (lane == 0) mbar_arrive(s_empty);               // the MMA warp may overwrite S with the next item's scores
             if (warp_rows) {
                 // ---- row maximum over the real, unmasked columns (Eq. (6)); padding and masked pairs become
                 //      kNoScore, a bias is added in place, so that the next step needs no case analysis
-                int mx = INT_MIN;
+                int mx = INT_MIN, mx1 = INT_MIN, mx2 = INT_MIN, mx3 = INT_MIN;
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     if (i < nch) {
@@ -323,32 +325,44 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                                 v[i][j] = (uint32_t)(use ? sc : kNoScore);
                             }
                         }
+                        // four running maxima: one chain of 64 dependent min/max instructions would leave the
+                        // thread waiting on itself
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) mx = max(mx, (int)v[i][j]);
+                        for (int j = 0; j < 16; j += 4) {
+                            mx = max(mx, (int)v[i][j]);     mx1 = max(mx1, (int)v[i][j + 1]);
+                            mx2 = max(mx2, (int)v[i][j + 2]); mx3 = max(mx3, (int)v[i][j + 3]);
+                        }
                     }
                 }
+                mx = max(max(mx, mx1), max(mx2, mx3));
                 xch_max[part * 128 + rloc] = mx;
                 named_barrier(1 + quad, 128);
                 mx = max(max(xch_max[rloc], xch_max[128 + rloc]), max(xch_max[256 + rloc], xch_max[384 + rloc]));
                 // ---- integer exponentials (Eqs. (7)-(14)), in place, and their sum
-                unsigned sum = 0;
+                unsigned sum = 0, sum1 = 0, sum2 = 0, sum3 = 0;         // four partial sums, as for the maximum
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     if (i < nch) {
+                        if (USE_LUT) {
+                            // table addresses first, then the 16 reads back to back, then the sums
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            unsigned e;
-                            if (USE_LUT) {
-                                const unsigned d = min((unsigned)mx - v[i][j], (unsigned)p.lut_n);
-                                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(e) : "r"(lut_addr + 2u * d));
-                            } else {
-                                e = exp_core_nd<VARIANT>(exp_distance(mx, (int)v[i][j]), p.ex);
-                            }
-                            sum += e;
-                            v[i][j] = e;
+                            for (int j = 0; j < 16; ++j)
+                                v[i][j] = lut_addr + 2u * min((unsigned)mx - v[i][j], (unsigned)p.lut_n);
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v[i][j]) : "r"(v[i][j]));
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                v[i][j] = exp_core_nd<VARIANT>(exp_distance(mx, (int)v[i][j]), p.ex);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4) {
+                            sum += v[i][j]; sum1 += v[i][j + 1]; sum2 += v[i][j + 2]; sum3 += v[i][j + 3];
                         }
                     }
                 }
+                sum = (sum + sum1) + (sum2 + sum3);
                 xch_sum[part * 128 + rloc] = sum;
                 named_barrier(1 + quad, 128);
                 sum = (xch_sum[rloc] + xch_sum[128 + rloc]) + (xch_sum[256 + rloc] + xch_sum[384 + rloc]);
@@ -416,7 +430,8 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     st_shared_v4(p_row + (uint32_t)(p.p_plane + (c0 >> 7) * 16384 + ((chunk ^ (rloc & 7)) << 4)), 0u, 0u, 0u, 0u);
             }
             fence_proxy_async_smem();            // generic-proxy stores -> visible to the tensor core's reads
-            mbar_arrive(&p_ready[k & 1]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&p_ready[k & 1]);
             // ---- output of the previous item: its P V product was issued right after that item's Softmax
             if (k > 0 && !epilogue(k - 1, pb, phd, pmt)) { ok = false; break; }
             pb = b; phd = h; pmt = mt;

@@ -62,10 +62,10 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
         for (int s = 0; s < ST; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
         for (int g = 0; g < G; ++g) {
             mbar_init(&s_full[g], 1);
-            mbar_init(&s_empty[g], 128);
-            mbar_init(&p_ready[g], 128);
+            mbar_init(&s_empty[g], 4);                     // one arrival per warp of the group
+            mbar_init(&p_ready[g], 4);
             mbar_init(&o_full[g], 1);
-            mbar_init(&o_empty[g], 128);
+            mbar_init(&o_empty[g], 4);
         }
         ctl->abort = 0;
         fence_barrier_init();
@@ -246,7 +246,8 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
                 if (warp_rows && i < nch) tmem_ld16(tS + (uint32_t)(i * 16), v[i]);
             tmem_wait_ld();
             tc_fence_before_sync();
-            mbar_arrive(&s_empty[g]);                          // the MMA warp may overwrite S with the group's next item
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s_empty[g]);           // the MMA warp may overwrite S with the group's next item
             int mx = INT_MIN;
             // most windows of a shifted layout lie inside one region: all labels equal, nothing to mask (the labels
             // were requested before the wait for the scores and are first looked at here)
@@ -348,7 +349,8 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
                 }
             }
             fence_proxy_async_smem();            // generic-proxy stores -> visible to the tensor core's reads
-            mbar_arrive(&p_ready[g]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&p_ready[g]);
             // ---- output of this item: the other groups' items fill the time the P V product takes
             if (!mbar_wait(&o_full[g], (uint32_t)n & 1u, ctl, p.status, 26)) break;
             tc_fence_after_sync();
@@ -384,7 +386,8 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
                 }
             }
             tc_fence_before_sync();
-            mbar_arrive(&o_empty[g]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&o_empty[g]);
         }
     }
 
