@@ -204,10 +204,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         const int tpp = p.TN >> 2;                             // tokens per part: 16, 32, 48 or 64
         const int nchunks = tpp >> 4;                          // 16-token chunks: 1..4
         uint8_t* out_blk = smem + ew * (tpp * 32);            // [tpp tokens][32 channels] int8
-        const uint32_t out_lane = smem_u32(out_blk) + (uint32_t)lane;
+        // where this lane's words go after the transpose: token (lane % 4) of a group of four, channels 4 (lane / 4) ..
+        const uint32_t out_word = smem_u32(out_blk) + (uint32_t)((lane & 3) * 32 + (lane >> 2) * 4);
+        const unsigned sel1 = (lane & 1) ? 0x3715u : 0x6240u, sel2 = (lane & 2) ? 0x3276u : 0x5410u;
         uint8_t* res_blk = smem + p.off_res + ew * (tpp * 32);
         const uint32_t res_lane = smem_u32(res_blk) + (uint32_t)lane;
         uint32_t res_ph = 0;
+        // the byte pack of the store saturates to int8: narrower ranges (activations below 8 bits) are clamped first
+        const bool sat8 = EPI == EPI_GELU ? (p.gelu.out.qmin == -128 && p.gelu.out.qmax == 127) : (p.qmin == -128 && p.qmax == 127);
         const uint32_t tab_mid = smem_u32(smem + p.off_tab) + 32768u;      // address of table[0 + 32768]
         if (EPI == EPI_GELU_TAB) {
             // the GELU table is static data: copy it while the previous kernel may still be running
@@ -291,12 +295,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                                 v[j] = max(-32768, min(32767, v[j]));
                             } else if (EPI == EPI_GELU) {
                                 v[j] = requant_nosat(gelu_core<GELU_VARIANT>(v[j], p.gelu), p.gelu.out);
-                                v[j] = max(p.gelu.out.qmin, min(p.gelu.out.qmax, v[j]));
+                                if (!sat8) v[j] = max(p.gelu.out.qmin, min(p.gelu.out.qmax, v[j]));
                             } else if (EPI == EPI_RESIDUAL) {
                                 v[j] += requant_core(r[j] * 65536 - p.res_off, p.res_mult, p.res_rnd, p.res_shift) + p.out_zp;
-                                v[j] = max(p.qmin, min(p.qmax, v[j]));
+                                if (!sat8) v[j] = max(p.qmin, min(p.qmax, v[j]));
                             } else {
-                                v[j] = max(p.qmin, min(p.qmax, v[j] + p.out_zp));
+                                v[j] += p.out_zp;
+                                if (!sat8) v[j] = max(p.qmin, min(p.qmax, v[j]));
                             }
                         }
                         if (EPI == EPI_GELU_TAB) {
@@ -304,9 +309,18 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                             for (int j = 0; j < 16; ++j)
                                 asm volatile("ld.shared.s8 %0, [%1];" : "=r"(v[j]) : "r"(tab_mid + (uint32_t)v[j]));
                         }
+                        // Four tokens of this lane's channel are packed into a word (saturating to int8), then a 4 x 4
+                        // byte transpose over the four lanes of a group (two shuffle + byte-permute rounds) leaves
+                        // lane m of the group with token m of the four for the group's four channels: one 32-bit
+                        // store per four outputs, every lane of the warp on its own bank (byte stores of four lanes
+                        // into one word took 2.7 shared-memory passes each).
 #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            asm volatile("st.shared.u8 [%0], %1;" ::"r"(out_lane + (uint32_t)((ch * 16 + j) * 32)), "r"(v[j]) : "memory");
+                        for (int g = 0; g < 4; ++g) {
+                            unsigned w = pack4_sat_s8(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                            w = __byte_perm(w, __shfl_xor_sync(0xffffffffu, w, 1), sel1);
+                            w = __byte_perm(w, __shfl_xor_sync(0xffffffffu, w, 2), sel2);
+                            asm volatile("st.shared.b32 [%0], %1;" ::"r"(out_word + (uint32_t)((ch * 16 + 4 * g) * 32)), "r"(w) : "memory");
+                        }
                     }
                 }
             }
