@@ -480,6 +480,17 @@ def run_ours(args):
     del hbuf, dbuf, graphs, blks, xd, yd
 
     clock_summary = clocks.summary(windows)
+    if args.headline_only:
+        # for profiler captures: the headline step alone (no other configuration, no CPU oracle)
+        clocks.stop()
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+                              "ms_per_step": total_ms / K, "config": {"workload": WORKLOAD}, "headline_only": True,
+                              "e2e": {"value": e2e_value, "unit": UNIT}, "sustained": sustained, "clocks": clock_summary,
+                              "stage_us": dict(zip(api.BLOCK_STAGES, [1e3 * t for t in stage_ms]))}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
     if rank != 0:
         clocks.stop()
         if world > 1:
@@ -873,6 +884,8 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="time the headline step only and print a short line (for profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
