@@ -91,16 +91,31 @@ struct GemmParams {
 };
 
 // The i-th tile of this CTA: tiles are numbered with the channel tile fastest, so that CTAs running side by side
-// share an activation tile in L2.
-__device__ __forceinline__ bool gemm_tile(const GemmParams& p, int i, int& tt, int& ct)
+// share an activation tile in L2.  A CTA pair takes two neighbouring channel tiles of one token tile (the odd CTA's
+// may lie past N when the number of channel tiles is odd: its weight rows then read as zeros and nothing is stored).
+template <bool PAIR>
+__device__ __forceinline__ bool gemm_tile(const GemmParams& p, int i, uint32_t rank, int& tt, int& ct)
 {
-    const int t = (int)blockIdx.x + i * (int)gridDim.x;
-    tt = t / p.n_ct;
-    ct = t - tt * p.n_ct;
+    if (PAIR) {
+        const int t = (int)cluster_id_x() + i * (int)cluster_count_x();
+        const int ncp = (p.n_ct + 1) >> 1;
+        tt = t / ncp;
+        ct = 2 * (t - tt * ncp) + (int)rank;
+    } else {
+        const int t = (int)blockIdx.x + i * (int)gridDim.x;
+        tt = t / p.n_ct;
+        ct = t - tt * p.n_ct;
+    }
     return tt < p.n_tt;
 }
 
-template <int EPI, int GELU_VARIANT>
+// PAIR: two CTAs of a cluster compute 256 channels x TN tokens with one MMA stream (cta_group::2).  Each stages its
+// own 128 weight rows and HALF of the activation tile (TN / 2 tokens), which lowers the operand traffic per SM from
+// (128 + TN) to (128 + TN / 2) rows per 128-byte block of K; each receives its 128 channels x TN tokens in its own
+// TMEM, so the epilogue is the same as without pairs.  The even CTA issues the MMAs: its `full` barriers count the
+// bytes of both CTAs' copies, its `acc_empty` barriers the epilogue warps of both, and its commits signal the
+// `empty` and `acc_full` barriers of both.
+template <int EPI, int GELU_VARIANT, bool PAIR>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_res,
@@ -121,10 +136,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     const int lane = threadIdx.x & 31;
     const int kblocks = (p.K + BK - 1) / BK;
     const int stages = p.stages;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EPI_WARPS); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], PAIR ? 2 * EPI_WARPS : EPI_WARPS); }
         for (int w = 0; w < EPI_WARPS; ++w) mbar_init(&res_bar[w], 1);
         ctl->abort = 0;
         fence_barrier_init();
@@ -134,11 +150,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         if (EPI == EPI_RESIDUAL) prefetch_tensormap(&map_res);
     }
     if (warp == 1) {
-        tmem_alloc(tmem_slot, TMEM_COLS);
-        tmem_relinquish();
+        if (PAIR) { tmem_alloc_pair(tmem_slot, TMEM_COLS); tmem_relinquish_pair(); }
+        else { tmem_alloc(tmem_slot, TMEM_COLS); tmem_relinquish(); }
     }
     tc_fence_before_sync();
     __syncthreads();
+    if (PAIR) cluster_sync();                                  // the peer's barriers exist before anything signals them
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     grid_dep_launch();
@@ -149,14 +166,23 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             grid_dep_wait();                                   // the activations (and unpacked weights) come from earlier kernels
             int s = 0; uint32_t ph = 0;
             int tt, ct;
-            for (int i = 0; gemm_tile(p, i, tt, ct); ++i) {
+            for (int i = 0; gemm_tile<PAIR>(p, i, rank, tt, ct); ++i) {
                 bool ok = true;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(&empty_bar[s], ph ^ 1u, ctl, p.status, 1)) { ok = false; break; }
                     uint8_t* st = ring + s * p.stage_bytes;
-                    mbar_expect_tx(&full_bar[s], (uint32_t)p.stage_bytes);
-                    tma_load_2d(st, &map_w, &full_bar[s], kb * BK, ct * CT);
-                    tma_load_2d(st + W_BYTES, &map_x, &full_bar[s], kb * BK, tt * p.TN);
+                    if (PAIR) {
+                        // both CTAs' bytes are counted on the even CTA's barrier (a copy of the odd CTA that lands
+                        // before the expectation is set only makes the pending count negative for a while)
+                        const uint32_t full0 = map_to_cta(smem_u32(&full_bar[s]), 0);
+                        if (rank == 0) mbar_expect_tx(&full_bar[s], 2u * (uint32_t)p.stage_bytes);
+                        tma_load_2d_pair(st, &map_w, full0, kb * BK, ct * CT);
+                        tma_load_2d_pair(st + W_BYTES, &map_x, full0, kb * BK, tt * p.TN + (int)rank * (p.TN >> 1));
+                    } else {
+                        mbar_expect_tx(&full_bar[s], (uint32_t)p.stage_bytes);
+                        tma_load_2d(st, &map_w, &full_bar[s], kb * BK, ct * CT);
+                        tma_load_2d(st + W_BYTES, &map_x, &full_bar[s], kb * BK, tt * p.TN);
+                    }
                     if (++s == stages) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
@@ -164,11 +190,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (elect_one()) {
-            const uint32_t idesc = umma_idesc_i8(CT, p.TN, true, true, false, false);
+        if ((!PAIR || rank == 0) && elect_one()) {
+            const uint32_t idesc = umma_idesc_i8(PAIR ? 2 * CT : CT, p.TN, true, true, false, false);
             int s = 0; uint32_t ph = 0;
             int tt, ct;
-            for (int it = 0; gemm_tile(p, it, tt, ct); ++it) {
+            for (int it = 0; gemm_tile<PAIR>(p, it, rank, tt, ct); ++it) {
                 const int ab = it & 1;
                 // the epilogue warps have pulled this accumulator's previous contents into registers
                 if (!mbar_wait(&acc_empty[ab], ((uint32_t)(it >> 1) & 1u) ^ 1u, ctl, p.status, 2)) break;
@@ -185,13 +211,15 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart; a k-step is 32 bytes
                         const uint64_t da = umma_smem_desc(w_addr + k * 32, 16, 1024, 128);
                         const uint64_t db = umma_smem_desc(x_addr + k * 32, 16, 1024, 128);
-                        umma_i8(tacc, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+                        if (PAIR) umma_i8_pair(tacc, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+                        else umma_i8(tacc, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
                     }
-                    umma_commit(&empty_bar[s]);               // frees the stage once these MMAs have read it
+                    // frees the stage (in both CTAs of a pair) once these MMAs have read it
+                    if (PAIR) umma_commit_pair(&empty_bar[s], 3); else umma_commit(&empty_bar[s]);
                     if (++s == stages) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit(&acc_full[ab]);                   // accumulator complete
+                if (PAIR) umma_commit_pair(&acc_full[ab], 3); else umma_commit(&acc_full[ab]);   // accumulator complete
             }
         }
     } else {
@@ -239,8 +267,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 tma_load_2d(res_blk, &map_res, &res_bar[ew], c0_, tok0_);
             }
         };
+        const uint32_t acc_empty0 = PAIR ? map_to_cta(smem_u32(&acc_empty[0]), 0) : 0u;   // the even CTA's pair of barriers
         int tt, ct;
-        bool have = gemm_tile(p, 0, tt, ct);
+        bool have = gemm_tile<PAIR>(p, 0, rank, tt, ct);
         int cm, cs, cb;
         if (have) {
             load_consts(ct, cm, cs, cb);
@@ -248,7 +277,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         }
         for (int it = 0; have; ++it) {
             int ntt, nct, ncm, ncs, ncb;
-            const bool nhave = gemm_tile(p, it + 1, ntt, nct);
+            const bool nhave = gemm_tile<PAIR>(p, it + 1, rank, ntt, nct);
             if (nhave) load_consts(nct, ncm, ncs, ncb);        // in flight during this tile
             const int ab = it & 1;
             const uint32_t abph = (uint32_t)(it >> 1) & 1u;
@@ -277,7 +306,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     } else {
                         tc_fence_before_sync();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(&acc_empty[ab]);   // the MMA warp may refill this accumulator
+                        if (lane == 0) {                       // the MMA warp may refill this accumulator
+                            if (PAIR) mbar_arrive_cluster(acc_empty0 + (uint32_t)(ab * 8)); else mbar_arrive(&acc_empty[ab]);
+                        }
                     }
                     if (active) {
                         // Three passes over the chunk, so that the shared-memory reads (volatile, hence kept in
@@ -350,9 +381,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         for (int i = 0; i < 64; ++i) __nanosleep(2000);
         __syncthreads();
     }
+    if (PAIR) cluster_sync();                                  // neither CTA leaves while the other may still reach into it
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        if (PAIR) tmem_dealloc_pair(tmem_base, TMEM_COLS); else tmem_dealloc(tmem_base, TMEM_COLS);
     }
 }
 
@@ -453,11 +485,11 @@ int unpack_int4_launch(const void* packed, int8_t* out, int64_t n_elems, cudaStr
 }
 
 // ---------------------------------------------------------------- launcher
-template <int EPI, int GV>
-static int launch_gemm(const CUtensorMap& mw, const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& mr,
-                       const GemmParams& p, int grid, int smem_bytes, cudaStream_t st)
+template <int EPI, int GV, bool PAIR>
+static int launch_gemm_as(const CUtensorMap& mw, const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& mr,
+                          const GemmParams& p, int grid, int smem_bytes, cudaStream_t st)
 {
-    auto kern = gemm_i8_kernel<EPI, GV>;
+    auto kern = gemm_i8_kernel<EPI, GV, PAIR>;
     static bool configured[64];               // one attribute call per instantiation and device
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return IPTQ_ERR_CUDA;
@@ -466,9 +498,18 @@ static int launch_gemm(const CUtensorMap& mw, const CUtensorMap& mx, const CUten
             return IPTQ_ERR_CUDA;
         configured[dev] = true;
     }
-    launch_kernel(kern, grid, GEMM_THREADS, smem_bytes, st, mw, mx, my, mr, p);
+    if (PAIR) launch_kernel_cluster(kern, grid, GEMM_THREADS, smem_bytes, st, 2u, mw, mx, my, mr, p);
+    else launch_kernel(kern, grid, GEMM_THREADS, smem_bytes, st, mw, mx, my, mr, p);
     note_launch();
     return last_launch_status();
+}
+
+template <int EPI, int GV>
+static int launch_gemm(const CUtensorMap& mw, const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& mr,
+                       const GemmParams& p, bool pair, int grid, int smem_bytes, cudaStream_t st)
+{
+    return pair ? launch_gemm_as<EPI, GV, true>(mw, mx, my, mr, p, grid, smem_bytes, st)
+                : launch_gemm_as<EPI, GV, false>(mw, mx, my, mr, p, grid, smem_bytes, st);
 }
 
 int linear_check(const LinearArgs& a)
@@ -493,7 +534,7 @@ int linear_check(const LinearArgs& a)
 
 // Shared-memory layout for a tile width: output blocks, residual blocks, GELU table, barriers, then as many ring
 // stages as fit.  Returns the number of stages (0: does not fit).
-static int gemm_layout(GemmParams& p, int TN, bool residual, bool table, int kblocks, int* smem_bytes)
+static int gemm_layout(GemmParams& p, int TN, bool pair, bool residual, bool table, int kblocks, int* smem_bytes)
 {
     const int blocks = EPI_WARPS * (TN / 4) * 32;             // = 128 TN bytes
     p.TN = TN;
@@ -501,7 +542,7 @@ static int gemm_layout(GemmParams& p, int TN, bool residual, bool table, int kbl
     p.off_tab = p.off_res + (residual ? blocks : 0);
     p.off_bar = p.off_tab + (table ? IPTQ_GELU_TABLE_SIZE : 0);
     p.off_ring = (p.off_bar + (2 * MAX_STAGES + 4 + EPI_WARPS) * 8 + 16 + 1023) & ~1023;
-    p.stage_bytes = W_BYTES + TN * BK;
+    p.stage_bytes = W_BYTES + (pair ? TN / 2 : TN) * BK;      // a CTA of a pair stages half of the activation tile
     const int room = SMEM_LIMIT - 1024 - p.off_ring;          // 1024: slack for the alignment of the dynamic base
     if (room < 0) return 0;
     int stages = std::min(MAX_STAGES, room / p.stage_bytes);
@@ -511,6 +552,14 @@ static int gemm_layout(GemmParams& p, int TN, bool residual, bool table, int kbl
     p.stages = stages;
     *smem_bytes = p.off_ring + stages * p.stage_bytes + 1024;
     return stages;
+}
+
+// CTA pairs pay where the mainloop waits for operands: a long reduction (the epilogue of a tile hides under the next
+// tile's K loop), 256 tokens per tile, at least two channel tiles, and enough tiles that every pair of SMs has one.
+static bool use_pairs(const LinearArgs& a, int n_ct, int kblocks, int sms)
+{
+    return kblocks >= 12 && a.M > 192 && n_ct >= 2 && sms >= 2 &&
+           (int64_t)((n_ct + 1) / 2) * ((a.M + 255) / 256) >= sms / 2;
 }
 
 int linear_launch(const LinearArgs& a, cudaStream_t st)
@@ -542,21 +591,24 @@ int linear_launch(const LinearArgs& a, cudaStream_t st)
     // the last round of tiles half empty.
     const int kblocks = (a.K + BK - 1) / BK;
     const int sms = sm_count();
+    bool pair = use_pairs(a, p.n_ct, kblocks, sms);
     int best_tn = 0, smem_bytes = 0;
-    for (int TN : {256, 192, 128, 64}) {
+    if (pair) best_tn = 256;
+    else for (int TN : {256, 192, 128, 64}) {
         GemmParams q = p;
         int sb;
         if (TN > 64 && a.M <= TN - 64) continue;              // a narrower tile covers all tokens
-        if (gemm_layout(q, TN, a.residual != nullptr, table, kblocks, &sb) < std::min(3, kblocks + 1)) continue;
+        if (gemm_layout(q, TN, false, a.residual != nullptr, table, kblocks, &sb) < std::min(3, kblocks + 1)) continue;
         best_tn = TN;
         break;
     }
     if (best_tn == 0) return IPTQ_ERR_SHAPE;
-    gemm_layout(p, best_tn, a.residual != nullptr, table, kblocks, &smem_bytes);
+    gemm_layout(p, best_tn, pair, a.residual != nullptr, table, kblocks, &smem_bytes);
     const int64_t n_tt = (a.M + p.TN - 1) / p.TN;
     if ((int64_t)p.n_ct * n_tt > (int64_t)1 << 30) return IPTQ_ERR_SHAPE;
     p.n_tt = (int)n_tt;
-    const int grid = (int)std::min<int64_t>((int64_t)p.n_ct * n_tt, sms);
+    const int grid = pair ? 2 * (int)std::min<int64_t>((int64_t)((p.n_ct + 1) / 2) * n_tt, sms / 2)
+                          : (int)std::min<int64_t>((int64_t)p.n_ct * n_tt, sms);
 
     CUtensorMap mw, mx, my, mr;
     int rc;
@@ -569,7 +621,7 @@ int linear_launch(const LinearArgs& a, cudaStream_t st)
     {
         const uint64_t dims[2] = {(uint64_t)a.K, (uint64_t)a.M};
         const uint64_t str[1] = {(uint64_t)a.K};
-        const uint32_t box[2] = {BK, (uint32_t)p.TN};
+        const uint32_t box[2] = {BK, (uint32_t)(pair ? p.TN / 2 : p.TN)};
         if ((rc = make_tensor_map_u8(&mx, a.x, 2, dims, str, box, 128)) != IPTQ_OK) return rc;
     }
     {
@@ -580,16 +632,16 @@ int linear_launch(const LinearArgs& a, cudaStream_t st)
         if ((rc = make_tensor_map_u8(&my, a.y, 2, dims, str, box, 0)) != IPTQ_OK) return rc;
         if ((rc = make_tensor_map_u8(&mr, a.residual ? a.residual : a.y, 2, dims, str, box, 0)) != IPTQ_OK) return rc;
     }
-    if (table) return launch_gemm<EPI_GELU_TAB, 0>(mw, mx, my, mr, p, grid, smem_bytes, st);   // the variant is in the table
+    if (table) return launch_gemm<EPI_GELU_TAB, 0>(mw, mx, my, mr, p, pair, grid, smem_bytes, st);   // the variant is in the table
     if (a.gelu) {
         switch (a.gelu->variant) {
-            case IPTQ_GELU_POLY4: return launch_gemm<EPI_GELU, IPTQ_GELU_POLY4>(mw, mx, my, mr, p, grid, smem_bytes, st);
-            case IPTQ_GELU_POLY2: return launch_gemm<EPI_GELU, IPTQ_GELU_POLY2>(mw, mx, my, mr, p, grid, smem_bytes, st);
-            default: return launch_gemm<EPI_GELU, IPTQ_GELU_SHIFT>(mw, mx, my, mr, p, grid, smem_bytes, st);
+            case IPTQ_GELU_POLY4: return launch_gemm<EPI_GELU, IPTQ_GELU_POLY4>(mw, mx, my, mr, p, pair, grid, smem_bytes, st);
+            case IPTQ_GELU_POLY2: return launch_gemm<EPI_GELU, IPTQ_GELU_POLY2>(mw, mx, my, mr, p, pair, grid, smem_bytes, st);
+            default: return launch_gemm<EPI_GELU, IPTQ_GELU_SHIFT>(mw, mx, my, mr, p, pair, grid, smem_bytes, st);
         }
     }
-    if (a.residual) return launch_gemm<EPI_RESIDUAL, 0>(mw, mx, my, mr, p, grid, smem_bytes, st);
-    return launch_gemm<EPI_REQUANT, 0>(mw, mx, my, mr, p, grid, smem_bytes, st);
+    if (a.residual) return launch_gemm<EPI_RESIDUAL, 0>(mw, mx, my, mr, p, pair, grid, smem_bytes, st);
+    return launch_gemm<EPI_REQUANT, 0>(mw, mx, my, mr, p, pair, grid, smem_bytes, st);
 }
 
 static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
