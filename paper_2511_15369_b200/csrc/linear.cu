@@ -192,7 +192,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         // ------------------------------------------------------------ MMA issuer
         if ((!PAIR || rank == 0) && elect_one()) {
             const uint32_t idesc = umma_idesc_i8(PAIR ? 2 * CT : CT, p.TN, true, true, false, false);
-            int s = 0; uint32_t ph = 0;
+            // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart.  The address field of a descriptor counts
+            // 16-byte units from the start of shared memory (all of it fits the field), so the descriptor of stage s,
+            // k-step k is the ring's descriptor plus (s * stage_bytes + 32 k) / 16: the loop below adds, it does not
+            // rebuild
+            const uint64_t desc_ring = umma_smem_desc(smem_u32(ring), 16, 1024, 128);
+            const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4;
+            int s = 0; uint32_t ph = 0, soff = 0;
             int tt, ct;
             for (int it = 0; gemm_tile<PAIR>(p, it, rank, tt, ct); ++it) {
                 const int ab = it & 1;
@@ -204,19 +210,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(&full_bar[s], ph, ctl, p.status, 3)) { ok = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t w_addr = smem_u32(ring + s * p.stage_bytes);
-                    const uint32_t x_addr = w_addr + W_BYTES;
+                    const uint64_t da0 = desc_ring + soff, db0 = da0 + (W_BYTES >> 4);
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k) {
-                        // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart; a k-step is 32 bytes
-                        const uint64_t da = umma_smem_desc(w_addr + k * 32, 16, 1024, 128);
-                        const uint64_t db = umma_smem_desc(x_addr + k * 32, 16, 1024, 128);
+                        const uint64_t da = da0 + 2 * k, db = db0 + 2 * k;      // a k-step is 32 bytes
                         if (PAIR) umma_i8_pair(tacc, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
                         else umma_i8(tacc, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
                     }
                     // frees the stage (in both CTAs of a pair) once these MMAs have read it
                     if (PAIR) umma_commit_pair(&empty_bar[s], 3); else umma_commit(&empty_bar[s]);
-                    if (++s == stages) { s = 0; ph ^= 1u; }
+                    soff += stage16;
+                    if (++s == stages) { s = 0; soff = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
                 if (PAIR) umma_commit_pair(&acc_full[ab], 3); else umma_commit(&acc_full[ab]);   // accumulator complete

@@ -621,7 +621,8 @@ static int launch_ln(const int8_t* x, int8_t* y, int64_t rows, const int32_t* gq
     constexpr int RW = NW == 1 ? 8 : NW <= 4 ? 4 : NW <= 8 ? 2 : 1;
     const int threads = 256;
     const int64_t want = ((rows + RW - 1) / RW + 7) / 8;
-    const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 8);
+    // two waves of the two CTAs an SM holds: with more, a warp has a single group and nothing to prefetch
+    const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 4);
     const bool sat8 = c.out.qmin == -128 && c.out.qmax == 127;
     const bool exact = c.dim == 128 * NW;
     // fold the zero point into the rounding constant when the sum stays clear of 32-bit overflow (|hi32| < 2^30)
@@ -630,7 +631,7 @@ static int launch_ln(const int8_t* x, int8_t* y, int64_t rows, const int32_t* gq
     const bool zpf = rz > -(1ll << 30) && rz < (1ll << 30);
     if (zpf) { cc.out.rnd = (int)rz; cc.out.zp = 0; }
     const bool ptf = c.variant == IPTQ_LN_PTF;
-    const bool pf = (rows + RW - 1) / RW >= (int64_t)4 * grid * (threads / 32);     // several groups per warp
+    const bool pf = (rows + RW - 1) / RW >= (int64_t)2 * grid * (threads / 32);     // two or more groups per warp
 #define IPTQ_LN_GO(P, S8, EX, ZF)                                                                                        \
     do {                                                                                                                 \
         if (pf) launch_kernel(layernorm_rows_kernel<NW, RW, P, S8, EX, ZF, true>, grid, threads, 0, st, x, y, rows, gq, bq, ptf_ptr, cc);  \

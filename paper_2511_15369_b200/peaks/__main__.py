@@ -1,6 +1,7 @@
 """Builds and runs the micro-benchmarks that give the ceilings `bench.py` reports against (dense INT8 tensor rate of
-a bare `tcgen05.mma.kind::i8` issue loop, integer instruction issue rates, TMEM load rate, cost of a satisfied
-mbarrier wait) and samples the SM clock and the power meanwhile.
+a bare `tcgen05.mma.kind::i8` issue loop, alone and as a CTA pair, integer instruction issue rates, TMEM load rate
+alone and beside running MMAs, the rate at which copies from L2 refill shared memory beside running MMAs, cost of a
+satisfied mbarrier wait) and samples the SM clock and the power meanwhile.
 
     python -m paper_2511_15369_b200.peaks [--sustained]
 
@@ -24,7 +25,7 @@ NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 def build():
     os.makedirs(OUT, exist_ok=True)
     exes = []
-    for name in ("probe", "probe_wait"):
+    for name in ("probe", "probe_wait", "probe_feed"):
         exe = os.path.join(OUT, name)
         subprocess.check_call([NVCC, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
                                "-I", os.path.join(ROOT, "include"), "-I", os.path.join(os.path.dirname(HERE), "csrc"),
