@@ -878,6 +878,30 @@ def bench_assignment(api, torch, dev):
             "oracle_first_block": {"evaluations": compared, "agree_within_1e-9": agree, "seconds": t_cpu}}
 
 
+def run_section(args):
+    """One part of the benchmark alone, on one GPU, for profiler captures (small footprint, few launches):
+    `nonlinear` = the stand-alone Softmax / GELU / LayerNorm kernels, `cfg3` = the Swin-Tiny stage-1 window block."""
+    import torch
+    from paper_2511_15369_b200 import api
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    api.lib()
+    peaks, peak_kind = measured_peaks()
+    if args.section == "nonlinear":
+        result = bench_nonlinear(api, torch, dev, peaks, peak_kind)
+    else:
+        shape = synth.CONFIGS["cfg3"]
+        spec = synth.make_block(shape, seed=0, calib_images=8)
+        blk = api.EncoderBlock(spec, TABLE, dev)
+        x = torch.from_numpy(spec.x).to(dev)
+        y = torch.empty_like(x)
+        flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+        ms = time_graph(torch, flush, lambda: blk(x, y), reps=max(3, args.steps))
+        blk.ws.check()
+        result = {"config": "cfg3", "us_per_step": 1e3 * ms, "tops": shape.gemm_ops() / (ms * 1e-3) / 1e12}
+    print(json.dumps({"section": args.section, "result": result}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -886,8 +910,12 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--headline-only", action="store_true",
                     help="time the headline step only and print a short line (for profiler captures)")
+    ap.add_argument("--section", choices=["nonlinear", "cfg3"],
+                    help="run one part of the benchmark alone and print its entries (for profiler captures)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.section:
+        run_section(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
