@@ -477,7 +477,29 @@ def run_ours(args):
     dbuf = torch.empty(64 << 20, dtype=torch.uint8, device=dev)
     link = {"h2d_gbs": link_gbs(dbuf, hbuf), "d2h_gbs": link_gbs(hbuf, dbuf)}
     link["floor_ms_per_step"] = 1e3 * max(xh.numel() / (link["h2d_gbs"] * 1e9), yh[0].numel() / (link["d2h_gbs"] * 1e9))
-    del hbuf, dbuf, graphs, blks, xd, yd
+    # both directions at once, as the pipelined steps use the link: 64 MiB each way on two streams
+    hbuf2 = torch.empty(64 << 20, dtype=torch.uint8).pin_memory()
+    dbuf2 = torch.empty(64 << 20, dtype=torch.uint8, device=dev)
+    s_up, s_dn = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    both = []
+    for _ in range(4):
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        s_up.wait_event(a)
+        s_dn.wait_event(a)
+        with torch.cuda.stream(s_up):
+            dbuf.copy_(hbuf, non_blocking=True)
+        with torch.cuda.stream(s_dn):
+            hbuf2.copy_(dbuf2, non_blocking=True)
+        torch.cuda.current_stream().wait_stream(s_up)
+        torch.cuda.current_stream().wait_stream(s_dn)
+        b.record()
+        torch.cuda.synchronize()
+        both.append(a.elapsed_time(b))
+    link["both_ways_gbs_each"] = hbuf.numel() / (min(both) * 1e-3) / 1e9
+    link["floor_ms_per_step_both_ways"] = 1e3 * xh.numel() / (link["both_ways_gbs_each"] * 1e9)
+    del hbuf, dbuf, hbuf2, dbuf2, graphs, blks, xd, yd
 
     clock_summary = clocks.summary(windows)
     if args.headline_only:

@@ -85,6 +85,15 @@ __device__ __forceinline__ int mad_hi(int a, int b, int c)
     asm("mad.hi.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
     return d;
 }
+// hi32(a * b + c) with a 64-bit addend (IMAD.WIDE; the value is the high word of its result).  With
+// c = bias * b + (rnd << 32) this is hi32((a + bias) * b) + rnd exactly: the 64-bit sum cannot overflow for 32-bit
+// a, bias and a multiplier below 2^31, and adding a multiple of 2^32 before the floor adds it after the floor.
+__device__ __forceinline__ int mad_wide_hi(int a, int b, long long c)
+{
+    long long d;
+    asm("mad.wide.s32 %0, %1, %2, %3;" : "=l"(d) : "r"(a), "r"(b), "l"(c));
+    return (int)(d >> 32);
+}
 // Logical right shift that yields 0 for shift amounts >= 32 (PTX shr clamps the amount).
 __device__ __forceinline__ unsigned shr_clamp(unsigned v, unsigned n)
 {

@@ -288,7 +288,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const int c0 = ct * CT + quad * 32;               // first channel of this warp
             const int tok0 = tt * p.TN + part * tpp;          // first token of this warp
             const bool active = c0 < p.N && tok0 < p.M;       // warp-uniform
-            const int crnd = 1 << (cs - 1);
+            // bias and rounding constant of this lane's channel as one 64-bit addend of the requantising multiply
+            const long long c64 = (long long)cb * (long long)cm + ((long long)(1 << (cs - 1)) << 32);
             if (!mbar_wait(&acc_full[ab], abph, ctl, p.status, 4)) break;
             tc_fence_after_sync();
             // the previous tile's store has read the output block (it was issued a whole K loop ago)
@@ -325,7 +326,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         }
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
-                            v[j] = requant_core((int)acc[ch & 1][j] + cb, cm, crnd, cs);
+                            v[j] = mad_wide_hi((int)acc[ch & 1][j], cm, c64) >> cs;
                             if (EPI == EPI_GELU_TAB) {
                                 v[j] = max(-32768, min(32767, v[j]));
                             } else if (EPI == EPI_GELU) {
