@@ -217,6 +217,16 @@ int iptq_layernorm(const int8_t* x, int8_t* y, int64_t rows, int dim, const int3
  * n_elems even (IPTQ_ERR_SHAPE otherwise). */
 int iptq_unpack_int4(const void* packed, int8_t* out, int64_t n_elems, iptq_stream_t stream);
 size_t iptq_linear_workspace_bytes(int64_t M, int N, int K, int w_bits);
+/* How iptq_linear() would tile an [M, K] x [N, K]^T product (no counterpart in the paper; host arithmetic only, for
+ * capacity planning and tests): tokens per tile (64, 128, 192 or 256), depth of the operand ring, whether CTA pairs
+ * (clusters of two, one 256-channel MMA stream) are used, dynamic shared memory per CTA, grid size, and the tile
+ * counts.  has_residual / has_gelu_table: the epilogue's staging needs; sm_count: SMs to plan for, 0 = those of the
+ * current device (the only case that touches CUDA).  IPTQ_ERR_SHAPE for sizes iptq_linear() rejects. */
+typedef struct {
+    int32_t tile_tokens, stages, cta_pairs, smem_bytes, grid, channel_tiles, token_tiles;
+} iptq_linear_plan_info;
+int iptq_linear_plan(int64_t M, int N, int K, int has_residual, int has_gelu_table, int sm_count,
+                     iptq_linear_plan_info* out);
 int iptq_linear(const int8_t* x, const void* w, int w_bits, const int32_t* bias, const int32_t* mult,
                 const int8_t* shift, int32_t out_zp, const int8_t* residual, const iptq_requant* residual_rq,
                 int8_t* y, int64_t M, int N, int K, void* ws, size_t ws_bytes, iptq_stream_t stream);

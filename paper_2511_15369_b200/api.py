@@ -73,6 +73,11 @@ class BlockParams(C.Structure):
     ]
 
 
+class LinearPlan(C.Structure):
+    _fields_ = [("tile_tokens", C.c_int32), ("stages", C.c_int32), ("cta_pairs", C.c_int32), ("smem_bytes", C.c_int32),
+                ("grid", C.c_int32), ("channel_tiles", C.c_int32), ("token_tiles", C.c_int32)]
+
+
 class IptqError(RuntimeError):
     def __init__(self, status, what):
         self.status = status
@@ -113,6 +118,7 @@ def lib():
         L.iptq_layernorm.argtypes = [_vp, _vp, C.c_int64, C.c_int, _vp, _vp, _vp, C.POINTER(LnConsts), _vp]
         L.iptq_linear_workspace_bytes.restype = C.c_size_t
         L.iptq_linear_workspace_bytes.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
+        L.iptq_linear_plan.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(LinearPlan)]
         L.iptq_linear.argtypes = [_vp, _vp, C.c_int, _vp, _vp, _vp, C.c_int32, _vp, C.POINTER(Requant), _vp,
                                   C.c_int64, C.c_int, C.c_int, _vp, C.c_size_t, _vp]
         L.iptq_linear_bits.argtypes = [_vp, _vp, C.c_int, _vp, _vp, _vp, C.c_int32, _vp, C.POINTER(Requant), _vp,
@@ -162,7 +168,7 @@ def exported_symbols():
     """Names declared in include/iptq.h (used by the CPU-side load test)."""
     return ["iptq_requant_prepare", "iptq_channel_requant_prepare", "iptq_softmax_prepare", "iptq_softmax", "iptq_softmax_table",
             "iptq_gelu_prepare", "iptq_gelu", "iptq_gelu_table", "iptq_gelu_fit", "iptq_gelu_prepare_coeffs", "iptq_layernorm_prepare", "iptq_layernorm",
-            "iptq_unpack_int4", "iptq_linear_workspace_bytes", "iptq_linear", "iptq_linear_bits", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_patchify", "iptq_attention_workspace_bytes", "iptq_attention_bias_bytes", "iptq_attention_bias_prepare", "iptq_attention_block",
+            "iptq_unpack_int4", "iptq_linear_workspace_bytes", "iptq_linear_plan", "iptq_linear", "iptq_linear_bits", "iptq_linear_w4_static", "iptq_gather_rows", "iptq_patchify", "iptq_attention_workspace_bytes", "iptq_attention_bias_bytes", "iptq_attention_bias_prepare", "iptq_attention_block",
             "iptq_mlp_workspace_bytes", "iptq_mlp_block", "iptq_encoder_block_workspace_bytes",
             "iptq_encoder_block", "iptq_encoder_block_profiled", "iptq_workspace_init", "iptq_check", "iptq_workspace_set_wait_limit", "iptq_selftest_wait_timeout", "iptq_strerror", "iptq_launch_count",
             "iptq_metric_softmax", "iptq_metric_gelu", "iptq_metric_layernorm", "iptq_softplus", "iptq_sqnr_db",
@@ -403,6 +409,13 @@ def unpack_int4(w_packed):
     n, k2 = w_packed.shape
     out = torch.empty((n, 2 * k2), dtype=torch.int8, device=w_packed.device)
     _chk(lib().iptq_unpack_int4(_dp(w_packed), _dp(out), n * 2 * k2, _stream()), "iptq_unpack_int4")
+    return out
+
+
+def linear_plan(M, N, K, residual=False, gelu_table=False, sm_count=0) -> LinearPlan:
+    """How ``linear`` would tile the product (host arithmetic; ``sm_count=0`` asks the current device)."""
+    out = LinearPlan()
+    _chk(lib().iptq_linear_plan(M, N, K, int(residual), int(gelu_table), sm_count, C.byref(out)), "iptq_linear_plan")
     return out
 
 

@@ -567,6 +567,38 @@ static bool use_pairs(const LinearArgs& a, int n_ct, int kblocks, int sms)
            (int64_t)((n_ct + 1) / 2) * ((a.M + 255) / 256) >= sms / 2;
 }
 
+// Tile width, ring depth, single CTAs or pairs, grid: fills p.TN, p.n_tt and the shared-memory layout.  Single CTAs
+// take the widest tile that fits beside a ring of at least three stages and is not mostly padding: a wide tile
+// amortises the weight tile (the operand bytes per MMA clock fall from 128 B at 128 tokens to 96 B at 256) and beat
+// every narrower one that was measured, even where it leaves the last round of tiles half empty.
+static int gemm_plan(GemmParams& p, int64_t M, bool residual, bool table, int sms, bool* pair_out, int* smem_bytes,
+                     int* grid)
+{
+    const int kblocks = (p.K + BK - 1) / BK;
+    LinearArgs shape{};
+    shape.M = M;
+    const bool pair = use_pairs(shape, p.n_ct, kblocks, sms);
+    int best_tn = 0;
+    if (pair) best_tn = 256;
+    else for (int TN : {256, 192, 128, 64}) {
+        GemmParams q = p;
+        int sb;
+        if (TN > 64 && M <= TN - 64) continue;                // a narrower tile covers all tokens
+        if (gemm_layout(q, TN, false, residual, table, kblocks, &sb) < std::min(3, kblocks + 1)) continue;
+        best_tn = TN;
+        break;
+    }
+    if (best_tn == 0) return IPTQ_ERR_SHAPE;
+    if (gemm_layout(p, best_tn, pair, residual, table, kblocks, smem_bytes) < 2) return IPTQ_ERR_SHAPE;
+    const int64_t n_tt = (M + p.TN - 1) / p.TN;
+    if ((int64_t)p.n_ct * n_tt > (int64_t)1 << 30) return IPTQ_ERR_SHAPE;
+    p.n_tt = (int)n_tt;
+    *grid = pair ? 2 * (int)std::min<int64_t>((int64_t)((p.n_ct + 1) / 2) * n_tt, sms / 2)
+                 : (int)std::min<int64_t>((int64_t)p.n_ct * n_tt, sms);
+    *pair_out = pair;
+    return IPTQ_OK;
+}
+
 int linear_launch(const LinearArgs& a, cudaStream_t st)
 {
     const int rc0 = linear_check(a);
@@ -589,31 +621,12 @@ int linear_launch(const LinearArgs& a, cudaStream_t st)
     const bool table = a.gelu && a.gelu->table;
     p.gelu_tab = table ? a.gelu->table : nullptr;
 
-    // Tile width: the widest that fits beside a ring of at least three stages and is not mostly padding.  What
-    // bounds a tile is shared-memory bandwidth (128 bytes per clock): every operand byte is written once by the
-    // copy engine and read once by the tensor core, (16 KB + 128 TN) bytes per 128-byte block of K each way, so a
-    // wide tile, which amortises the weight tile, beat every narrower one that was measured, even where it leaves
-    // the last round of tiles half empty.
     const int kblocks = (a.K + BK - 1) / BK;
-    const int sms = sm_count();
-    bool pair = use_pairs(a, p.n_ct, kblocks, sms);
-    int best_tn = 0, smem_bytes = 0;
-    if (pair) best_tn = 256;
-    else for (int TN : {256, 192, 128, 64}) {
-        GemmParams q = p;
-        int sb;
-        if (TN > 64 && a.M <= TN - 64) continue;              // a narrower tile covers all tokens
-        if (gemm_layout(q, TN, false, a.residual != nullptr, table, kblocks, &sb) < std::min(3, kblocks + 1)) continue;
-        best_tn = TN;
-        break;
-    }
-    if (best_tn == 0) return IPTQ_ERR_SHAPE;
-    gemm_layout(p, best_tn, pair, a.residual != nullptr, table, kblocks, &smem_bytes);
-    const int64_t n_tt = (a.M + p.TN - 1) / p.TN;
-    if ((int64_t)p.n_ct * n_tt > (int64_t)1 << 30) return IPTQ_ERR_SHAPE;
-    p.n_tt = (int)n_tt;
-    const int grid = pair ? 2 * (int)std::min<int64_t>((int64_t)((p.n_ct + 1) / 2) * n_tt, sms / 2)
-                          : (int)std::min<int64_t>((int64_t)p.n_ct * n_tt, sms);
+    bool pair = false;
+    int smem_bytes = 0, grid = 0;
+    const int rcp = gemm_plan(p, a.M, a.residual != nullptr, table, sm_count(), &pair, &smem_bytes, &grid);
+    if (rcp != IPTQ_OK) return rcp;
+    (void)kblocks;
 
     CUtensorMap mw, mx, my, mr;
     int rc;
@@ -685,6 +698,26 @@ size_t iptq_linear_workspace_bytes(int64_t M, int N, int K, int w_bits)
     size_t b = kStatusBytes;
     if (w_bits == 4 && N > 0 && K > 0) b += align256((size_t)N * (size_t)K);
     return b;
+}
+
+int iptq_linear_plan(int64_t M, int N, int K, int has_residual, int has_gelu_table, int sm_count_in,
+                     iptq_linear_plan_info* out)
+{
+    if (!out) return IPTQ_ERR_NULL;
+    if (M < 1 || M > (int64_t)1 << 30 || N < 16 || K < 16 || K > 4096 || (N & 15) || (K & 15)) return IPTQ_ERR_SHAPE;
+    const int sms = sm_count_in > 0 ? sm_count_in : sm_count();
+    if (sms < 1) return IPTQ_ERR_CUDA;
+    GemmParams p{};
+    p.M = (int)M; p.N = N; p.K = K;
+    p.n_ct = (N + CT - 1) / CT;
+    bool pair = false;
+    int smem_bytes = 0, grid = 0;
+    const int rc = gemm_plan(p, M, has_residual != 0, has_gelu_table != 0, sms, &pair, &smem_bytes, &grid);
+    if (rc != IPTQ_OK) return rc;
+    out->tile_tokens = p.TN; out->stages = p.stages; out->cta_pairs = pair ? 1 : 0;
+    out->smem_bytes = smem_bytes; out->grid = grid;
+    out->channel_tiles = p.n_ct; out->token_tiles = p.n_tt;
+    return IPTQ_OK;
 }
 
 int iptq_linear(const int8_t* x, const void* w, int w_bits, const int32_t* bias, const int32_t* mult,

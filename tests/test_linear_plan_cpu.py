@@ -1,0 +1,59 @@
+"""Host-side tiling plan of the INT8 linear layer (`iptq_linear_plan`): no GPU is touched when the SM count is given.
+The plan must fit the SM for every admissible shape, and the choices documented for it must hold: the widest tile
+that leaves a ring of three stages (or one per block of K plus one), CTA pairs only for long reductions with enough
+tiles, an even grid for pairs, never more CTAs than SMs."""
+import itertools
+
+import pytest
+
+from paper_2511_15369_b200 import api
+
+SMEM_LIMIT = 227 * 1024
+
+
+def plan(M, N, K, **kw):
+    return api.linear_plan(M, N, K, sm_count=kw.pop("sm_count", 148), **kw)
+
+
+@pytest.mark.parametrize("residual,table", [(False, False), (True, False), (False, True)])
+def test_every_admissible_shape_gets_a_plan_that_fits_the_sm(residual, table):
+    Ms = [1, 5, 64, 65, 128, 192, 193, 197, 256, 257, 1000, 12608, 25216, 200704]
+    Ns = [16, 96, 144, 288, 384, 768, 1008, 1152, 2304, 3072]
+    Ks = [16, 96, 144, 272, 384, 768, 1536, 1552, 3072, 4096]
+    for M, N, K in itertools.product(Ms, Ns, Ks):
+        p = plan(M, N, K, residual=residual, gelu_table=table)
+        kblocks = (K + 127) // 128
+        assert p.tile_tokens in (64, 128, 192, 256)
+        assert 1024 < p.smem_bytes <= SMEM_LIMIT, (M, N, K, p.smem_bytes)
+        assert 2 <= p.stages <= 8
+        assert p.stages >= min(3, kblocks + 1) or p.cta_pairs, (M, N, K, p.stages)
+        assert p.channel_tiles == (N + 127) // 128
+        assert p.token_tiles == (M + p.tile_tokens - 1) // p.tile_tokens
+        assert 1 <= p.grid <= 148
+        if p.cta_pairs:
+            assert p.tile_tokens == 256 and p.grid % 2 == 0 and kblocks >= 12 and p.channel_tiles >= 2
+            assert ((p.channel_tiles + 1) // 2) * p.token_tiles >= 74      # every pair of SMs has a tile
+        else:
+            assert p.grid == min(148, p.channel_tiles * p.token_tiles)
+        if M <= 64:
+            assert p.tile_tokens == 64          # a wider tile would be mostly padding
+
+
+def test_the_configurations_of_the_benchmark():
+    # ViT-Base batch 128: QKV, proj, FC1 (GELU table) on single CTAs, FC2 on pairs
+    assert (plan(25216, 2304, 768).tile_tokens, plan(25216, 2304, 768).cta_pairs) == (256, 0)
+    assert plan(25216, 768, 768, residual=True).cta_pairs == 0
+    assert plan(25216, 3072, 768, gelu_table=True).cta_pairs == 0
+    fc2 = plan(25216, 768, 3072, residual=True)
+    assert (fc2.tile_tokens, fc2.cta_pairs, fc2.grid) == (256, 1, 148)
+    # DeiT-Small batch 64: FC2 has 12 blocks of K
+    assert plan(12608, 384, 1536, residual=True).cta_pairs == 1
+    # a small device gets a smaller grid, and no pairs on a single SM
+    assert plan(25216, 768, 3072, residual=True, sm_count=1).cta_pairs == 0
+    assert plan(25216, 768, 3072, residual=True, sm_count=20).grid == 20
+
+
+def test_shapes_the_layer_rejects_are_rejected_by_the_plan():
+    for M, N, K in [(0, 128, 128), (128, 8, 128), (128, 128, 8), (128, 130, 128), (128, 128, 4112), (128, 128, 100)]:
+        with pytest.raises(api.IptqError):
+            plan(M, N, K)
