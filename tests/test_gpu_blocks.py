@@ -40,10 +40,11 @@ def _linear_case(rng, M, N, K, w_bits=8):
 
 
 # the last two shapes are long and large enough for CTA pairs: an odd number of channel tiles whose last one is ragged
-# (1808 = 14 x 128 + 16), and a ragged last token tile with a reduction that ends inside a 128-byte block
+# (2064 = 16 x 128 + 16), and a ragged last token tile with a reduction that ends inside a 128-byte block; the one
+# before them is a long reduction over few tiles, which takes half-width tiles
 @pytest.mark.parametrize("M,N,K", [(128, 128, 128), (197, 384, 384), (300, 1152, 384), (1000, 384, 1536),
                                    (77, 96, 96), (130, 288, 96), (256, 16, 16), (5, 144, 272),
-                                   (2600, 1808, 1536), (9500, 512, 1552)])
+                                   (2600, 384, 1536), (7100, 2064, 1536), (29000, 512, 1552)])
 def test_linear_parity(api, orc, M, N, K):
     rng = np.random.default_rng(M + N + K)
     x, w, bias, ratios = _linear_case(rng, M, N, K)
@@ -163,8 +164,9 @@ def test_linear_errors(api):
 
 @pytest.mark.parametrize("variant", [0, 1, 2])
 # hidden widths that are multiples of the 128-channel tile (768, 1536, 384) and one that is not (288)
-# (4800, 1536, 1024): FC1 with a reduction long enough for CTA pairs (both GELU epilogues on the pair kernel)
-@pytest.mark.parametrize("M,D,Dh", [(197, 192, 768), (333, 384, 1536), (64, 96, 384), (130, 96, 288), (4800, 1536, 1024)])
+# (14300, 1536, 1024): FC1 with a reduction long enough, and enough tiles, for CTA pairs (both GELU epilogues on the
+# pair kernel)
+@pytest.mark.parametrize("M,D,Dh", [(197, 192, 768), (333, 384, 1536), (64, 96, 384), (130, 96, 288), (14300, 1536, 1024)])
 def test_mlp_parity(api, orc, variant, M, D, Dh):
     rng = np.random.default_rng(M + variant)
     x = rng.integers(-128, 128, size=(M, D)).astype(np.int8)
