@@ -169,7 +169,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             for (int i = 0; gemm_tile<PAIR>(p, i, rank, tt, ct); ++i) {
                 bool ok = true;
                 for (int kb = 0; kb < kblocks; ++kb) {
-                    if (!mbar_wait(&empty_bar[s], ph ^ 1u, ctl, p.status, 1)) { ok = false; break; }
+                    if (!mbar_wait_relaxed(&empty_bar[s], ph ^ 1u, ctl, p.status, 1)) { ok = false; break; }
                     uint8_t* st = ring + s * p.stage_bytes;
                     if (PAIR) {
                         // both CTAs' bytes are counted on the even CTA's barrier (a copy of the odd CTA that lands
