@@ -109,6 +109,13 @@ __device__ __forceinline__ bool gemm_tile(const GemmParams& p, int i, uint32_t r
     return tt < p.n_tt;
 }
 
+// Tokens the MMAs of token tile tt cover: all TN, or, for the ragged last tile, what is left of M rounded up to 32
+// (the MMA's N).  The last round of tiles is usually made of such tiles; they then cost their share of a full one.
+__device__ __forceinline__ int tile_tokens(const GemmParams& p, int tt)
+{
+    return min(p.TN, (p.M - tt * p.TN + 31) & ~31);
+}
+
 // PAIR: two CTAs of a cluster compute 256 channels x TN tokens with one MMA stream (cta_group::2).  Each stages its
 // own 128 weight rows and HALF of the activation tile (TN / 2 tokens), which lowers the operand traffic per SM from
 // (128 + TN) to (128 + TN / 2) rows per 128-byte block of K; each receives its 128 channels x TN tokens in its own
@@ -177,7 +184,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         const uint32_t full0 = map_to_cta(smem_u32(&full_bar[s]), 0);
                         if (rank == 0) mbar_expect_tx(&full_bar[s], 2u * (uint32_t)p.stage_bytes);
                         tma_load_2d_pair(st, &map_w, full0, kb * BK, ct * CT);
-                        tma_load_2d_pair(st + W_BYTES, &map_x, full0, kb * BK, tt * p.TN + (int)rank * (p.TN >> 1));
+                        // the activation rows of a tile are split evenly between the two CTAs, also in a ragged tile
+                        tma_load_2d_pair(st + W_BYTES, &map_x, full0, kb * BK, tt * p.TN + (int)rank * (tile_tokens(p, tt) >> 1));
                     } else {
                         mbar_expect_tx(&full_bar[s], (uint32_t)p.stage_bytes);
                         tma_load_2d(st, &map_w, &full_bar[s], kb * BK, ct * CT);
@@ -191,7 +199,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if ((!PAIR || rank == 0) && elect_one()) {
-            const uint32_t idesc = umma_idesc_i8(PAIR ? 2 * CT : CT, p.TN, true, true, false, false);
+            const uint32_t idesc_full = umma_idesc_i8(PAIR ? 2 * CT : CT, p.TN, true, true, false, false);
             // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart.  The address field of a descriptor counts
             // 16-byte units from the start of shared memory (all of it fits the field), so the descriptor of stage s,
             // k-step k is the ring's descriptor plus (s * stage_bytes + 32 k) / 16: the loop below adds, it does not
@@ -203,9 +211,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             for (int it = 0; gemm_tile<PAIR>(p, it, rank, tt, ct); ++it) {
                 const int ab = it & 1;
                 // the epilogue warps have pulled this accumulator's previous contents into registers
-                if (!mbar_wait(&acc_empty[ab], ((uint32_t)(it >> 1) & 1u) ^ 1u, ctl, p.status, 2)) break;
+                // (when this wait is not satisfied at once the epilogue is what paces the kernel: sleep between tries)
+                if (!mbar_wait_relaxed(&acc_empty[ab], ((uint32_t)(it >> 1) & 1u) ^ 1u, ctl, p.status, 2)) break;
                 tc_fence_after_sync();
                 const uint32_t tacc = tmem_base + (uint32_t)(ab * ACC_COLS);
+                const int nt = tile_tokens(p, tt);
+                const uint32_t idesc = nt == p.TN ? idesc_full
+                                                  : umma_idesc_i8(PAIR ? 2 * CT : CT, nt, true, true, false, false);
                 bool ok = true;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(&full_bar[s], ph, ctl, p.status, 3)) { ok = false; break; }
