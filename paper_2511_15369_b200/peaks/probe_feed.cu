@@ -25,22 +25,22 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
                  :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
-// warp 0: TMEM; warp 1: MMA loop (operands at the start of shared memory); warp 2: copies into a 3-deep ring behind
+// warp 0: TMEM; warp 1: MMA loop (operands at the start of shared memory); warp 2: copies into a `depth`-deep ring behind
 // them; warps 4..: TMEM loads from columns 256.. until the MMA loop has ended
-__global__ void __launch_bounds__(640, 1) mix_kernel(int N, int iters, int copy_bytes, int ld_warps, const uint8_t* src,
-                                                     MixOut* out, int* sink)
+__global__ void __launch_bounds__(640, 1) mix_kernel(int N, int iters, int copy_bytes, int depth, int ld_warps,
+                                                     const uint8_t* src, MixOut* out, int* sink)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* ring = smem + STAGE;
-    __shared__ uint64_t bar, rbar[3];
+    __shared__ uint64_t bar, rbar[4];
     __shared__ uint32_t tmem_slot;
     __shared__ CtaControl ctl;
     __shared__ volatile int mma_done;
     for (int i = threadIdx.x; i < STAGE / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(smem)[i] = 0x01010101u;
     if (threadIdx.x == 0) {
         mbar_init(&bar, 1);
-        for (int i = 0; i < 3; ++i) mbar_init(&rbar[i], 1);
+        for (int i = 0; i < 4; ++i) mbar_init(&rbar[i], 1);
         ctl.abort = 0; mma_done = 0;
         fence_barrier_init();
     }
@@ -74,13 +74,13 @@ __global__ void __launch_bounds__(640, 1) mix_kernel(int N, int iters, int copy_
             const unsigned long long c0 = clock64();
             bool ok = true;
             for (int it = 0; it < iters && ok; ++it) {
-                const int s = it % 3;
-                if (it >= 3) ok = mbar_wait(&rbar[s], (uint32_t)((it / 3) - 1) & 1u, &ctl, nullptr, 2);
+                const int s = it % depth;
+                if (it >= depth) ok = mbar_wait(&rbar[s], (uint32_t)((it / depth) - 1) & 1u, &ctl, nullptr, 2);
                 mbar_expect_tx(&rbar[s], (uint32_t)copy_bytes);
-                bulk_load(ring + s * STAGE, base + (size_t)(it % 10) * STAGE, (uint32_t)copy_bytes, &rbar[s]);
+                bulk_load(ring + s * copy_bytes, base + (size_t)(it % 10) * STAGE, (uint32_t)copy_bytes, &rbar[s]);
             }
-            for (int it = max(iters - 3, 0); it < iters && ok; ++it)
-                ok = mbar_wait(&rbar[it % 3], (uint32_t)(it / 3) & 1u, &ctl, nullptr, 3);
+            for (int it = max(iters - depth, 0); it < iters && ok; ++it)
+                ok = mbar_wait(&rbar[it % depth], (uint32_t)(it / depth) & 1u, &ctl, nullptr, 3);
             out[blockIdx.x].copy_clocks = clock64() - c0;
             if (!ok) out[blockIdx.x].ok = 0;
         }
@@ -159,10 +159,10 @@ int main()
     int* sink; CK(cudaMalloc(&sink, 64));
     std::vector<MixOut> h(sms);
     const int iters = 4000;
-    auto run = [&](int N, int copy_bytes, int ld_warps, int grid) {
+    auto run = [&](int N, int copy_bytes, int ld_warps, int grid, int depth = 3) {
         CK(cudaMemset(out, 0, sizeof(MixOut) * sms));
         for (int rep = 0; rep < 2; ++rep) {
-            mix_kernel<<<grid, 640, smem>>>(N, iters, copy_bytes, ld_warps, src, out, sink);
+            mix_kernel<<<grid, 640, smem>>>(N, iters, copy_bytes, depth, ld_warps, src, out, sink);
             CK(cudaDeviceSynchronize());
         }
         CK(cudaMemcpy(h.data(), out, sizeof(MixOut) * sms, cudaMemcpyDeviceToHost));
@@ -174,7 +174,7 @@ int main()
         std::sort(m.begin(), m.end()); std::sort(t.begin(), t.end());
         const double mm = m[grid / 2], tt = t[grid / 2];
         printf("feed: MMA N=%3d on %3d SMs", N, grid);
-        if (copy_bytes) printf(", copies of %d B: %.0f clocks each = %.1f B/clk/SM (%.1f KB/clk in all)", copy_bytes, tt,
+        if (copy_bytes) printf(", %d copies of %d B in flight: %.0f clocks each = %.1f B/clk/SM (%.1f KB/clk in all)", depth, copy_bytes, tt,
                                copy_bytes / tt, copy_bytes / tt * grid / 1024.0);
         if (ld_warps) printf(", %2d warps of TMEM loads: one 32x32b.x16 per %.0f clocks per warp = %.0f B/clk/SM", ld_warps,
                              mm * iters * 4.0 / (ldi / grid), 2048.0 * ld_warps * (ldi / grid) / (mm * iters * 4.0));
@@ -187,6 +187,8 @@ int main()
         run(N, 0, 16, sms);
         run(N, 16384 + 128 * N, 16, sms);
     }
+    // is the rate with all SMs copying a limit of bandwidth or of bytes in flight?  2, 3 and 4 copies of 36 KB
+    for (int depth : {2, 3, 4}) run(256, 36864, 0, sms, depth);
     // CTA pairs
     const int psmem = 32768 + 1024;
     CK(cudaFuncSetAttribute(pair_loop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, psmem));
