@@ -117,7 +117,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             grid_dep_wait();                                   // q/k/v come from the previous kernel
             int s = 0; uint32_t ph = 0;
             for (;;) {
-                if (!mbar_wait_relaxed(&kv_empty[s], ph ^ 1u, ctl, p.status, 11)) break;
+                if (!mbar_wait(&kv_empty[s], ph ^ 1u, ctl, p.status, 11)) break;
                 const int it = atomicAdd(&p.status->work_next, 1);
                 if (it >= p.items) {
                     item_of[s] = -1;
@@ -152,9 +152,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             int s = 0; uint32_t ph = 0;
             int s_prev = 0;
             auto issue_pv = [&](int k) -> bool {                // k = item count index of the item whose P is ready
-                // the longest wait of this warp (a whole Softmax); the product is not needed before the next item's
-                // Softmax is over, so the warp may sleep between tries
-                if (!mbar_wait_relaxed(&p_ready[k & 1], (uint32_t)(k >> 1) & 1u, ctl, p.status, 14)) return false;
+                if (!mbar_wait(&p_ready[k & 1], (uint32_t)(k >> 1) & 1u, ctl, p.status, 14)) return false;
                 if (!mbar_wait(o_empty, ((uint32_t)k & 1u) ^ 1u, ctl, p.status, 12)) return false;   // previous O has been read
                 tc_fence_after_sync();
                 const uint32_t p_addr = smem_u32(sP + (k & 1) * p.p_bytes);

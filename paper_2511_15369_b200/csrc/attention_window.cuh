@@ -90,7 +90,7 @@ window_attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_
             int s = 0; uint32_t ph = 0;
             int stops = 0;                                     // stop marks written so far (every group needs one)
             for (;;) {
-                if (!mbar_wait_relaxed(&kv_empty[s], ph ^ 1u, ctl, p.status, 21)) break;
+                if (!mbar_wait(&kv_empty[s], ph ^ 1u, ctl, p.status, 21)) break;
                 const int it = stops ? p.items : atomicAdd(&p.status->work_next, 1);
                 if (it >= p.items) {
                     item_of[s] = -1;

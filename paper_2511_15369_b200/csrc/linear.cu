@@ -176,7 +176,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             for (int i = 0; gemm_tile<PAIR>(p, i, rank, tt, ct); ++i) {
                 bool ok = true;
                 for (int kb = 0; kb < kblocks; ++kb) {
-                    if (!mbar_wait_relaxed(&empty_bar[s], ph ^ 1u, ctl, p.status, 1)) { ok = false; break; }
+                    if (!mbar_wait(&empty_bar[s], ph ^ 1u, ctl, p.status, 1)) { ok = false; break; }
                     uint8_t* st = ring + s * p.stage_bytes;
                     if (PAIR) {
                         // both CTAs' bytes are counted on the even CTA's barrier (a copy of the odd CTA that lands
@@ -211,8 +211,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             for (int it = 0; gemm_tile<PAIR>(p, it, rank, tt, ct); ++it) {
                 const int ab = it & 1;
                 // the epilogue warps have pulled this accumulator's previous contents into registers
-                // (when this wait is not satisfied at once the epilogue is what paces the kernel: sleep between tries)
-                if (!mbar_wait_relaxed(&acc_empty[ab], ((uint32_t)(it >> 1) & 1u) ^ 1u, ctl, p.status, 2)) break;
+                if (!mbar_wait(&acc_empty[ab], ((uint32_t)(it >> 1) & 1u) ^ 1u, ctl, p.status, 2)) break;
                 tc_fence_after_sync();
                 const uint32_t tacc = tmem_base + (uint32_t)(ab * ACC_COLS);
                 const int nt = tile_tokens(p, tt);

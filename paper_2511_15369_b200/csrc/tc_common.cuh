@@ -71,8 +71,7 @@ __device__ __forceinline__ uint64_t global_timer_ns()
 
 // Bounded wait.  Returns false when the wait ran out or another role already aborted; the first
 // waiter to give up records (where, blockIdx) in the status block.
-static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, CtaControl* ctl, StatusBlock* status, int where,
-                                                   uint32_t nap_ns = 0)
+static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, CtaControl* ctl, StatusBlock* status, int where)
 {
     uint64_t t0 = 0;
     // 16 tries in a row cost nothing but the tries; the abort flag and the clock are looked at between such runs
@@ -80,7 +79,6 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parit
 #pragma unroll 1
         for (int i = 0; i < 16; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (nap_ns) __nanosleep(nap_ns);
         if (ctl->abort) return false;
         if ((run & 63u) == 63u) {
             const uint64_t t = global_timer_ns();
@@ -106,16 +104,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, CtaCon
 {
     if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, ctl, status, where);
-}
-
-// The same wait for a role that runs far ahead of what it waits for (a copy producer waiting for a ring stage to be
-// freed): between runs of tries the warp sleeps, so that its polling does not take issue slots from the warps that
-// share its scheduler; waking up a few hundred nanoseconds late costs such a role nothing.
-__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity, CtaControl* ctl, StatusBlock* status,
-                                                  int where)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, ctl, status, where, 200u);
 }
 
 // The same wait for a whole (converged) warp: one lane polls, the others learn the outcome from a shuffle, which
