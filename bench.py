@@ -550,6 +550,9 @@ def run_ours(args):
     stage_ops = {"qkv": 2 * T * D * 3 * D, "attention": 4 * B * H * N * N * dh, "proj": 2 * T * D * D,
                  "fc1_gelu": 2 * T * D * Dh, "fc2": 2 * T * Dh * D}
     stage_bytes = {"ln1": 2 * T * D, "ln2": 2 * T * D}
+    # (output channels, reduction length, residual epilogue, GELU table epilogue) of the four linear layers
+    gemm_shapes = {"qkv": (3 * D, D, False, False), "proj": (D, D, True, False), "fc1_gelu": (Dh, D, False, True),
+                   "fc2": (D, Dh, True, False)}
     int8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
     stages = []
     for name, t in zip(api.BLOCK_STAGES, stage_ms):
@@ -557,6 +560,12 @@ def run_ours(args):
         if name in stage_ops:
             s["tops"] = stage_ops[name] / (t * 1e-3) / 1e12
             s.update(int8_fracs(s["tops"], peaks))
+            if name in gemm_shapes:
+                n_out, k_red, res, tab = gemm_shapes[name]
+                pl = api.linear_plan(T, n_out, k_red, residual=res, gelu_table=tab)
+                s["tiling"] = {"tile_tokens": pl.tile_tokens, "ring_stages": pl.stages, "cta_pairs": bool(pl.cta_pairs),
+                               "smem_bytes": pl.smem_bytes, "grid": pl.grid,
+                               "tiles": pl.channel_tiles * pl.token_tiles}
         else:
             s["gbs"] = stage_bytes[name] / (t * 1e-3) / 1e9
             s["frac_hbm"] = s["gbs"] / peaks["hbm_gbs"]

@@ -345,3 +345,12 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_workspace_recovers(api
     got = api.linear(_cu(x), _cu(w), _cu(bias), _cu(ma), _cu(sa), ws, out_zp=3).cpu().numpy()
     ws.check()
     assert (got == orc.linear(x, w, bias, ma, sa, out_zp=3)).all()
+
+
+def test_the_plan_for_the_current_device_is_the_plan_that_runs(api):
+    """`linear_plan` with sm_count = 0 reads the device; on the part this library targets that is 148 SMs."""
+    import torch
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for shape in [(25216, 2304, 768), (25216, 768, 3072), (12608, 384, 1536), (197, 192, 192)]:
+        here, given = api.linear_plan(*shape, residual=True), api.linear_plan(*shape, residual=True, sm_count=sms)
+        assert [getattr(here, f) for f, _ in here._fields_] == [getattr(given, f) for f, _ in given._fields_]
