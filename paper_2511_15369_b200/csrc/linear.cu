@@ -570,11 +570,12 @@ static int gemm_layout(GemmParams& p, int TN, bool pair, bool residual, bool tab
     return stages;
 }
 
-// CTA pairs pay where the mainloop waits for operands: a long reduction (the epilogue of a tile hides under the next
-// tile's K loop), 256 tokens per tile, at least two channel tiles, and enough tiles that every pair of SMs has one.
+// CTA pairs pay where the mainloop waits for operands: a reduction of six blocks of K or more (measured on ViT-Base:
+// QKV 40.3 -> 37.6 us, FC1 + GELU 66.5 -> 58.5 us, FC2 62.6 -> 49.7 us; at three blocks, DeiT-Small, pairs lose),
+// 256 tokens per tile, at least two channel tiles, and three rounds of pair tiles or more.
 static bool use_pairs(const LinearArgs& a, int n_ct, int kblocks, int sms)
 {
-    return kblocks >= 12 && a.M > 192 && n_ct >= 2 && sms >= 2 &&
+    return kblocks >= 6 && a.M > 192 && n_ct >= 2 && sms >= 2 &&
            (int64_t)((n_ct + 1) / 2) * ((a.M + 255) / 256) >= 3 * (int64_t)(sms / 2);   // three rounds of pair tiles
 }
 
