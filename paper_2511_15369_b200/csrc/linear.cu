@@ -90,24 +90,32 @@ struct GemmParams {
     StatusBlock* status;
 };
 
-// The i-th tile of this CTA: tiles are numbered with the channel tile fastest, so that CTAs running side by side
+// The tiles of this CTA, round by round: tiles are numbered with the channel tile fastest, so that CTAs running side by side
 // share an activation tile in L2.  A CTA pair takes two neighbouring channel tiles of one token tile (the odd CTA's
 // may lie past N when the number of channel tiles is odd: its weight rows then read as zeros and nothing is stored).
 template <bool PAIR>
-__device__ __forceinline__ bool gemm_tile(const GemmParams& p, int i, uint32_t rank, int& tt, int& ct)
-{
-    if (PAIR) {
-        const int t = (int)cluster_id_x() + i * (int)cluster_count_x();
-        const int ncp = (p.n_ct + 1) >> 1;
-        tt = t / ncp;
-        ct = 2 * (t - tt * ncp) + (int)rank;
-    } else {
-        const int t = (int)blockIdx.x + i * (int)gridDim.x;
-        tt = t / p.n_ct;
-        ct = t - tt * p.n_ct;
+struct TileWalk {
+    int tt, ct;                  // the current tile: token tile, channel tile
+    int c, dtt, dc, nc, rank;    // channel unit (tile, or pair of tiles), step per round in both coordinates, units per row
+    __device__ __forceinline__ void start(const GemmParams& p, uint32_t rank_)
+    {
+        rank = (int)rank_;
+        nc = PAIR ? (p.n_ct + 1) >> 1 : p.n_ct;
+        const int first = PAIR ? (int)cluster_id_x() : (int)blockIdx.x;
+        const int stride = PAIR ? (int)cluster_count_x() : (int)gridDim.x;
+        tt = first / nc; c = first - tt * nc;
+        dtt = stride / nc; dc = stride - dtt * nc;
+        ct = PAIR ? 2 * c + rank : c;
     }
-    return tt < p.n_tt;
-}
+    // one round further (no division in the roles' loops)
+    __device__ __forceinline__ void next()
+    {
+        tt += dtt; c += dc;
+        if (c >= nc) { c -= nc; ++tt; }
+        ct = PAIR ? 2 * c + rank : c;
+    }
+    __device__ __forceinline__ bool valid(const GemmParams& p) const { return tt < p.n_tt; }
+};
 
 // Tokens the MMAs of token tile tt cover: all TN, or, for the ragged last tile, what is left of M rounded up to 32
 // (the MMA's N).  The last round of tiles is usually made of such tiles; they then cost their share of a full one.
@@ -172,8 +180,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         if (elect_one()) {
             grid_dep_wait();                                   // the activations (and unpacked weights) come from earlier kernels
             int s = 0; uint32_t ph = 0;
-            int tt, ct;
-            for (int i = 0; gemm_tile<PAIR>(p, i, rank, tt, ct); ++i) {
+            TileWalk<PAIR> tw;
+            for (tw.start(p, rank); tw.valid(p); tw.next()) {
+                const int tt = tw.tt, ct = tw.ct;
                 bool ok = true;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(&empty_bar[s], ph ^ 1u, ctl, p.status, 1)) { ok = false; break; }
@@ -207,8 +216,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const uint64_t desc_ring = umma_smem_desc(smem_u32(ring), 16, 1024, 128);
             const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4;
             int s = 0; uint32_t ph = 0, soff = 0;
-            int tt, ct;
-            for (int it = 0; gemm_tile<PAIR>(p, it, rank, tt, ct); ++it) {
+            TileWalk<PAIR> tw;
+            tw.start(p, rank);
+            for (int it = 0; tw.valid(p); ++it, tw.next()) {
+                const int tt = tw.tt;
                 const int ab = it & 1;
                 // the epilogue warps have pulled this accumulator's previous contents into registers
                 if (!mbar_wait(&acc_empty[ab], ((uint32_t)(it >> 1) & 1u) ^ 1u, ctl, p.status, 2)) break;
@@ -283,16 +294,20 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             }
         };
         const uint32_t acc_empty0 = PAIR ? map_to_cta(smem_u32(&acc_empty[0]), 0) : 0u;   // the even CTA's pair of barriers
-        int tt, ct;
-        bool have = gemm_tile<PAIR>(p, 0, rank, tt, ct);
+        TileWalk<PAIR> tw;
+        tw.start(p, rank);
+        int tt = tw.tt, ct = tw.ct;
+        bool have = tw.valid(p);
         int cm, cs, cb;
         if (have) {
             load_consts(ct, cm, cs, cb);
             if (EPI == EPI_RESIDUAL) request_residual(tt, ct);
         }
         for (int it = 0; have; ++it) {
-            int ntt, nct, ncm, ncs, ncb;
-            const bool nhave = gemm_tile<PAIR>(p, it + 1, rank, ntt, nct);
+            int ncm, ncs, ncb;
+            tw.next();
+            const int ntt = tw.tt, nct = tw.ct;
+            const bool nhave = tw.valid(p);
             if (nhave) load_consts(nct, ncm, ncs, ncb);        // in flight during this tile
             const int ab = it & 1;
             const uint32_t abph = (uint32_t)(it >> 1) & 1u;
