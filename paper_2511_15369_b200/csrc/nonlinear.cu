@@ -512,7 +512,7 @@ layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int6
 // four lanes, and every lane then runs the scalar part (variance, square root, reciprocal) of its own row, so the
 // hundred dependent instructions of that part are shared by eight rows without any broadcast.
 template <int WPL, bool PTF, bool SAT8, bool ZPF>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 layernorm_short_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int64_t rows,
                             const int32_t* __restrict__ gamma_q, const int32_t* __restrict__ beta_q,
                             const uint8_t* __restrict__ ptf, const LnDev c)
@@ -524,15 +524,19 @@ layernorm_short_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const int64_t steps = (rows + 7) / 8;
-    int4 g[WPL], b[WPL];
+    // The per-channel parameters live in shared memory (the four lanes of a row read four addresses, the eight rows of
+    // a warp the same four: no bank conflict).  In registers they are 48 per thread and halve the resident warps, and
+    // resident warps are what hides a row's chain of dependent steps (load, two reductions, square root, divide):
+    // 64 registers and four CTAs per SM instead of 98 and two took the 96-channel case from 25.0 to 20.8 us.
+    __shared__ int4 g[4 * WPL], b[4 * WPL];
     unsigned sh[WPL];
-#pragma unroll
-    for (int k = 0; k < WPL; ++k) {
-        const int wi = q + 4 * k;
-        g[k] = __ldg(reinterpret_cast<const int4*>(gamma_q) + wi);
-        b[k] = __ldg(reinterpret_cast<const int4*>(beta_q) + wi);
-        sh[k] = PTF ? __ldg(reinterpret_cast<const unsigned*>(ptf) + wi) : 0u;
+    for (int i = threadIdx.x; i < 4 * WPL; i += blockDim.x) {
+        g[i] = __ldg(reinterpret_cast<const int4*>(gamma_q) + i);
+        b[i] = __ldg(reinterpret_cast<const int4*>(beta_q) + i);
     }
+#pragma unroll
+    for (int k = 0; k < WPL; ++k) sh[k] = PTF ? __ldg(reinterpret_cast<const unsigned*>(ptf) + q + 4 * k) : 0u;
+    __syncthreads();
     grid_dep_wait();                                          // gamma / beta above are static; the rows come from the previous kernel
     const int om = c.out.mult, ornd = c.out.rnd, osh = c.out.shift, ozp = c.out.zp;
     for (int64_t step = warp; step < steps; step += nwarps) {
@@ -578,10 +582,11 @@ layernorm_short_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y
                 if (!SAT8) o = max(c.out.qmin, min(c.out.qmax, o));
                 return o;
             };
-            const int o0 = elem(sext_byte<0>(wk), 0, g[k].x, b[k].x);
-            const int o1 = elem(sext_byte<1>(wk), 1, g[k].y, b[k].y);
-            const int o2 = elem(sext_byte<2>(wk), 2, g[k].z, b[k].z);
-            const int o3 = elem(sext_byte<3>(wk), 3, g[k].w, b[k].w);
+            const int4 gk = g[q + 4 * k], bk = b[q + 4 * k];
+            const int o0 = elem(sext_byte<0>(wk), 0, gk.x, bk.x);
+            const int o1 = elem(sext_byte<1>(wk), 1, gk.y, bk.y);
+            const int o2 = elem(sext_byte<2>(wk), 2, gk.z, bk.z);
+            const int o3 = elem(sext_byte<3>(wk), 3, gk.w, bk.w);
             out[k] = SAT8 ? (int)pack4_sat_s8(o0, o1, o2, o3) : (int)pack4_s8(o0, o1, o2, o3);
         }
         if (live) {
@@ -621,8 +626,12 @@ static int launch_ln(const int8_t* x, int8_t* y, int64_t rows, const int32_t* gq
     constexpr int RW = NW == 1 ? 8 : NW <= 4 ? 4 : NW <= 8 ? 2 : 1;
     const int threads = 256;
     const int64_t want = ((rows + RW - 1) / RW + 7) / 8;
-    // two waves of the two CTAs an SM holds: with more, a warp has a single group and nothing to prefetch
-    const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 4);
+    // Wide rows (640 channels and more: two CTAs per SM): two waves, and the next rows prefetched from two groups per
+    // warp on; with more CTAs a warp has a single group and nothing to prefetch (ViT-Base LayerNorm 16.7 -> 15.3 us).
+    // Narrower rows: four waves and prefetch only for long loops; there the prefetch costs more than it hides
+    // (192 channels, 50 176 rows: 15.2 us against 16.4 - 17.2 us).
+    constexpr int kCtasPerSm = NW >= 5 ? 4 : 8, kPrefetchFrom = NW >= 5 ? 2 : 4;
+    const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * kCtasPerSm);
     const bool sat8 = c.out.qmin == -128 && c.out.qmax == 127;
     const bool exact = c.dim == 128 * NW;
     // fold the zero point into the rounding constant when the sum stays clear of 32-bit overflow (|hi32| < 2^30)
@@ -631,7 +640,7 @@ static int launch_ln(const int8_t* x, int8_t* y, int64_t rows, const int32_t* gq
     const bool zpf = rz > -(1ll << 30) && rz < (1ll << 30);
     if (zpf) { cc.out.rnd = (int)rz; cc.out.zp = 0; }
     const bool ptf = c.variant == IPTQ_LN_PTF;
-    const bool pf = (rows + RW - 1) / RW >= (int64_t)2 * grid * (threads / 32);     // two or more groups per warp
+    const bool pf = (rows + RW - 1) / RW >= (int64_t)kPrefetchFrom * grid * (threads / 32);   // groups per warp
 #define IPTQ_LN_GO(P, S8, EX, ZF)                                                                                        \
     do {                                                                                                                 \
         if (pf) launch_kernel(layernorm_rows_kernel<NW, RW, P, S8, EX, ZF, true>, grid, threads, 0, st, x, y, rows, gq, bq, ptf_ptr, cc);  \
