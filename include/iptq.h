@@ -202,7 +202,8 @@ int iptq_layernorm(const int8_t* x, int8_t* y, int64_t rows, int dim, const int3
                    iptq_stream_t stream);
 
 /* ------------------------------------------------------------------ INT8 GEMM carrier
- * Linear ops run in integer arithmetic (Sec. 3.1): acc[m,n] = sum_k x[m,k] w[n,k] + bias[n];
+ * Linear ops run in integer arithmetic (Sec. 3.1): acc[m,n] = sum_k x[m,k] w[n,k] + bias[n], which must fit int32
+ * (K <= 4096 keeps the sum below 2^26 in magnitude);
  * y = clamp(R_n(acc) + R_res((residual - residual_rq.zp) << 16) + out_zp, -128, 127), where R_n uses
  * (mult[n], shift[n]) without zero point/clamp and the residual term is present only if residual != NULL.
  * x: dev int8 [M, K]; w: dev int8 [N, K] (w_bits = 8) or packed int4 [N, K/2] (w_bits = 4: element k in
@@ -219,11 +220,13 @@ int iptq_unpack_int4(const void* packed, int8_t* out, int64_t n_elems, iptq_stre
 size_t iptq_linear_workspace_bytes(int64_t M, int N, int K, int w_bits);
 /* How iptq_linear() would tile an [M, K] x [N, K]^T product (no counterpart in the paper; host arithmetic only, for
  * capacity planning and tests): tokens per tile (64, 128, 192 or 256), depth of the operand ring, whether CTA pairs
- * (clusters of two, one 256-channel MMA stream) are used, dynamic shared memory per CTA, grid size, and the tile
- * counts.  has_residual / has_gelu_table: the epilogue's staging needs; sm_count: SMs to plan for, 0 = those of the
- * current device (the only case that touches CUDA).  IPTQ_ERR_SHAPE for sizes iptq_linear() rejects. */
+ * (clusters of two, one 256-channel MMA stream) are used, dynamic shared memory per CTA, grid size, the tile
+ * counts, and whether the epilogue stages outputs and residuals in one buffer per warp or in two used by alternate
+ * tiles (two where they cost no ring stage).  has_residual / has_gelu_table: the epilogue's staging needs;
+ * sm_count: SMs to plan for, 0 = those of the current device (the only case that touches CUDA).  IPTQ_ERR_SHAPE
+ * for sizes iptq_linear() rejects. */
 typedef struct {
-    int32_t tile_tokens, stages, cta_pairs, smem_bytes, grid, channel_tiles, token_tiles;
+    int32_t tile_tokens, stages, cta_pairs, smem_bytes, grid, channel_tiles, token_tiles, staging_buffers;
 } iptq_linear_plan_info;
 int iptq_linear_plan(int64_t M, int N, int K, int has_residual, int has_gelu_table, int sm_count,
                      iptq_linear_plan_info* out);

@@ -75,7 +75,8 @@ class BlockParams(C.Structure):
 
 class LinearPlan(C.Structure):
     _fields_ = [("tile_tokens", C.c_int32), ("stages", C.c_int32), ("cta_pairs", C.c_int32), ("smem_bytes", C.c_int32),
-                ("grid", C.c_int32), ("channel_tiles", C.c_int32), ("token_tiles", C.c_int32)]
+                ("grid", C.c_int32), ("channel_tiles", C.c_int32), ("token_tiles", C.c_int32),
+                ("staging_buffers", C.c_int32)]
 
 
 class IptqError(RuntimeError):

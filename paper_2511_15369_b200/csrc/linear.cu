@@ -8,6 +8,7 @@
 // epilogue.  The accumulator is double-buffered in TMEM so that the epilogue of tile i overlaps the mainloop of
 // tile i+1.
 #include <algorithm>
+#include <climits>
 #include <mutex>
 
 #include "tc_common.cuh"
@@ -80,6 +81,7 @@ struct GemmParams {
     int TN;                                           // tokens per tile: 64, 128, 192 or 256
     int n_ct, n_tt;                                   // channel tiles, token tiles
     int stages, stage_bytes;                          // TMA ring
+    int epi_bufs;                                     // staging buffers of the epilogue (output, residual): 1 or 2
     int off_res, off_tab, off_bar, off_ring;          // shared-memory layout (the output blocks start at 0)
     const int32_t* bias; const int32_t* mult; const int8_t* shift;
     int out_zp;
@@ -88,6 +90,7 @@ struct GemmParams {
     GeluDev gelu;
     const int8_t* gelu_tab;                           // device table of the integer GELU (EPI_GELU_TAB)
     StatusBlock* status;
+    int acc_floor;                                    // INT_MIN, as a value the compiler cannot see (epilogue, bias add)
 };
 
 // The tiles of this CTA, round by round: tiles are numbered with the channel tile fastest, so that CTAs running side by side
@@ -143,8 +146,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     uint64_t* empty_bar = full_bar + MAX_STAGES;
     uint64_t* acc_full = empty_bar + MAX_STAGES;  // [2]
     uint64_t* acc_empty = acc_full + 2;           // [2]
-    uint64_t* res_bar = acc_empty + 2;            // [EPI_WARPS]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(res_bar + EPI_WARPS);
+    uint64_t* res_bar = acc_empty + 2;            // [EPI_WARPS][2]: one per warp and staging buffer
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(res_bar + 2 * EPI_WARPS);
     CtaControl* ctl = reinterpret_cast<CtaControl*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5;
@@ -156,7 +159,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], PAIR ? 2 * EPI_WARPS : EPI_WARPS); }
-        for (int w = 0; w < EPI_WARPS; ++w) mbar_init(&res_bar[w], 1);
+        for (int w = 0; w < 2 * EPI_WARPS; ++w) mbar_init(&res_bar[w], 1);
         ctl->abort = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_w);
@@ -257,13 +260,19 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         const int part = ew >> 2;
         const int tpp = p.TN >> 2;                             // tokens per part: 16, 32, 48 or 64
         const int nchunks = tpp >> 4;                          // 16-token chunks: 1..4
-        uint8_t* out_blk = smem + ew * (tpp * 32);            // [tpp tokens][32 channels] int8
+        // Staging blocks of this warp, [tpp tokens][32 channels] int8 each: one for the outputs and one for the
+        // residual, or two of each used by alternate tiles.  With two, a tile neither waits for the copy engine to
+        // have read the previous tile's outputs nor for a residual block that could only be requested once the
+        // previous one had been consumed; it pays where the K loop is too short to cover those latencies.
+        const int two = p.epi_bufs - 1;                        // 0 or 1
+        const uint32_t buf_bytes = (uint32_t)(EPI_WARPS * tpp * 32);
+        uint8_t* out_blk0 = smem + ew * (tpp * 32);
         // where this lane's words go after the transpose: token (lane % 4) of a group of four, channels 4 (lane / 4) ..
-        const uint32_t out_word = smem_u32(out_blk) + (uint32_t)((lane & 3) * 32 + (lane >> 2) * 4);
+        const uint32_t out_word0 = smem_u32(out_blk0) + (uint32_t)((lane & 3) * 32 + (lane >> 2) * 4);
         const unsigned sel1 = (lane & 1) ? 0x3715u : 0x6240u, sel2 = (lane & 2) ? 0x3276u : 0x5410u;
-        uint8_t* res_blk = smem + p.off_res + ew * (tpp * 32);
-        const uint32_t res_lane = smem_u32(res_blk) + (uint32_t)lane;
-        uint32_t res_ph = 0;
+        uint8_t* res_blk0 = smem + p.off_res + ew * (tpp * 32);
+        const uint32_t res_lane0 = smem_u32(res_blk0) + (uint32_t)lane;
+        uint32_t res_ph = 0;                                   // bit b: phase of staging buffer b's barrier
         // the byte pack of the store saturates to int8: narrower ranges (activations below 8 bits) are clamped first
         const bool sat8 = EPI == EPI_GELU ? (p.gelu.out.qmin == -128 && p.gelu.out.qmax == 127) : (p.qmin == -128 && p.qmax == 127);
         const uint32_t tab_mid = smem_u32(smem + p.off_tab) + 32768u;      // address of table[0 + 32768]
@@ -286,11 +295,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 cb_ = p.bias ? __ldg(p.bias + c) : 0;
             }
         };
-        auto request_residual = [&](int tt_, int ct_) {
+        auto request_residual = [&](int tt_, int ct_, int b_) {
             const int c0_ = ct_ * CT + quad * 32, tok0_ = tt_ * p.TN + part * tpp;
             if (c0_ < p.N && tok0_ < p.M && lane == 0) {
-                mbar_expect_tx(&res_bar[ew], (uint32_t)(tpp * 32));
-                tma_load_2d(res_blk, &map_res, &res_bar[ew], c0_, tok0_);
+                mbar_expect_tx(&res_bar[2 * ew + b_], (uint32_t)(tpp * 32));
+                tma_load_2d(res_blk0 + (uint32_t)b_ * buf_bytes, &map_res, &res_bar[2 * ew + b_], c0_, tok0_);
             }
         };
         const uint32_t acc_empty0 = PAIR ? map_to_cta(smem_u32(&acc_empty[0]), 0) : 0u;   // the even CTA's pair of barriers
@@ -301,7 +310,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         int cm, cs, cb;
         if (have) {
             load_consts(ct, cm, cs, cb);
-            if (EPI == EPI_RESIDUAL) request_residual(tt, ct);
+            if (EPI == EPI_RESIDUAL) request_residual(tt, ct, 0);
         }
         for (int it = 0; have; ++it) {
             int ncm, ncs, ncb;
@@ -309,21 +318,30 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const int ntt = tw.tt, nct = tw.ct;
             const bool nhave = tw.valid(p);
             if (nhave) load_consts(nct, ncm, ncs, ncb);        // in flight during this tile
+            const int sb = it & two;                           // staging buffer of this tile
+            // the other buffer's residual bytes were consumed a tile ago (every lane has passed that tile's end)
+            if (EPI == EPI_RESIDUAL && two && nhave) request_residual(ntt, nct, sb ^ 1);
+            const uint32_t out_word = out_word0 + (uint32_t)sb * buf_bytes, res_lane = res_lane0 + (uint32_t)sb * buf_bytes;
             const int ab = it & 1;
             const uint32_t abph = (uint32_t)(it >> 1) & 1u;
             const int c0 = ct * CT + quad * 32;               // first channel of this warp
             const int tok0 = tt * p.TN + part * tpp;          // first token of this warp
             const bool active = c0 < p.N && tok0 < p.M;       // warp-uniform
-            // bias and rounding constant of this lane's channel as one 64-bit addend of the requantising multiply
+            // The output zero point, which is added after the shift, goes into the rounding constant, shifted left,
+            // where every channel of the warp has a shift small enough for that (the sum stays below 2^31).
+            const bool fold = EPI == EPI_REQUANT && __all_sync(0xffffffffu, cs <= 20);
+            const int crnd = (1 << (cs - 1)) + (fold ? p.out_zp << cs : 0);
+            // the residual epilogue, whose other half already is an add and a high multiply per output, is faster with
+            // bias and rounding constant in the 64-bit addend of one wide multiply-add (measured: 5 % at K = 96)
             const long long c64 = (long long)cb * (long long)cm + ((long long)(1 << (cs - 1)) << 32);
             if (!mbar_wait(&acc_full[ab], abph, ctl, p.status, 4)) break;
             tc_fence_after_sync();
-            // the previous tile's store has read the output block (it was issued a whole K loop ago)
-            if (lane == 0) bulk_wait_read_all();
+            // the store that last used this tile's output block has read it (one or two K loops ago)
+            if (lane == 0) { if (two) bulk_wait_read_but_one(); else bulk_wait_read_all(); }
             __syncwarp();
             if (EPI == EPI_RESIDUAL && active) {
-                if (!mbar_wait(&res_bar[ew], res_ph, ctl, p.status, 5)) break;
-                res_ph ^= 1u;
+                if (!mbar_wait(&res_bar[2 * ew + sb], (res_ph >> sb) & 1u, ctl, p.status, 5)) break;
+                res_ph ^= 1u << sb;
             }
             const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * ACC_COLS + part * tpp);
             uint32_t acc[2][16];
@@ -350,11 +368,22 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                             for (int j = 0; j < 16; ++j)
                                 asm volatile("ld.shared.s8 %0, [%1];" : "=r"(r[j]) : "r"(res_lane + (uint32_t)((ch * 16 + j) * 32)));
                         }
+                        // R of the header: hi32((acc + bias) * mult) + rounding constant, shifted.  The bias add is
+                        // written as add-then-max against INT_MIN: a plain add is moved to the multiplier's pipe by the
+                        // assembler, which is the pipe this loop is short of.
+                        if (fold) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                v[j] = mad_hi(__viaddmax_s32((int)acc[ch & 1][j], cb, p.acc_floor), cm, crnd) >> cs;
+                                if (!sat8) v[j] = max(p.qmin, min(p.qmax, v[j]));
+                            }
+                        } else
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
-                            v[j] = mad_wide_hi((int)acc[ch & 1][j], cm, c64) >> cs;
+                            if (EPI == EPI_RESIDUAL) v[j] = mad_wide_hi((int)acc[ch & 1][j], cm, c64) >> cs;
+                            else v[j] = mad_hi(__viaddmax_s32((int)acc[ch & 1][j], cb, p.acc_floor), cm, crnd) >> cs;
                             if (EPI == EPI_GELU_TAB) {
-                                v[j] = max(-32768, min(32767, v[j]));
+                                v[j] = max(-32768, min(32767, v[j])) + (int)tab_mid;
                             } else if (EPI == EPI_GELU) {
                                 v[j] = requant_nosat(gelu_core<GELU_VARIANT>(v[j], p.gelu), p.gelu.out);
                                 if (!sat8) v[j] = max(p.gelu.out.qmin, min(p.gelu.out.qmax, v[j]));
@@ -369,7 +398,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         if (EPI == EPI_GELU_TAB) {
 #pragma unroll
                             for (int j = 0; j < 16; ++j)
-                                asm volatile("ld.shared.s8 %0, [%1];" : "=r"(v[j]) : "r"(tab_mid + (uint32_t)v[j]));
+                                asm volatile("ld.shared.s8 %0, [%1];" : "=r"(v[j]) : "r"((uint32_t)v[j]));
                         }
                         // Four tokens of this lane's channel are packed into a word (saturating to int8), then a 4 x 4
                         // byte transpose over the four lanes of a group (two shuffle + byte-permute rounds) leaves
@@ -390,14 +419,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 fence_proxy_async_smem();                     // this lane's shared-memory stores -> visible to the TMA engine
                 __syncwarp();
                 if (lane == 0) {
-                    tma_store_2d(&map_y, out_blk, c0, tok0);  // clipped at N and M
+                    tma_store_2d(&map_y, out_blk0 + (uint32_t)sb * buf_bytes, c0, tok0);  // clipped at N and M
                     bulk_commit();
                 }
             }
-            if (EPI == EPI_RESIDUAL && nhave) {
-                __syncwarp();                                  // every lane has read its residual bytes of this tile
-                request_residual(ntt, nct);
-            }
+            __syncwarp();                                      // every lane has read its residual bytes of this tile
+            if (EPI == EPI_RESIDUAL && !two && nhave) request_residual(ntt, nct, 0);
             have = nhave; tt = ntt; ct = nct; cm = ncm; cs = ncs; cb = ncb;
         }
         if (lane == 0) bulk_wait_all();                       // stores complete before shared memory goes away
@@ -565,14 +592,16 @@ int linear_check(const LinearArgs& a)
 
 // Shared-memory layout for a tile width: output blocks, residual blocks, GELU table, barriers, then as many ring
 // stages as fit.  Returns the number of stages (0: does not fit).
-static int gemm_layout(GemmParams& p, int TN, bool pair, bool residual, bool table, int kblocks, int* smem_bytes)
+static int gemm_layout(GemmParams& p, int TN, bool pair, bool residual, bool table, int kblocks, int epi_bufs,
+                       int* smem_bytes)
 {
-    const int blocks = EPI_WARPS * (TN / 4) * 32;             // = 128 TN bytes
+    const int blocks = epi_bufs * EPI_WARPS * (TN / 4) * 32;  // = 128 TN bytes per buffer
     p.TN = TN;
+    p.epi_bufs = epi_bufs;
     p.off_res = blocks;
     p.off_tab = p.off_res + (residual ? blocks : 0);
     p.off_bar = p.off_tab + (table ? IPTQ_GELU_TABLE_SIZE : 0);
-    p.off_ring = (p.off_bar + (2 * MAX_STAGES + 4 + EPI_WARPS) * 8 + 16 + 1023) & ~1023;
+    p.off_ring = (p.off_bar + (2 * MAX_STAGES + 4 + 2 * EPI_WARPS) * 8 + 16 + 1023) & ~1023;
     p.stage_bytes = W_BYTES + (pair ? TN / 2 : TN) * BK;      // a CTA of a pair stages half of the activation tile
     const int room = SMEM_LIMIT - 1024 - p.off_ring;          // 1024: slack for the alignment of the dynamic base
     if (room < 0) return 0;
@@ -617,12 +646,21 @@ static int gemm_plan(GemmParams& p, int64_t M, bool residual, bool table, int sm
         GemmParams q = p;
         int sb;
         if (TN > 64 && M <= TN - 64) continue;                // a narrower tile covers all tokens
-        if (gemm_layout(q, TN, false, residual, table, kblocks, &sb) < std::min(3, kblocks + 1)) continue;
+        if (gemm_layout(q, TN, false, residual, table, kblocks, 1, &sb) < std::min(3, kblocks + 1)) continue;
         best_tn = TN;
         break;
     }
     if (best_tn == 0) return IPTQ_ERR_SHAPE;
-    if (gemm_layout(p, best_tn, pair, residual, table, kblocks, smem_bytes) < 2) return IPTQ_ERR_SHAPE;
+    // Two staging buffers per epilogue warp where they cost no ring stage (short reductions, whose K loop does not
+    // cover the latency of the output store and of the residual load).
+    int epi_bufs = 1;
+    {
+        GemmParams q1 = p, q2 = p;
+        int sb1, sb2;
+        if (gemm_layout(q2, best_tn, pair, residual, table, kblocks, 2, &sb2) >=
+            gemm_layout(q1, best_tn, pair, residual, table, kblocks, 1, &sb1)) epi_bufs = 2;
+    }
+    if (gemm_layout(p, best_tn, pair, residual, table, kblocks, epi_bufs, smem_bytes) < 2) return IPTQ_ERR_SHAPE;
     const int64_t n_tt = (M + p.TN - 1) / p.TN;
     if ((int64_t)p.n_ct * n_tt > (int64_t)1 << 30) return IPTQ_ERR_SHAPE;
     p.n_tt = (int)n_tt;
@@ -642,6 +680,7 @@ int linear_launch(const LinearArgs& a, cudaStream_t st)
     p.M = (int)a.M; p.N = a.N; p.K = a.K;
     p.n_ct = (a.N + CT - 1) / CT;
     p.bias = a.bias; p.mult = a.mult; p.shift = a.shift; p.out_zp = a.out_zp;
+    p.acc_floor = INT_MIN;
     p.qmin = -(1 << (a.out_bits - 1)); p.qmax = (1 << (a.out_bits - 1)) - 1;
     p.res_mult = p.res_rnd = p.res_shift = p.res_off = 0;
     if (a.residual) {
@@ -749,7 +788,7 @@ int iptq_linear_plan(int64_t M, int N, int K, int has_residual, int has_gelu_tab
     if (rc != IPTQ_OK) return rc;
     out->tile_tokens = p.TN; out->stages = p.stages; out->cta_pairs = pair ? 1 : 0;
     out->smem_bytes = smem_bytes; out->grid = grid;
-    out->channel_tiles = p.n_ct; out->token_tiles = p.n_tt;
+    out->channel_tiles = p.n_ct; out->token_tiles = p.n_tt; out->staging_buffers = p.epi_bufs;
     return IPTQ_OK;
 }
 

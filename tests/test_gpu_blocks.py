@@ -71,6 +71,30 @@ def test_linear_parity(api, orc, M, N, K):
     assert (got == want).all(), _mismatch(got, want)
 
 
+@pytest.mark.parametrize("M,N,K", [(300, 160, 96), (2600, 384, 1536)])
+def test_linear_large_shifts_and_biases(api, orc, M, N, K):
+    """Channel groups whose shifts are all small, all large and mixed (the epilogue treats the zero point differently
+    when every channel of a 32-channel group has a small shift), with biases that dwarf the sums."""
+    rng = np.random.default_rng(M)
+    x, w, _, _ = _linear_case(rng, M, N, K)
+    ratios = 2.0 ** rng.uniform(-12, -7, size=N)
+    ratios[32:64] = 2.0 ** rng.uniform(-27, -23, size=32)           # shifts of 23 .. 27 beyond the 32 of hi32
+    ratios[64:96:3] = 2.0 ** rng.uniform(-26, -22, size=len(ratios[64:96:3]))
+    bias = rng.integers(-3000, 3000, size=N).astype(np.int32)
+    bias[32:96] = rng.integers(-(1 << 30), 1 << 30, size=64).astype(np.int32)
+    bias[100] = (1 << 31) - 1 - (1 << 26)
+    bias[101] = -(1 << 31) + (1 << 26)
+    ma, sa = api.channel_requant_prepare(ratios)
+    assert sa[32:64].min() >= 22 and sa[:32].max() <= 12
+    ws = api.Workspace(api.linear_workspace_bytes(M, N, K))
+    for zp in (3, -128, 127):
+        want = orc.linear(x, w, bias, ma, sa, out_zp=zp)
+        got = api.linear(_cu(x), _cu(w), _cu(bias), _cu(ma), _cu(sa), ws, out_zp=zp).cpu().numpy()
+        ws.check()
+        assert (got == want).all(), _mismatch(got, want)
+    assert len(np.unique(want[:, 32:96])) > 20
+
+
 @pytest.mark.parametrize("out_bits", [6, 4])
 def test_linear_narrow_outputs(api, orc, out_bits):
     """Outputs clamped to a signed range narrower than 8 bits (W6A6 activations), plain and residual epilogue."""

@@ -26,6 +26,7 @@ def test_every_admissible_shape_gets_a_plan_that_fits_the_sm(residual, table):
         assert p.tile_tokens in (64, 128, 192, 256)
         assert 1024 < p.smem_bytes <= SMEM_LIMIT, (M, N, K, p.smem_bytes)
         assert 2 <= p.stages <= 8
+        assert p.staging_buffers in (1, 2)
         assert p.stages >= min(3, kblocks + 1) or p.cta_pairs, (M, N, K, p.stages)
         assert p.channel_tiles == (N + 127) // 128
         assert p.token_tiles == (M + p.tile_tokens - 1) // p.tile_tokens
@@ -40,6 +41,9 @@ def test_every_admissible_shape_gets_a_plan_that_fits_the_sm(residual, table):
 
 
 def test_the_configurations_of_the_benchmark():
+    # short reductions have room for two staging buffers per epilogue warp, the long ones of ViT-Base keep their ring
+    assert plan(200704, 96, 96, residual=True).staging_buffers == 2 and plan(200704, 288, 96).staging_buffers == 2
+    assert plan(25216, 768, 3072, residual=True).staging_buffers == 1 and plan(25216, 2304, 768).staging_buffers == 1
     # ViT-Base batch 128: all four linear layers on CTA pairs
     assert (plan(25216, 2304, 768).tile_tokens, plan(25216, 2304, 768).cta_pairs) == (256, 1)
     assert plan(25216, 768, 768, residual=True).cta_pairs == 1
