@@ -81,6 +81,15 @@ __device__ __forceinline__ int one_op(int a, int b, int c)
     else if (OP == 7) asm volatile("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));     // PRMT
     else if (OP == 8) { asm volatile("{ .reg .s32 t; max.s32 t, %1, %2; min.s32 %0, t, %3; }" : "=r"(d) : "r"(a), "r"(b), "r"(c)); }   // 3-input min/max
     else if (OP == 9) asm volatile("mul.hi.u32 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));               // IMAD.HI.U32 no addend
+    else if (OP == 11) { asm volatile("{ .reg .s32 t; add.s32 t, %1, %2; max.s32 %0, t, %3; }" : "=r"(d) : "r"(a), "r"(b), "r"(c)); }  // add, then max
+    else if (OP == 12) asm volatile("dp4a.s32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));          // IDP.4A
+    else if (OP == 13) asm volatile("dp2a.lo.s32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));       // IDP.2A
+    else if (OP == 14) asm volatile("shfl.sync.bfly.b32 %0, %1, 1, 0x1f, 0xffffffff;" : "=r"(d) : "r"(a));       // SHFL
+    // pairs of independent-pipe candidates, two instructions per call: does one hide behind the other?
+    else if (OP == 20) { int t; asm volatile("mad.hi.s32 %0, %1, %2, %3;" : "=r"(t) : "r"(a), "r"(b), "r"(c)); asm volatile("shr.s32 %0, %1, %2;" : "=r"(d) : "r"(t), "r"(b & 7)); }
+    else if (OP == 21) { int t; asm volatile("mad.lo.s32 %0, %1, %2, %3;" : "=r"(t) : "r"(a), "r"(b), "r"(c)); asm volatile("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(t), "r"(b), "r"(c)); }
+    else if (OP == 22) { int t; asm volatile("mad.hi.s32 %0, %1, %2, %3;" : "=r"(t) : "r"(a), "r"(b), "r"(c)); asm volatile("add.s32 %0, %1, %2;" : "=r"(d) : "r"(t), "r"(c)); }
+    else if (OP == 23) { int t; asm volatile("shr.s32 %0, %1, %2;" : "=r"(t) : "r"(a), "r"(b & 7)); asm volatile("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(t), "r"(b), "r"(c)); }
     else { long long w; asm volatile("mul.wide.s32 %0, %1, %2;" : "=l"(w) : "r"(a), "r"(b)); d = (int)(w >> 32) ^ (int)w; }
     return d;
 }
@@ -212,7 +221,7 @@ __global__ void __launch_bounds__(512, 1) store_kernel(uint8_t* out, long long b
 }
 
 template <int OP>
-static void run_int(const char* name, int* sink, unsigned long long* dclk, int sms)
+static void run_int(const char* name, int* sink, unsigned long long* dclk, int sms, int instr_per_op = 1)
 {
     const int iters = 4096;
     int_rate_kernel<OP><<<sms, 1024>>>(iters, 12345, sink, dclk);
@@ -226,7 +235,7 @@ static void run_int(const char* name, int* sink, unsigned long long* dclk, int s
     std::vector<unsigned long long> h(sms);
     CK(cudaMemcpy(h.data(), dclk, sms * 8, cudaMemcpyDeviceToHost));
     std::sort(h.begin(), h.end());
-    const double warp_instr = (double)iters * 32 * 32;       // per SM: 32 warps x iters x 32 ops
+    const double warp_instr = (double)iters * 32 * 32 * instr_per_op;       // per SM: 32 warps x iters x 32 ops
     printf("int %-10s median clocks %llu  warp-instr/clk/SM %.3f  (per sub-partition %.3f)  kernel %.3f ms\n", name,
            h[sms / 2], warp_instr / (double)h[sms / 2], warp_instr / (double)h[sms / 2] / 4, ms);
 }
@@ -297,6 +306,14 @@ int main(int argc, char** argv)
     run_int<6>("I2IP", sink, dclk, sms);
     run_int<7>("PRMT", sink, dclk, sms);
     run_int<10>("IMAD.WIDE", sink, dclk, sms);
+    run_int<11>("ADD+MAX", sink, dclk, sms);
+    run_int<12>("DP4A", sink, dclk, sms);
+    run_int<13>("DP2A", sink, dclk, sms);
+    run_int<14>("SHFL", sink, dclk, sms);
+    run_int<20>("IMAD.HI,SHF", sink, dclk, sms, 2);
+    run_int<21>("IMAD,PRMT", sink, dclk, sms, 2);
+    run_int<22>("IMAD.HI,IADD", sink, dclk, sms, 2);
+    run_int<23>("SHF,PRMT", sink, dclk, sms, 2);
 
     // (3) TMEM loads
     for (int nw : {1, 4, 8, 16}) {
