@@ -16,8 +16,9 @@
 // warp computes the next item's scores while the Softmax of the current one runs.
 //
 // Work item = (batch, head, 128-row query tile), handed out dynamically (full tiles first) through a counter in
-// the workspace status block.  One CTA per SM, 18 warps: warp 0 = TMA producer (3-stage ring of Q/K/V tiles),
-// warp 1 = MMA issuer, warps 2..17 = Softmax + output (warp w may only touch TMEM lanes 32*(w%4)..).
+// the workspace status block.  One CTA per SM, 20 warps: warps 0..15 = Softmax + output (warp w may only
+// touch TMEM lanes 32*(w%4)..), warp 16 = TMA producer (3-stage ring of Q/K/V tiles), warp 17 = MMA issuer, warps
+// 18 and 19 idle (they complete the group of four whose registers go to the Softmax warps).
 // The output of item k is requantised after the Softmax of item k+1, when its P V product is certainly done.
 #include <algorithm>
 
@@ -25,8 +26,16 @@
 
 namespace iptq {
 
-constexpr int ATT_THREADS = 576;
-constexpr int ATT_SOFTMAX_THREADS = 512;
+constexpr int ATT_SOFTMAX_THREADS = 512;                 // warps 0..15
+constexpr int ATT_SVC_WARP = ATT_SOFTMAX_THREADS / 32;   // the service group: TMA producer, MMA issuer, two idle warps
+constexpr int ATT_THREADS = ATT_SOFTMAX_THREADS + 128;
+// Registers per thread once the roles have split (setmaxnreg).  The CTA's pool is what it was launched with, 640
+// threads x 96 registers; the service group keeps 32 per thread and the Softmax warps, which hold a quarter of a
+// score row each, take 112 (16 x 112 + 4 x 32 = 20 x 96: all of the pool and no more).  At 96 the Softmax code
+// spills 16-22 registers into its loops; at 112, one or two (ViT-Base attention 84.5 -> 76.5 us).
+constexpr int ATT_LAUNCH_REGS = 96, ATT_SOFTMAX_REGS = 112, ATT_SVC_REGS = 32;
+static_assert((ATT_SOFTMAX_THREADS / 32) * ATT_SOFTMAX_REGS + 4 * ATT_SVC_REGS <= (ATT_THREADS / 32) * ATT_LAUNCH_REGS,
+              "the register counts after the split exceed the CTA's pool: reg_alloc would wait for ever");
 constexpr int ATT_STAGES = 3;              // upper bound of the Q/K/V ring depth
 
 struct AttnParams {
@@ -101,7 +110,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         prefetch_tensormap(&map_k);
         prefetch_tensormap(&map_v);
     }
-    if (warp == 1) {
+    if (warp == ATT_SVC_WARP + 1) {
         tmem_alloc(tmem_slot, p.tmem_cols);
         tmem_relinquish();
     }
@@ -111,96 +120,101 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t tmem_base = *tmem_slot;
     grid_dep_launch();
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer + work distribution
-        if (elect_one()) {
-            grid_dep_wait();                                   // q/k/v come from the previous kernel
-            int s = 0; uint32_t ph = 0;
-            for (;;) {
-                if (!mbar_wait(&kv_empty[s], ph ^ 1u, ctl, p.status, 11)) break;
-                const int it = atomicAdd(&p.status->work_next, 1);
-                if (it >= p.items) {
-                    item_of[s] = -1;
-                    mbar_arrive(&kv_full[s]);                  // release: the consumers see the stop mark
-                    break;
+    if (warp >= ATT_SVC_WARP) {
+        // the service group: its four warps give registers back at one place, then two of them take a role
+        reg_dealloc<ATT_SVC_REGS>();
+        if (warp == ATT_SVC_WARP) {
+            // ------------------------------------------------------------ TMA producer + work distribution
+            if (elect_one()) {
+                grid_dep_wait();                                   // q/k/v come from the previous kernel
+                int s = 0; uint32_t ph = 0;
+                for (;;) {
+                    if (!mbar_wait_nocall(&kv_empty[s], ph ^ 1u, ctl, p.status, 11)) break;
+                    const int it = atomicAdd(&p.status->work_next, 1);
+                    if (it >= p.items) {
+                        item_of[s] = -1;
+                        mbar_arrive(&kv_full[s]);                  // release: the consumers see the stop mark
+                        break;
+                    }
+                    int bh, mt;
+                    decode_item(p, it, bh, mt);
+                    const int h = bh % p.H, b = bh / p.H;
+                    item_of[s] = it;
+                    uint8_t* st = smem + s * p.stage_bytes;
+                    mbar_expect_tx(&kv_full[s], (uint32_t)((128 + p.npad_s + p.kpad) * DH));   // bytes of the three full boxes
+                    tma_load_4d(st, &map_q, &kv_full[s], 0, mt * 128, h, b);
+                    tma_load_4d(st + p.q_bytes, &map_k, &kv_full[s], 0, 0, h, b);
+                    tma_load_4d(st + p.q_bytes + p.k_bytes, &map_v, &kv_full[s], 0, 0, h, b);
+                    if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
-                int bh, mt;
-                decode_item(p, it, bh, mt);
-                const int h = bh % p.H, b = bh / p.H;
-                item_of[s] = it;
-                uint8_t* st = smem + s * p.stage_bytes;
-                mbar_expect_tx(&kv_full[s], (uint32_t)((128 + p.npad_s + p.kpad) * DH));   // bytes of the three full boxes
-                tma_load_4d(st, &map_q, &kv_full[s], 0, mt * 128, h, b);
-                tma_load_4d(st + p.q_bytes, &map_k, &kv_full[s], 0, 0, h, b);
-                tma_load_4d(st + p.q_bytes + p.k_bytes, &map_v, &kv_full[s], 0, 0, h, b);
-                if (++s == p.stages) { s = 0; ph ^= 1u; }
-            }
-            // the last CTA to finish re-arms the counters for the next launch that uses this workspace
-            __threadfence();
-            if (atomicAdd(&p.status->work_done, 1) == (int)gridDim.x - 1) {
-                p.status->work_next = 0;
-                p.status->work_done = 0;
+                // the last CTA to finish re-arms the counters for the next launch that uses this workspace
                 __threadfence();
+                if (atomicAdd(&p.status->work_done, 1) == (int)gridDim.x - 1) {
+                    p.status->work_next = 0;
+                    p.status->work_done = 0;
+                    __threadfence();
+                }
             }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer: S(k), then P V of item k-1
-        if (elect_one()) {
-            const uint32_t idesc_s = umma_idesc_i8(128, p.npad_s, true, true, false, false);
-            const uint32_t idesc_o = umma_idesc_i8(128, DH, false, true, false, true);     // u8 P (K-major) x s8 V (MN-major)
-            const uint32_t tmem_o = tmem_base + (uint32_t)p.o_col;
-            int s = 0; uint32_t ph = 0;
-            int s_prev = 0;
-            auto issue_pv = [&](int k) -> bool {                // k = item count index of the item whose P is ready
-                if (!mbar_wait(&p_ready[k & 1], (uint32_t)(k >> 1) & 1u, ctl, p.status, 14)) return false;
-                if (!mbar_wait(o_empty, ((uint32_t)k & 1u) ^ 1u, ctl, p.status, 12)) return false;   // previous O has been read
-                tc_fence_after_sync();
-                const uint32_t p_addr = smem_u32(sP + (k & 1) * p.p_bytes);
-                const uint32_t v_addr = smem_u32(smem + s_prev * p.stage_bytes) + p.q_bytes + p.k_bytes;
-                for (int ks = 0; ks < p.kpad / 32; ++ks) {
-                    // A = P: K-major, 128-byte swizzle, column blocks of 128 keys are 16 KB apart
-                    const uint64_t da = umma_smem_desc(p_addr + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, 128);
-                    // B = V [keys, DH]: MN-major (DH contiguous), DH-byte swizzle, 8-key groups 8*DH apart
-                    const uint64_t db = umma_smem_desc(v_addr + ks * 32 * DH, 8 * DH, 8 * DH, DH);
-                    umma_i8(tmem_o, da, db, idesc_o, ks != 0 ? 1u : 0u);
-                    if constexpr (VARIANT == IPTQ_SM_LOG2) {
-                        // low-order plane (probabilities 2^-8 .. 2^-15) into its own accumulator behind the first
-                        const uint64_t da2 = umma_smem_desc(p_addr + p.p_plane + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, 128);
-                        umma_i8(tmem_o + (uint32_t)DH, da2, db, idesc_o, ks != 0 ? 1u : 0u);
-                    }
-                }
-                umma_commit(&kv_empty[s_prev]);                // the stage may be refilled
-                umma_commit(o_full);
-                return true;
-            };
-            int k = 0;
-            for (;; ++k) {
-                if (!mbar_wait(&kv_full[s], ph, ctl, p.status, 13)) break;
-                const bool stop = item_of[s] < 0;
-                if (!stop) {
-                    if (!mbar_wait(s_empty, ((uint32_t)k & 1u) ^ 1u, ctl, p.status, 18)) break;   // S(k-1) is in registers
+        } else if (warp == ATT_SVC_WARP + 1) {
+            // ------------------------------------------------------------ MMA issuer: S(k), then P V of item k-1
+            if (elect_one()) {
+                const uint32_t idesc_s = umma_idesc_i8(128, p.npad_s, true, true, false, false);
+                const uint32_t idesc_o = umma_idesc_i8(128, DH, false, true, false, true);     // u8 P (K-major) x s8 V (MN-major)
+                const uint32_t tmem_o = tmem_base + (uint32_t)p.o_col;
+                int s = 0; uint32_t ph = 0;
+                int s_prev = 0;
+                auto issue_pv = [&](int k) -> bool {                // k = item count index of the item whose P is ready
+                    if (!mbar_wait_nocall(&p_ready[k & 1], (uint32_t)(k >> 1) & 1u, ctl, p.status, 14)) return false;
+                    if (!mbar_wait_nocall(o_empty, ((uint32_t)k & 1u) ^ 1u, ctl, p.status, 12)) return false;   // previous O has been read
                     tc_fence_after_sync();
-                    const uint32_t q_addr = smem_u32(smem + s * p.stage_bytes);
-                    const uint32_t k_addr = q_addr + p.q_bytes;
-                    // S = Q K^T: both operands K-major with DH-byte rows (DH-byte swizzle, 8-row groups 8*DH apart)
-#pragma unroll
-                    for (int kk = 0; kk < DH / 32; ++kk) {
-                        const uint64_t da = umma_smem_desc(q_addr + kk * 32, 16, 8 * DH, DH);
-                        const uint64_t db = umma_smem_desc(k_addr + kk * 32, 16, 8 * DH, DH);
-                        umma_i8(tmem_base, da, db, idesc_s, kk != 0 ? 1u : 0u);
+                    const uint32_t p_addr = smem_u32(sP + (k & 1) * p.p_bytes);
+                    const uint32_t v_addr = smem_u32(smem + s_prev * p.stage_bytes) + p.q_bytes + p.k_bytes;
+                    for (int ks = 0; ks < p.kpad / 32; ++ks) {
+                        // A = P: K-major, 128-byte swizzle, column blocks of 128 keys are 16 KB apart
+                        const uint64_t da = umma_smem_desc(p_addr + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, 128);
+                        // B = V [keys, DH]: MN-major (DH contiguous), DH-byte swizzle, 8-key groups 8*DH apart
+                        const uint64_t db = umma_smem_desc(v_addr + ks * 32 * DH, 8 * DH, 8 * DH, DH);
+                        umma_i8(tmem_o, da, db, idesc_o, ks != 0 ? 1u : 0u);
+                        if constexpr (VARIANT == IPTQ_SM_LOG2) {
+                            // low-order plane (probabilities 2^-8 .. 2^-15) into its own accumulator behind the first
+                            const uint64_t da2 = umma_smem_desc(p_addr + p.p_plane + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, 128);
+                            umma_i8(tmem_o + (uint32_t)DH, da2, db, idesc_o, ks != 0 ? 1u : 0u);
+                        }
                     }
-                    umma_commit(s_full);
+                    umma_commit(&kv_empty[s_prev]);                // the stage may be refilled
+                    umma_commit(o_full);
+                    return true;
+                };
+                int k = 0;
+                for (;; ++k) {
+                    if (!mbar_wait_nocall(&kv_full[s], ph, ctl, p.status, 13)) break;
+                    const bool stop = item_of[s] < 0;
+                    if (!stop) {
+                        if (!mbar_wait_nocall(s_empty, ((uint32_t)k & 1u) ^ 1u, ctl, p.status, 18)) break;   // S(k-1) is in registers
+                        tc_fence_after_sync();
+                        const uint32_t q_addr = smem_u32(smem + s * p.stage_bytes);
+                        const uint32_t k_addr = q_addr + p.q_bytes;
+                        // S = Q K^T: both operands K-major with DH-byte rows (DH-byte swizzle, 8-row groups 8*DH apart)
+    #pragma unroll
+                        for (int kk = 0; kk < DH / 32; ++kk) {
+                            const uint64_t da = umma_smem_desc(q_addr + kk * 32, 16, 8 * DH, DH);
+                            const uint64_t db = umma_smem_desc(k_addr + kk * 32, 16, 8 * DH, DH);
+                            umma_i8(tmem_base, da, db, idesc_s, kk != 0 ? 1u : 0u);
+                        }
+                        umma_commit(s_full);
+                    }
+                    if (k > 0 && !issue_pv(k - 1)) break;
+                    if (stop) break;
+                    s_prev = s;
+                    if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
-                if (k > 0 && !issue_pv(k - 1)) break;
-                if (stop) break;
-                s_prev = s;
-                if (++s == p.stages) { s = 0; ph ^= 1u; }
             }
         }
     } else {
         // ------------------------------------------------------------ softmax + output warps
+        reg_alloc<ATT_SOFTMAX_REGS>();
         const int quad = warp & 3;                             // TMEM lane quadrant this warp may touch
-        const int part = (warp - 2) >> 2;                      // which quarter of the columns
+        const int part = warp >> 2;                            // which quarter of the columns
         const int rloc = quad * 32 + lane;                     // row inside the 128-row tile
         const uint32_t trow = tmem_base + ((uint32_t)(quad * 32) << 16);
         const uint32_t p_row0 = smem_u32(sP) + (uint32_t)((rloc >> 3) * 1024 + (rloc & 7) * 128);
@@ -218,9 +232,9 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 // written and fenced by iptq_softmax_table(): safe to read ahead of the dependency wait
                 const int4* src = reinterpret_cast<const int4*>(p.lut_src);
                 int4* dst = reinterpret_cast<int4*>(lut);
-                for (int i = (int)threadIdx.x - 64; i < (p.lut_n + 8) / 8; i += ATT_SOFTMAX_THREADS) dst[i] = __ldg(src + i);
+                for (int i = (int)threadIdx.x; i < (p.lut_n + 8) / 8; i += ATT_SOFTMAX_THREADS) dst[i] = __ldg(src + i);
             } else {
-                for (int d = (int)threadIdx.x - 64; d <= p.lut_n; d += ATT_SOFTMAX_THREADS)
+                for (int d = (int)threadIdx.x; d <= p.lut_n; d += ATT_SOFTMAX_THREADS)
                     lut[d] = d < p.lut_n ? (uint16_t)exp_core_nd<VARIANT>(-d, p.ex) : (uint16_t)0;
             }
             named_barrier(5, ATT_SOFTMAX_THREADS);              // the table is complete before anyone reads it
@@ -229,7 +243,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
         // requantises and stores this thread's share of the output tile of item (b, h, mt), count index k
         auto epilogue = [&](int k, int b, int h, int mt) -> bool {
-            if (!mbar_wait(o_full, (uint32_t)k & 1u, ctl, p.status, 16)) return false;
+            if (!mbar_wait_nocall(o_full, (uint32_t)k & 1u, ctl, p.status, 16)) return false;
             tc_fence_after_sync();
             const int row = mt * 128 + rloc;
             constexpr int OPARTS = DH / 16;                    // threads of a row that hold 16 output columns each
@@ -272,7 +286,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         for (;; ++k) {
             // the four warps of a quadrant meet at two named barriers per item: a warp that gives up before them
             // arrives without waiting, so that a bounded wait running out can never strand the others
-            if (!mbar_wait(&kv_full[s], ph, ctl, p.status, 17)) {   // acquire: the item number is visible
+            if (!mbar_wait_nocall(&kv_full[s], ph, ctl, p.status, 17)) {   // acquire: the item number is visible
                 named_barrier_arrive(1 + quad, 128); named_barrier_arrive(1 + quad, 128);
                 ok = false;
                 break;
@@ -291,7 +305,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const unsigned my_id = HAS_MASK ? mrow[valid ? row : 0] : 0u;
             const uint32_t p_row = p_row0 + (uint32_t)((k & 1) * p.p_bytes);
 
-            if (!mbar_wait(s_full, (uint32_t)k & 1u, ctl, p.status, 15)) {
+            if (!mbar_wait_nocall(s_full, (uint32_t)k & 1u, ctl, p.status, 15)) {
                 named_barrier_arrive(1 + quad, 128); named_barrier_arrive(1 + quad, 128);
                 ok = false;
                 break;
@@ -447,7 +461,7 @@ attention_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         for (int i = 0; i < 64; ++i) __nanosleep(2000);
         __syncthreads();
     }
-    if (warp == 1) {
+    if (warp == ATT_SVC_WARP + 1) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, p.tmem_cols);
     }

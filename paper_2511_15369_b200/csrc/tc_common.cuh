@@ -71,7 +71,7 @@ __device__ __forceinline__ uint64_t global_timer_ns()
 
 // Bounded wait.  Returns false when the wait ran out or another role already aborted; the first
 // waiter to give up records (where, blockIdx) in the status block.
-static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, CtaControl* ctl, StatusBlock* status, int where)
+__device__ __forceinline__ bool mbar_wait_poll(uint64_t* bar, uint32_t parity, CtaControl* ctl, StatusBlock* status, int where)
 {
     uint64_t t0 = 0;
     // 16 tries in a row cost nothing but the tries; the abort flag and the clock are looked at between such runs
@@ -97,6 +97,10 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parit
     __threadfence();
     return false;
 }
+static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, CtaControl* ctl, StatusBlock* status, int where)
+{
+    return mbar_wait_poll(bar, parity, ctl, status, where);
+}
 // A wait that is already satisfied -- the common case for a consumer that runs behind its producer -- is one
 // try (about 30 clocks); the loop with its bookkeeping is a call (measured: 200 clocks and more when inlined).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, CtaControl* ctl, StatusBlock* status,
@@ -104,6 +108,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, CtaCon
 {
     if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, ctl, status, where);
+}
+// The same with the polling loop inline, for kernels whose warp groups change their register count (setmaxnreg): a
+// called function would have to fit the smallest of the counts, and the assembler refuses the mix.
+__device__ __forceinline__ bool mbar_wait_nocall(uint64_t* bar, uint32_t parity, CtaControl* ctl, StatusBlock* status,
+                                                 int where)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_poll(bar, parity, ctl, status, where);
 }
 
 // The same wait for a whole (converged) warp: one lane polls, the others learn the outcome from a shuffle, which
@@ -153,6 +165,14 @@ __device__ __forceinline__ void bulk_wait_read_but_one() { asm volatile("cp.asyn
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // generic-proxy writes to shared memory -> visible to the async proxy (UMMA / TMA reads)
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// ---------------------------------------------------------------- registers per thread, per warp group
+// All four warps of an aligned group of four execute the same one of these.  reg_alloc waits until the CTA's pool
+// (the registers it was launched with, threads x registers per thread) has room and never gives up: the counts of
+// all groups must add up to no more than that pool (assert it at compile time), and the warps that give registers
+// back must do so unconditionally.
+template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
 // ---------------------------------------------------------------- TMEM
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_result, uint32_t ncols)
