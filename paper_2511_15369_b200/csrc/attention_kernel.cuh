@@ -479,11 +479,16 @@ int launch_attn(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap&
         auto kern = attention_kernel<DH, VARIANT, HB, HM, PS, LT>;                                                \
         static int configured[64];          /* largest dynamic shared memory size set so far, per device */     \
         if (configured[dev] < smem_bytes) {                                                                       \
+            /* the register counts the roles take after the split are sized for a launch with ATT_LAUNCH_REGS: a   \
+               build that starts this kernel with fewer would leave its Softmax warps waiting for registers */     \
+            cudaFuncAttributes fa;                                                                                \
+            if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess || ((fa.numRegs + 7) & ~7) != ATT_LAUNCH_REGS)   \
+                return IPTQ_ERR_CUDA;                                                                             \
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) \
                 return IPTQ_ERR_CUDA;                                                                             \
             configured[dev] = smem_bytes;                                                                         \
         }                                                                                                         \
-        launch_kernel(kern, grid, ATT_THREADS, smem_bytes, st, mq, mk, mv, p);                                               \
+        launch_kernel(kern, grid, ATT_THREADS, smem_bytes, st, mq, mk, mv, p);                                    \
     } while (0)
 #define IPTQ_ATT_LAUNCH2(HB, HM, PS)                                                                              \
     do {                                                                                                          \
