@@ -40,6 +40,17 @@ def test_every_admissible_shape_gets_a_plan_that_fits_the_sm(residual, table):
             assert p.tile_tokens == 64          # a wider tile would be mostly padding
 
 
+def test_small_batches_take_narrow_tiles():
+    # less than one round of 256-token tiles: the narrowest tile that still fits one round of 148 SMs, else 128
+    assert plan(197, 576, 192).tile_tokens == 64 and plan(197, 192, 768, residual=True).tile_tokens == 64
+    assert plan(1576, 1152, 384).tile_tokens == 128                      # 9 x 25 tiles of 64 tokens are too many
+    assert plan(1576, 384, 1536, residual=True).tile_tokens == 64        # 3 x 25 fit
+    assert plan(1576, 768, 3072, residual=True).tile_tokens == 128
+    assert plan(1576, 2304, 768).tile_tokens == 128 and plan(1576, 2304, 768).cta_pairs == 0
+    # one round or more at 256 tokens: unchanged
+    assert plan(12608, 384, 384, residual=True).tile_tokens == 256
+
+
 def test_the_configurations_of_the_benchmark():
     # short reductions have room for two staging buffers per epilogue warp, the long ones of ViT-Base keep their ring
     assert plan(200704, 96, 96, residual=True).staging_buffers == 2 and plan(200704, 288, 96).staging_buffers == 2
