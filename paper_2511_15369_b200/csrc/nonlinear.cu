@@ -507,45 +507,48 @@ layernorm_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int6
     }
 }
 
-// Short rows (dim <= 128, dim % 16 == 0: the first Swin stage): four lanes share a row, so a warp step covers eight
-// rows.  Lane q of a row takes words q, q + 4, ... (WPL = dim / 16 words); row sums are two xor-shuffles over the
-// four lanes, and every lane then runs the scalar part (variance, square root, reciprocal) of its own row, so the
-// hundred dependent instructions of that part are shared by eight rows without any broadcast.
-template <int WPL, bool PTF, bool SAT8, bool ZPF>
+// Short rows (dim <= 128, dim % 16 == 0: the first Swin stage): LPR lanes share a row, so a warp step covers 32 / LPR
+// rows.  Lane q of a row takes words q, q + LPR, ... (WPL = dim / (4 LPR) words); row sums are xor-shuffles over the
+// LPR lanes, and every lane then runs the scalar part (variance, square root, reciprocal) of its own row, so the
+// hundred dependent instructions of that part are shared by 32 / LPR rows without any broadcast.  Two lanes per row
+// up to 96 channels (16 rows per scalar part: 96 channels 20.8 -> 19.5 us, 64 channels 17.4 -> 15.1 us on 200 k rows),
+// four at 128, where twelve more words per lane would spill.
+template <int LPR, int WPL, bool PTF, bool SAT8, bool ZPF>
 __global__ void __launch_bounds__(256, 4)
 layernorm_short_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y, int64_t rows,
                             const int32_t* __restrict__ gamma_q, const int32_t* __restrict__ beta_q,
                             const uint8_t* __restrict__ ptf, const LnDev c)
 {
     const int lane = threadIdx.x & 31;
-    const int q = lane & 3;                                   // position inside the row's four lanes
+    constexpr int RPW = 32 / LPR;                             // rows per warp step
+    const int q = lane & (LPR - 1);                           // position inside the row's lanes
     const int D = c.dim;                                      // = 16 * WPL
     grid_dep_launch();
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    const int64_t steps = (rows + 7) / 8;
-    // The per-channel parameters live in shared memory (the four lanes of a row read four addresses, the eight rows of
-    // a warp the same four: no bank conflict).  In registers they are 48 per thread and halve the resident warps, and
+    const int64_t steps = (rows + RPW - 1) / RPW;
+    // The per-channel parameters live in shared memory (the lanes of a row read consecutive addresses, the rows of a
+    // warp the same ones: no bank conflict).  In registers they are 48 per thread and halve the resident warps, and
     // resident warps are what hides a row's chain of dependent steps (load, two reductions, square root, divide):
     // 64 registers and four CTAs per SM instead of 98 and two took the 96-channel case from 25.0 to 20.8 us.
-    __shared__ int4 g[4 * WPL], b[4 * WPL];
+    __shared__ int4 g[LPR * WPL], b[LPR * WPL];
     unsigned sh[WPL];
-    for (int i = threadIdx.x; i < 4 * WPL; i += blockDim.x) {
+    for (int i = threadIdx.x; i < LPR * WPL; i += blockDim.x) {
         g[i] = __ldg(reinterpret_cast<const int4*>(gamma_q) + i);
         b[i] = __ldg(reinterpret_cast<const int4*>(beta_q) + i);
     }
 #pragma unroll
-    for (int k = 0; k < WPL; ++k) sh[k] = PTF ? __ldg(reinterpret_cast<const unsigned*>(ptf) + q + 4 * k) : 0u;
+    for (int k = 0; k < WPL; ++k) sh[k] = PTF ? __ldg(reinterpret_cast<const unsigned*>(ptf) + q + LPR * k) : 0u;
     __syncthreads();
     grid_dep_wait();                                          // gamma / beta above are static; the rows come from the previous kernel
     const int om = c.out.mult, ornd = c.out.rnd, osh = c.out.shift, ozp = c.out.zp;
     for (int64_t step = warp; step < steps; step += nwarps) {
-        const int64_t row = step * 8 + (lane >> 2);
+        const int64_t row = step * RPW + lane / LPR;
         const bool live = row < rows;
         const int* xr = reinterpret_cast<const int*>(x + (live ? row : 0) * D);
         int w[WPL];
 #pragma unroll
-        for (int k = 0; k < WPL; ++k) w[k] = live ? __ldcs(xr + q + 4 * k) : 0;
+        for (int k = 0; k < WPL; ++k) w[k] = live ? __ldcs(xr + q + LPR * k) : 0;
         int s1 = 0;
         unsigned s2 = 0;
 #pragma unroll
@@ -563,7 +566,7 @@ layernorm_short_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y
             }
         }
         s1 += __shfl_xor_sync(kFull, s1, 1); s2 += __shfl_xor_sync(kFull, s2, 1);
-        s1 += __shfl_xor_sync(kFull, s1, 2); s2 += __shfl_xor_sync(kFull, s2, 2);
+        if (LPR == 4) { s1 += __shfl_xor_sync(kFull, s1, 2); s2 += __shfl_xor_sync(kFull, s2, 2); }
         const long long V = (long long)D * (long long)s2 - (long long)s1 * (long long)s1;            // D^2 var, exact
         const unsigned long long rt = isqrt_variant((unsigned long long)V, c.variant);                // D * std
         const long long F = rt ? (long long)floor_div_f64(1099511627776.0, (double)rt) : 0;          // floor(2^40 / rt)
@@ -582,7 +585,7 @@ layernorm_short_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y
                 if (!SAT8) o = max(c.out.qmin, min(c.out.qmax, o));
                 return o;
             };
-            const int4 gk = g[q + 4 * k], bk = b[q + 4 * k];
+            const int4 gk = g[q + LPR * k], bk = b[q + LPR * k];
             const int o0 = elem(sext_byte<0>(wk), 0, gk.x, bk.x);
             const int o1 = elem(sext_byte<1>(wk), 1, gk.y, bk.y);
             const int o2 = elem(sext_byte<2>(wk), 2, gk.z, bk.z);
@@ -592,24 +595,26 @@ layernorm_short_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ y
         if (live) {
             int* yr = reinterpret_cast<int*>(y + row * D);
 #pragma unroll
-            for (int k = 0; k < WPL; ++k) __stcs(yr + q + 4 * k, out[k]);
+            for (int k = 0; k < WPL; ++k) __stcs(yr + q + LPR * k, out[k]);
         }
     }
 }
 
-template <int WPL>
+// W16 = dim / 16
+template <int W16>
 static int launch_ln_short(const int8_t* x, int8_t* y, int64_t rows, const int32_t* gq, const int32_t* bq,
                            const uint8_t* ptf_in, const LnDev& c, cudaStream_t st)
 {
     const int threads = 256;
-    const int64_t want = ((rows + 7) / 8 + 7) / 8;
+    constexpr int LPR = W16 <= 6 ? 2 : 4, WPL = 4 * W16 / LPR;
+    const int64_t want = ((rows + 32 / LPR - 1) / (32 / LPR) + 7) / 8;
     const int grid = (int)std::min<int64_t>(want, (int64_t)sm_count() * 8);
     const bool sat8 = c.out.qmin == -128 && c.out.qmax == 127;
     LnDev cc = c;
     const long long rz = (long long)c.out.rnd + ((long long)c.out.zp << c.out.shift);
     const bool zpf = rz > -(1ll << 30) && rz < (1ll << 30);
     if (zpf) { cc.out.rnd = (int)rz; cc.out.zp = 0; }
-#define IPTQ_LNS_GO(P, S8, ZF) launch_kernel(layernorm_short_rows_kernel<WPL, P, S8, ZF>, grid, threads, 0, st, x, y, rows, gq, bq, ptf_in, cc)
+#define IPTQ_LNS_GO(P, S8, ZF) launch_kernel(layernorm_short_rows_kernel<LPR, WPL, P, S8, ZF>, grid, threads, 0, st, x, y, rows, gq, bq, ptf_in, cc)
     if (c.variant == IPTQ_LN_PTF) { if (sat8) IPTQ_LNS_GO(true, true, false); else IPTQ_LNS_GO(true, false, false); }
     else if (!sat8)               { IPTQ_LNS_GO(false, false, false); }
     else if (zpf)                 { IPTQ_LNS_GO(false, true, true); }
@@ -677,7 +682,7 @@ int layernorm_launch(const int8_t* x, int8_t* y, int64_t rows, int dim, const in
     LnDev c;
     c.variant = consts->variant; c.dim = dim; c.out = to_dev(consts->out);
     if ((dim & 15) == 0 && dim <= 128 && rows >= 64) {
-        switch (dim / 16) {                                   // words per lane with four lanes per row
+        switch (dim / 16) {
             case 1: return launch_ln_short<1>(x, y, rows, gq, bq, ptf, c, st);
             case 2: return launch_ln_short<2>(x, y, rows, gq, bq, ptf, c, st);
             case 3: return launch_ln_short<3>(x, y, rows, gq, bq, ptf, c, st);

@@ -274,7 +274,7 @@ def test_layernorm_parity(api, orc, variant, rows, dim):
     assert (got == want).all()
 
 
-@pytest.mark.parametrize("dim,rows", [(192, 40), (96, 75), (128, 64), (16, 100), (48, 333)])
+@pytest.mark.parametrize("dim,rows", [(192, 40), (96, 75), (128, 64), (16, 100), (48, 333), (64, 201), (32, 129)])
 def test_layernorm_degenerate_rows(api, orc, dim, rows):
     """Constant rows, extreme variances, a ragged last step -- for the general kernel (dim 192) and for the
     four-lanes-per-row kernel of short rows (dim <= 128, at least 64 rows)."""
