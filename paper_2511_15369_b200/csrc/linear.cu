@@ -96,10 +96,17 @@ struct GemmParams {
 // The tiles of this CTA, round by round: tiles are numbered with the channel tile fastest, so that CTAs running side by side
 // share an activation tile in L2.  A CTA pair takes two neighbouring channel tiles of one token tile (the odd CTA's
 // may lie past N when the number of channel tiles is odd: its weight rows then read as zeros and nothing is stored).
-template <bool PAIR>
+// Rounds alternate in direction: CTA j of S takes tile r S + j in even rounds and r S + (S - 1 - j) in odd ones.  The
+// ragged last token tile is narrower and its tiles come last, so the few tiles of a final, partly filled round then
+// go to the CTAs whose previous tile was a short one too, instead of to those that have only had full ones
+// (ViT-Base proj 22.1 -> 21.4 us, FC2 48.6 -> 47.9 us, DeiT-Small FC2 12.1 -> 11.3 us).  ALTERNATE = false keeps every
+// round in the same direction: the tabulated-GELU kernel on single CTAs is 7-10 % slower with the longer walk state.
+template <bool PAIR, bool ALTERNATE>
 struct TileWalk {
     int tt, ct;                  // the current tile: token tile, channel tile
-    int c, dtt, dc, nc, rank;    // channel unit (tile, or pair of tiles), step per round in both coordinates, units per row
+    int c, nc, rank;             // channel unit (tile, or pair of tiles), units per row of tiles
+    int dtt0, dc0, dtt1, dc1;    // step to the next round's tile after an even and after an odd round
+    int odd;                     // parity of the current round
     __device__ __forceinline__ void start(const GemmParams& p, uint32_t rank_)
     {
         rank = (int)rank_;
@@ -107,13 +114,17 @@ struct TileWalk {
         const int first = PAIR ? (int)cluster_id_x() : (int)blockIdx.x;
         const int stride = PAIR ? (int)cluster_count_x() : (int)gridDim.x;
         tt = first / nc; c = first - tt * nc;
-        dtt = stride / nc; dc = stride - dtt * nc;
+        const int s0 = ALTERNATE ? 2 * (stride - 1 - first) + 1 : stride, s1 = ALTERNATE ? 2 * first + 1 : stride;
+        dtt0 = s0 / nc; dc0 = s0 - dtt0 * nc;
+        dtt1 = s1 / nc; dc1 = s1 - dtt1 * nc;
+        odd = 0;
         ct = PAIR ? 2 * c + rank : c;
     }
     // one round further (no division in the roles' loops)
     __device__ __forceinline__ void next()
     {
-        tt += dtt; c += dc;
+        if (ALTERNATE) { tt += odd ? dtt1 : dtt0; c += odd ? dc1 : dc0; odd ^= 1; }
+        else { tt += dtt0; c += dc0; }
         if (c >= nc) { c -= nc; ++tt; }
         ct = PAIR ? 2 * c + rank : c;
     }
@@ -183,7 +194,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         if (elect_one()) {
             grid_dep_wait();                                   // the activations (and unpacked weights) come from earlier kernels
             int s = 0; uint32_t ph = 0;
-            TileWalk<PAIR> tw;
+            TileWalk<PAIR, PAIR || EPI != EPI_GELU_TAB> tw;
             for (tw.start(p, rank); tw.valid(p); tw.next()) {
                 const int tt = tw.tt, ct = tw.ct;
                 bool ok = true;
@@ -219,7 +230,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const uint64_t desc_ring = umma_smem_desc(smem_u32(ring), 16, 1024, 128);
             const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4;
             int s = 0; uint32_t ph = 0, soff = 0;
-            TileWalk<PAIR> tw;
+            TileWalk<PAIR, PAIR || EPI != EPI_GELU_TAB> tw;
             tw.start(p, rank);
             for (int it = 0; tw.valid(p); ++it, tw.next()) {
                 const int tt = tw.tt;
@@ -303,7 +314,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             }
         };
         const uint32_t acc_empty0 = PAIR ? map_to_cta(smem_u32(&acc_empty[0]), 0) : 0u;   // the even CTA's pair of barriers
-        TileWalk<PAIR> tw;
+        TileWalk<PAIR, PAIR || EPI != EPI_GELU_TAB> tw;
         tw.start(p, rank);
         int tt = tw.tt, ct = tw.ct;
         bool have = tw.valid(p);
