@@ -294,6 +294,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             for (int i = ew * 32 + lane; i < IPTQ_GELU_TABLE_SIZE / 16; i += EPI_WARPS * 32) dst[i] = __ldg(src + i);
             named_barrier(1, EPI_WARPS * 32);
         }
+        // The residual term R_res((res - zp) << 16) depends on the residual byte alone: its 256 values are tabulated
+        // once per CTA, with the arithmetic the epilogue would otherwise run per output, and an output then costs a
+        // second shared-memory read instead of a high multiply and a shift.
+        const uint32_t rlut_mid = smem_u32(smem + p.off_tab) + 512u;        // address of the entry of residual byte 0
+        if (EPI == EPI_RESIDUAL) {
+            int* rl = reinterpret_cast<int*>(smem + p.off_tab);
+            const int i = ew * 32 + lane;
+            if (i < 256) rl[i] = requant_core((i - 128) * 65536 - p.res_off, p.res_mult, p.res_rnd, p.res_shift);
+            named_barrier(1, EPI_WARPS * 32);
+        }
         grid_dep_wait();                                       // residual reads and output writes come after this
         // Nothing in a tile's epilogue waits for something that was started in the same tile: the channel constants
         // and the residual block of tile i + 1 are requested during tile i.
@@ -378,6 +388,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 #pragma unroll
                             for (int j = 0; j < 16; ++j)
                                 asm volatile("ld.shared.s8 %0, [%1];" : "=r"(r[j]) : "r"(res_lane + (uint32_t)((ch * 16 + j) * 32)));
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(r[j]) : "r"(rlut_mid + (uint32_t)(r[j] * 4)));
                         }
                         // R of the header: hi32((acc + bias) * mult) + rounding constant, shifted.  The bias add is
                         // written as add-then-max against INT_MIN: a plain add is moved to the multiplier's pipe by the
@@ -399,7 +412,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                                 v[j] = requant_nosat(gelu_core<GELU_VARIANT>(v[j], p.gelu), p.gelu.out);
                                 if (!sat8) v[j] = max(p.gelu.out.qmin, min(p.gelu.out.qmax, v[j]));
                             } else if (EPI == EPI_RESIDUAL) {
-                                v[j] += requant_core(r[j] * 65536 - p.res_off, p.res_mult, p.res_rnd, p.res_shift) + p.out_zp;
+                                v[j] += r[j] + p.out_zp;
                                 if (!sat8) v[j] = max(p.qmin, min(p.qmax, v[j]));
                             } else {
                                 v[j] += p.out_zp;
@@ -611,7 +624,7 @@ static int gemm_layout(GemmParams& p, int TN, bool pair, bool residual, bool tab
     p.epi_bufs = epi_bufs;
     p.off_res = blocks;
     p.off_tab = p.off_res + (residual ? blocks : 0);
-    p.off_bar = p.off_tab + (table ? IPTQ_GELU_TABLE_SIZE : 0);
+    p.off_bar = p.off_tab + (table ? IPTQ_GELU_TABLE_SIZE : residual ? 1024 : 0);   // GELU table, or residual terms
     p.off_ring = (p.off_bar + (2 * MAX_STAGES + 4 + 2 * EPI_WARPS) * 8 + 16 + 1023) & ~1023;
     p.stage_bytes = W_BYTES + (pair ? TN / 2 : TN) * BK;      // a CTA of a pair stages half of the activation tile
     const int room = SMEM_LIMIT - 1024 - p.off_ring;          // 1024: slack for the alignment of the dynamic base
